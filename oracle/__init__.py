@@ -1,0 +1,257 @@
+"""CPU oracle for the OBRS token pass (TEST INFRASTRUCTURE ONLY).
+
+A thin ctypes loader around ``obrs_oracle.cpp`` plus :func:`forward`, which
+strings the oracle's steps together in the paper's order (log-softmax and
+gathers, the two top-k lists, lambda, acceptance and decision, Z_approx and
+exact Z, batch correction, weights).  Only tests, the smoke check and the
+benchmark's CPU-baseline leg may import this package; the product path never
+does, and this package never imports the CUDA path.
+
+Arrays are numpy.  bf16 logits travel as ``uint16`` bit patterns
+(``dtype="bf16"``); fp32 logits as ``float32``.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "obrs_oracle.cpp")
+_LIB = os.path.join(_HERE, "liboracle.so")
+_lib = None
+
+BF16, F32 = 0, 1
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with g++ (no fast-math: summation order is part of it)."""
+    if (not force and os.path.exists(_LIB)
+            and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
+        return _LIB
+    cmd = ["g++", "-O2", "-std=c++17", "-fopenmp", "-fPIC", "-shared", "-o", _LIB, _SRC]
+    subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def _p(a, ct):
+    return None if a is None else a.ctypes.data_as(ctypes.POINTER(ct))
+
+
+def _vp(a):
+    return None if a is None else ctypes.c_void_p(a.ctypes.data)
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        build()
+        _lib = ctypes.CDLL(_LIB)
+        _lib.jo_uniform.restype = ctypes.c_float
+        _lib.jo_uniform.argtypes = [ctypes.c_uint64, ctypes.c_uint64]
+        _lib.jo_lambda_from_budget.restype = ctypes.c_double
+        _lib.jo_loss.restype = ctypes.c_double
+        _lib.jo_num_threads.restype = ctypes.c_int
+    return _lib
+
+
+def num_threads() -> int:
+    return int(lib().jo_num_threads())
+
+
+def set_num_threads(n: int) -> None:
+    lib().jo_set_num_threads(ctypes.c_int(n))
+
+
+def _dtype_code(z: np.ndarray) -> int:
+    if z.dtype == np.uint16:
+        return BF16
+    if z.dtype == np.float32:
+        return F32
+    raise TypeError("logits must be uint16 (bf16 bits) or float32")
+
+
+def _check2d(z):
+    assert z.ndim == 2 and z.flags.c_contiguous
+    return z.shape[0], z.shape[1]
+
+
+def philox4x32_10(ctr, key):
+    c = np.asarray(ctr, dtype=np.uint32)
+    k = np.asarray(key, dtype=np.uint32)
+    out = np.zeros(4, dtype=np.uint32)
+    lib().jo_philox4x32_10(_p(c, ctypes.c_uint32), _p(k, ctypes.c_uint32), _p(out, ctypes.c_uint32))
+    return out
+
+
+def uniform(seed: int, g: int) -> float:
+    return float(lib().jo_uniform(ctypes.c_uint64(seed), ctypes.c_uint64(g)))
+
+
+def lse_gather(za, zp, tokens, mask=None):
+    T, V = _check2d(za)
+    dt = _dtype_code(za)
+    tokens = np.ascontiguousarray(tokens, dtype=np.int32)
+    out = dict(lse_a=np.zeros(T), lse_p=np.zeros(T), lq64=np.zeros(T), lp64=np.zeros(T),
+               lq=np.zeros(T, np.float32), lp=np.zeros(T, np.float32), bad=np.zeros(T, np.uint8))
+    lib().jo_lse_gather(ctypes.c_int64(T), ctypes.c_int64(V), ctypes.c_int64(V), ctypes.c_int(dt),
+                        _vp(za), _vp(zp), _p(tokens, ctypes.c_int32), _p(mask, ctypes.c_uint8),
+                        _p(out["lse_a"], ctypes.c_double), _p(out["lse_p"], ctypes.c_double),
+                        _p(out["lq64"], ctypes.c_double), _p(out["lp64"], ctypes.c_double),
+                        _p(out["lq"], ctypes.c_float), _p(out["lp"], ctypes.c_float),
+                        _p(out["bad"], ctypes.c_uint8))
+    return out
+
+
+def topk(z, k, mask=None):
+    T, V = _check2d(z)
+    idx = np.zeros((T, k), dtype=np.int32)
+    lib().jo_topk(ctypes.c_int64(T), ctypes.c_int64(V), ctypes.c_int64(V), ctypes.c_int(_dtype_code(z)),
+                  _vp(z), _p(mask, ctypes.c_uint8), ctypes.c_int(k), _p(idx, ctypes.c_int32))
+    return idx
+
+
+def lambda_from_budget(lq, lp, budget, mask=None, bad=None):
+    lq = np.ascontiguousarray(lq, np.float32)
+    lp = np.ascontiguousarray(lp, np.float32)
+    return float(lib().jo_lambda_from_budget(ctypes.c_int64(lq.shape[0]), _p(lq, ctypes.c_float),
+                                             _p(lp, ctypes.c_float), _p(mask, ctypes.c_uint8),
+                                             _p(bad, ctypes.c_uint8), ctypes.c_double(budget)))
+
+
+def accept(lq, lp, lam, seed, token_offset=0, mask=None, bad=None):
+    T = lq.shape[0]
+    a = np.zeros(T, np.float32)
+    u = np.zeros(T, np.float32)
+    acc = np.zeros(T, np.uint8)
+    lib().jo_accept(ctypes.c_int64(T), _p(lq, ctypes.c_float), _p(lp, ctypes.c_float),
+                    _p(mask, ctypes.c_uint8), _p(bad, ctypes.c_uint8), ctypes.c_float(lam),
+                    ctypes.c_uint64(seed), ctypes.c_int64(token_offset),
+                    _p(a, ctypes.c_float), _p(u, ctypes.c_float), _p(acc, ctypes.c_uint8))
+    return a, u, acc
+
+
+def z_topk(za, zp, idx_a, idx_p, lse_a, lse_p, lam, mask=None, bad=None):
+    T, V = _check2d(za)
+    k = idx_a.shape[1]
+    zk = np.zeros(T)
+    lib().jo_z_topk(ctypes.c_int64(T), ctypes.c_int64(V), ctypes.c_int64(V), ctypes.c_int(_dtype_code(za)),
+                    _vp(za), _vp(zp), _p(mask, ctypes.c_uint8), _p(bad, ctypes.c_uint8), ctypes.c_int(k),
+                    _p(np.ascontiguousarray(idx_a), ctypes.c_int32),
+                    _p(np.ascontiguousarray(idx_p), ctypes.c_int32),
+                    _p(lse_a, ctypes.c_double), _p(lse_p, ctypes.c_double), ctypes.c_double(lam),
+                    _p(zk, ctypes.c_double))
+    return zk
+
+
+def z_exact(za, zp, lse_a, lse_p, lam, mask=None, bad=None):
+    T, V = _check2d(za)
+    z = np.zeros(T)
+    lib().jo_z_exact(ctypes.c_int64(T), ctypes.c_int64(V), ctypes.c_int64(V), ctypes.c_int(_dtype_code(za)),
+                     _vp(za), _vp(zp), _p(mask, ctypes.c_uint8), _p(bad, ctypes.c_uint8),
+                     _p(lse_a, ctypes.c_double), _p(lse_p, ctypes.c_double), ctypes.c_double(lam),
+                     _p(z, ctypes.c_double))
+    return z
+
+
+_STAT_KEYS = ("n_valid", "n_accept", "alpha_hat", "mean_accept_prob", "z_approx_mean", "kappa",
+              "lambda_used")
+
+
+def batch_weights(lq, lp, acc, a, zk, lam, c1=0.0, mask=None, bad=None):
+    T = lq.shape[0]
+    w = np.zeros(T, np.float32)
+    w64 = np.zeros(T)
+    st = np.zeros(8)
+    lib().jo_batch_weights(ctypes.c_int64(T), _p(lq, ctypes.c_float), _p(lp, ctypes.c_float),
+                           _p(mask, ctypes.c_uint8), _p(bad, ctypes.c_uint8), _p(acc, ctypes.c_uint8),
+                           _p(a, ctypes.c_float), _p(zk, ctypes.c_double), ctypes.c_double(lam),
+                           ctypes.c_double(c1), _p(w, ctypes.c_float), _p(w64, ctypes.c_double),
+                           _p(st, ctypes.c_double))
+    stats = {k: float(st[i]) for i, k in enumerate(_STAT_KEYS)}
+    stats["n_valid"] = int(stats["n_valid"])
+    stats["n_accept"] = int(stats["n_accept"])
+    return w, w64, stats
+
+
+def grad_rows(rows, za, zp, tokens, acc, weight, lse_a, lse_p, n_valid, mask=None, adv=None,
+              grad_out=1.0, lambda_distill=0.0):
+    T, V = _check2d(za)
+    rows = np.ascontiguousarray(rows, dtype=np.int64)
+    tokens = np.ascontiguousarray(tokens, dtype=np.int32)
+    da = np.zeros((rows.shape[0], V))
+    dp = np.zeros((rows.shape[0], V))
+    adv32 = None if adv is None else np.ascontiguousarray(adv, np.float32)
+    lib().jo_grad_rows(ctypes.c_int64(rows.shape[0]), _p(rows, ctypes.c_int64), ctypes.c_int64(V),
+                       ctypes.c_int64(V), ctypes.c_int(_dtype_code(za)), _vp(za), _vp(zp),
+                       _p(tokens, ctypes.c_int32), _p(mask, ctypes.c_uint8), _p(acc, ctypes.c_uint8),
+                       _p(np.ascontiguousarray(weight, np.float32), ctypes.c_float),
+                       _p(adv32, ctypes.c_float), _p(lse_a, ctypes.c_double), _p(lse_p, ctypes.c_double),
+                       ctypes.c_double(n_valid), ctypes.c_double(grad_out), ctypes.c_double(lambda_distill),
+                       _p(da, ctypes.c_double), _p(dp, ctypes.c_double))
+    return da, dp
+
+
+def loss(za64, zp64, tokens, acc, weight64, adv64, logp_ref, logq_ref, pfix, lambda_distill, mask=None):
+    T, V = za64.shape
+    tokens = np.ascontiguousarray(tokens, dtype=np.int32)
+    args = [np.ascontiguousarray(x, np.float64) for x in (za64, zp64)]
+    return float(lib().jo_loss(ctypes.c_int64(T), ctypes.c_int64(V), _p(args[0], ctypes.c_double),
+                               _p(args[1], ctypes.c_double), _p(tokens, ctypes.c_int32),
+                               _p(mask, ctypes.c_uint8), _p(acc, ctypes.c_uint8),
+                               _p(np.ascontiguousarray(weight64, np.float64), ctypes.c_double),
+                               _p(None if adv64 is None else np.ascontiguousarray(adv64, np.float64),
+                                  ctypes.c_double),
+                               _p(np.ascontiguousarray(logp_ref, np.float64), ctypes.c_double),
+                               _p(np.ascontiguousarray(logq_ref, np.float64), ctypes.c_double),
+                               _p(np.ascontiguousarray(pfix, np.float64), ctypes.c_double),
+                               ctypes.c_double(lambda_distill)))
+
+
+def kl_rows(za, zp, lse_a, lse_p, mask=None):
+    T, V = _check2d(za)
+    kl = np.zeros(T)
+    lib().jo_kl_rows(ctypes.c_int64(T), ctypes.c_int64(V), ctypes.c_int64(V), ctypes.c_int(_dtype_code(za)),
+                     _vp(za), _vp(zp), _p(mask, ctypes.c_uint8), _p(lse_a, ctypes.c_double),
+                     _p(lse_p, ctypes.c_double), _p(kl, ctypes.c_double))
+    return kl
+
+
+def forward(za, zp, tokens, mask=None, *, lam=None, budget=None, k=20, seed=0, token_offset=0,
+            c1=0.0, exact=False, want_kl=False):
+    """All forward steps in the paper's order on whole arrays.
+
+    Exactly one of ``lam`` (fixed lambda) and ``budget`` (acceptance budget) is
+    given.  ``k >= V`` makes Z_approx the exact Z.  ``exact=True`` also returns
+    the brute-force full-vocabulary Z beside Z_approx.
+    """
+    assert (lam is None) != (budget is None)
+    T, V = _check2d(za)
+    mask = None if mask is None else np.ascontiguousarray(mask, np.uint8)
+    r = lse_gather(za, zp, tokens, mask)
+    bad = r["bad"]
+    kk = min(k, V)
+    if kk < V:
+        r["topk_idx_a"] = topk(za, kk, mask)
+        r["topk_idx_p"] = topk(zp, kk, mask)
+    if budget is not None:
+        lam = float(np.float32(lambda_from_budget(r["lq"], r["lp"], budget, mask, bad)))
+    lam = float(np.float32(lam))
+    r["lambda"] = lam
+    r["a"], r["u"], r["accept"] = accept(r["lq"], r["lp"], lam, seed, token_offset, mask, bad)
+    if exact or kk >= V:
+        r["z_exact"] = z_exact(za, zp, r["lse_a"], r["lse_p"], lam, mask, bad)
+    if kk < V:
+        r["zk"] = z_topk(za, zp, r["topk_idx_a"], r["topk_idx_p"], r["lse_a"], r["lse_p"], lam, mask, bad)
+    else:
+        r["zk"] = r["z_exact"]
+    r["w"], r["w64"], r["stats"] = batch_weights(r["lq"], r["lp"], r["accept"], r["a"], r["zk"], lam,
+                                                 c1, mask, bad)
+    r["stats"]["n_bad_token"] = int(bad.sum())
+    if want_kl:
+        kl = kl_rows(za, zp, r["lse_a"], r["lse_p"], mask)
+        n = max(r["stats"]["n_valid"], 1)
+        r["stats"]["mean_kl_p_q"] = float(kl.sum() / n)
+    return r
