@@ -1,0 +1,204 @@
+/* libjackpot: the OBRS token pass of Jackpot on one B200 (sm_100a).
+ *
+ * One pass over actor (rollout model, p_inf = q) and policy (p_target = p) logits
+ * of shape [T, V].  Per token it computes both log-softmaxes and the sampled
+ * token's log-probabilities, the two top-k sets, the OBRS acceptance probability
+ * (Eq. obrs_accept), a Bernoulli accept/reject decision from a counter-based
+ * generator, the top-k estimate of the normaliser Z (Section 4.4.1), the
+ * batch-level bias correction kappa (Section 4.4.2) and the OBRS weights
+ * (Algorithm 1, step 3).  A second call writes the gradient of the joint
+ * objective (Eq. sys_joint_obj) with respect to both logit tensors.
+ *
+ * Conventions for every call
+ *   - C linkage, plain pointers and sizes, no exceptions cross the boundary.
+ *   - Unless a parameter says HOST, every data pointer is DEVICE memory on the
+ *     context's device, owned by the caller, 16-byte aligned for logits and
+ *     gradients.  The library never frees or keeps caller memory.
+ *   - All work is enqueued on the context's stream; calls return after launch
+ *     and never synchronise the device (the *_host variants do: they copy).
+ *   - The context owns one workspace (per-token records), allocated with
+ *     cudaMalloc on first use or by jp_reserve; it grows, never shrinks.
+ *   - Return value: JP_OK or a negative jp_status; jp_last_error(ctx) gives a
+ *     sentence.  Conditions found on the device (token id out of range,
+ *     non-finite rows) never trap: they are counted in jp_stats.
+ *   - A context is thread-compatible, not thread-safe.
+ *   - Rows with mask[t] == 0 are not read; their outputs are accept = 0,
+ *     weight = 0, logp = 0 and zero gradient rows.
+ */
+#ifndef JACKPOT_H_
+#define JACKPOT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct jp_ctx jp_ctx;
+
+typedef enum {
+  JP_OK = 0,
+  JP_ERR_INVALID_ARG = -1,
+  JP_ERR_ALIGNMENT = -2,
+  JP_ERR_UNSUPPORTED = -3,
+  JP_ERR_WORKSPACE = -4,
+  JP_ERR_CUDA = -5,
+  JP_ERR_TIMEOUT = -6,
+  JP_ERR_STATE = -7
+} jp_status;
+
+typedef enum { JP_BF16 = 0, JP_F32 = 1 } jp_dtype;
+typedef enum { JP_LAMBDA_FIXED = 0, JP_LAMBDA_FROM_BUDGET = 1 } jp_lambda_mode;
+
+enum { JP_MAX_TOPK = 128 };
+
+/* Shapes, dtype, mode and optional outputs of one forward / backward call.
+ * Zero-initialise, then set T, V and what differs from the defaults. */
+typedef struct {
+  int64_t T;             /* rows (token positions) in this call                          */
+  int64_t V;             /* vocabulary size                                              */
+  int64_t ld;            /* leading dimension of the logit (and gradient) rows in
+                            elements; 0 means V.  ld * element size must be a multiple
+                            of 16 bytes (for JP_F32 logits with a backward call: ld % 8 == 0) */
+  int32_t dtype;         /* jp_dtype of the logits; gradients are always bf16            */
+  int32_t lambda_mode;   /* jp_lambda_mode: meaning of lambda_or_budget                  */
+  float c1;              /* clip on w_OBRS (Algorithm 1, step 3); <= 0 means no clip     */
+  int32_t reserved0;
+  int64_t token_offset;  /* global index of row 0: the accept draw of row t is keyed on
+                            (seed, token_offset + t)                                     */
+  /* Optional per-token outputs (device pointers, NULL to skip). */
+  int32_t* topk_idx_actor;   /* [T,k] top-k(p_inf) indices, best first, ties by lower index */
+  int32_t* topk_idx_policy;  /* [T,k] top-k(p_target)                                     */
+  float* topk_val_actor;     /* [T,k] the actor logits at topk_idx_actor, as fp32         */
+  float* topk_val_policy;    /* [T,k] the policy logits at topk_idx_policy                */
+  float* accept_prob;        /* [T] a(x_t), Eq. obrs_accept                               */
+  float* uniform;            /* [T] the uniform each decision compared against            */
+  float* z_approx;           /* [T] Z_approx before the kappa correction (= Z when k >= V)*/
+  float* z_exact;            /* [T] full-vocabulary Z (costs a second pass over the rows) */
+  float* lse_actor;          /* [T] log sum_v exp(actor logit)                            */
+  float* lse_policy;         /* [T]                                                       */
+} jp_obrs_desc;
+
+/* Batch statistics, written to DEVICE memory by the last kernel of a forward. */
+typedef struct {
+  int64_t n_valid;       /* N: rows with mask != 0 and a token id inside [0, V)            */
+  int64_t n_accept;      /* accepted among them                                           */
+  int64_t n_bad_token;   /* unmasked rows whose token id was outside [0, V): treated as masked */
+  int64_t n_nonfinite;   /* valid rows whose log-sum-exp came out non-finite              */
+  double alpha_hat;      /* n_accept / n_valid (Section 4.4.2)                            */
+  double mean_accept_prob; /* mean of a(x_t) over valid rows                              */
+  double z_approx_mean;  /* mean of Z_approx over valid rows                              */
+  double kappa;          /* alpha_hat / z_approx_mean; 1 if n_valid == 0 or the mean is 0 */
+  double lambda_used;    /* the fixed lambda, or the one solved from the budget           */
+  double reserved;
+  int32_t status;        /* 0, or a jp_status raised on the device                        */
+  int32_t pad;
+} jp_stats;
+
+/* Creates a context bound to `device` and to `cuda_stream` (a cudaStream_t cast
+ * to void*, NULL = the default stream).  Allocates a few hundred bytes. */
+jp_status jp_create(jp_ctx** out_ctx, int device, void* cuda_stream);
+jp_status jp_destroy(jp_ctx* ctx);
+/* Rebinds the stream later calls enqueue on. */
+jp_status jp_set_stream(jp_ctx* ctx, void* cuda_stream);
+
+/* Bytes of workspace that T_max rows with top-k size k need. */
+size_t jp_obrs_workspace_bytes(int64_t T_max, int64_t V, int k);
+/* Grows the workspace now (cudaMalloc) so that later calls allocate nothing. */
+jp_status jp_reserve(jp_ctx* ctx, int64_t T_max, int64_t V, int k);
+
+/* Forward pass over one [T,V] pair (Eq. obrs_accept, Eq. obrs_dist, Sections
+ * 4.4.1-4.4.2, Algorithm 1 steps 2-3, Algorithm 2's accept test).
+ *   actor_logits, policy_logits : [T, ld] of desc->dtype, each row read once
+ *                                 (twice if desc->z_exact is set or k >= V)
+ *   tokens  : [T] int32 sampled token ids a_t ~ p_inf
+ *   mask    : [T] uint8, 0 = padding; NULL = all valid
+ *   lambda_or_budget : lambda > 0 (JP_LAMBDA_FIXED) or the target mean acceptance
+ *                      in (0,1] from which one batch-level lambda is solved
+ *                      (Theorem 3.4 applied to the batch's sampled tokens)
+ *   k       : 1..JP_MAX_TOPK selects the top-k estimate of Z; k >= V the exact
+ *             sum over the vocabulary; JP_MAX_TOPK < k < V is JP_ERR_UNSUPPORTED
+ *   seed    : key of the Philox4x32-10 stream of accept draws
+ *   out_accept [T] uint8, out_weight [T] fp32 (min(kappa Z_approx max(lambda,
+ *   p/q), c1) for every valid row, accepted or not), out_logp_actor /
+ *   out_logp_policy [T] fp32 log-probabilities of the sampled token,
+ *   out_stats : one jp_stats in device memory (may be NULL).
+ * The per-token records stay in the context until the next forward or
+ * jp_batch_begin; jp_obrs_backward reads them. */
+jp_status jp_obrs_forward(jp_ctx* ctx, const jp_obrs_desc* desc, const void* actor_logits,
+                          const void* policy_logits, const int32_t* tokens, const uint8_t* mask,
+                          float lambda_or_budget, int k, uint64_t seed, uint8_t* out_accept,
+                          float* out_weight, float* out_logp_actor, float* out_logp_policy,
+                          jp_stats* out_stats);
+
+/* Parameters of the backward pass (Eq. obrs_ppo, Eq. ppo_rollout, Eq.
+ * distill_loss combined as Eq. sys_joint_obj; the PPO terms are maximised and
+ * the distillation term minimised, so the loss is
+ *   J = -L^{PPO-OBRS}(theta) - L^{PPO}(omega) + lambda_distill L^{distill}(omega),
+ * a mean over the batch's N valid proposed tokens, evaluated where the ratios
+ * r_theta = r_omega = 1 and F = 1). */
+typedef struct {
+  const float* advantages;  /* [T] A_t; NULL means 1                                   */
+  float lambda_distill;     /* >= 0                                                    */
+  float grad_out;           /* upstream scalar dL/dJ; 0 means 1                        */
+  int64_t n_valid;          /* N of the whole batch; 0 = take it from the context's
+                               last forward / jp_batch_finalize                        */
+  int64_t record_offset;    /* index of row 0 in the context's records (the chunk's
+                               token_offset for chunked batches, else 0)               */
+} jp_obrs_bwd_desc;
+
+/* Writes dJ/d(actor logits) and dJ/d(policy logits), both [T, ld] bf16:
+ *   d_policy[t,v] = -(g/N) accept_t w_t A_t (1[v = x_t] - p_t(v))
+ *   d_actor[t,v]  = -(g/N) A_t (1[v = x_t] - q_t(v)) + (g lambda_distill/N)(q_t(v) - p_t(v))
+ * accept / weight are the forward's outputs.  The log-sum-exps come from the
+ * context's records of the matching forward (JP_ERR_STATE if there are none).
+ * For bf16 logits d_actor_logits may alias actor_logits and d_policy_logits may
+ * alias policy_logits (each element is read before it is overwritten). */
+jp_status jp_obrs_backward(jp_ctx* ctx, const jp_obrs_desc* desc, const jp_obrs_bwd_desc* bwd,
+                           const void* actor_logits, const void* policy_logits,
+                           const int32_t* tokens, const uint8_t* mask, const uint8_t* accept,
+                           const float* weight, void* d_actor_logits, void* d_policy_logits);
+
+/* Chunked batches: kappa and a budget-derived lambda span the whole batch while
+ * the logits exist one chunk at a time (Section 4.4.2: the calibration factor is
+ * batch-wide).  begin -> chunk x n (rows stream once, records accumulate at
+ * desc->token_offset .. +T) -> finalize (lambda, decisions, Z_approx, kappa,
+ * weights for all T_total rows; outputs are [T_total]).  Rows no chunk covered
+ * count as masked.  Exact mode (k >= V) needs a fixed lambda given at begin. */
+jp_status jp_batch_begin(jp_ctx* ctx, int64_t T_total, int64_t V, int32_t dtype, int k,
+                         float fixed_lambda_for_exact_mode);
+jp_status jp_batch_chunk(jp_ctx* ctx, const jp_obrs_desc* desc, const void* actor_logits,
+                         const void* policy_logits, const int32_t* tokens, const uint8_t* mask);
+jp_status jp_batch_finalize(jp_ctx* ctx, const jp_obrs_desc* desc_outputs, float lambda_or_budget,
+                            int32_t lambda_mode, uint64_t seed, uint8_t* out_accept,
+                            float* out_weight, float* out_logp_actor, float* out_logp_policy,
+                            jp_stats* out_stats);
+
+/* Same forward with every pointer in HOST memory (pinned memory makes the
+ * copies asynchronous): the library stages the rows through device buffers it
+ * owns, chunk by chunk with copies overlapping compute, writes the outputs back
+ * and synchronises before returning.  chunk_rows = 0 picks a default.
+ * Optional outputs of desc are not supported here and must be NULL. */
+jp_status jp_obrs_forward_host(jp_ctx* ctx, const jp_obrs_desc* desc, const void* actor_logits,
+                               const void* policy_logits, const int32_t* tokens,
+                               const uint8_t* mask, float lambda_or_budget, int k, uint64_t seed,
+                               uint8_t* out_accept, float* out_weight, float* out_logp_actor,
+                               float* out_logp_policy, jp_stats* out_stats, int64_t chunk_rows);
+
+const char* jp_status_string(jp_status s);
+const char* jp_last_error(jp_ctx* ctx);
+/* Number of kernel launches this context has enqueued so far. */
+int64_t jp_launch_count(jp_ctx* ctx);
+/* Per-launch device time of the row-stream kernel.  While timing is on, every
+ * stream-kernel launch is bracketed by CUDA events on the context's stream (a
+ * ring of 256 pairs).  jp_stream_kernel_times waits for the newest n of them,
+ * writes their durations in milliseconds to out_ms (HOST memory, oldest first)
+ * and returns how many it wrote.  Enabling or disabling restarts the count. */
+jp_status jp_enable_kernel_timing(jp_ctx* ctx, int on);
+int64_t jp_stream_kernel_times(jp_ctx* ctx, float* out_ms, int64_t n);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* JACKPOT_H_ */

@@ -1,0 +1,122 @@
+// Internal launch interface between the C-ABI host code and the sm_100a kernels.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "jackpot.h"
+
+namespace jp {
+
+// Per-token records kept in the context's workspace (struct of arrays, indexed
+// by record row r = record_offset + t).
+struct Records {
+  int32_t* idx;     // [cap, 2k]  top-k(p_inf) then top-k(p_target) indices, -1 = empty
+  float* za;        // [cap, 2k]  actor logit of every candidate
+  float* zp;        // [cap, 2k]  policy logit of every candidate
+  float* lse_a;     // [cap]
+  float* lse_p;     // [cap]
+  float* lq;        // [cap] log p_inf(a_t)
+  float* lp;        // [cap] log p_target(a_t)
+  float* zk;        // [cap] Z_approx (or exact Z when k >= V)
+  float* zx;        // [cap] exact Z when asked for beside Z_approx
+  float* a;         // [cap] acceptance probability
+  uint8_t* flag;    // [cap] 1 = valid row with records, 0 = masked / bad / never streamed
+  double* ratio;    // [cap] p(a_t)/q(a_t) in double, compacted, for the budget solve
+  float* dval;      // [cap] lp - lq of the compacted valid rows
+};
+
+// Device scalars shared by the kernels of one forward.
+struct Scalars {
+  int32_t row_counter;     // persistent-CTA work queue of the stream kernel
+  int32_t row_counter2;    // same for the exact-Z / gradient kernels
+  int32_t n_compact;       // number of valid rows found by the ratio kernel
+  int32_t status;
+  unsigned long long n_bad_token;
+  unsigned long long n_nonfinite;
+  float lambda;            // lambda in use (fixed, or written by the budget solve)
+  float pad;
+  double lambda64;
+  jp_stats stats;          // the last forward's batch statistics
+};
+
+constexpr int kMaxPartials = 256;
+struct Partials {
+  long long n_valid[kMaxPartials];
+  long long n_accept[kMaxPartials];
+  double sum_zk[kMaxPartials];
+  double sum_a[kMaxPartials];
+};
+
+struct StreamArgs {
+  const void* za;
+  const void* zp;
+  const int32_t* tokens;
+  const uint8_t* mask;
+  int64_t T, V, ld;
+  int32_t dtype;
+  int32_t k;               // 0 = no top-k (exact mode)
+  int64_t record_offset;
+  Records rec;
+  Scalars* sc;
+};
+
+struct ExactZArgs {
+  const void* za;
+  const void* zp;
+  int64_t T, V, ld;
+  int32_t dtype;
+  int64_t record_offset;
+  Records rec;
+  Scalars* sc;
+  float* out;              // rec.zk or rec.zx
+};
+
+struct EpilogueArgs {
+  int64_t T;               // record rows to finalise
+  int32_t k;               // 0 = zk already holds the exact Z
+  uint64_t seed;
+  int64_t rng_base;        // accept draw of record row r uses counter rng_base + r
+  float c1;
+  Records rec;
+  Scalars* sc;
+  Partials* part;
+  int32_t n_part;
+  // outputs, all [T] (any may be null)
+  uint8_t* out_accept;
+  float* out_weight;
+  float* out_lq;
+  float* out_lp;
+  jp_stats* out_stats;
+  int32_t* aux_idx_a; int32_t* aux_idx_p; float* aux_val_a; float* aux_val_p;
+  float* aux_a; float* aux_u; float* aux_zk; float* aux_zx; float* aux_lse_a; float* aux_lse_p;
+};
+
+struct GradArgs {
+  const void* za;
+  const void* zp;
+  const int32_t* tokens;
+  const uint8_t* mask;
+  const uint8_t* accept;
+  const float* weight;
+  const float* adv;
+  void* d_actor;
+  void* d_policy;
+  int64_t T, V, ld;
+  int32_t dtype;
+  int64_t record_offset;
+  float lambda_distill, grad_out;
+  int64_t n_valid;         // 0 = read sc->stats.n_valid on the device
+  Records rec;
+  Scalars* sc;
+};
+
+int stream_grid_size(int device);   // number of SMs
+cudaError_t launch_stream(const StreamArgs& a, cudaStream_t s, int sms);
+cudaError_t launch_exact_z(const ExactZArgs& a, cudaStream_t s, int sms);
+cudaError_t launch_reset(Scalars* sc, float lambda_fixed, cudaStream_t s);
+cudaError_t launch_clear_flags(uint8_t* flag, int64_t n, cudaStream_t s);
+cudaError_t launch_budget_solve(const EpilogueArgs& a, double budget, cudaStream_t s, int* n_launch);
+cudaError_t launch_epilogue(const EpilogueArgs& a, cudaStream_t s, int* n_launch);
+cudaError_t launch_grad(const GradArgs& a, cudaStream_t s, int sms);
+
+}  // namespace jp
