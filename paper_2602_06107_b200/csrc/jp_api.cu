@@ -20,6 +20,7 @@ struct jp_ctx {
   int cap_k = 0;
   Records rec{};
   Scalars* sc = nullptr;
+  int32_t* list = nullptr;
   Partials* part = nullptr;
   // state of the records
   bool have_records = false;
@@ -48,7 +49,7 @@ namespace {
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
-  size_t scalars, partials, idx, za, zp, f[7], flag, ratio, dval, total;
+  size_t scalars, partials, idx, za, zp, f[7], flag, ratio, dval, list, total;
 };
 
 Layout layout_for(int64_t rows, int k) {
@@ -65,6 +66,7 @@ Layout layout_for(int64_t rows, int k) {
   L.flag = take((size_t)rows);
   L.ratio = take((size_t)rows * 8);
   L.dval = take((size_t)rows * 4);
+  L.list = take((size_t)rows * 4);
   L.total = off;
   return L;
 }
@@ -119,6 +121,7 @@ jp_status ensure_workspace(jp_ctx* c, int64_t rows, int k) {
   c->rec.flag = (uint8_t*)(b + L.flag);
   c->rec.ratio = (double*)(b + L.ratio);
   c->rec.dval = (float*)(b + L.dval);
+  c->list = (int32_t*)(b + L.list);
   return JP_OK;
 }
 
@@ -162,7 +165,7 @@ jp_status stream_rows(jp_ctx* c, const jp_obrs_desc* d, int64_t ld, int k_eff, i
   StreamArgs a{};
   a.za = za; a.zp = zp; a.tokens = tokens; a.mask = mask;
   a.T = d->T; a.V = d->V; a.ld = ld; a.dtype = d->dtype; a.k = k_eff;
-  a.record_offset = record_offset; a.rec = c->rec; a.sc = c->sc;
+  a.record_offset = record_offset; a.rec = c->rec; a.sc = c->sc; a.list = c->list;
   const int slot = (int)(c->ev_count % jp_ctx::kEvRing);
   if (c->timing) {
     if (!c->ev0[slot]) { cudaEventCreate(&c->ev0[slot]); cudaEventCreate(&c->ev1[slot]); }
@@ -171,7 +174,7 @@ jp_status stream_rows(jp_ctx* c, const jp_obrs_desc* d, int64_t ld, int k_eff, i
   cudaError_t e = launch_stream(a, c->stream, c->sms);
   if (c->timing) { cudaEventRecord(c->ev1[slot], c->stream); c->ev_count += 1; }
   if (e != cudaSuccess) return cuda_fail(c, e, "stream kernel launch");
-  c->launches += 1;
+  c->launches += 2;
   if (exact_now) {
     ExactZArgs x{};
     x.za = za; x.zp = zp; x.T = d->T; x.V = d->V; x.ld = ld; x.dtype = d->dtype;
@@ -387,8 +390,8 @@ jp_status jp_batch_chunk(jp_ctx* c, const jp_obrs_desc* d, const void* za, const
   if (d->token_offset < 0 || d->token_offset + d->T > c->rec_rows)
     return fail(c, JP_ERR_INVALID_ARG, "chunk rows fall outside [0, T_total)");
   cudaSetDevice(c->device);
-  // the row queue restarts for every chunk; the other scalars accumulate
-  cudaError_t e = cudaMemsetAsync(&c->sc->row_counter, 0, 2 * sizeof(int32_t), c->stream);
+  // the row list restarts for every chunk; the other scalars accumulate
+  cudaError_t e = cudaMemsetAsync(&c->sc->n_list, 0, 2 * sizeof(int32_t), c->stream);
   if (e != cudaSuccess) return cuda_fail(c, e, "cudaMemsetAsync");
   return stream_rows(c, d, ld, c->rec_k, d->token_offset, za, zp, tokens, mask, c->batch_exact, false);
 }

@@ -11,7 +11,7 @@
 namespace jp {
 
 __global__ void reset_kernel(Scalars* sc, float lambda_fixed) {
-  sc->row_counter = 0;
+  sc->n_list = 0;
   sc->row_counter2 = 0;
   sc->n_compact = 0;
   sc->status = 0;

@@ -27,8 +27,8 @@ struct Records {
 
 // Device scalars shared by the kernels of one forward.
 struct Scalars {
-  int32_t row_counter;     // persistent-CTA work queue of the stream kernel
-  int32_t row_counter2;    // same for the exact-Z / gradient kernels
+  int32_t n_list;          // valid rows of the call being streamed (length of the row list)
+  int32_t row_counter2;    // persistent-CTA work queue of the exact-Z / gradient kernels
   int32_t n_compact;       // number of valid rows found by the ratio kernel
   int32_t status;
   unsigned long long n_bad_token;
@@ -58,6 +58,7 @@ struct StreamArgs {
   int64_t record_offset;
   Records rec;
   Scalars* sc;
+  int32_t* list;           // [T] scratch: the call's valid rows, in no particular order
 };
 
 struct ExactZArgs {

@@ -4,37 +4,116 @@
 // union of top-k(p_inf) and top-k(p_new)), each candidate carrying both logits.
 // A second kernel sums the exact normaliser Z over the vocabulary (Eq. obrs_dist).
 //
-// Work split: persistent CTAs pull rows from an atomic counter; one CTA owns one
-// row at a time; a thread owns 16-byte vectors strided by the CTA width, so every
-// warp-level load is one contiguous 512-byte segment.
+// Shape of the stream kernel (one persistent CTA per SM, one row pair at a time):
 //
-// Top-k: the total order is (logit desc, index asc), encoded in one 64-bit key.
-// A threshold tau (the current k-th best key) filters the stream: one compare
-// per 16-byte vector (its max against tau's logit) in the hot loop, exact key
-// compares only for vectors that pass.  Survivors go to a shared-memory
-// candidate buffer that is bitonic-sorted together with the current list when
-// it fills, which tightens tau.  The first tile has no tau yet: the k-th
-// largest of the per-thread maxima bounds it from below.
+//   producer warp   one lane issues 1-D bulk async copies (global -> shared,
+//                   completion counted on an mbarrier) of the next tile of both
+//                   rows into a ring of STAGES shared-memory stages;
+//   consumer warps  wait for a stage, pull their 16-byte vectors into registers,
+//                   release the stage, then update the online (max, sum) of both
+//                   rows and test each vector's maximum against the row's current
+//                   top-k threshold tau; a vector that may hold a top-k entry is
+//                   pushed BY INDEX into a small shared-memory queue;
+//   top-k warps     four of them, one per (tensor, row slot): they drain the
+//                   queue while the consumers keep streaming, re-read the few
+//                   candidate vectors from L2, keep the sorted list in registers
+//                   (bitonic sort / merge across the lanes, or single inserts)
+//                   and publish the tightened tau; at the end of the row they
+//                   finish the log-sum-exp, gather the sampled token's logit and
+//                   write the row's record.
+//
+// Rows alternate between two "slots" (queue, tau, partial sums, barriers), so the
+// consumers start the next row while the top-k warps finish the previous one.
+// The total order of the top-k is (logit desc, index asc), one 64-bit key; the
+// result does not depend on the order in which candidates arrive.
+//
+// Every wait is bounded: a wait that runs out raises the CTA's abort flag, the
+// status word gets JP_ERR_TIMEOUT and every warp leaves its loop.
 #include "jp_common.cuh"
 #include "jp_internal.h"
 
 namespace jp {
 
-constexpr int NT = 256;                 // threads per CTA
-constexpr int NWARP = NT / 32;
-constexpr int UNROLL = 4;               // vectors per thread per tensor per tile
-constexpr int PMAX = 512;               // list + candidate slots per tensor
-constexpr int CTAS_PER_SM = 2;
+constexpr int NC = 8;                     // consumer warps
+constexpr int VPL = 4;                    // 16-byte vectors per lane per tensor per tile
+constexpr int TV = NC * 32 * VPL;         // vectors per tensor per tile
+constexpr int STAGES = 5;
+constexpr int QCAP = 2048;                // candidate-vector queue entries per (slot, tensor)
+constexpr int SCAP = 512;                 // staged keys per top-k warp
+constexpr int NTOPK = 4;                  // top-k warps: (tensor, slot)
+constexpr int NWARPS = 1 + NC + NTOPK;
+constexpr int NTHREADS = NWARPS * 32;
+constexpr uint32_t QEMPTY = 0xffffffffu;
+constexpr long long kSpinLimit = 4000000000ll;   // clock cycles a wait may last (about 2 s)
 
-struct __align__(16) StreamSmem {
-  unsigned long long buf[2][PMAX];      // [0,K): current list, best first; [K,PMAX): candidates
-  unsigned long long tau_key[2];
-  int cnt[2];
-  float red_m[2][NWARP];
-  float red_s[2][NWARP];
-  float warp_bound[2][NWARP];
-  int row;
+struct __align__(128) StreamSmem {
+  uint4 ring[STAGES][2][TV];              // [stage][tensor][vector]
+  unsigned long long skeys[2][2][SCAP];   // [slot][tensor] keys waiting to be merged
+  uint32_t queue[2][2][QCAP];             // [slot][tensor] candidate vector indices
+  unsigned long long full[STAGES], empty[STAGES];
+  unsigned long long row_done[2], slot_free[2], bound_ready[2];
+  int qcnt[2][2];
+  float tau[2][2];                        // published threshold (a logit value)
+  float warp_bound[2][2][NC];
+  float part_mL[2][2][NC];
+  float part_s[2][2][NC];
+  int abort;
 };
+
+// ---- mbarrier / bulk-copy wrappers ----------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(unsigned long long* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait; false = gave up (or another warp did).
+__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity, volatile int* abort) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*abort) return false;
+    if (clock64() - t0 > kSpinLimit) { *abort = 1; return false; }
+  }
+}
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, unsigned long long* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(dst)),
+               "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ float lds_volatile_f32(const float* p) {
+  float v;
+  asm volatile("ld.volatile.shared.f32 %0, [%1];" : "=f"(v) : "r"(smem_u32(p)) : "memory");
+  return v;
+}
+__device__ __forceinline__ uint32_t lds_volatile_u32(const void* p) {
+  uint32_t v;
+  asm volatile("ld.volatile.shared.u32 %0, [%1];" : "=r"(v) : "r"(smem_u32(p)) : "memory");
+  return v;
+}
+__device__ __forceinline__ void sts_volatile_f32(float* p, float v) {
+  asm volatile("st.volatile.shared.f32 [%0], %1;" ::"r"(smem_u32(p)), "f"(v) : "memory");
+}
 
 // ---- packed fp32x2 arithmetic (two lanes of one 64-bit register pair) ------
 __device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
@@ -60,21 +139,6 @@ __device__ __forceinline__ unsigned long long fmul2(unsigned long long a, unsign
   unsigned long long d;
   asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
   return d;
-}
-
-// r-th largest (1-based) of the 32 lane values: shuffle bitonic sort, descending.
-__device__ __forceinline__ float warp_rth_largest(float v, int r, int lane) {
-#pragma unroll
-  for (int size = 2; size <= 32; size <<= 1) {
-#pragma unroll
-    for (int stride = size >> 1; stride > 0; stride >>= 1) {
-      float o = __shfl_xor_sync(0xffffffffu, v, stride);
-      bool lower = (lane & stride) == 0;
-      bool desc = (lane & size) == 0;
-      v = (lower == desc) ? fmaxf(v, o) : fminf(v, o);
-    }
-  }
-  return __shfl_sync(0xffffffffu, v, r - 1);
 }
 
 // 2^d for an integer-valued d <= 0, exact (built from the exponent field).
@@ -137,252 +201,324 @@ __device__ __forceinline__ void accumulate(const uint4& v, float vm, Online& o) 
   }
 }
 
-// Element `e` (runtime) of a vector held as four words.
+// The ragged end of a row (fewer than one 16-byte vector) as a -inf padded vector.
 template <int DT>
-__device__ __forceinline__ float vec_elem(uint32_t x, uint32_t y, uint32_t z, uint32_t w, int e) {
-  if (DT == JP_BF16) {
-    const int wi = e >> 1;
-    uint32_t word = wi == 0 ? x : wi == 1 ? y : wi == 2 ? z : w;
-    return __uint_as_float((e & 1) ? (word & 0xffff0000u) : (word << 16));
-  }
-  return __uint_as_float(e == 0 ? x : e == 1 ? y : e == 2 ? z : w);
+__device__ __forceinline__ uint4 load_tail_vector(const char* row, int64_t first, int tail) {
+  uint4 v = Vec<DT>::neg_inf();
+#pragma unroll
+  for (int e = 0; e < Vec<DT>::N - 1; ++e)
+    if (e < tail) Vec<DT>::set(v, e, Vec<DT>::load_scalar(row, first + e));
+  return v;
 }
 
-// Warp-cooperative append.  `pass` marks the lanes whose vector may hold an entry
-// that beats tau.  For each such lane the vector is broadcast, lanes 0..N-1 each
-// test one entry exactly (64-bit key against tau) and the winners take
-// consecutive slots of the CTA's candidate buffer.  Control flow is warp-uniform.
-// `done` (owner lane's bits 0..N-1) marks entries appended earlier in this tile;
-// the function returns the updated bits for the calling lane's own vector and
-// sets `flag` when the CTA should merge (soft limit passed, or no slot left).
-template <int DT>
-__device__ __forceinline__ uint32_t push_warp(StreamSmem& sm, int t, const uint4& v, bool pass,
-                                              uint32_t idx0, uint32_t V, unsigned long long tau,
-                                              uint32_t done, int K, int lane, bool& flag) {
-  constexpr int N = Vec<DT>::N;
-  uint32_t mask = __ballot_sync(0xffffffffu, pass);
-  const int cap = PMAX - K;
-  const int soft = cap >> 1;
-  while (mask) {
-    const int L = __ffs(mask) - 1;
-    mask &= mask - 1;
-    const uint32_t x = __shfl_sync(0xffffffffu, v.x, L), y = __shfl_sync(0xffffffffu, v.y, L);
-    const uint32_t z = __shfl_sync(0xffffffffu, v.z, L), w = __shfl_sync(0xffffffffu, v.w, L);
-    const uint32_t i0 = __shfl_sync(0xffffffffu, idx0, L);
-    const uint32_t dn = __shfl_sync(0xffffffffu, done, L);
-    const uint32_t idx = i0 + lane;
-    bool win = false;
-    unsigned long long key = 0ull;
-    if (lane < N && idx < V && !((dn >> lane) & 1u)) {
-      key = make_key(vec_elem<DT>(x, y, z, w, lane), idx);
-      win = key > tau;
-    }
-    const uint32_t wmask = __ballot_sync(0xffffffffu, win);
-    if (wmask) {
-      int base = 0;
-      if (lane == 0) base = atomicAdd(&sm.cnt[t], __popc(wmask));
-      base = __shfl_sync(0xffffffffu, base, 0);
-      const int slot = base + __popc(wmask & ((1u << lane) - 1u));
-      const bool stored = win && slot < cap;
-      if (stored) sm.buf[t][K + slot] = key;
-      const uint32_t smask = __ballot_sync(0xffffffffu, stored);
-      if (lane == L) done |= smask;
-      if (smask != wmask || base + __popc(wmask) > soft) flag = true;
-    }
+// r-th largest (1-based) of the 32 lane values; -inf when fewer than r lanes hold a number.
+__device__ __forceinline__ float warp_rth_largest(float v, int r, int lane) {
+  uint32_t ob = f32_order_bits(v);
+  uint32_t mx = 0u;
+  for (int i = 0; i < r; ++i) {
+    mx = __reduce_max_sync(0xffffffffu, ob);
+    const uint32_t holders = __ballot_sync(0xffffffffu, ob == mx);
+    if (lane == __ffs(holders) - 1) ob = 0u;     // retire one holder of the maximum
   }
-  return done;
+  return mx <= 0x007fffffu ? JP_NEG_INF : order_bits_f32(mx);
 }
 
-// Bitonic sort (descending) of buf[0..P) by ONE warp, then keep the best k, clear
-// the rest and publish tau and the reset count.  P is a power of two >= 2.
-__device__ __forceinline__ void warp_sort_list(unsigned long long* buf, int P, int k, int lane,
-                                               unsigned long long* tau_out, int* cnt_out) {
-  for (int size = 2; size <= P; size <<= 1) {
-    for (int stride = size >> 1; stride > 0; stride >>= 1) {
-      for (int j = lane; j < (P >> 1); j += 32) {
-        const int lo = ((j & ~(stride - 1)) << 1) | (j & (stride - 1));
-        const int hi = lo | stride;
-        const bool desc = (lo & size) == 0;
-        const unsigned long long a = buf[lo], b = buf[hi];
-        if ((a < b) == desc) { buf[lo] = b; buf[hi] = a; }
+// ---- the sorted list of a top-k warp ---------------------------------------
+// 32*KPL keys, sorted descending, position p = lane*KPL + j in register j of a lane.
+__device__ __forceinline__ unsigned long long u64max(unsigned long long a, unsigned long long b) { return a > b ? a : b; }
+__device__ __forceinline__ unsigned long long u64min(unsigned long long a, unsigned long long b) { return a < b ? a : b; }
+
+// One compare-exchange layer of a bitonic network at distance `stride` (in
+// positions).  `asc_of(p)` gives the direction of the block position p is in.
+template <int KPL, int STRIDE>
+__device__ __forceinline__ void bitonic_layer(unsigned long long (&x)[KPL], int lane, int size, bool all_desc) {
+  if (STRIDE < KPL) {
+#pragma unroll
+    for (int j = 0; j < KPL; ++j) {
+      if ((j & STRIDE) == 0) {
+        const int p = lane * KPL + j;
+        const bool asc = all_desc ? false : ((p & size) == 0);
+        const unsigned long long a = x[j], b = x[j | STRIDE];
+        const unsigned long long lo = u64min(a, b), hi = u64max(a, b);
+        x[j] = asc ? lo : hi;
+        x[j | STRIDE] = asc ? hi : lo;
       }
-      __syncwarp();
+    }
+  } else {
+    constexpr int LS = STRIDE / KPL;            // lane distance
+    const bool lower = (lane & LS) == 0;
+#pragma unroll
+    for (int j = 0; j < KPL; ++j) {
+      const int p = lane * KPL + j;
+      const bool asc = all_desc ? false : ((p & size) == 0);
+      const unsigned long long o = __shfl_xor_sync(0xffffffffu, x[j], LS);
+      x[j] = (lower == asc) ? u64min(x[j], o) : u64max(x[j], o);
     }
   }
-  for (int i = k + lane; i < P; i += 32) buf[i] = 0ull;
+}
+
+template <int KPL, int STRIDE>
+struct BitonicDown {   // layers STRIDE, STRIDE/2, ..., 1
+  static __device__ __forceinline__ void run(unsigned long long (&x)[KPL], int lane, int size, bool all_desc) {
+    bitonic_layer<KPL, STRIDE>(x, lane, size, all_desc);
+    BitonicDown<KPL, STRIDE / 2>::run(x, lane, size, all_desc);
+  }
+};
+template <int KPL>
+struct BitonicDown<KPL, 0> {
+  static __device__ __forceinline__ void run(unsigned long long (&)[KPL], int, int, bool) {}
+};
+
+template <int KPL, int SIZE>
+struct BitonicSort {   // full sort, ascending, of 32*KPL keys
+  static __device__ __forceinline__ void run(unsigned long long (&x)[KPL], int lane) {
+    BitonicSort<KPL, SIZE / 2>::run(x, lane);
+    BitonicDown<KPL, SIZE / 2>::run(x, lane, SIZE, false);
+  }
+};
+template <int KPL>
+struct BitonicSort<KPL, 1> {
+  static __device__ __forceinline__ void run(unsigned long long (&)[KPL], int) {}
+};
+
+// Folds up to 32*KPL keys taken from the end of the staging buffer into the list.
+template <int KPL>
+__device__ __forceinline__ void merge_staged(unsigned long long (&L)[KPL], const unsigned long long* stg,
+                                             int& staged, int lane) {
+  constexpr int NL = 32 * KPL;
+  const int m = staged < NL ? staged : NL;
+  unsigned long long nw[KPL];
+#pragma unroll
+  for (int j = 0; j < KPL; ++j) {
+    const int i = lane * KPL + j;
+    nw[j] = i < m ? stg[staged - m + i] : 0ull;
+  }
+  BitonicSort<KPL, NL>::run(nw, lane);                       // ascending
+#pragma unroll
+  for (int j = 0; j < KPL; ++j) L[j] = u64max(L[j], nw[j]);    // the NL largest of the union, bitonic
+  BitonicDown<KPL, NL / 2>::run(L, lane, NL, true);          // descending
+  staged -= m;
+}
+
+// Inserts one key into the descending list, dropping the smallest.
+template <int KPL>
+__device__ __forceinline__ void insert_one(unsigned long long (&L)[KPL], unsigned long long key, int lane) {
+  unsigned long long up = __shfl_up_sync(0xffffffffu, L[KPL - 1], 1);
+  if (lane == 0) up = ~0ull;
+#pragma unroll
+  for (int j = KPL - 1; j >= 0; --j) {
+    const unsigned long long before = j == 0 ? up : L[j - 1];
+    L[j] = L[j] > key ? L[j] : (before > key ? key : before);
+  }
+}
+
+template <int KPL>
+__device__ __forceinline__ unsigned long long kth_key(const unsigned long long (&L)[KPL], int k) {
+  unsigned long long v = L[0];
+#pragma unroll
+  for (int j = 1; j < KPL; ++j)
+    if (((k - 1) % KPL) == j) v = L[j];
+  return __shfl_sync(0xffffffffu, v, (k - 1) / KPL);
+}
+
+// Tests the entries of one vector per lane against tau and appends the winners'
+// keys to the staging buffer; returns the new number of staged keys.
+template <int DT>
+__device__ __forceinline__ int filter_vector(const uint4& v, uint32_t vi, bool have, int64_t V,
+                                             unsigned long long tau_key, unsigned long long* stg, int staged,
+                                             int lane) {
+  constexpr int N = Vec<DT>::N;
+  unsigned long long key[N];
+  uint32_t pass = 0u;
+#pragma unroll
+  for (int e = 0; e < N; ++e) {
+    const uint32_t idx = vi * N + e;
+    key[e] = make_key(Vec<DT>::get(v, e), idx);
+    if (have && (int64_t)idx < V && key[e] > tau_key) pass |= 1u << e;
+  }
+  const int c = __popc(pass);
+  int incl = c;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int n = __shfl_up_sync(0xffffffffu, incl, off);
+    if (lane >= off) incl += n;
+  }
+  const int total = __shfl_sync(0xffffffffu, incl, 31);
+  int pos = staged + incl - c;
+#pragma unroll
+  for (int e = 0; e < N; ++e)
+    if ((pass >> e) & 1u) stg[pos++] = key[e];
   __syncwarp();
-  if (lane == 0) { *tau_out = buf[k - 1]; *cnt_out = 0; }
+  return staged + total;
 }
 
-// Folds the candidates of both tensors into their lists: warp 0 sorts the actor
-// side, warp 1 the policy side, everyone else waits.  Called by all threads
-// after a barrier that ordered every append before it; ends with a barrier.
-__device__ __forceinline__ void merge_lists(StreamSmem& sm, int k, int K, int warp, int lane) {
-  if (warp < 2) {
-    const int cap = PMAX - K;
-    const int n = min(sm.cnt[warp], cap);
-    int P = K < 2 ? 2 : K;
-    while (P < K + n) P <<= 1;
-    if (n > 0) warp_sort_list(sm.buf[warp], P, k, lane, &sm.tau_key[warp], &sm.cnt[warp]);
-    else if (lane == 0) sm.tau_key[warp] = sm.buf[warp][k - 1];
+// Empties the staging buffer into the list and returns the new tau key.
+template <int KPL>
+__device__ __forceinline__ unsigned long long drain_staged(unsigned long long (&L)[KPL],
+                                                           const unsigned long long* stg, int& staged, int k,
+                                                           int lane) {
+  constexpr int SORT_MIN = 6 * KPL;       // below this, single inserts are cheaper than a sort + merge
+  while (staged >= SORT_MIN) merge_staged<KPL>(L, stg, staged, lane);
+  while (staged > 0) {
+    insert_one<KPL>(L, stg[staged - 1], lane);
+    --staged;
   }
-  __syncthreads();
+  __syncwarp();
+  return kth_key<KPL>(L, k);
 }
 
-__device__ __forceinline__ float tau_value(unsigned long long key) {
-  return key == 0ull ? JP_NEG_INF : key_value(key);
+__device__ __forceinline__ void raise_timeout(StreamSmem& sm, Scalars* sc) {
+  sm.abort = 1;
+  atomicExch(&sc->status, (int)JP_ERR_TIMEOUT);
 }
 
+// ---- producer ---------------------------------------------------------------
 template <int DT>
-__device__ __forceinline__ void load_tile(uint4 (&va)[UNROLL], uint4 (&vp)[UNROLL], const char* ra,
-                                          const char* rp, int64_t v0, int64_t nvec, int tail,
-                                          int tid) {
-#pragma unroll
-  for (int j = 0; j < UNROLL; ++j) {
-    int64_t vi = v0 + (int64_t)j * NT + tid;
-    if (vi < nvec) {
-      va[j] = ldg_stream((const uint4*)ra + vi);
-      vp[j] = ldg_stream((const uint4*)rp + vi);
-    } else {
-      va[j] = Vec<DT>::neg_inf();
-      vp[j] = Vec<DT>::neg_inf();
-      if (vi == nvec && tail > 0) {       // ragged end of the row: scalar loads, -inf padding
-#pragma unroll
-        for (int e = 0; e < Vec<DT>::N - 1; ++e) {
-          if (e < tail) {
-            Vec<DT>::set(va[j], e, Vec<DT>::load_scalar(ra, nvec * Vec<DT>::N + e));
-            Vec<DT>::set(vp[j], e, Vec<DT>::load_scalar(rp, nvec * Vec<DT>::N + e));
-          }
-        }
-      }
-    }
-  }
-}
-
-template <int DT, bool TOPK>
-__global__ void __launch_bounds__(NT, CTAS_PER_SM) stream_kernel(StreamArgs A) {
-  __shared__ StreamSmem sm;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+__device__ void producer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows) {
   constexpr int N = Vec<DT>::N;
-  const int k = A.k;
-  int K = 1;
-  while (K < k) K <<= 1;
   const int64_t nvec = A.V / N;
-  const int tail = (int)(A.V - nvec * N);
-  const int64_t nvt = nvec + (tail > 0 ? 1 : 0);
-  constexpr int64_t TILE = (int64_t)NT * UNROLL;
-
-  if (TOPK) {
-    for (int i = tid; i < 2 * PMAX; i += NT) (&sm.buf[0][0])[i] = 0ull;
-    if (tid < 2) { sm.cnt[tid] = 0; sm.tau_key[tid] = 0ull; }
-  }
-  __syncthreads();
-
-  for (;;) {
-    if (tid == 0) sm.row = atomicAdd(&A.sc->row_counter, 1);
-    __syncthreads();
-    const int64_t row = sm.row;
-    __syncthreads();
-    if (row >= A.T) break;
-    const int64_t rrow = A.record_offset + row;
-    bool valid = A.mask == nullptr || A.mask[row] != 0;
-    const int32_t x = valid ? A.tokens[row] : 0;
-    if (valid && (x < 0 || (int64_t)x >= A.V)) {
-      valid = false;
-      if (tid == 0) atomicAdd(&A.sc->n_bad_token, 1ull);
-    }
-    if (!valid) {
-      if (tid == 0) {
-        A.rec.flag[rrow] = 0;
-        A.rec.lse_a[rrow] = 0.f; A.rec.lse_p[rrow] = 0.f;
-        A.rec.lq[rrow] = 0.f; A.rec.lp[rrow] = 0.f;
-      }
-      continue;
-    }
+  const int ntiles = nvec > 0 ? (int)((nvec + TV - 1) / TV) : 1;
+  long long g = 0;
+  bool ok = true;
+  for (int64_t it = blockIdx.x; it < n_rows && ok; it += gridDim.x) {
+    const int64_t row = A.list[it];
     const char* ra = (const char*)A.za + row * A.ld * Vec<DT>::ESIZE;
     const char* rp = (const char*)A.zp + row * A.ld * Vec<DT>::ESIZE;
+    for (int tile = 0; tile < ntiles; ++tile, ++g) {
+      const int s = (int)(g % STAGES);
+      const uint32_t ph = (uint32_t)((g / STAGES) & 1);
+      if (!mbar_wait(&sm.empty[s], ph ^ 1u, &sm.abort)) { ok = false; break; }
+      const int64_t v0 = (int64_t)tile * TV;
+      const int64_t nv = nvec - v0 < TV ? nvec - v0 : TV;
+      const uint32_t bytes = (uint32_t)(nv > 0 ? nv * 16 : 0);
+      if (bytes > 0) {
+        mbar_arrive_expect_tx(&sm.full[s], 2u * bytes);
+        bulk_g2s(&sm.ring[s][0][0], ra + v0 * 16, bytes, &sm.full[s]);
+        bulk_g2s(&sm.ring[s][1][0], rp + v0 * 16, bytes, &sm.full[s]);
+      } else {
+        mbar_arrive(&sm.full[s]);
+      }
+    }
+  }
+  if (!ok) {
+    // Leave no copy in flight: every stage this lane armed and nobody consumed
+    // completes once its bytes have landed.
+    raise_timeout(sm, A.sc);
+    for (long long h = g > STAGES ? g - STAGES : 0; h < g; ++h) {
+      const long long t0 = clock64();
+      while (!mbar_try_wait(&sm.full[h % STAGES], (uint32_t)((h / STAGES) & 1)))
+        if (clock64() - t0 > kSpinLimit) break;
+    }
+  }
+}
+
+// ---- consumers ----------------------------------------------------------------
+template <int DT, bool TOPK>
+__device__ void consumer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, int cw, int lane) {
+  constexpr int N = Vec<DT>::N;
+  const int64_t nvec = A.V / N;
+  const int tail = (int)(A.V - nvec * N);
+  const int ntiles = nvec > 0 ? (int)((nvec + TV - 1) / TV) : 1;
+  const int r = (A.k + NC - 1) / NC;
+  long long g = 0;
+  int lr = 0;
+  for (int64_t it = blockIdx.x; it < n_rows; it += gridDim.x, ++lr) {
+    const int p = lr & 1;
+    const uint32_t ph = (uint32_t)((lr >> 1) & 1);
+    // the slot's queue, tau and partial sums are free once both of its top-k warps
+    // have finished the row that used it before
+    if (!mbar_wait(&sm.slot_free[p], ph ^ 1u, &sm.abort)) { raise_timeout(sm, A.sc); return; }
 
     Online oa{JP_NEG_INF, 0.f, 0ull}, op{JP_NEG_INF, 0.f, 0ull};
-    unsigned long long tkey_a = 0ull, tkey_p = 0ull;
-    float tval_a = JP_NEG_INF, tval_p = JP_NEG_INF;
+    float tau0_a = JP_NEG_INF, tau0_p = JP_NEG_INF;
 
-    uint4 ca[UNROLL], cp[UNROLL], na[UNROLL], np_[UNROLL];
-    load_tile<DT>(ca, cp, ra, rp, 0, nvec, tail, tid);
-    int tile = 0;
-    for (int64_t v0 = 0; v0 < nvt; v0 += TILE, ++tile) {
-      const bool more = v0 + TILE < nvt;
-      if (more) load_tile<DT>(na, np_, ra, rp, v0 + TILE, nvec, tail, tid);
-
-      float vm_a[UNROLL], vm_p[UNROLL];
+    for (int tile = 0; tile < ntiles; ++tile, ++g) {
+      const int s = (int)(g % STAGES);
+      if (!mbar_wait(&sm.full[s], (uint32_t)((g / STAGES) & 1), &sm.abort)) { raise_timeout(sm, A.sc); return; }
+      const int64_t v0 = (int64_t)tile * TV;
+      const uint4* sa = &sm.ring[s][0][cw * 32 + lane];
+      const uint4* sp = &sm.ring[s][1][cw * 32 + lane];
+      uint4 va[VPL], vp[VPL];
+      uint32_t okm = 0u;
+      if (v0 + TV <= nvec) {
 #pragma unroll
-      for (int j = 0; j < UNROLL; ++j) {
-        vm_a[j] = Vec<DT>::vmax(ca[j]);
-        vm_p[j] = Vec<DT>::vmax(cp[j]);
-        accumulate<DT>(ca[j], vm_a[j], oa);
-        accumulate<DT>(cp[j], vm_p[j], op);
+        for (int j = 0; j < VPL; ++j) { va[j] = sa[j * NC * 32]; vp[j] = sp[j * NC * 32]; }
+        okm = (1u << VPL) - 1u;
+      } else {
+#pragma unroll
+        for (int j = 0; j < VPL; ++j) {
+          const bool in = v0 + j * NC * 32 + cw * 32 + lane < nvec;
+          va[j] = in ? sa[j * NC * 32] : Vec<DT>::neg_inf();
+          vp[j] = in ? sp[j * NC * 32] : Vec<DT>::neg_inf();
+          okm |= in ? (1u << j) : 0u;
+        }
       }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sm.empty[s]);       // the vectors are in registers: stage free
 
+      float vm_a[VPL], vm_p[VPL];
+#pragma unroll
+      for (int j = 0; j < VPL; ++j) { vm_a[j] = Vec<DT>::vmax(va[j]); vm_p[j] = Vec<DT>::vmax(vp[j]); }
+
+      float tval_a, tval_p;
+      if (TOPK && tile == 0) {
+        // No threshold yet.  With r = ceil(k / warps), the smallest over the warps of
+        // each warp's r-th largest per-lane maximum has at least k row entries at or
+        // above it, so it bounds the k-th best logit of the row from below.
+        float tm_a = vm_a[0], tm_p = vm_p[0];
+#pragma unroll
+        for (int j = 1; j < VPL; ++j) { tm_a = fmaxf(tm_a, vm_a[j]); tm_p = fmaxf(tm_p, vm_p[j]); }
+        const float ba = warp_rth_largest(tm_a, r, lane);
+        const float bp = warp_rth_largest(tm_p, r, lane);
+        if (lane == 0) { sm.warp_bound[p][0][cw] = ba; sm.warp_bound[p][1][cw] = bp; }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.bound_ready[p]);
+      }
+#pragma unroll
+      for (int j = 0; j < VPL; ++j) {
+        accumulate<DT>(va[j], vm_a[j], oa);
+        accumulate<DT>(vp[j], vm_p[j], op);
+      }
       if (TOPK) {
-        // Merge after tiles 0, 1, 3, 7, ... (whenever the number of tiles seen
-        // doubles): the expected number of later candidates falls like 1/seen.
-        bool force = ((tile + 1) & tile) == 0;
         if (tile == 0) {
-          // No threshold yet.  With r = ceil(k / warps), the smallest over the
-          // warps of each warp's r-th largest per-thread maximum has at least k
-          // row entries at or above it, so it bounds the k-th best logit from below.
-          float tm_a = vm_a[0], tm_p = vm_p[0];
+          if (!mbar_wait(&sm.bound_ready[p], ph, &sm.abort)) { raise_timeout(sm, A.sc); return; }
+          tau0_a = sm.warp_bound[p][0][0]; tau0_p = sm.warp_bound[p][1][0];
 #pragma unroll
-          for (int j = 1; j < UNROLL; ++j) { tm_a = fmaxf(tm_a, vm_a[j]); tm_p = fmaxf(tm_p, vm_p[j]); }
-          const int r = (k + NWARP - 1) / NWARP;
-          float wa = warp_rth_largest(tm_a, r, lane);
-          float wp = warp_rth_largest(tm_p, r, lane);
-          if (lane == 0) { sm.warp_bound[0][warp] = wa; sm.warp_bound[1][warp] = wp; }
-          __syncthreads();
-          float ba = sm.warp_bound[0][0], bp = sm.warp_bound[1][0];
-#pragma unroll
-          for (int w = 1; w < NWARP; ++w) { ba = fminf(ba, sm.warp_bound[0][w]); bp = fminf(bp, sm.warp_bound[1][w]); }
-          tval_a = ba; tval_p = bp;
-          tkey_a = (unsigned long long)f32_order_bits(ba) << 32;   // below every entry with logit >= ba
-          tkey_p = (unsigned long long)f32_order_bits(bp) << 32;
-        }
-        uint32_t pushed_a = 0u, pushed_p = 0u;
-        for (;;) {
-          bool flag = force;
-          bool any_a = false, any_p = false;
-#pragma unroll
-          for (int j = 0; j < UNROLL; ++j) { any_a |= vm_a[j] >= tval_a; any_p |= vm_p[j] >= tval_p; }
-          if (__any_sync(0xffffffffu, any_a)) {
-#pragma unroll
-            for (int j = 0; j < UNROLL; ++j) {
-              const uint32_t idx0 = (uint32_t)((v0 + (int64_t)j * NT + tid) * N);
-              const uint32_t d = push_warp<DT>(sm, 0, ca[j], vm_a[j] >= tval_a, idx0, (uint32_t)A.V, tkey_a,
-                                               (pushed_a >> (j * N)) & ((1u << N) - 1u), K, lane, flag);
-              pushed_a |= d << (j * N);
-            }
+          for (int w = 1; w < NC; ++w) {
+            tau0_a = fminf(tau0_a, sm.warp_bound[p][0][w]);
+            tau0_p = fminf(tau0_p, sm.warp_bound[p][1][w]);
           }
-          if (__any_sync(0xffffffffu, any_p)) {
-#pragma unroll
-            for (int j = 0; j < UNROLL; ++j) {
-              const uint32_t idx0 = (uint32_t)((v0 + (int64_t)j * NT + tid) * N);
-              const uint32_t d = push_warp<DT>(sm, 1, cp[j], vm_p[j] >= tval_p, idx0, (uint32_t)A.V, tkey_p,
-                                               (pushed_p >> (j * N)) & ((1u << N) - 1u), K, lane, flag);
-              pushed_p |= d << (j * N);
-            }
-          }
-          if (!__syncthreads_or(flag)) break;
-          merge_lists(sm, k, K, warp, lane);
-          tkey_a = sm.tau_key[0]; tkey_p = sm.tau_key[1];
-          tval_a = tau_value(tkey_a); tval_p = tau_value(tkey_p);
-          force = false;
+          tval_a = tau0_a; tval_p = tau0_p;
+        } else {
+          tval_a = fmaxf(tau0_a, lds_volatile_f32(&sm.tau[p][0]));
+          tval_p = fmaxf(tau0_p, lds_volatile_f32(&sm.tau[p][1]));
         }
-      }
-      if (more) {
 #pragma unroll
-        for (int j = 0; j < UNROLL; ++j) { ca[j] = na[j]; cp[j] = np_[j]; }
+        for (int j = 0; j < VPL; ++j) {
+          const uint32_t vi = (uint32_t)(v0 + j * NC * 32 + cw * 32 + lane);
+          if (((okm >> j) & 1u) && vm_a[j] >= tval_a) {
+            const int pos = atomicAdd(&sm.qcnt[p][0], 1);
+            if (pos < QCAP) sm.queue[p][0][pos] = vi;
+          }
+          if (((okm >> j) & 1u) && vm_p[j] >= tval_p) {
+            const int pos = atomicAdd(&sm.qcnt[p][1], 1);
+            if (pos < QCAP) sm.queue[p][1][pos] = vi;
+          }
+        }
       }
     }
 
-    // ---- row epilogue: merge the per-thread (max, sum) pairs in a fixed tree
+    if (tail > 0 && cw == 0 && lane == 0) {     // ragged end of the row: scalar loads
+      const int64_t row = A.list[it];
+      const char* ra = (const char*)A.za + row * A.ld * Vec<DT>::ESIZE;
+      const char* rp = (const char*)A.zp + row * A.ld * Vec<DT>::ESIZE;
+      const uint4 ta = load_tail_vector<DT>(ra, nvec * N, tail);
+      const uint4 tp = load_tail_vector<DT>(rp, nvec * N, tail);
+      accumulate<DT>(ta, Vec<DT>::vmax(ta), oa);
+      accumulate<DT>(tp, Vec<DT>::vmax(tp), op);
+    }
+
+    // per-warp (max, sum) pairs, merged in a fixed tree
     float mL_a = oa.mL, mL_p = op.mL, s_a, s_p;
     {
       float s0, s1;
@@ -397,59 +533,235 @@ __global__ void __launch_bounds__(NT, CTAS_PER_SM) stream_kernel(StreamArgs A) {
       merge_scaled(mL_p, s_p, __shfl_xor_sync(0xffffffffu, mL_p, off), __shfl_xor_sync(0xffffffffu, s_p, off));
     }
     if (lane == 0) {
-      sm.red_m[0][warp] = mL_a; sm.red_s[0][warp] = s_a;
-      sm.red_m[1][warp] = mL_p; sm.red_s[1][warp] = s_p;
+      sm.part_mL[p][0][cw] = mL_a; sm.part_s[p][0][cw] = s_a;
+      sm.part_mL[p][1][cw] = mL_p; sm.part_s[p][1][cw] = s_p;
     }
-    __syncthreads();
-    if (TOPK) merge_lists(sm, k, K, warp, lane);          // folds whatever the last tiles appended
-    if (tid < 2) {
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sm.row_done[p]);
+  }
+}
+
+// ---- top-k warps ---------------------------------------------------------------
+template <int DT, int KPL>
+__device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, int t, int p, int lane) {
+  constexpr int N = Vec<DT>::N;
+  constexpr bool TOPK = KPL > 0;
+  constexpr int KL = KPL > 0 ? KPL : 1;
+  const int64_t nvec = A.V / N;
+  const int tail = (int)(A.V - nvec * N);
+  const int k = A.k;
+  unsigned long long* stg = sm.skeys[p][t];
+  int lr = p;
+  for (int64_t it = (int64_t)blockIdx.x + (int64_t)p * gridDim.x; it < n_rows; it += 2ll * gridDim.x, lr += 2) {
+    const uint32_t ph = (uint32_t)((lr >> 1) & 1);
+    const int64_t row = A.list[it];
+    const int64_t rrow = A.record_offset + row;
+    const char* rmine = (const char*)(t == 0 ? A.za : A.zp) + row * A.ld * Vec<DT>::ESIZE;
+    const char* ra = (const char*)A.za + row * A.ld * Vec<DT>::ESIZE;
+    const char* rp = (const char*)A.zp + row * A.ld * Vec<DT>::ESIZE;
+    unsigned long long L[KL];
+#pragma unroll
+    for (int j = 0; j < KL; ++j) L[j] = 0ull;
+    unsigned long long tau_key = 0ull;
+    int staged = 0, head = 0;
+    bool overflow = false;
+    int n_seen = 0;
+    const long long t0 = clock64();
+    for (;;) {
+      // probe the end of the row first: if the consumers are done, the count read
+      // after it is final
+      int done = 0;
+      if (lane == 0) done = mbar_try_wait(&sm.row_done[p], ph) ? 1 : 0;
+      done = __shfl_sync(0xffffffffu, done, 0);
+      if (TOPK) {
+        int n = (int)lds_volatile_u32(&sm.qcnt[p][t]);
+        if (n > QCAP) { overflow = true; n = QCAP; }
+        n_seen = n;
+        if (head < n && !overflow) {
+          const int nb = n - head < 32 ? n - head : 32;
+          uint32_t vi = QEMPTY;
+          if (lane < nb) {
+            int spins = 0;
+            do { vi = lds_volatile_u32(&sm.queue[p][t][head + lane]); } while (vi == QEMPTY && ++spins < (1 << 22));
+          }
+          if (__any_sync(0xffffffffu, lane < nb && vi == QEMPTY)) { raise_timeout(sm, A.sc); return; }
+          uint4 v = Vec<DT>::neg_inf();
+          if (lane < nb) v = ldg_stream((const uint4*)rmine + vi);
+          staged = filter_vector<DT>(v, vi, lane < nb, A.V, tau_key, stg, staged, lane);
+          if (staged > 0) {
+            const unsigned long long nt = drain_staged<KL>(L, stg, staged, k, lane);
+            if (nt != tau_key) {
+              tau_key = nt;
+              if (lane == 0 && nt != 0ull) sts_volatile_f32(&sm.tau[p][t], key_value(nt));
+            }
+          }
+          head += nb;
+          continue;
+        }
+      }
+      if (done) break;
+      if (*(volatile int*)&sm.abort) return;
+      if (clock64() - t0 > kSpinLimit) { raise_timeout(sm, A.sc); return; }
+      __nanosleep(100);
+    }
+
+    if (TOPK) {
+      if (overflow) {
+        // The queue could not hold the row's candidates (an ascending ramp, a row of
+        // equal logits): start over and scan the whole row from memory.
+#pragma unroll
+        for (int j = 0; j < KL; ++j) L[j] = 0ull;
+        tau_key = 0ull;
+        staged = 0;
+        for (int64_t b = 0; b < nvec; b += 32) {
+          const int64_t vi = b + lane;
+          uint4 v = Vec<DT>::neg_inf();
+          if (vi < nvec) v = ldg_stream((const uint4*)rmine + vi);
+          staged = filter_vector<DT>(v, (uint32_t)vi, vi < nvec, A.V, tau_key, stg, staged, lane);
+          if (staged > 0) tau_key = drain_staged<KL>(L, stg, staged, k, lane);
+        }
+      }
+      if (tail > 0) {
+        uint4 v = Vec<DT>::neg_inf();
+        if (lane == 0) v = load_tail_vector<DT>(rmine, nvec * N, tail);
+        staged = filter_vector<DT>(v, (uint32_t)nvec, lane == 0, A.V, tau_key, stg, staged, lane);
+        if (staged > 0) tau_key = drain_staged<KL>(L, stg, staged, k, lane);
+      }
+      // the record: this tensor's list, best first, every entry with both logits
+#pragma unroll
+      for (int j = 0; j < KL; ++j) {
+        const int pos = lane * KL + j;
+        if (pos < k) {
+          const int64_t o = rrow * (2 * k) + (int64_t)t * k + pos;
+          const unsigned long long key = L[j];
+          if (key != 0ull) {
+            const uint32_t idx = key_index(key);
+            A.rec.idx[o] = (int32_t)idx;
+            A.rec.za[o] = Vec<DT>::load_scalar(ra, idx);
+            A.rec.zp[o] = Vec<DT>::load_scalar(rp, idx);
+          } else {
+            A.rec.idx[o] = -1; A.rec.za[o] = 0.f; A.rec.zp[o] = 0.f;
+          }
+        }
+      }
+      // hand the slot back clean
+      for (int i = lane; i < n_seen; i += 32) sm.queue[p][t][i] = QEMPTY;
+      if (lane == 0) { sm.qcnt[p][t] = 0; sts_volatile_f32(&sm.tau[p][t], JP_NEG_INF); }
+    }
+
+    if (lane == 0) {
       // log-sum-exp = ln2 (M + log2 S).  S = 2^e f with f in [1,2): logf(f) is good to an
       // ulp of a number below 0.7, and the large part (M + e) ln2 is formed in double, so
       // the published fp32 values are rounded once.
-      float M = sm.red_m[tid][0];
-      for (int w = 1; w < NWARP; ++w) M = fmaxf(M, sm.red_m[tid][w]);
+      float M = sm.part_mL[p][t][0];
+      for (int w = 1; w < NC; ++w) M = fmaxf(M, sm.part_mL[p][t][w]);
       float S = 0.f;
-      for (int w = 0; w < NWARP; ++w)
-        if (sm.red_m[tid][w] != JP_NEG_INF) S += sm.red_s[tid][w] * exp2_int(sm.red_m[tid][w] - M);
+      for (int w = 0; w < NC; ++w)
+        if (sm.part_mL[p][t][w] != JP_NEG_INF) S += sm.part_s[p][t][w] * exp2_int(sm.part_mL[p][t][w] - M);
       int e;
       const float f = 2.f * frexpf(S, &e);                // S = f * 2^(e-1)
       const double lse = ((double)M + (double)(e - 1)) * 0.6931471805599453 + (double)logf(f);
       const float lsef = (float)lse;
-      const char* rowp = tid == 0 ? ra : rp;
-      const float zx = Vec<DT>::load_scalar(rowp, x);
+      const int32_t x = A.tokens[row];
+      const float zx = Vec<DT>::load_scalar(rmine, x);
       const float lpx = (float)((double)zx - lse);
-      if (tid == 0) { A.rec.lse_a[rrow] = lsef; A.rec.lq[rrow] = lpx; A.rec.flag[rrow] = 1; }
-      else          { A.rec.lse_p[rrow] = lsef; A.rec.lp[rrow] = lpx; }
+      if (t == 0) { A.rec.lse_a[rrow] = lsef; A.rec.lq[rrow] = lpx; A.rec.flag[rrow] = 1; }
+      else        { A.rec.lse_p[rrow] = lsef; A.rec.lp[rrow] = lpx; }
       if (!isfinite(lsef)) atomicAdd(&A.sc->n_nonfinite, 1ull);
     }
-    if (TOPK) {
-      if (tid < 2 * k) {
-        int t = tid >= k;
-        int j = tid - t * k;
-        unsigned long long key = sm.buf[t][j];
-        int64_t o = rrow * (2 * k) + tid;
-        if (key != 0ull) {
-          uint32_t idx = key_index(key);
-          A.rec.idx[o] = (int32_t)idx;
-          A.rec.za[o] = Vec<DT>::load_scalar(ra, idx);
-          A.rec.zp[o] = Vec<DT>::load_scalar(rp, idx);
-        } else {
-          A.rec.idx[o] = -1; A.rec.za[o] = 0.f; A.rec.zp[o] = 0.f;
-        }
-      }
-      __syncthreads();
-      for (int i = tid; i < 2 * K; i += NT) sm.buf[i >= K][i - (i >= K) * K] = 0ull;
-      if (tid < 2) sm.tau_key[tid] = 0ull;
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sm.slot_free[p]);
+  }
+}
+
+template <int DT, int KPL>
+__global__ void __launch_bounds__(NTHREADS, 1) stream_kernel(StreamArgs A) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  StreamSmem& sm = *reinterpret_cast<StreamSmem*>(smem_raw);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  for (int i = tid; i < 2 * 2 * QCAP; i += NTHREADS) (&sm.queue[0][0][0])[i] = QEMPTY;
+  if (tid == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], NC); }
+    for (int p = 0; p < 2; ++p) {
+      mbar_init(&sm.row_done[p], NC);
+      mbar_init(&sm.slot_free[p], 2);
+      mbar_init(&sm.bound_ready[p], NC);
+      for (int t = 0; t < 2; ++t) { sm.qcnt[p][t] = 0; sm.tau[p][t] = JP_NEG_INF; }
     }
-    __syncthreads();
+    sm.abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const int64_t n_rows = A.sc->n_list;
+
+  if (warp == 0) {
+    if (lane == 0) producer_loop<DT>(A, sm, n_rows);
+  } else if (warp <= NC) {
+    consumer_loop<DT, (KPL > 0)>(A, sm, n_rows, warp - 1, lane);
+  } else {
+    const int tw = warp - 1 - NC;
+    topk_loop<DT, KPL>(A, sm, n_rows, tw & 1, tw >> 1, lane);
+  }
+}
+
+// Splits the rows of one call into the list of valid rows the stream kernel walks
+// and the masked / out-of-range ones, whose records are cleared here.
+__global__ void __launch_bounds__(256) prep_rows_kernel(StreamArgs A) {
+  const int64_t row = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  const int lane = threadIdx.x & 31;
+  bool valid = false, bad = false;
+  if (row < A.T) {
+    valid = A.mask == nullptr || A.mask[row] != 0;
+    if (valid) {
+      const int32_t x = A.tokens[row];
+      if (x < 0 || (int64_t)x >= A.V) { valid = false; bad = true; }
+    }
+    if (!valid) {
+      const int64_t rrow = A.record_offset + row;
+      A.rec.flag[rrow] = 0;
+      A.rec.lse_a[rrow] = 0.f; A.rec.lse_p[rrow] = 0.f;
+      A.rec.lq[rrow] = 0.f; A.rec.lp[rrow] = 0.f;
+    }
+  }
+  const uint32_t vm = __ballot_sync(0xffffffffu, valid), bm = __ballot_sync(0xffffffffu, bad);
+  int base = 0;
+  if (lane == 0 && vm) base = atomicAdd(&A.sc->n_list, __popc(vm));
+  base = __shfl_sync(0xffffffffu, base, 0);
+  if (valid) A.list[base + __popc(vm & ((1u << lane) - 1u))] = (int32_t)row;
+  if (lane == 0 && bm) atomicAdd(&A.sc->n_bad_token, (unsigned long long)__popc(bm));
+}
+
+// ---- exact normaliser -----------------------------------------------------------
+constexpr int XNT = 256;
+constexpr int XNWARP = XNT / 32;
+constexpr int XUNROLL = 4;
+constexpr int XCTAS_PER_SM = 2;
+
+template <int DT>
+__device__ __forceinline__ void load_tile(uint4 (&va)[XUNROLL], uint4 (&vp)[XUNROLL], const char* ra,
+                                          const char* rp, int64_t v0, int64_t nvec, int tail, int tid) {
+#pragma unroll
+  for (int j = 0; j < XUNROLL; ++j) {
+    int64_t vi = v0 + (int64_t)j * XNT + tid;
+    if (vi < nvec) {
+      va[j] = ldg_stream((const uint4*)ra + vi);
+      vp[j] = ldg_stream((const uint4*)rp + vi);
+    } else if (vi == nvec && tail > 0) {
+      va[j] = load_tail_vector<DT>(ra, nvec * Vec<DT>::N, tail);
+      vp[j] = load_tail_vector<DT>(rp, nvec * Vec<DT>::N, tail);
+    } else {
+      va[j] = Vec<DT>::neg_inf();
+      vp[j] = Vec<DT>::neg_inf();
+    }
   }
 }
 
 // Exact normaliser: Z_t = sum_v min(q_t(v), p_t(v)/lambda), one more pass over the
 // row with the log-sum-exps known (Eq. obrs_dist; Appendix A, Z_C).
 template <int DT>
-__global__ void __launch_bounds__(NT, CTAS_PER_SM) exact_z_kernel(ExactZArgs A) {
-  __shared__ float red[NWARP];
+__global__ void __launch_bounds__(XNT, XCTAS_PER_SM) exact_z_kernel(ExactZArgs A) {
+  __shared__ float red[XNWARP];
   __shared__ int s_row;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   constexpr int N = Vec<DT>::N;
@@ -473,11 +785,11 @@ __global__ void __launch_bounds__(NT, CTAS_PER_SM) exact_z_kernel(ExactZArgs A) 
     const float ca = A.rec.lse_a[rrow] * kLog2e;
     const float cp = A.rec.lse_p[rrow] * kLog2e + log2_lambda;
     float acc = 0.f;
-    for (int64_t v0 = 0; v0 < nvt; v0 += (int64_t)NT * UNROLL) {
-      uint4 va[UNROLL], vp[UNROLL];
+    for (int64_t v0 = 0; v0 < nvt; v0 += (int64_t)XNT * XUNROLL) {
+      uint4 va[XUNROLL], vp[XUNROLL];
       load_tile<DT>(va, vp, ra, rp, v0, nvec, tail, tid);
 #pragma unroll
-      for (int j = 0; j < UNROLL; ++j) {
+      for (int j = 0; j < XUNROLL; ++j) {
 #pragma unroll
         for (int e = 0; e < N; ++e) {
           float q = ex2_approx(fmaf(Vec<DT>::get(va[j], e), kLog2e, -ca));
@@ -492,7 +804,7 @@ __global__ void __launch_bounds__(NT, CTAS_PER_SM) exact_z_kernel(ExactZArgs A) 
     __syncthreads();
     if (tid == 0) {
       double S = 0.0;
-      for (int w = 0; w < NWARP; ++w) S += (double)red[w];
+      for (int w = 0; w < XNWARP; ++w) S += (double)red[w];
       A.out[rrow] = (float)S;
     }
     __syncthreads();
@@ -505,26 +817,45 @@ int stream_grid_size(int device) {
   return sms;
 }
 
+template <int DT, int KPL>
+static cudaError_t launch_stream_variant(const StreamArgs& a, cudaStream_t s, int grid) {
+  // per device, and cheap: set on every launch rather than cached per process
+  cudaError_t e = cudaFuncSetAttribute(stream_kernel<DT, KPL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)sizeof(StreamSmem));
+  if (e != cudaSuccess) return e;
+  stream_kernel<DT, KPL><<<grid, NTHREADS, sizeof(StreamSmem), s>>>(a);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_stream(const StreamArgs& a, cudaStream_t s, int sms) {
   if (a.T <= 0) return cudaSuccess;
-  const int grid = sms * CTAS_PER_SM;
-  int g = (int)(a.T < grid ? a.T : grid);
+  prep_rows_kernel<<<(unsigned)((a.T + 255) / 256), 256, 0, s>>>(a);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  const int grid = (int)(a.T < sms ? a.T : sms);
+  const int kpl = a.k <= 0 ? 0 : a.k <= 32 ? 1 : a.k <= 64 ? 2 : 4;
   if (a.dtype == JP_BF16) {
-    if (a.k > 0) stream_kernel<JP_BF16, true><<<g, NT, 0, s>>>(a);
-    else stream_kernel<JP_BF16, false><<<g, NT, 0, s>>>(a);
-  } else {
-    if (a.k > 0) stream_kernel<JP_F32, true><<<g, NT, 0, s>>>(a);
-    else stream_kernel<JP_F32, false><<<g, NT, 0, s>>>(a);
+    switch (kpl) {
+      case 0: return launch_stream_variant<JP_BF16, 0>(a, s, grid);
+      case 1: return launch_stream_variant<JP_BF16, 1>(a, s, grid);
+      case 2: return launch_stream_variant<JP_BF16, 2>(a, s, grid);
+      default: return launch_stream_variant<JP_BF16, 4>(a, s, grid);
+    }
   }
-  return cudaGetLastError();
+  switch (kpl) {
+    case 0: return launch_stream_variant<JP_F32, 0>(a, s, grid);
+    case 1: return launch_stream_variant<JP_F32, 1>(a, s, grid);
+    case 2: return launch_stream_variant<JP_F32, 2>(a, s, grid);
+    default: return launch_stream_variant<JP_F32, 4>(a, s, grid);
+  }
 }
 
 cudaError_t launch_exact_z(const ExactZArgs& a, cudaStream_t s, int sms) {
   if (a.T <= 0) return cudaSuccess;
-  const int grid = sms * CTAS_PER_SM;
+  const int grid = sms * XCTAS_PER_SM;
   int g = (int)(a.T < grid ? a.T : grid);
-  if (a.dtype == JP_BF16) exact_z_kernel<JP_BF16><<<g, NT, 0, s>>>(a);
-  else exact_z_kernel<JP_F32><<<g, NT, 0, s>>>(a);
+  if (a.dtype == JP_BF16) exact_z_kernel<JP_BF16><<<g, XNT, 0, s>>>(a);
+  else exact_z_kernel<JP_F32><<<g, XNT, 0, s>>>(a);
   return cudaGetLastError();
 }
 
