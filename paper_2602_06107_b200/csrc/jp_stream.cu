@@ -13,14 +13,17 @@
 //                   release the stage, then update the online (max, sum) of both
 //                   rows and test each vector's maximum against the row's current
 //                   top-k threshold tau; a vector that may hold a top-k entry is
-//                   pushed BY INDEX into a small shared-memory queue;
+//                   copied, with its index, into a small shared-memory ring queue;
 //   top-k warps     four of them, one per (tensor, row slot): they drain the
-//                   queue while the consumers keep streaming, re-read the few
-//                   candidate vectors from L2, keep the sorted list in registers
-//                   (bitonic sort / merge across the lanes, or single inserts)
-//                   and publish the tightened tau; at the end of the row they
-//                   finish the log-sum-exp, gather the sampled token's logit and
-//                   write the row's record.
+//                   queue while the consumers keep streaming.  Every entry at or
+//                   above tau is counted in a histogram over the 16-bit order code
+//                   of its logit and its 64-bit key is appended to a buffer; the
+//                   histogram gives the running tau (the highest code with at least
+//                   k entries at or above it) without sorting anything.  At the end
+//                   of the row the buffered keys at or above the final tau are
+//                   sorted into the list (bitonic sort / merge across the lanes),
+//                   the warp finishes the log-sum-exp, gathers the sampled token's
+//                   logit and writes the row's record.
 //
 // Rows alternate between two "slots" (queue, tau, partial sums, barriers), so the
 // consumers start the next row while the top-k warps finish the previous one.
@@ -29,17 +32,38 @@
 //
 // Every wait is bounded: a wait that runs out raises the CTA's abort flag, the
 // status word gets JP_ERR_TIMEOUT and every warp leaves its loop.
+#include <type_traits>
+
 #include "jp_common.cuh"
 #include "jp_internal.h"
 
 namespace jp {
 
-constexpr int NC = 8;                     // consumer warps
-constexpr int VPL = 4;                    // 16-byte vectors per lane per tensor per tile
-constexpr int TV = NC * 32 * VPL;         // vectors per tensor per tile
-constexpr int STAGES = 5;
-constexpr int QCAP = 2048;                // candidate-vector queue entries per (slot, tensor)
-constexpr int SCAP = 512;                 // staged keys per top-k warp
+#ifndef JP_NC
+#define JP_NC 16
+#endif
+#ifndef JP_VPL
+#define JP_VPL 4
+#endif
+#ifndef JP_TOPK_SLEEP_NS
+#define JP_TOPK_SLEEP_NS 300
+#endif
+#ifndef JP_STAGES
+#define JP_STAGES 5
+#endif
+#ifndef JP_NG
+#define JP_NG 2
+#endif
+constexpr int NC = JP_NC;                 // consumer warps
+constexpr int NG = JP_NG;                 // consumer groups: group q takes tiles q, q + NG, ...
+constexpr int WPT = NC / NG;              // warps that share one tile
+constexpr int VPL = JP_VPL;               // 16-byte vectors per lane per tensor per tile
+constexpr int TV = WPT * 32 * VPL;        // vectors per tensor per tile
+static_assert(NC % NG == 0 && NG < JP_STAGES, "consumer groups must divide the warps and fit the ring");
+constexpr int STAGES = JP_STAGES;
+constexpr int QCAP = 256;                 // candidate-vector ring entries per (slot, tensor); power of two
+constexpr int SCAP = 512;                 // buffered keys per top-k warp
+constexpr int NB = 1024;                  // histogram bins (16-bit order codes above the row's first bound)
 constexpr int NTOPK = 4;                  // top-k warps: (tensor, slot)
 constexpr int NWARPS = 1 + NC + NTOPK;
 constexpr int NTHREADS = NWARPS * 32;
@@ -48,11 +72,14 @@ constexpr long long kSpinLimit = 4000000000ll;   // clock cycles a wait may last
 
 struct __align__(128) StreamSmem {
   uint4 ring[STAGES][2][TV];              // [stage][tensor][vector]
-  unsigned long long skeys[2][2][SCAP];   // [slot][tensor] keys waiting to be merged
-  uint32_t queue[2][2][QCAP];             // [slot][tensor] candidate vector indices
+  uint4 qdata[2][2][QCAP];                // [slot][tensor] candidate vectors ...
+  unsigned long long skeys[2][2][SCAP];   // [slot][tensor] keys of entries at or above tau
+  uint32_t qidx[2][2][QCAP];              // ... and their vector index (QEMPTY = not written yet)
+  uint32_t hist[2][2][NB];                // [slot][tensor] entries seen per order code
   unsigned long long full[STAGES], empty[STAGES];
   unsigned long long row_done[2], slot_free[2], bound_ready[2];
-  int qcnt[2][2];
+  int qtail[2][2];                        // next ring position to reserve (consumers)
+  int qhead[2][2];                        // first position not yet drained (top-k warp)
   float tau[2][2];                        // published threshold (a logit value)
   float warp_bound[2][2][NC];
   float part_mL[2][2][NC];
@@ -85,14 +112,31 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, uint32_t 
       : "memory");
   return ok != 0;
 }
-// Bounded wait; false = gave up (or another warp did).
+// Same, but the thread may stay suspended for up to `ns` nanoseconds before it answers.
+__device__ __forceinline__ bool mbar_try_wait_for(unsigned long long* bar, uint32_t parity, uint32_t ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(ns)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait; false = gave up (or another warp did).  The clock is read once in
+// 64 polls, each of which may itself suspend the thread for a while.
 __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity, volatile int* abort) {
   if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  for (;;) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if (*abort) return false;
-    if (clock64() - t0 > kSpinLimit) { *abort = 1; return false; }
+  long long t0 = 0;
+  for (uint32_t i = 0;; ++i) {
+    if (mbar_try_wait_for(bar, parity, 2000u)) return true;
+    if ((i & 63u) == 0u) {
+      if (*abort) return false;
+      const long long now = clock64();
+      if (i == 0u) t0 = now;
+      else if (now - t0 > kSpinLimit) { *abort = 1; return false; }
+    }
   }
 }
 __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, unsigned long long* bar) {
@@ -165,6 +209,37 @@ struct Online {
   unsigned long long s2;
 };
 
+#ifndef JP_POLY_WORDS
+#define JP_POLY_WORDS 0
+#endif
+// 2^x for two x <= ~0 without the special-function unit, folded into the running
+// sums: returns s + 2^x (both lanes).  x is rounded to the nearest integer n with the
+// 1.5 * 2^23 trick, 2^(x - n) comes from a degree-5 polynomial on [-0.5, 0.5] (fitted
+// for the smallest maximum relative error, 1.7e-7, about that of ex2.approx) and 2^n
+// is built in the exponent field.  x is clamped at -125 so that the exponent stays
+// valid: terms below 2^-125 count as 2^-125, far below one ulp of any sum that holds
+// a term near 1.  A NaN stays a NaN.
+__device__ __forceinline__ unsigned long long add_exp2_poly2(unsigned long long s2, unsigned long long x2) {
+  float x0, x1;
+  unpack2(x2, x0, x1);
+  asm("max.NaN.f32 %0, %0, %1;" : "+f"(x0) : "f"(-125.f));
+  asm("max.NaN.f32 %0, %0, %1;" : "+f"(x1) : "f"(-125.f));
+  x2 = pack2(x0, x1);
+  const unsigned long long t2 = fadd2(x2, pack2(12582912.f, 12582912.f));
+  const unsigned long long n2 = fadd2(t2, pack2(-12582912.f, -12582912.f));
+  const unsigned long long f2 = ffma2(n2, pack2(-1.f, -1.f), x2);
+  unsigned long long p2 = ffma2(pack2(1.326462603e-03f, 1.326462603e-03f), f2, pack2(9.671481326e-03f, 9.671481326e-03f));
+  p2 = ffma2(p2, f2, pack2(5.550733581e-02f, 5.550733581e-02f));
+  p2 = ffma2(p2, f2, pack2(2.402224243e-01f, 2.402224243e-01f));
+  p2 = ffma2(p2, f2, pack2(6.931470037e-01f, 6.931470037e-01f));
+  p2 = ffma2(p2, f2, pack2(1.f, 1.f));
+  float t0, t1;
+  unpack2(t2, t0, t1);
+  const float sc0 = __int_as_float((__float_as_int(t0) << 23) + 0x3f800000);
+  const float sc1 = __int_as_float((__float_as_int(t1) << 23) + 0x3f800000);
+  return ffma2(p2, pack2(sc0, sc1), s2);
+}
+
 // One 16-byte vector into the online (max, sum).
 template <int DT>
 __device__ __forceinline__ void accumulate(const uint4& v, float vm, Online& o) {
@@ -179,6 +254,28 @@ __device__ __forceinline__ void accumulate(const uint4& v, float vm, Online& o) 
     o.m = vm;
     o.mL = nmL;
   }
+#ifdef JP_SCALAR_ACC
+  {
+    float s0, s1;
+    unpack2(o.s2, s0, s1);
+    const float nm = -o.mL;
+    if (DT == JP_BF16) {
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        s0 += ex2_approx(fmaf(__uint_as_float(w[i] << 16), kLog2e, nm));
+        s1 += ex2_approx(fmaf(__uint_as_float(w[i] & 0xffff0000u), kLog2e, nm));
+      }
+    } else {
+      s0 += ex2_approx(fmaf(__uint_as_float(v.x), kLog2e, nm));
+      s1 += ex2_approx(fmaf(__uint_as_float(v.y), kLog2e, nm));
+      s0 += ex2_approx(fmaf(__uint_as_float(v.z), kLog2e, nm));
+      s1 += ex2_approx(fmaf(__uint_as_float(v.w), kLog2e, nm));
+    }
+    o.s2 = pack2(s0, s1);
+    return;
+  }
+#endif
   const unsigned long long L2 = pack2(kLog2e, kLog2e);
   const unsigned long long nm2 = pack2(-o.mL, -o.mL);
   if (DT == JP_BF16) {
@@ -186,9 +283,15 @@ __device__ __forceinline__ void accumulate(const uint4& v, float vm, Online& o) 
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       unsigned long long a = ffma2(pack2(__uint_as_float(w[i] << 16), __uint_as_float(w[i] & 0xffff0000u)), L2, nm2);
-      float a0, a1;
-      unpack2(a, a0, a1);
-      o.s2 = fadd2(o.s2, pack2(ex2_approx(a0), ex2_approx(a1)));
+      if (i >= 4 - JP_POLY_WORDS) {
+        // a share of the exponentials runs on the FMA pipe: one ex2 per logit would
+        // saturate the special-function unit before HBM
+        o.s2 = add_exp2_poly2(o.s2, a);
+      } else {
+        float a0, a1;
+        unpack2(a, a0, a1);
+        o.s2 = fadd2(o.s2, pack2(ex2_approx(a0), ex2_approx(a1)));
+      }
     }
   } else {
     unsigned long long a = ffma2(pack2(__uint_as_float(v.x), __uint_as_float(v.y)), L2, nm2);
@@ -321,12 +424,28 @@ __device__ __forceinline__ unsigned long long kth_key(const unsigned long long (
   return __shfl_sync(0xffffffffu, v, (k - 1) / KPL);
 }
 
-// Tests the entries of one vector per lane against tau and appends the winners'
-// keys to the staging buffer; returns the new number of staged keys.
+// The running threshold of one (row, tensor): `code` is the highest 16-bit order
+// code with at least k of the entries seen so far at or above it (so the k-th
+// best logit of the row is at or above the low edge of that code's bin); `cnt`
+// counts the entries seen at or above it.  `key` is the exact k-th best key of
+// the sorted list once a merge has happened (0 before).
+struct Tau {
+  uint32_t code;
+  int cnt;
+  unsigned long long key;
+};
+
+__device__ __forceinline__ uint32_t order_code(float v) { return f32_order_bits(v) >> 16; }
+// low edge of a code's bin, as a logit
+__device__ __forceinline__ float code_value(uint32_t code) { return order_bits_f32(code << 16); }
+
+// Tests the entries of one vector per lane against tau; every entry at or above
+// it is counted in the histogram and its key appended to the buffer.  Returns
+// the new number of buffered keys.
 template <int DT>
-__device__ __forceinline__ int filter_vector(const uint4& v, uint32_t vi, bool have, int64_t V,
-                                             unsigned long long tau_key, unsigned long long* stg, int staged,
-                                             int lane) {
+__device__ __forceinline__ int filter_vector(const uint4& v, uint32_t vi, bool have, int64_t V, Tau& tau,
+                                             uint32_t base, uint32_t* hist, unsigned long long* stg,
+                                             int staged, int lane) {
   constexpr int N = Vec<DT>::N;
   unsigned long long key[N];
   uint32_t pass = 0u;
@@ -334,30 +453,80 @@ __device__ __forceinline__ int filter_vector(const uint4& v, uint32_t vi, bool h
   for (int e = 0; e < N; ++e) {
     const uint32_t idx = vi * N + e;
     key[e] = make_key(Vec<DT>::get(v, e), idx);
-    if (have && (int64_t)idx < V && key[e] > tau_key) pass |= 1u << e;
+    const uint32_t code = (uint32_t)(key[e] >> 48);
+    if (have && (int64_t)idx < V && code >= tau.code) {
+      const uint32_t bin = code - base < (uint32_t)(NB - 1) ? code - base : (uint32_t)(NB - 1);
+      atomicAdd(&hist[bin], 1u);
+      if (key[e] > tau.key) pass |= 1u << e;
+    }
+  }
+  // entries counted but below the exact key (ties that a merge already ruled out) still
+  // count toward tau.cnt: they are entries of the row at or above the code
+  uint32_t counted = 0u;
+#pragma unroll
+  for (int e = 0; e < N; ++e) {
+    const uint32_t idx = vi * N + e;
+    if (have && (int64_t)idx < V && (uint32_t)(key[e] >> 48) >= tau.code) counted += 1u;
   }
   const int c = __popc(pass);
-  int incl = c;
+  int incl = c | ((int)counted << 16);       // two prefix sums in one shuffle chain
 #pragma unroll
   for (int off = 1; off < 32; off <<= 1) {
     const int n = __shfl_up_sync(0xffffffffu, incl, off);
     if (lane >= off) incl += n;
   }
   const int total = __shfl_sync(0xffffffffu, incl, 31);
-  int pos = staged + incl - c;
+  int pos = staged + (incl & 0xffff) - c;
 #pragma unroll
   for (int e = 0; e < N; ++e)
     if ((pass >> e) & 1u) stg[pos++] = key[e];
+  tau.cnt += total >> 16;
   __syncwarp();
-  return staged + total;
+  return staged + (total & 0xffff);
 }
 
-// Empties the staging buffer into the list and returns the new tau key.
+// Raises tau.code while at least k counted entries stay at or above it.
+__device__ __forceinline__ bool advance_tau(Tau& tau, uint32_t base, const uint32_t* hist, int k) {
+  bool moved = false;
+  for (;;) {
+    const uint32_t bin = tau.code - base;
+    if (bin >= (uint32_t)(NB - 1)) break;
+    const int h = (int)lds_volatile_u32(&hist[bin]);
+    if (tau.cnt - h < k) break;
+    tau.cnt -= h;
+    tau.code += 1u;
+    moved = true;
+  }
+  return moved;
+}
+
+// Drops buffered keys that can no longer be among the k best.
+__device__ __forceinline__ int compact_keys(unsigned long long* stg, int staged, const Tau& tau, int lane) {
+  int out = 0;
+  for (int b = 0; b < staged; b += 32) {
+    const int i = b + lane;
+    unsigned long long key = 0ull;
+    bool keep = false;
+    if (i < staged) {
+      key = stg[i];
+      keep = (uint32_t)(key >> 48) >= tau.code && key > tau.key;
+    }
+    const uint32_t m = __ballot_sync(0xffffffffu, keep);
+    __syncwarp();
+    if (keep) stg[out + __popc(m & ((1u << lane) - 1u))] = key;
+    out += __popc(m);
+    __syncwarp();
+  }
+  return out;
+}
+
+// Folds every buffered key into the sorted list; returns the list's k-th key.
 template <int KPL>
-__device__ __forceinline__ unsigned long long drain_staged(unsigned long long (&L)[KPL],
-                                                           const unsigned long long* stg, int& staged, int k,
-                                                           int lane) {
+__device__ __forceinline__ unsigned long long merge_all(unsigned long long (&L)[KPL],
+                                                        const unsigned long long* stg, int& staged, int k,
+                                                        int lane) {
   constexpr int SORT_MIN = 6 * KPL;       // below this, single inserts are cheaper than a sort + merge
+  __syncwarp();
   while (staged >= SORT_MIN) merge_staged<KPL>(L, stg, staged, lane);
   while (staged > 0) {
     insert_one<KPL>(L, stg[staged - 1], lane);
@@ -370,6 +539,21 @@ __device__ __forceinline__ unsigned long long drain_staged(unsigned long long (&
 __device__ __forceinline__ void raise_timeout(StreamSmem& sm, Scalars* sc) {
   sm.abort = 1;
   atomicExch(&sc->status, (int)JP_ERR_TIMEOUT);
+}
+
+// A consumer lane hands one vector that may hold a top-k entry to the slot's
+// top-k warp: reserve a ring position, wait (bounded) until the ring has room,
+// write the vector, then publish it by writing its index.
+__device__ __forceinline__ void push_candidate(StreamSmem& sm, int p, int t, const uint4& v, uint32_t vi) {
+  const int pos = atomicAdd(&sm.qtail[p][t], 1);
+  int spins = 0;
+  while (pos - (int)lds_volatile_u32(&sm.qhead[p][t]) >= QCAP) {
+    if (++spins > (1 << 24) || *(volatile int*)&sm.abort) { sm.abort = 1; return; }
+  }
+  const int slot = pos & (QCAP - 1);
+  sm.qdata[p][t][slot] = v;
+  __threadfence_block();
+  asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(smem_u32(&sm.qidx[p][t][slot])), "r"(vi) : "memory");
 }
 
 // ---- producer ---------------------------------------------------------------
@@ -418,11 +602,13 @@ __device__ void consumer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_row
   constexpr int N = Vec<DT>::N;
   const int64_t nvec = A.V / N;
   const int tail = (int)(A.V - nvec * N);
-  const int ntiles = nvec > 0 ? (int)((nvec + TV - 1) / TV) : 1;
+  const uint32_t ntiles = nvec > 0 ? (uint32_t)((nvec + TV - 1) / TV) : 1u;
   const int r = (A.k + NC - 1) / NC;
-  long long g = 0;
+  const int gq = cw / WPT;              // this warp's group: it takes tiles gq, gq + NG, ...
+  const int wq = cw % WPT;              // its place among the warps that share a tile
+  uint32_t g0 = 0;                      // ring position of the current row's tile 0
   int lr = 0;
-  for (int64_t it = blockIdx.x; it < n_rows; it += gridDim.x, ++lr) {
+  for (int64_t it = blockIdx.x; it < n_rows; it += gridDim.x, ++lr, g0 += ntiles) {
     const int p = lr & 1;
     const uint32_t ph = (uint32_t)((lr >> 1) & 1);
     // the slot's queue, tau and partial sums are free once both of its top-k warps
@@ -432,26 +618,23 @@ __device__ void consumer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_row
     Online oa{JP_NEG_INF, 0.f, 0ull}, op{JP_NEG_INF, 0.f, 0ull};
     float tau0_a = JP_NEG_INF, tau0_p = JP_NEG_INF;
 
-    for (int tile = 0; tile < ntiles; ++tile, ++g) {
-      const int s = (int)(g % STAGES);
-      if (!mbar_wait(&sm.full[s], (uint32_t)((g / STAGES) & 1), &sm.abort)) { raise_timeout(sm, A.sc); return; }
-      const int64_t v0 = (int64_t)tile * TV;
-      const uint4* sa = &sm.ring[s][0][cw * 32 + lane];
-      const uint4* sp = &sm.ring[s][1][cw * 32 + lane];
+    // One tile of both rows.  FULL = every vector of the tile lies inside the row;
+    // first = this warp's first tile of the row.
+    auto consume_tile = [&](uint32_t tile, bool first, auto full_c) -> bool {
+      constexpr bool FULL = decltype(full_c)::value;
+      const uint32_t g = g0 + tile;
+      const uint32_t s = g % STAGES;
+      if (!mbar_wait(&sm.full[s], (g / STAGES) & 1u, &sm.abort)) return false;
+      const uint32_t v0 = tile * TV + wq * 32 + lane;
+      const uint4* sa = &sm.ring[s][0][wq * 32 + lane];
+      const uint4* sp = &sm.ring[s][1][wq * 32 + lane];
       uint4 va[VPL], vp[VPL];
-      uint32_t okm = 0u;
-      if (v0 + TV <= nvec) {
+      bool in[VPL];
 #pragma unroll
-        for (int j = 0; j < VPL; ++j) { va[j] = sa[j * NC * 32]; vp[j] = sp[j * NC * 32]; }
-        okm = (1u << VPL) - 1u;
-      } else {
-#pragma unroll
-        for (int j = 0; j < VPL; ++j) {
-          const bool in = v0 + j * NC * 32 + cw * 32 + lane < nvec;
-          va[j] = in ? sa[j * NC * 32] : Vec<DT>::neg_inf();
-          vp[j] = in ? sp[j * NC * 32] : Vec<DT>::neg_inf();
-          okm |= in ? (1u << j) : 0u;
-        }
+      for (int j = 0; j < VPL; ++j) {
+        in[j] = FULL || (int64_t)(v0 + j * WPT * 32) < nvec;
+        va[j] = in[j] ? sa[j * WPT * 32] : Vec<DT>::neg_inf();
+        vp[j] = in[j] ? sp[j * WPT * 32] : Vec<DT>::neg_inf();
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(&sm.empty[s]);       // the vectors are in registers: stage free
@@ -460,11 +643,10 @@ __device__ void consumer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_row
 #pragma unroll
       for (int j = 0; j < VPL; ++j) { vm_a[j] = Vec<DT>::vmax(va[j]); vm_p[j] = Vec<DT>::vmax(vp[j]); }
 
-      float tval_a, tval_p;
-      if (TOPK && tile == 0) {
+      if (TOPK && first) {
         // No threshold yet.  With r = ceil(k / warps), the smallest over the warps of
-        // each warp's r-th largest per-lane maximum has at least k row entries at or
-        // above it, so it bounds the k-th best logit of the row from below.
+        // each warp's r-th largest per-lane maximum (over its first tile) has at least k
+        // row entries at or above it, so it bounds the k-th best logit of the row from below.
         float tm_a = vm_a[0], tm_p = vm_p[0];
 #pragma unroll
         for (int j = 1; j < VPL; ++j) { tm_a = fmaxf(tm_a, vm_a[j]); tm_p = fmaxf(tm_p, vm_p[j]); }
@@ -480,32 +662,39 @@ __device__ void consumer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_row
         accumulate<DT>(vp[j], vm_p[j], op);
       }
       if (TOPK) {
-        if (tile == 0) {
-          if (!mbar_wait(&sm.bound_ready[p], ph, &sm.abort)) { raise_timeout(sm, A.sc); return; }
+        float tval_a, tval_p;
+        if (first) {
+          if (!mbar_wait(&sm.bound_ready[p], ph, &sm.abort)) return false;
           tau0_a = sm.warp_bound[p][0][0]; tau0_p = sm.warp_bound[p][1][0];
 #pragma unroll
           for (int w = 1; w < NC; ++w) {
             tau0_a = fminf(tau0_a, sm.warp_bound[p][0][w]);
             tau0_p = fminf(tau0_p, sm.warp_bound[p][1][w]);
           }
-          tval_a = tau0_a; tval_p = tau0_p;
-        } else {
-          tval_a = fmaxf(tau0_a, lds_volatile_f32(&sm.tau[p][0]));
-          tval_p = fmaxf(tau0_p, lds_volatile_f32(&sm.tau[p][1]));
         }
+        tval_a = fmaxf(tau0_a, lds_volatile_f32(&sm.tau[p][0]));
+        tval_p = fmaxf(tau0_p, lds_volatile_f32(&sm.tau[p][1]));
 #pragma unroll
         for (int j = 0; j < VPL; ++j) {
-          const uint32_t vi = (uint32_t)(v0 + j * NC * 32 + cw * 32 + lane);
-          if (((okm >> j) & 1u) && vm_a[j] >= tval_a) {
-            const int pos = atomicAdd(&sm.qcnt[p][0], 1);
-            if (pos < QCAP) sm.queue[p][0][pos] = vi;
-          }
-          if (((okm >> j) & 1u) && vm_p[j] >= tval_p) {
-            const int pos = atomicAdd(&sm.qcnt[p][1], 1);
-            if (pos < QCAP) sm.queue[p][1][pos] = vi;
-          }
+          const uint32_t vi = v0 + j * WPT * 32;
+          if (in[j] && vm_a[j] >= tval_a) push_candidate(sm, p, 0, va[j], vi);
+          if (in[j] && vm_p[j] >= tval_p) push_candidate(sm, p, 1, vp[j], vi);
         }
       }
+      return true;
+    };
+    bool first = true;
+    for (uint32_t tile = gq; tile < ntiles; tile += NG) {
+      const bool ok = ((int64_t)(tile + 1) * TV <= nvec) ? consume_tile(tile, first, std::true_type{})
+                                                         : consume_tile(tile, first, std::false_type{});
+      if (!ok) { raise_timeout(sm, A.sc); return; }
+      first = false;
+    }
+    if (TOPK && first) {
+      // a short row gave this warp no tile: it still takes part in the bound exchange
+      if (lane == 0) { sm.warp_bound[p][0][cw] = JP_NEG_INF; sm.warp_bound[p][1][cw] = JP_NEG_INF; }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sm.bound_ready[p]);
     }
 
     if (tail > 0 && cw == 0 && lane == 0) {     // ragged end of the row: scalar loads
@@ -551,82 +740,97 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
   const int tail = (int)(A.V - nvec * N);
   const int k = A.k;
   unsigned long long* stg = sm.skeys[p][t];
+  uint32_t* hist = sm.hist[p][t];
   int lr = p;
   for (int64_t it = (int64_t)blockIdx.x + (int64_t)p * gridDim.x; it < n_rows; it += 2ll * gridDim.x, lr += 2) {
     const uint32_t ph = (uint32_t)((lr >> 1) & 1);
     const int64_t row = A.list[it];
     const int64_t rrow = A.record_offset + row;
     const char* rmine = (const char*)(t == 0 ? A.za : A.zp) + row * A.ld * Vec<DT>::ESIZE;
-    const char* ra = (const char*)A.za + row * A.ld * Vec<DT>::ESIZE;
-    const char* rp = (const char*)A.zp + row * A.ld * Vec<DT>::ESIZE;
     unsigned long long L[KL];
 #pragma unroll
     for (int j = 0; j < KL; ++j) L[j] = 0ull;
-    unsigned long long tau_key = 0ull;
+    Tau tau{0u, 0, 0ull};
+    uint32_t base = 0u;
     int staged = 0, head = 0;
-    bool overflow = false;
-    int n_seen = 0;
-    const long long t0 = clock64();
+
+    if (TOPK) {
+      for (int i = lane; i < NB; i += 32) hist[i] = 0u;
+      // the consumers' first bound on the k-th best logit starts the histogram
+      if (!mbar_wait(&sm.bound_ready[p], ph, &sm.abort)) { raise_timeout(sm, A.sc); return; }
+      float tau0 = sm.warp_bound[p][t][0];
+#pragma unroll
+      for (int w = 1; w < NC; ++w) tau0 = fminf(tau0, sm.warp_bound[p][t][w]);
+      base = order_code(tau0);
+      tau.code = base;
+      __syncwarp();
+    }
+
+    long long t0 = 0;
+    uint32_t idle = 0;
     for (;;) {
-      // probe the end of the row first: if the consumers are done, the count read
+      // probe the end of the row first: if the consumers are done, the tail read
       // after it is final
       int done = 0;
       if (lane == 0) done = mbar_try_wait(&sm.row_done[p], ph) ? 1 : 0;
       done = __shfl_sync(0xffffffffu, done, 0);
       if (TOPK) {
-        int n = (int)lds_volatile_u32(&sm.qcnt[p][t]);
-        if (n > QCAP) { overflow = true; n = QCAP; }
-        n_seen = n;
-        if (head < n && !overflow) {
-          const int nb = n - head < 32 ? n - head : 32;
+        const int tailv = (int)lds_volatile_u32(&sm.qtail[p][t]);
+        int avail = tailv - head;
+        if (avail > 32) avail = 32;
+        if (avail > 0) {
+          const int slot = (head + lane) & (QCAP - 1);
           uint32_t vi = QEMPTY;
-          if (lane < nb) {
-            int spins = 0;
-            do { vi = lds_volatile_u32(&sm.queue[p][t][head + lane]); } while (vi == QEMPTY && ++spins < (1 << 22));
-          }
-          if (__any_sync(0xffffffffu, lane < nb && vi == QEMPTY)) { raise_timeout(sm, A.sc); return; }
-          uint4 v = Vec<DT>::neg_inf();
-          if (lane < nb) v = ldg_stream((const uint4*)rmine + vi);
-          staged = filter_vector<DT>(v, vi, lane < nb, A.V, tau_key, stg, staged, lane);
-          if (staged > 0) {
-            const unsigned long long nt = drain_staged<KL>(L, stg, staged, k, lane);
-            if (nt != tau_key) {
-              tau_key = nt;
-              if (lane == 0 && nt != 0ull) sts_volatile_f32(&sm.tau[p][t], key_value(nt));
+          if (lane < avail) vi = lds_volatile_u32(&sm.qidx[p][t][slot]);
+          const uint32_t ready = __ballot_sync(0xffffffffu, vi != QEMPTY);
+          const int n = ready == 0xffffffffu ? 32 : __ffs(~ready) - 1;     // written entries, in order
+          if (n > 0) {
+            __threadfence_block();
+            uint4 v = Vec<DT>::neg_inf();
+            if (lane < n) {
+              v = sm.qdata[p][t][slot];
+              sm.qidx[p][t][slot] = QEMPTY;
             }
+            __syncwarp();
+            __threadfence_block();
+            head += n;
+            if (lane == 0) asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(smem_u32(&sm.qhead[p][t])), "r"(head) : "memory");
+            staged = filter_vector<DT>(v, vi, lane < n, A.V, tau, base, hist, stg, staged, lane);
+            if (advance_tau(tau, base, hist, k) && lane == 0)
+              sts_volatile_f32(&sm.tau[p][t], code_value(tau.code));
+            if (staged > SCAP - 32 * N) {
+              // the buffer is filling up: drop what tau has ruled out; if ties keep it
+              // full, sort it into the list and go on with the exact k-th key
+              staged = compact_keys(stg, staged, tau, lane);
+              if (staged > SCAP / 2) tau.key = merge_all<KL>(L, stg, staged, k, lane);
+            }
+            continue;
           }
-          head += nb;
-          continue;
         }
+        if (done && tailv == head) break;
+      } else if (done) {
+        break;
       }
-      if (done) break;
-      if (*(volatile int*)&sm.abort) return;
-      if (clock64() - t0 > kSpinLimit) { raise_timeout(sm, A.sc); return; }
-      __nanosleep(100);
+      if ((idle++ & 63u) == 0u) {
+        if (*(volatile int*)&sm.abort) return;
+        const long long now = clock64();
+        if (idle == 1u) t0 = now;
+        else if (now - t0 > kSpinLimit) { raise_timeout(sm, A.sc); return; }
+      }
+      __nanosleep(JP_TOPK_SLEEP_NS);
     }
 
     if (TOPK) {
-      if (overflow) {
-        // The queue could not hold the row's candidates (an ascending ramp, a row of
-        // equal logits): start over and scan the whole row from memory.
-#pragma unroll
-        for (int j = 0; j < KL; ++j) L[j] = 0ull;
-        tau_key = 0ull;
-        staged = 0;
-        for (int64_t b = 0; b < nvec; b += 32) {
-          const int64_t vi = b + lane;
-          uint4 v = Vec<DT>::neg_inf();
-          if (vi < nvec) v = ldg_stream((const uint4*)rmine + vi);
-          staged = filter_vector<DT>(v, (uint32_t)vi, vi < nvec, A.V, tau_key, stg, staged, lane);
-          if (staged > 0) tau_key = drain_staged<KL>(L, stg, staged, k, lane);
-        }
-      }
+      const char* ra = (const char*)A.za + row * A.ld * Vec<DT>::ESIZE;
+      const char* rp = (const char*)A.zp + row * A.ld * Vec<DT>::ESIZE;
       if (tail > 0) {
         uint4 v = Vec<DT>::neg_inf();
         if (lane == 0) v = load_tail_vector<DT>(rmine, nvec * N, tail);
-        staged = filter_vector<DT>(v, (uint32_t)nvec, lane == 0, A.V, tau_key, stg, staged, lane);
-        if (staged > 0) tau_key = drain_staged<KL>(L, stg, staged, k, lane);
+        staged = filter_vector<DT>(v, (uint32_t)nvec, lane == 0, A.V, tau, base, hist, stg, staged, lane);
+        advance_tau(tau, base, hist, k);
       }
+      staged = compact_keys(stg, staged, tau, lane);
+      merge_all<KL>(L, stg, staged, k, lane);
       // the record: this tensor's list, best first, every entry with both logits
 #pragma unroll
       for (int j = 0; j < KL; ++j) {
@@ -644,9 +848,11 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
           }
         }
       }
-      // hand the slot back clean
-      for (int i = lane; i < n_seen; i += 32) sm.queue[p][t][i] = QEMPTY;
-      if (lane == 0) { sm.qcnt[p][t] = 0; sts_volatile_f32(&sm.tau[p][t], JP_NEG_INF); }
+      // hand the slot back clean (every ring entry was reset as it was drained)
+      if (lane == 0) {
+        sm.qtail[p][t] = 0; sm.qhead[p][t] = 0;
+        sts_volatile_f32(&sm.tau[p][t], JP_NEG_INF);
+      }
     }
 
     if (lane == 0) {
@@ -680,14 +886,14 @@ __global__ void __launch_bounds__(NTHREADS, 1) stream_kernel(StreamArgs A) {
   StreamSmem& sm = *reinterpret_cast<StreamSmem*>(smem_raw);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-  for (int i = tid; i < 2 * 2 * QCAP; i += NTHREADS) (&sm.queue[0][0][0])[i] = QEMPTY;
+  for (int i = tid; i < 2 * 2 * QCAP; i += NTHREADS) (&sm.qidx[0][0][0])[i] = QEMPTY;
   if (tid == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], NC); }
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], WPT); }
     for (int p = 0; p < 2; ++p) {
       mbar_init(&sm.row_done[p], NC);
       mbar_init(&sm.slot_free[p], 2);
       mbar_init(&sm.bound_ready[p], NC);
-      for (int t = 0; t < 2; ++t) { sm.qcnt[p][t] = 0; sm.tau[p][t] = JP_NEG_INF; }
+      for (int t = 0; t < 2; ++t) { sm.qtail[p][t] = 0; sm.qhead[p][t] = 0; sm.tau[p][t] = JP_NEG_INF; }
     }
     sm.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
