@@ -175,6 +175,16 @@ jp_status jp_batch_finalize(jp_ctx* ctx, const jp_obrs_desc* desc_outputs, float
                             float* out_weight, float* out_logp_actor, float* out_logp_policy,
                             jp_stats* out_stats);
 
+/* Weights with a calibration factor supplied by the caller (Section 4.4.2: kappa
+ * is a batch-wide scalar).  A batch whose rows are spread over several devices
+ * runs the forward on each shard, sums (n_valid, n_accept, n_valid *
+ * z_approx_mean) of the shards' jp_stats over all of them, forms
+ * kappa = (sum n_accept / sum n_valid) / (sum of Z_approx / sum n_valid) and
+ * calls this on every shard: out_weight [rows of the last forward / batch] fp32
+ * gets min(kappa Z_approx max(lambda, p/q), c1) from the context's records
+ * (c1 <= 0: no clip).  JP_ERR_STATE without records. */
+jp_status jp_obrs_apply_kappa(jp_ctx* ctx, double kappa, float c1, float* out_weight);
+
 /* Same forward with every pointer in HOST memory (pinned memory makes the
  * copies asynchronous): the library stages the rows through device buffers it
  * owns, chunk by chunk with copies overlapping compute, writes the outputs back

@@ -6,4 +6,4 @@ The work is done by hand-written sm_100a kernels behind a C ABI
 seeded synthetic workloads.  Importing the package loads nothing; the first
 binding call loads ``libjackpot.so`` and raises if it is missing.
 """
-__all__ = ["binding", "runner", "inputs", "build"]
+__all__ = ["binding", "runner", "inputs", "build", "parallel"]

@@ -22,7 +22,7 @@ JP_MAX_TOPK = 128
 EXPORTS = (
     "jp_create", "jp_destroy", "jp_set_stream", "jp_obrs_workspace_bytes", "jp_reserve",
     "jp_obrs_forward", "jp_obrs_backward", "jp_batch_begin", "jp_batch_chunk", "jp_batch_finalize",
-    "jp_obrs_forward_host", "jp_status_string", "jp_last_error", "jp_launch_count",
+    "jp_obrs_forward_host", "jp_obrs_apply_kappa", "jp_status_string", "jp_last_error", "jp_launch_count",
     "jp_enable_kernel_timing", "jp_stream_kernel_times",
 )
 
@@ -92,6 +92,7 @@ def load():
     lib.jp_obrs_forward_host.argtypes = lib.jp_obrs_forward.argtypes + [i64]
     lib.jp_obrs_backward.argtypes = [vp, ctypes.POINTER(jp_obrs_desc), ctypes.POINTER(jp_obrs_bwd_desc),
                                      vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.jp_obrs_apply_kappa.argtypes = [vp, ctypes.c_double, f32, vp]
     lib.jp_batch_begin.argtypes = [vp, i64, i64, i32, ctypes.c_int, f32]
     lib.jp_batch_chunk.argtypes = [vp, ctypes.POINTER(jp_obrs_desc), vp, vp, vp, vp]
     lib.jp_batch_finalize.argtypes = [vp, ctypes.POINTER(jp_obrs_desc), f32, i32, u64, vp, vp, vp, vp, vp]
@@ -205,6 +206,10 @@ def jp_obrs_backward(ctx: Context, desc: jp_obrs_desc, bwd: jp_obrs_bwd_desc, ac
     ctx.check(ctx.lib.jp_obrs_backward(ctx.h, ctypes.byref(desc), ctypes.byref(bwd), _ptr(actor_logits),
                                        _ptr(policy_logits), _ptr(tokens), _ptr(mask), _ptr(accept),
                                        _ptr(weight), _ptr(d_actor_logits), _ptr(d_policy_logits)))
+
+
+def jp_obrs_apply_kappa(ctx: Context, kappa: float, c1: float, out_weight):
+    ctx.check(ctx.lib.jp_obrs_apply_kappa(ctx.h, kappa, c1, _ptr(out_weight)))
 
 
 def jp_batch_begin(ctx: Context, T_total: int, V: int, dtype: int, k: int, fixed_lambda_for_exact_mode=0.0):

@@ -427,6 +427,18 @@ jp_status jp_batch_finalize(jp_ctx* c, const jp_obrs_desc* dout, float lambda_or
   return JP_OK;
 }
 
+jp_status jp_obrs_apply_kappa(jp_ctx* c, double kappa, float c1, float* out_weight) {
+  if (!c) return JP_ERR_INVALID_ARG;
+  if (!c->have_records) return fail(c, JP_ERR_STATE, "no forward records in this context: run the forward (or finalize the batch) first");
+  if (!(kappa >= 0.0) || !(kappa < 1e300)) return fail(c, JP_ERR_INVALID_ARG, "kappa must be finite and >= 0");
+  if (!out_weight && c->rec_rows > 0) return fail(c, JP_ERR_INVALID_ARG, "out_weight is NULL");
+  cudaSetDevice(c->device);
+  cudaError_t e = launch_reweight(c->rec_rows, c->rec, c->sc, kappa, c1, out_weight, c->stream);
+  if (e != cudaSuccess) return cuda_fail(c, e, "reweight launch");
+  if (c->rec_rows > 0) c->launches += 1;
+  return JP_OK;
+}
+
 jp_status jp_obrs_backward(jp_ctx* c, const jp_obrs_desc* d, const jp_obrs_bwd_desc* b,
                            const void* za, const void* zp, const int32_t* tokens,
                            const uint8_t* mask, const uint8_t* accept, const float* weight,

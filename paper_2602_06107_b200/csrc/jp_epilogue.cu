@@ -267,6 +267,31 @@ __global__ void __launch_bounds__(EPI_NT) finalize_kernel(EpilogueArgs A) {
   if (A.out_weight) A.out_weight[r] = w;
 }
 
+// The weights again, with a calibration factor the caller supplies: a batch that
+// is spread over several devices sums (N, accepted, sum of Z_approx) over all of
+// them (Section 4.4.2: kappa is batch-wide) and hands the resulting kappa back.
+__global__ void __launch_bounds__(EPI_NT) reweight_kernel(int64_t T, Records rec, const Scalars* sc, double kappa,
+                                                          float c1, float* out_weight) {
+  const int64_t r = (int64_t)blockIdx.x * EPI_NT + threadIdx.x;
+  if (r >= T) return;
+  const float lambda = sc->lambda;
+  float w = 0.f;
+  if (rec.flag[r]) {
+    float d = rec.lp[r] - rec.lq[r];
+    double wt = kappa * (double)rec.zk[r] * fmax((double)lambda, exp((double)d));
+    if (c1 > 0.f) wt = fmin(wt, (double)c1);
+    w = (float)wt;
+  }
+  out_weight[r] = w;
+}
+
+cudaError_t launch_reweight(int64_t T, const Records& rec, const Scalars* sc, double kappa, float c1,
+                            float* out_weight, cudaStream_t s) {
+  if (T <= 0) return cudaSuccess;
+  reweight_kernel<<<(unsigned)((T + EPI_NT - 1) / EPI_NT), EPI_NT, 0, s>>>(T, rec, sc, kappa, c1, out_weight);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_reset(Scalars* sc, float lambda_fixed, cudaStream_t s) {
   reset_kernel<<<1, 1, 0, s>>>(sc, lambda_fixed);
   return cudaGetLastError();

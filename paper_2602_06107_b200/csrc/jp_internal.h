@@ -118,6 +118,8 @@ cudaError_t launch_reset(Scalars* sc, float lambda_fixed, cudaStream_t s);
 cudaError_t launch_clear_flags(uint8_t* flag, int64_t n, cudaStream_t s);
 cudaError_t launch_budget_solve(const EpilogueArgs& a, double budget, cudaStream_t s, int* n_launch);
 cudaError_t launch_epilogue(const EpilogueArgs& a, cudaStream_t s, int* n_launch);
+cudaError_t launch_reweight(int64_t T, const Records& rec, const Scalars* sc, double kappa, float c1,
+                            float* out_weight, cudaStream_t s);
 cudaError_t launch_grad(const GradArgs& a, cudaStream_t s, int sms);
 
 }  // namespace jp

@@ -1,0 +1,55 @@
+"""Rows over several GPUs: one process per GPU, `torch.distributed` for the plumbing.
+
+Token rows are independent (rejection is per token), so a batch shards over
+ranks by contiguous row ranges and every rank streams its own rows.  The
+accept draw of a row is keyed on its global index (desc.token_offset), so the
+decisions do not depend on how the batch was split.  The one batch-wide
+quantity is the calibration factor kappa (Section 4.4.2): 24 bytes per rank,
+summed with one all-reduce, after which every rank rewrites its weights with
+jp_obrs_apply_kappa.  Nothing here does arithmetic on per-token data.
+"""
+from __future__ import annotations
+
+import torch
+import torch.distributed as dist
+
+
+def shard_rows(T: int, world: int, rank: int):
+    """Contiguous, balanced row range [lo, hi) of rank `rank` (the first T % world ranks get one row more)."""
+    if world < 1 or not (0 <= rank < world) or T < 0:
+        raise ValueError("need world >= 1, 0 <= rank < world, T >= 0")
+    q, r = divmod(T, world)
+    lo = rank * q + min(rank, r)
+    return lo, lo + q + (1 if rank < r else 0)
+
+
+def batch_totals(stats: dict) -> torch.Tensor:
+    """The three sums kappa is made of, from one shard's jp_stats (float64; counts below 2^53 are exact)."""
+    n = float(stats["n_valid"])
+    return torch.tensor([n, float(stats["n_accept"]), n * float(stats["z_approx_mean"])], dtype=torch.float64)
+
+
+def kappa_from_totals(tot) -> float:
+    n, acc, szk = (float(x) for x in tot)
+    if n <= 0 or szk <= 0:
+        return 1.0
+    return (acc / n) / (szk / n)
+
+
+def global_kappa(stats: dict, group=None, device=None) -> tuple[float, torch.Tensor]:
+    """All-reduces the shard totals; returns (kappa of the whole batch, the summed totals)."""
+    tot = batch_totals(stats)
+    if device is not None:
+        tot = tot.to(device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
+        dist.all_reduce(tot, op=dist.ReduceOp.SUM, group=group)
+    tot = tot.cpu()
+    return kappa_from_totals(tot), tot
+
+
+def max_over_ranks(value: float, group=None, device=None) -> float:
+    """A timing is the slowest rank's."""
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX, group=group)
+    return float(t.item())

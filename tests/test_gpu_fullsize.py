@@ -1,0 +1,152 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times.
+
+The oracle cannot run the whole [4096, 151936] batch in test time, so it runs
+on sampled blocks of rows (per-row quantities are independent of the rest of
+the batch) and on properties that hold at any size: kappa * mean(Z_approx) ==
+alpha_hat, every weight equals kappa * Z_approx * max(lambda, p/q), the accept
+count equals the sum of the accept bits.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2602_06107_b200 import binding as B
+from paper_2602_06107_b200 import build as jp_build
+from paper_2602_06107_b200 import runner
+from paper_2602_06107_b200.inputs import CONFIGS, LogitRecipe, make_lengths_mask, make_logits, to_numpy_bits
+
+pytestmark = pytest.mark.gpu
+RTOL, ATOL = 1e-5, 1e-6
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    jp_build.build()
+    c = B.Context(0)
+    yield c
+    c.close()
+
+
+def close(a, b, rtol=RTOL, atol=ATOL):
+    a = np.asarray(a, np.float64)
+    b = np.asarray(b, np.float64)
+    bad = np.abs(a - b) > atol + rtol * np.abs(b)
+    assert not bad.any(), f"{bad.sum()} of {bad.size} differ; worst {np.abs(a - b).max():.3e}"
+
+
+def check_blocks(out, za, zp, tok, mask, lam, k, seed, blocks, block_rows=8):
+    """Oracle on blocks of consecutive rows; the accept draw of row t is keyed on
+    its global index, which the oracle gets through token_offset."""
+    flips = 0
+    for b0 in blocks:
+        sl = slice(b0, b0 + block_rows)
+        m = None if mask is None else mask[sl].cpu().numpy()
+        ref = oracle.forward(to_numpy_bits(za[sl]), to_numpy_bits(zp[sl]), tok[sl].cpu().numpy(), m, lam=lam, k=k,
+                             seed=seed, token_offset=b0)
+        valid = np.ones(block_rows, bool) if m is None else m != 0
+        g = {n: out[n][sl].cpu().numpy() for n in ("logp_actor", "logp_policy", "lse_actor", "lse_policy",
+                                                   "accept_prob", "uniform", "z_approx", "accept", "weight",
+                                                   "topk_idx_actor", "topk_idx_policy")}
+        close(g["logp_actor"], ref["lq64"])
+        close(g["logp_policy"], ref["lp64"])
+        close(g["lse_actor"][valid], ref["lse_a"][valid])
+        close(g["lse_policy"][valid], ref["lse_p"][valid])
+        assert np.array_equal(g["topk_idx_actor"][valid], ref["topk_idx_a"][valid])
+        assert np.array_equal(g["topk_idx_policy"][valid], ref["topk_idx_p"][valid])
+        assert np.array_equal(g["uniform"], ref["u"])
+        close(g["accept_prob"], ref["a"])
+        close(g["z_approx"], ref["zk"])
+        diff = g["accept"] != ref["accept"]
+        near = np.abs(ref["u"].astype(np.float64) - ref["a"].astype(np.float64)) < 1e-6
+        assert not (diff & ~near).any()
+        flips += int(diff.sum())
+        # weight = kappa * Z_approx * max(lambda, p/q) with the batch's kappa
+        d = (ref["lp"] - ref["lq"]).astype(np.float64)
+        w_ref = out["stats"]["kappa"] * ref["zk"] * np.maximum(lam, np.exp(d))
+        close(g["weight"][valid], w_ref[valid])
+    return flips
+
+
+def batch_properties(out, mask):
+    st = out["stats"]
+    acc = out["accept"].cpu().numpy()
+    zk = out["z_approx"].cpu().numpy().astype(np.float64)
+    valid = np.ones(acc.shape[0], bool) if mask is None else mask.cpu().numpy() != 0
+    assert st["status"] == 0 and st["n_nonfinite"] == 0
+    assert st["n_valid"] == int(valid.sum())
+    assert st["n_accept"] == int(acc.sum()) and not acc[~valid].any()
+    close(st["z_approx_mean"], zk[valid].mean(), rtol=1e-6)
+    close(st["kappa"] * st["z_approx_mean"], st["alpha_hat"], rtol=1e-12)
+    a = out["accept_prob"].cpu().numpy()
+    assert np.all((a >= 0) & (a <= 1))
+    assert np.all(out["weight"].cpu().numpy()[~valid] == 0)
+
+
+def test_qwen3_shape_full_batch(ctx):
+    cfg = CONFIGS["cfg2_qwen3"]
+    za, zp, tok = make_logits(cfg["recipe"], "cuda")
+    T = za.shape[0]
+    out = runner.forward(ctx, za, zp, tok, None, lam=cfg["lam"], k=cfg["k"], seed=cfg["seed"])
+    batch_properties(out, None)
+    blocks = list(range(0, T, 296))[:14] + [T - 8]           # rows of every part of the grid's row walk, and the tail
+    flips = check_blocks(out, za, zp, tok, None, cfg["lam"], cfg["k"], cfg["seed"], blocks)
+    print("near-threshold accept flips in the sample:", flips)
+    # the same call twice gives the same bits
+    out2 = runner.forward(ctx, za, zp, tok, None, lam=cfg["lam"], k=cfg["k"], seed=cfg["seed"])
+    for n in ("accept", "weight", "logp_actor", "logp_policy", "z_approx", "topk_idx_policy"):
+        assert torch.equal(out[n], out2[n]), n
+
+
+def test_padded_batch_chunked_with_budget(ctx):
+    """The padded-batch shape at a quarter of its rows: responses of random length
+    padded to 2048, streamed in chunks, lambda from a budget of 0.6, k = 64."""
+    cfg = CONFIGS["cfg3_batch"]
+    r0 = cfg["recipe"]
+    n_resp, max_len, chunk = 4, 2048, 2048
+    T = n_resp * max_len
+    r = LogitRecipe(T=T, V=r0.V, dtype=r0.dtype, sigma0=r0.sigma0, peaks=r0.peaks, peak_lo=r0.peak_lo,
+                    peak_hi=r0.peak_hi, sigma=r0.sigma, seed=r0.seed)
+    za, zp, tok = make_logits(r, "cuda")
+    mask, lengths = make_lengths_mask(n_resp, max_len, cfg["min_len"], seed=cfg["seed"], device="cuda")
+    chunks = [(o, za[o:o + chunk], zp[o:o + chunk], tok[o:o + chunk], mask[o:o + chunk]) for o in range(0, T, chunk)]
+    out = runner.forward_chunked(ctx, chunks, T, r.V, B.JP_BF16, budget=cfg["budget"], k=cfg["k"], seed=cfg["seed"],
+                                 aux=True)
+    batch_properties(out, mask)
+    st = out["stats"]
+    assert abs(st["mean_accept_prob"] - cfg["budget"]) < 5e-6
+    # lambda against the oracle's exact solve on the library's own log-probs (fp32 inputs of the solve)
+    lam_ref = oracle.lambda_from_budget(out["logp_actor"].cpu().numpy(), out["logp_policy"].cpu().numpy(),
+                                        cfg["budget"], mask.cpu().numpy())
+    close(st["lambda_used"], np.float32(lam_ref))
+    # realised acceptance within 4 sigma of the budget
+    n = st["n_valid"]
+    assert abs(st["alpha_hat"] - cfg["budget"]) < 4 * np.sqrt(0.25 / n)
+    lam = float(np.float32(st["lambda_used"]))
+    starts = [int(i * max_len) for i in range(n_resp)]
+    ends = [min(int(i * max_len + lengths[i].item()) - 4, T - 8) for i in range(n_resp)]   # straddle each response's end
+    blocks = starts + ends
+    check_blocks(out, za, zp, tok, mask, lam, cfg["k"], cfg["seed"], blocks)
+
+
+@pytest.mark.parametrize("k", [8, 128])
+def test_sweep_shape_top_k_against_exact(ctx, k):
+    """One point of the exact-vs-estimate sweep: Z_approx <= Z, and exact mode
+    (k >= V) returns the full-vocabulary sum."""
+    cfg = CONFIGS["cfg4_sweep"]
+    r0 = cfg["recipe"]
+    r = LogitRecipe(T=1024, V=r0.V, dtype=r0.dtype, sigma0=r0.sigma0, peaks=r0.peaks, peak_lo=r0.peak_lo,
+                    peak_hi=r0.peak_hi, sigma=1.0, seed=r0.seed)
+    za, zp, tok = make_logits(r, "cuda")
+    out = runner.forward(ctx, za, zp, tok, None, lam=cfg["lam"], k=k, seed=cfg["seed"], want_exact=True)
+    ex = runner.forward(ctx, za, zp, tok, None, lam=cfg["lam"], k=r.V, seed=cfg["seed"])
+    zk, zx = out["z_approx"].cpu().numpy(), out["z_exact"].cpu().numpy()
+    assert np.all(zk <= zx * (1 + 1e-5) + 1e-6)
+    close(ex["z_approx"].cpu().numpy(), zx)
+    assert np.all(zx <= min(1.0, 1.0 / cfg["lam"]) * (1 + 1e-5))
+    sl = slice(500, 508)
+    ref = oracle.forward(to_numpy_bits(za[sl]), to_numpy_bits(zp[sl]), tok[sl].cpu().numpy(), None, lam=cfg["lam"],
+                         k=k, seed=cfg["seed"], token_offset=500, exact=True)
+    close(zx[sl], ref["z_exact"])
+    close(zk[sl], ref["zk"])
+    assert np.array_equal(out["topk_idx_actor"][sl].cpu().numpy(), ref["topk_idx_a"])

@@ -264,3 +264,37 @@ def test_argument_errors_are_reported_not_trapped(ctx):
     # the context is still usable
     out = runner.forward(ctx, za, zp, tok, None, lam=1.0, k=4)
     assert out["stats"]["n_valid"] == 4
+
+
+def test_row_shards_with_a_batch_wide_kappa_match_the_undivided_batch(ctx):
+    """Two shards of one batch (as two ranks would hold them): decisions are keyed on
+    the global row index, and the weights rewritten with the all-shard kappa equal
+    those of one call over the whole batch."""
+    from paper_2602_06107_b200 import parallel
+    T, V, k = 300, 6000, 12
+    r = LogitRecipe(T=T, V=V, dtype="bf16", sigma0=2.5, peaks=4, sigma=1.2, seed=61)
+    za, zp, tok = make_logits(r, "cuda")
+    mask = (torch.arange(T, device="cuda") % 4 != 1).to(torch.uint8)
+    whole = runner.forward(ctx, za, zp, tok, mask, lam=1.4, k=k, seed=3, c1=2.5)
+    ctxs = [B.Context(0), B.Context(0)]
+    outs, tot = [], torch.zeros(3, dtype=torch.float64)
+    for rank, c in enumerate(ctxs):
+        lo, hi = parallel.shard_rows(T, 2, rank)
+        o = runner.forward(c, za[lo:hi], zp[lo:hi], tok[lo:hi], mask[lo:hi], lam=1.4, k=k, seed=3, c1=2.5,
+                           token_offset=lo)
+        outs.append(o)
+        tot += parallel.batch_totals(o["stats"])
+    kappa = parallel.kappa_from_totals(tot)
+    close(kappa, whole["stats"]["kappa"], rtol=1e-12)
+    for c, o in zip(ctxs, outs):
+        B.jp_obrs_apply_kappa(c, kappa, 2.5, o["weight"])
+    torch.cuda.synchronize()
+    assert torch.equal(torch.cat([o["accept"] for o in outs]), whole["accept"])
+    w = torch.cat([o["weight"] for o in outs])
+    assert torch.equal(w, whole["weight"])
+    for c in ctxs:
+        c.close()
+    fresh = B.Context(0)
+    with pytest.raises(B.JackpotError, match="sequence"):
+        B.jp_obrs_apply_kappa(fresh, 1.0, 0.0, w)
+    fresh.close()

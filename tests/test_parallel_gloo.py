@@ -1,0 +1,87 @@
+"""The multi-rank path on CPU: two gloo ranks each take a contiguous share of a
+batch's rows, run the oracle on their share (standing in for the GPU forward of
+that shard), all-reduce the three batch totals and form the batch-wide kappa.
+It must equal the kappa of the undivided batch, and the accept decisions must
+not depend on the split (they are keyed on the global row index)."""
+import os
+import socket
+
+import numpy as np
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+import oracle
+from paper_2602_06107_b200 import parallel
+from paper_2602_06107_b200.inputs import LogitRecipe, make_logits, to_numpy_bits
+
+
+def test_shard_rows_partitions_exactly():
+    for T in (0, 1, 7, 4096, 131072 + 3):
+        for world in (1, 2, 3, 8):
+            spans = [parallel.shard_rows(T, world, r) for r in range(world)]
+            assert spans[0][0] == 0 and spans[-1][1] == T
+            assert all(a[1] == b[0] for a, b in zip(spans, spans[1:]))
+            sizes = [hi - lo for lo, hi in spans]
+            assert max(sizes) - min(sizes) <= 1
+    with pytest.raises(ValueError):
+        parallel.shard_rows(10, 2, 2)
+
+
+def test_kappa_from_totals_degenerate():
+    assert parallel.kappa_from_totals([0, 0, 0.0]) == 1.0
+    assert parallel.kappa_from_totals([10, 5, 0.0]) == 1.0
+    assert parallel.kappa_from_totals([10, 5, 2.5]) == pytest.approx(2.0)
+
+
+def _free_port():
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    return port
+
+
+def _worker(rank, world, port, T, V, out_q):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        r = LogitRecipe(T=T, V=V, dtype="bf16", sigma0=2.5, peaks=4, sigma=1.2, seed=9)
+        za, zp, tok = make_logits(r, "cpu", block_rows=T)
+        mask = (torch.arange(T) % 5 != 2).to(torch.uint8).numpy()
+        lo, hi = parallel.shard_rows(T, world, rank)
+        ref = oracle.forward(to_numpy_bits(za[lo:hi]), to_numpy_bits(zp[lo:hi]), tok[lo:hi].numpy(), mask[lo:hi],
+                             lam=1.4, k=8, seed=3, token_offset=lo)
+        kappa, tot = parallel.global_kappa(ref["stats"])
+        slow = parallel.max_over_ranks(float(rank + 1))
+        out_q.put((rank, lo, hi, kappa, tot.tolist(), slow, ref["accept"].tolist(), ref["zk"].tolist()))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_ranks_agree_with_the_undivided_batch():
+    T, V, world = 96, 2048, 2
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_worker, args=(r, world, port, T, V, q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    got = sorted(q.get(timeout=180) for _ in range(world))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    r = LogitRecipe(T=T, V=V, dtype="bf16", sigma0=2.5, peaks=4, sigma=1.2, seed=9)
+    za, zp, tok = make_logits(r, "cpu", block_rows=T)
+    mask = (torch.arange(T) % 5 != 2).to(torch.uint8).numpy()
+    whole = oracle.forward(to_numpy_bits(za), to_numpy_bits(zp), tok.numpy(), mask, lam=1.4, k=8, seed=3)
+    assert got[0][3] == got[1][3], "ranks disagree on kappa"
+    assert got[0][3] == pytest.approx(whole["stats"]["kappa"], rel=1e-12)
+    assert got[0][4][0] == whole["stats"]["n_valid"] and got[0][4][1] == whole["stats"]["n_accept"]
+    assert got[0][5] == got[1][5] == 2.0
+    acc = np.concatenate([np.asarray(g[6], np.uint8) for g in got])
+    zk = np.concatenate([np.asarray(g[7]) for g in got])
+    assert np.array_equal(acc, whole["accept"]), "decisions depend on the split"
+    assert np.array_equal(zk, whole["zk"])
