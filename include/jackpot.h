@@ -45,13 +45,15 @@ typedef enum {
   JP_ERR_WORKSPACE = -4,
   JP_ERR_CUDA = -5,
   JP_ERR_TIMEOUT = -6,
-  JP_ERR_STATE = -7
+  JP_ERR_STATE = -7,
+  JP_ERR_TOO_LARGE = -8
 } jp_status;
 
 typedef enum { JP_BF16 = 0, JP_F32 = 1 } jp_dtype;
 typedef enum { JP_LAMBDA_FIXED = 0, JP_LAMBDA_FROM_BUDGET = 1 } jp_lambda_mode;
 
 enum { JP_MAX_TOPK = 128 };
+enum { JP_STATIC_MAX_ROWS = 131072 };   /* row limit of jp_budget_lambda_static */
 
 /* Shapes, dtype, mode and optional outputs of one forward / backward call.
  * Zero-initialise, then set T, V and what differs from the defaults. */
@@ -195,6 +197,46 @@ jp_status jp_obrs_forward_host(jp_ctx* ctx, const jp_obrs_desc* desc, const void
                                const uint8_t* mask, float lambda_or_budget, int k, uint64_t seed,
                                uint8_t* out_accept, float* out_weight, float* out_logp_actor,
                                float* out_logp_policy, jp_stats* out_stats, int64_t chunk_rows);
+
+/* The batch-level lambda for an acceptance budget, for callers that cannot
+ * allocate device memory.  (The paper has no counterpart: this entry point exists
+ * for integration, not for the method.)
+ *
+ * Who this is for: code that runs where cudaMalloc is off limits.  Examples are a
+ * training step whose device memory is entirely owned and budgeted by a framework
+ * allocator, so that a hidden driver allocation could fail or fragment the pool; a
+ * serving plug-in that may allocate only while it initialises; a latency-critical
+ * loop, since cudaMalloc and cudaFree synchronise the device.  Every other entry
+ * point of this library keeps its scratch in a context workspace that it grows
+ * with cudaMalloc; this one calls no cudaMalloc, cudaFree or other allocating
+ * routine.  Its scratch is a fixed array of about 1.7 MB inside the library's
+ * device image, which every GPU that loads the library holds until the process
+ * ends.
+ *
+ *   logp_actor, logp_policy : [T] fp32, DEVICE, log-probabilities of the sampled
+ *                             tokens (outputs of jp_obrs_forward), read only
+ *   mask    : [T] uint8 DEVICE, 0 = row takes no part; NULL = all rows
+ *   T       : 0..JP_STATIC_MAX_ROWS; more rows return JP_ERR_TOO_LARGE and nothing
+ *             is launched
+ *   budget  : target mean acceptance in (0, 1]
+ *   out_lambda : one fp32 in DEVICE memory; receives the lambda with
+ *             (1/N) sum_t min(1, (p/q)(x_t) / lambda) = budget (1 if no row takes part)
+ *   cuda_stream : cudaStream_t as void*, NULL = default stream; the work is
+ *             enqueued on it on the CURRENT device and the call does not wait
+ *
+ * The first call on each device sets up: the driver loads the part of the library
+ * image that holds the array (with lazy module loading this is when the device's
+ * free memory drops by the array's size, once) and the array's device address is
+ * looked up (a driver query).  Make that first call before any stream capture
+ * begins.  Later calls change no allocation.
+ * All calls on a device share the one array, which keeps whatever the previous
+ * call left: each call rewrites what it reads, but two calls whose kernels overlap
+ * on the GPU (different streams, no ordering between them) race on it.  Order
+ * them, or use jp_obrs_forward with JP_LAMBDA_FROM_BUDGET, which has per-context
+ * scratch.  Returns JP_OK, JP_ERR_INVALID_ARG, JP_ERR_TOO_LARGE or JP_ERR_CUDA. */
+jp_status jp_budget_lambda_static(const float* logp_actor, const float* logp_policy,
+                                  const uint8_t* mask, int64_t T, float budget, float* out_lambda,
+                                  void* cuda_stream);
 
 const char* jp_status_string(jp_status s);
 const char* jp_last_error(jp_ctx* ctx);

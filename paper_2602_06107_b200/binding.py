@@ -18,11 +18,13 @@ LIB_PATH = os.path.join(_PKG, "libjackpot.so")
 JP_BF16, JP_F32 = 0, 1
 JP_LAMBDA_FIXED, JP_LAMBDA_FROM_BUDGET = 0, 1
 JP_MAX_TOPK = 128
+JP_STATIC_MAX_ROWS = 131072
+JP_ERR_TOO_LARGE = -8
 
 EXPORTS = (
     "jp_create", "jp_destroy", "jp_set_stream", "jp_obrs_workspace_bytes", "jp_reserve",
     "jp_obrs_forward", "jp_obrs_backward", "jp_batch_begin", "jp_batch_chunk", "jp_batch_finalize",
-    "jp_obrs_forward_host", "jp_obrs_apply_kappa", "jp_status_string", "jp_last_error", "jp_launch_count",
+    "jp_obrs_forward_host", "jp_obrs_apply_kappa", "jp_budget_lambda_static", "jp_status_string", "jp_last_error", "jp_launch_count",
     "jp_enable_kernel_timing", "jp_stream_kernel_times",
 )
 
@@ -93,6 +95,7 @@ def load():
     lib.jp_obrs_backward.argtypes = [vp, ctypes.POINTER(jp_obrs_desc), ctypes.POINTER(jp_obrs_bwd_desc),
                                      vp, vp, vp, vp, vp, vp, vp, vp]
     lib.jp_obrs_apply_kappa.argtypes = [vp, ctypes.c_double, f32, vp]
+    lib.jp_budget_lambda_static.argtypes = [vp, vp, vp, i64, f32, vp, vp]
     lib.jp_batch_begin.argtypes = [vp, i64, i64, i32, ctypes.c_int, f32]
     lib.jp_batch_chunk.argtypes = [vp, ctypes.POINTER(jp_obrs_desc), vp, vp, vp, vp]
     lib.jp_batch_finalize.argtypes = [vp, ctypes.POINTER(jp_obrs_desc), f32, i32, u64, vp, vp, vp, vp, vp]
@@ -210,6 +213,16 @@ def jp_obrs_backward(ctx: Context, desc: jp_obrs_desc, bwd: jp_obrs_bwd_desc, ac
 
 def jp_obrs_apply_kappa(ctx: Context, kappa: float, c1: float, out_weight):
     ctx.check(ctx.lib.jp_obrs_apply_kappa(ctx.h, kappa, c1, _ptr(out_weight)))
+
+
+def jp_budget_lambda_static(logp_actor, logp_policy, mask, T: int, budget: float, out_lambda, stream=None) -> int:
+    """Calls the allocation-free budget solve on the current device and returns its
+    status code (0 = ok) instead of raising, so that callers can test the limits."""
+    lib = load()
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    return int(lib.jp_budget_lambda_static(_ptr(logp_actor), _ptr(logp_policy), _ptr(mask), T, budget,
+                                           _ptr(out_lambda), ctypes.c_void_p(stream)))
 
 
 def jp_batch_begin(ctx: Context, T_total: int, V: int, dtype: int, k: int, fixed_lambda_for_exact_mode=0.0):

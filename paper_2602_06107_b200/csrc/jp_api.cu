@@ -220,6 +220,7 @@ const char* jp_status_string(jp_status s) {
     case JP_ERR_CUDA: return "CUDA error";
     case JP_ERR_TIMEOUT: return "device wait timed out";
     case JP_ERR_STATE: return "call out of sequence";
+    case JP_ERR_TOO_LARGE: return "size beyond the fixed maximum of this entry point";
   }
   return "unknown status";
 }
