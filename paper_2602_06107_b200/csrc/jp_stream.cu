@@ -59,11 +59,15 @@ constexpr int NG = JP_NG;                 // consumer groups: group q takes tile
 constexpr int WPT = NC / NG;              // warps that share one tile
 constexpr int VPL = JP_VPL;               // 16-byte vectors per lane per tensor per tile
 constexpr int TV = WPT * 32 * VPL;        // vectors per tensor per tile
+constexpr int HV = 2;                     // vectors per tensor a lane holds at a time
+static_assert(JP_VPL % HV == 0, "a tile is taken in passes of HV vectors");
+static_assert(NC <= 16, "one top-k warp polls two entries of up to 16 rings");
 static_assert(NC % NG == 0 && NG < JP_STAGES, "consumer groups must divide the warps and fit the ring");
 constexpr int STAGES = JP_STAGES;
-constexpr int QCAP = 256;                 // candidate-vector ring entries per (slot, tensor); power of two
-constexpr int SCAP = 512;                 // buffered keys per top-k warp
-constexpr int NB = 1024;                  // histogram bins (16-bit order codes above the row's first bound)
+constexpr int MQ = 16;                    // candidate-vector ring entries per (slot, tensor, consumer warp); power of two
+constexpr int SCAP = 384;                 // buffered keys per top-k warp (used while sorting survivors into the list)
+constexpr int SVCAP = 192;                // candidate vectors a top-k warp keeps until the row ends
+constexpr int NB = 512;                   // histogram bins (16-bit order codes above the row's first bound)
 constexpr int NTOPK = 4;                  // top-k warps: (tensor, slot)
 constexpr int NWARPS = 1 + NC + NTOPK;
 constexpr int NTHREADS = NWARPS * 32;
@@ -72,14 +76,15 @@ constexpr long long kSpinLimit = 4000000000ll;   // clock cycles a wait may last
 
 struct __align__(128) StreamSmem {
   uint4 ring[STAGES][2][TV];              // [stage][tensor][vector]
-  uint4 qdata[2][2][QCAP];                // [slot][tensor] candidate vectors ...
-  unsigned long long skeys[2][2][SCAP];   // [slot][tensor] keys of entries at or above tau
-  uint32_t qidx[2][2][QCAP];              // ... and their vector index (QEMPTY = not written yet)
-  uint32_t hist[2][2][NB];                // [slot][tensor] entries seen per order code
+  uint4 qdata[2][2][NC][MQ];              // [slot][tensor][consumer warp] candidate vectors ...
+  uint4 svdata[2][2][SVCAP];              // [slot][tensor] candidate vectors still alive under tau ...
+  unsigned long long skeys[2][2][SCAP];   // [slot][tensor] keys waiting to be sorted into the list
+  uint32_t qidx[2][2][NC][MQ];            // ... their vector index (QEMPTY = not written yet)
+  uint32_t svidx[2][2][SVCAP];            // ... and the kept vectors' indices
+  uint32_t hist[2][2][NB];                // [slot][tensor] candidate vectors seen per order code of their maximum
   unsigned long long full[STAGES], empty[STAGES];
   unsigned long long row_done[2], slot_free[2], bound_ready[2];
-  int qtail[2][2];                        // next ring position to reserve (consumers)
-  int qhead[2][2];                        // first position not yet drained (top-k warp)
+  int qhead[2][2][NC];                    // per ring: entries drained so far (top-k warp)
   float tau[2][2];                        // published threshold (a logit value)
   float warp_bound[2][2][NC];
   float part_mL[2][2][NC];
@@ -314,14 +319,26 @@ __device__ __forceinline__ uint4 load_tail_vector(const char* row, int64_t first
   return v;
 }
 
-// r-th largest (1-based) of the 32 lane values; -inf when fewer than r lanes hold a number.
-__device__ __forceinline__ float warp_rth_largest(float v, int r, int lane) {
-  uint32_t ob = f32_order_bits(v);
+// r-th largest (1-based) of the warp's 32 * NV values (NV per lane); -inf when
+// fewer than r of them are numbers above -inf.
+template <int NV>
+__device__ __forceinline__ float warp_rth_largest(const float (&v)[NV], int r, int lane) {
+  uint32_t ob[NV];
+#pragma unroll
+  for (int j = 0; j < NV; ++j) ob[j] = f32_order_bits(v[j]);
   uint32_t mx = 0u;
   for (int i = 0; i < r; ++i) {
-    mx = __reduce_max_sync(0xffffffffu, ob);
-    const uint32_t holders = __ballot_sync(0xffffffffu, ob == mx);
-    if (lane == __ffs(holders) - 1) ob = 0u;     // retire one holder of the maximum
+    uint32_t lm = ob[0];
+#pragma unroll
+    for (int j = 1; j < NV; ++j) lm = lm > ob[j] ? lm : ob[j];
+    mx = __reduce_max_sync(0xffffffffu, lm);
+    const uint32_t holders = __ballot_sync(0xffffffffu, lm == mx);
+    if (lane == __ffs(holders) - 1) {            // retire one copy of the maximum
+      bool gone = false;
+#pragma unroll
+      for (int j = 0; j < NV; ++j)
+        if (!gone && ob[j] == mx) { ob[j] = 0u; gone = true; }
+    }
   }
   return mx <= 0x007fffffu ? JP_NEG_INF : order_bits_f32(mx);
 }
@@ -424,11 +441,12 @@ __device__ __forceinline__ unsigned long long kth_key(const unsigned long long (
   return __shfl_sync(0xffffffffu, v, (k - 1) / KPL);
 }
 
-// The running threshold of one (row, tensor): `code` is the highest 16-bit order
-// code with at least k of the entries seen so far at or above it (so the k-th
-// best logit of the row is at or above the low edge of that code's bin); `cnt`
-// counts the entries seen at or above it.  `key` is the exact k-th best key of
-// the sorted list once a merge has happened (0 before).
+// The running threshold of one (row, tensor).  `code` is the highest 16-bit order
+// code with at least k of the candidate vectors seen so far having their maximum
+// at or above it: k different vectors hold k different entries, so the k-th best
+// logit of the row is at or above the low edge of that code's bin.  `cnt` counts
+// the vectors at or above it.  `key` is the exact k-th best key of the sorted
+// list once candidates have been sorted into it (0 before).
 struct Tau {
   uint32_t code;
   int cnt;
@@ -439,53 +457,15 @@ __device__ __forceinline__ uint32_t order_code(float v) { return f32_order_bits(
 // low edge of a code's bin, as a logit
 __device__ __forceinline__ float code_value(uint32_t code) { return order_bits_f32(code << 16); }
 
-// Tests the entries of one vector per lane against tau; every entry at or above
-// it is counted in the histogram and its key appended to the buffer.  Returns
-// the new number of buffered keys.
-template <int DT>
-__device__ __forceinline__ int filter_vector(const uint4& v, uint32_t vi, bool have, int64_t V, Tau& tau,
-                                             uint32_t base, uint32_t* hist, unsigned long long* stg,
-                                             int staged, int lane) {
-  constexpr int N = Vec<DT>::N;
-  unsigned long long key[N];
-  uint32_t pass = 0u;
-#pragma unroll
-  for (int e = 0; e < N; ++e) {
-    const uint32_t idx = vi * N + e;
-    key[e] = make_key(Vec<DT>::get(v, e), idx);
-    const uint32_t code = (uint32_t)(key[e] >> 48);
-    if (have && (int64_t)idx < V && code >= tau.code) {
-      const uint32_t bin = code - base < (uint32_t)(NB - 1) ? code - base : (uint32_t)(NB - 1);
-      atomicAdd(&hist[bin], 1u);
-      if (key[e] > tau.key) pass |= 1u << e;
-    }
-  }
-  // entries counted but below the exact key (ties that a merge already ruled out) still
-  // count toward tau.cnt: they are entries of the row at or above the code
-  uint32_t counted = 0u;
-#pragma unroll
-  for (int e = 0; e < N; ++e) {
-    const uint32_t idx = vi * N + e;
-    if (have && (int64_t)idx < V && (uint32_t)(key[e] >> 48) >= tau.code) counted += 1u;
-  }
-  const int c = __popc(pass);
-  int incl = c | ((int)counted << 16);       // two prefix sums in one shuffle chain
-#pragma unroll
-  for (int off = 1; off < 32; off <<= 1) {
-    const int n = __shfl_up_sync(0xffffffffu, incl, off);
-    if (lane >= off) incl += n;
-  }
-  const int total = __shfl_sync(0xffffffffu, incl, 31);
-  int pos = staged + (incl & 0xffff) - c;
-#pragma unroll
-  for (int e = 0; e < N; ++e)
-    if ((pass >> e) & 1u) stg[pos++] = key[e];
-  tau.cnt += total >> 16;
-  __syncwarp();
-  return staged + (total & 0xffff);
+// Can the vector with index vi and maximum order bits `ob` still hold one of the k best?
+__device__ __forceinline__ bool vector_alive(uint32_t ob, uint32_t vi, int n_per_vec, const Tau& tau) {
+  if ((ob >> 16) < tau.code) return false;
+  if (tau.key == 0ull) return true;
+  // its best possible entry: the maximum at the vector's first index
+  return (((unsigned long long)ob << 32) | (unsigned long long)(uint32_t)(~(vi * (uint32_t)n_per_vec))) > tau.key;
 }
 
-// Raises tau.code while at least k counted entries stay at or above it.
+// Raises tau.code while at least k counted vectors stay at or above it.
 __device__ __forceinline__ bool advance_tau(Tau& tau, uint32_t base, const uint32_t* hist, int k) {
   bool moved = false;
   for (;;) {
@@ -500,31 +480,58 @@ __device__ __forceinline__ bool advance_tau(Tau& tau, uint32_t base, const uint3
   return moved;
 }
 
-// Drops buffered keys that can no longer be among the k best.
-__device__ __forceinline__ int compact_keys(unsigned long long* stg, int staged, const Tau& tau, int lane) {
+// Drops the kept candidate vectors that tau has ruled out since they were kept.
+template <int DT>
+__device__ __noinline__ int compact_survivors(uint4* svd, uint32_t* svi, int nsv, Tau tau, int lane) {
   int out = 0;
-  for (int b = 0; b < staged; b += 32) {
+  for (int b = 0; b < nsv; b += 32) {
     const int i = b + lane;
-    unsigned long long key = 0ull;
+    uint4 v = Vec<DT>::neg_inf();
+    uint32_t vi = 0u;
     bool keep = false;
-    if (i < staged) {
-      key = stg[i];
-      keep = (uint32_t)(key >> 48) >= tau.code && key > tau.key;
+    if (i < nsv) {
+      v = svd[i];
+      vi = svi[i];
+      keep = vector_alive(f32_order_bits(Vec<DT>::vmax(v)), vi, Vec<DT>::N, tau);
     }
     const uint32_t m = __ballot_sync(0xffffffffu, keep);
     __syncwarp();
-    if (keep) stg[out + __popc(m & ((1u << lane) - 1u))] = key;
+    if (keep) {
+      const int o = out + __popc(m & ((1u << lane) - 1u));
+      svd[o] = v;
+      svi[o] = vi;
+    }
     out += __popc(m);
     __syncwarp();
   }
   return out;
 }
 
+// Appends to the key buffer the keys of one vector's entries (one vector per lane)
+// that can still be among the k best.  Returns the new number of buffered keys.
+template <int DT>
+__device__ __forceinline__ int stage_entries(const uint4& v, uint32_t vi, bool have, int64_t V, const Tau& tau,
+                                             unsigned long long* stg, int staged, int lane) {
+  constexpr int N = Vec<DT>::N;
+  const uint32_t lt = (1u << lane) - 1u;
+#pragma unroll
+  for (int e = 0; e < N; ++e) {
+    const uint32_t idx = vi * N + e;
+    const uint32_t ob = f32_order_bits(Vec<DT>::get(v, e));
+    const unsigned long long key = ((unsigned long long)ob << 32) | (unsigned long long)(uint32_t)(~idx);
+    const bool keep = have && (int64_t)idx < V && (ob >> 16) >= tau.code && key > tau.key;
+    const uint32_t bk = __ballot_sync(0xffffffffu, keep);
+    if (keep) stg[staged + __popc(bk & lt)] = key;
+    staged += __popc(bk);
+  }
+  __syncwarp();
+  return staged;
+}
+
 // Folds every buffered key into the sorted list; returns the list's k-th key.
 template <int KPL>
-__device__ __forceinline__ unsigned long long merge_all(unsigned long long (&L)[KPL],
-                                                        const unsigned long long* stg, int& staged, int k,
-                                                        int lane) {
+__device__ __noinline__ unsigned long long merge_all(unsigned long long (&L)[KPL], const unsigned long long* stg,
+                                                     int& staged, int k, int lane) {
   constexpr int SORT_MIN = 6 * KPL;       // below this, single inserts are cheaper than a sort + merge
   __syncwarp();
   while (staged >= SORT_MIN) merge_staged<KPL>(L, stg, staged, lane);
@@ -536,24 +543,86 @@ __device__ __forceinline__ unsigned long long merge_all(unsigned long long (&L)[
   return kth_key<KPL>(L, k);
 }
 
+// Sorts the entries of every kept vector into the list (exact from here on:
+// tau.key becomes the list's k-th key) and empties the survivor buffer.
+template <int DT, int KPL>
+__device__ __noinline__ void survivors_to_list(unsigned long long (&L)[KPL], const uint4* svd, const uint32_t* svi,
+                                               int& nsv, int64_t V, Tau& tau, unsigned long long* stg, int k,
+                                               int lane) {
+  int staged = 0;
+  for (int b = 0; b < nsv; b += 32) {
+    const int i = b + lane;
+    uint4 v = Vec<DT>::neg_inf();
+    uint32_t vi = 0u;
+    if (i < nsv) { v = svd[i]; vi = svi[i]; }
+    staged = stage_entries<DT>(v, vi, i < nsv, V, tau, stg, staged, lane);
+    if (staged > SCAP - 32 * Vec<DT>::N) tau.key = merge_all<KPL>(L, stg, staged, k, lane);
+  }
+  tau.key = merge_all<KPL>(L, stg, staged, k, lane);
+  nsv = 0;
+}
+
 __device__ __forceinline__ void raise_timeout(StreamSmem& sm, Scalars* sc) {
   sm.abort = 1;
   atomicExch(&sc->status, (int)JP_ERR_TIMEOUT);
 }
 
-// A consumer lane hands one vector that may hold a top-k entry to the slot's
-// top-k warp: reserve a ring position, wait (bounded) until the ring has room,
-// write the vector, then publish it by writing its index.
-__device__ __forceinline__ void push_candidate(StreamSmem& sm, int p, int t, const uint4& v, uint32_t vi) {
-  const int pos = atomicAdd(&sm.qtail[p][t], 1);
-  int spins = 0;
-  while (pos - (int)lds_volatile_u32(&sm.qhead[p][t]) >= QCAP) {
-    if (++spins > (1 << 24) || *(volatile int*)&sm.abort) { sm.abort = 1; return; }
+// A consumer warp hands the vectors that may hold a top-k entry (`cand` lanes) to
+// the slot's top-k warp through the warp's own small ring: no atomics, the tail
+// lives in a register.  The ring's head (entries the top-k warp has drained) is
+// re-read only when the ring looks full; that wait is bounded.  Each entry is
+// published by writing its index after its data.  Kept out of line: the streaming
+// loop only pays a ballot and a branch for a vector that is no candidate.
+// state.x = entries pushed so far, state.y = last head seen; returns the new state
+// (x < 0: the wait for room ran out).
+__device__ __noinline__ int2 push_candidates(uint4* qdata, uint32_t* qidx, const int* qhead, volatile int* abort,
+                                             uint32_t m, uint4 v, uint32_t vi, int2 state, int lane) {
+  int tail = state.x, head_known = state.y;
+  while (m) {
+    int room = MQ - (tail - head_known);
+    if (room <= 0) {
+      int spins = 0;
+      do {
+        head_known = (int)lds_volatile_u32(qhead);
+        room = MQ - (tail - head_known);
+      } while (room <= 0 && ++spins < (1 << 22) && !*abort);
+      if (room <= 0) { *abort = 1; return make_int2(-1, head_known); }
+    }
+    const int rank = __popc(m & ((1u << lane) - 1u));
+    const bool mine = ((m >> lane) & 1u) && rank < room;
+    if (mine) {
+      const int slot = (tail + rank) & (MQ - 1);
+      qdata[slot] = v;
+      __threadfence_block();
+      asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(smem_u32(&qidx[slot])), "r"(vi) : "memory");
+    }
+    const uint32_t took = __ballot_sync(0xffffffffu, mine);
+    m &= ~took;
+    tail += __popc(took);
   }
-  const int slot = pos & (QCAP - 1);
-  sm.qdata[p][t][slot] = v;
-  __threadfence_block();
-  asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(smem_u32(&sm.qidx[p][t][slot])), "r"(vi) : "memory");
+  return make_int2(tail, head_known);
+}
+
+// First tile of a row, first consumer group: no threshold exists yet.  Every warp
+// of the group takes the r-th largest of its vector maxima over the tile,
+// r = ceil(k / warps in the group); the smallest of these over the group has at
+// least k row entries at or above it (distinct vectors, r per warp), so it bounds
+// the k-th best logit of the row from below.  The vectors are only looked at here;
+// the streaming pass that follows reads them again from the stage.
+template <int DT>
+__device__ __noinline__ void first_tile_bound(const uint4* sa, const uint4* sp, uint32_t v0, int64_t nvec, int r,
+                                              float* bound_a, float* bound_p, int lane) {
+  float vm_a[VPL], vm_p[VPL];
+#pragma unroll
+  for (int j = 0; j < VPL; ++j) {
+    const bool in = (int64_t)(v0 + j * WPT * 32) < nvec;
+    vm_a[j] = in ? Vec<DT>::vmax(sa[j * WPT * 32]) : JP_NEG_INF;
+    vm_p[j] = in ? Vec<DT>::vmax(sp[j * WPT * 32]) : JP_NEG_INF;
+  }
+  const float ba = warp_rth_largest<VPL>(vm_a, r, lane);
+  const float bp = warp_rth_largest<VPL>(vm_p, r, lane);
+  if (lane == 0) { *bound_a = ba; *bound_p = bp; }
+  __syncwarp();
 }
 
 // ---- producer ---------------------------------------------------------------
@@ -603,7 +672,7 @@ __device__ void consumer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_row
   const int64_t nvec = A.V / N;
   const int tail = (int)(A.V - nvec * N);
   const uint32_t ntiles = nvec > 0 ? (uint32_t)((nvec + TV - 1) / TV) : 1u;
-  const int r = (A.k + NC - 1) / NC;
+  const int r = (A.k + WPT - 1) / WPT;
   const int gq = cw / WPT;              // this warp's group: it takes tiles gq, gq + NG, ...
   const int wq = cw % WPT;              // its place among the warps that share a tile
   uint32_t g0 = 0;                      // ring position of the current row's tile 0
@@ -617,84 +686,79 @@ __device__ void consumer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_row
 
     Online oa{JP_NEG_INF, 0.f, 0ull}, op{JP_NEG_INF, 0.f, 0ull};
     float tau0_a = JP_NEG_INF, tau0_p = JP_NEG_INF;
+    int2 q_a = make_int2(0, 0), q_p = make_int2(0, 0);  // this warp's rings: entries pushed, last head seen
 
-    // One tile of both rows.  FULL = every vector of the tile lies inside the row;
-    // first = this warp's first tile of the row.
-    auto consume_tile = [&](uint32_t tile, bool first, auto full_c) -> bool {
-      constexpr bool FULL = decltype(full_c)::value;
+    // One tile of both rows; first = this warp's first tile of the row.  The tile is
+    // taken in passes of HV vectors per tensor: a short loop body keeps the streaming
+    // code small enough for the instruction caches and the live registers few.
+    auto consume_tile = [&](uint32_t tile, bool first) -> bool {
       const uint32_t g = g0 + tile;
       const uint32_t s = g % STAGES;
       if (!mbar_wait(&sm.full[s], (g / STAGES) & 1u, &sm.abort)) return false;
       const uint32_t v0 = tile * TV + wq * 32 + lane;
       const uint4* sa = &sm.ring[s][0][wq * 32 + lane];
       const uint4* sp = &sm.ring[s][1][wq * 32 + lane];
-      uint4 va[VPL], vp[VPL];
-      bool in[VPL];
-#pragma unroll
-      for (int j = 0; j < VPL; ++j) {
-        in[j] = FULL || (int64_t)(v0 + j * WPT * 32) < nvec;
-        va[j] = in[j] ? sa[j * WPT * 32] : Vec<DT>::neg_inf();
-        vp[j] = in[j] ? sp[j * WPT * 32] : Vec<DT>::neg_inf();
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&sm.empty[s]);       // the vectors are in registers: stage free
-
-      float vm_a[VPL], vm_p[VPL];
-#pragma unroll
-      for (int j = 0; j < VPL; ++j) { vm_a[j] = Vec<DT>::vmax(va[j]); vm_p[j] = Vec<DT>::vmax(vp[j]); }
-
-      if (TOPK && first) {
-        // No threshold yet.  With r = ceil(k / warps), the smallest over the warps of
-        // each warp's r-th largest per-lane maximum (over its first tile) has at least k
-        // row entries at or above it, so it bounds the k-th best logit of the row from below.
-        float tm_a = vm_a[0], tm_p = vm_p[0];
-#pragma unroll
-        for (int j = 1; j < VPL; ++j) { tm_a = fmaxf(tm_a, vm_a[j]); tm_p = fmaxf(tm_p, vm_p[j]); }
-        const float ba = warp_rth_largest(tm_a, r, lane);
-        const float bp = warp_rth_largest(tm_p, r, lane);
-        if (lane == 0) { sm.warp_bound[p][0][cw] = ba; sm.warp_bound[p][1][cw] = bp; }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sm.bound_ready[p]);
-      }
-#pragma unroll
-      for (int j = 0; j < VPL; ++j) {
-        accumulate<DT>(va[j], vm_a[j], oa);
-        accumulate<DT>(vp[j], vm_p[j], op);
-      }
+      float tval_a = 0.f, tval_p = 0.f;
       if (TOPK) {
-        float tval_a, tval_p;
         if (first) {
+          if (gq == 0) {
+            first_tile_bound<DT>(sa, sp, v0, nvec, r, &sm.warp_bound[p][0][wq], &sm.warp_bound[p][1][wq], lane);
+            if (lane == 0) mbar_arrive(&sm.bound_ready[p]);
+          }
           if (!mbar_wait(&sm.bound_ready[p], ph, &sm.abort)) return false;
           tau0_a = sm.warp_bound[p][0][0]; tau0_p = sm.warp_bound[p][1][0];
 #pragma unroll
-          for (int w = 1; w < NC; ++w) {
+          for (int w = 1; w < WPT; ++w) {
             tau0_a = fminf(tau0_a, sm.warp_bound[p][0][w]);
             tau0_p = fminf(tau0_p, sm.warp_bound[p][1][w]);
           }
         }
         tval_a = fmaxf(tau0_a, lds_volatile_f32(&sm.tau[p][0]));
         tval_p = fmaxf(tau0_p, lds_volatile_f32(&sm.tau[p][1]));
+      }
+#pragma unroll 1
+      for (int h = 0; h < VPL / HV; ++h) {
+        uint4 va[HV], vp[HV];
+        bool in[HV];
 #pragma unroll
-        for (int j = 0; j < VPL; ++j) {
-          const uint32_t vi = v0 + j * WPT * 32;
-          if (in[j] && vm_a[j] >= tval_a) push_candidate(sm, p, 0, va[j], vi);
-          if (in[j] && vm_p[j] >= tval_p) push_candidate(sm, p, 1, vp[j], vi);
+        for (int j = 0; j < HV; ++j) {
+          const int o = (h * HV + j) * WPT * 32;
+          in[j] = (int64_t)(v0 + o) < nvec;
+          va[j] = in[j] ? sa[o] : Vec<DT>::neg_inf();
+          vp[j] = in[j] ? sp[o] : Vec<DT>::neg_inf();
+        }
+        if (h == VPL / HV - 1) {
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&sm.empty[s]);     // the last vectors are in registers: stage free
+        }
+#pragma unroll
+        for (int j = 0; j < HV; ++j) {
+          const float vm_a = Vec<DT>::vmax(va[j]), vm_p = Vec<DT>::vmax(vp[j]);
+          accumulate<DT>(va[j], vm_a, oa);
+          accumulate<DT>(vp[j], vm_p, op);
+          if (TOPK) {
+            const uint32_t vi = v0 + (h * HV + j) * WPT * 32;
+            const uint32_t ma = __ballot_sync(0xffffffffu, in[j] && vm_a >= tval_a);
+            if (ma) {
+              q_a = push_candidates(sm.qdata[p][0][cw], sm.qidx[p][0][cw], &sm.qhead[p][0][cw], &sm.abort, ma, va[j],
+                                    vi, q_a, lane);
+              if (q_a.x < 0) return false;
+            }
+            const uint32_t mp = __ballot_sync(0xffffffffu, in[j] && vm_p >= tval_p);
+            if (mp) {
+              q_p = push_candidates(sm.qdata[p][1][cw], sm.qidx[p][1][cw], &sm.qhead[p][1][cw], &sm.abort, mp, vp[j],
+                                    vi, q_p, lane);
+              if (q_p.x < 0) return false;
+            }
+          }
         }
       }
       return true;
     };
     bool first = true;
     for (uint32_t tile = gq; tile < ntiles; tile += NG) {
-      const bool ok = ((int64_t)(tile + 1) * TV <= nvec) ? consume_tile(tile, first, std::true_type{})
-                                                         : consume_tile(tile, first, std::false_type{});
-      if (!ok) { raise_timeout(sm, A.sc); return; }
+      if (!consume_tile(tile, first)) { raise_timeout(sm, A.sc); return; }
       first = false;
-    }
-    if (TOPK && first) {
-      // a short row gave this warp no tile: it still takes part in the bound exchange
-      if (lane == 0) { sm.warp_bound[p][0][cw] = JP_NEG_INF; sm.warp_bound[p][1][cw] = JP_NEG_INF; }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&sm.bound_ready[p]);
     }
 
     if (tail > 0 && cw == 0 && lane == 0) {     // ragged end of the row: scalar loads
@@ -752,15 +816,23 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
     for (int j = 0; j < KL; ++j) L[j] = 0ull;
     Tau tau{0u, 0, 0ull};
     uint32_t base = 0u;
-    int staged = 0, head = 0;
+    uint4* svd = sm.svdata[p][t];
+    uint32_t* svi = sm.svidx[p][t];
+    int nsv = 0;                                      // candidate vectors kept so far
+
+    // the sampled token's logit is needed only at the end of the row: fetch it now
+    float zx = 0.f;
+    if (lane == 0) zx = Vec<DT>::load_scalar(rmine, A.tokens[row]);
+    const int ring = lane & 15, off = lane >> 4;      // this lane polls entry `off` past the head of ring `ring`
+    int head_r = 0;
 
     if (TOPK) {
       for (int i = lane; i < NB; i += 32) hist[i] = 0u;
-      // the consumers' first bound on the k-th best logit starts the histogram
+      // the first consumer group's bound on the k-th best logit starts the histogram
       if (!mbar_wait(&sm.bound_ready[p], ph, &sm.abort)) { raise_timeout(sm, A.sc); return; }
       float tau0 = sm.warp_bound[p][t][0];
 #pragma unroll
-      for (int w = 1; w < NC; ++w) tau0 = fminf(tau0, sm.warp_bound[p][t][w]);
+      for (int w = 1; w < WPT; ++w) tau0 = fminf(tau0, sm.warp_bound[p][t][w]);
       base = order_code(tau0);
       tau.code = base;
       __syncwarp();
@@ -769,48 +841,60 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
     long long t0 = 0;
     uint32_t idle = 0;
     for (;;) {
-      // probe the end of the row first: if the consumers are done, the tail read
-      // after it is final
+      // probe the end of the row first: if the consumers are done, every entry they
+      // pushed is visible to the poll that follows
       int done = 0;
       if (lane == 0) done = mbar_try_wait(&sm.row_done[p], ph) ? 1 : 0;
       done = __shfl_sync(0xffffffffu, done, 0);
       if (TOPK) {
-        const int tailv = (int)lds_volatile_u32(&sm.qtail[p][t]);
-        int avail = tailv - head;
-        if (avail > 32) avail = 32;
-        if (avail > 0) {
-          const int slot = (head + lane) & (QCAP - 1);
-          uint32_t vi = QEMPTY;
-          if (lane < avail) vi = lds_volatile_u32(&sm.qidx[p][t][slot]);
-          const uint32_t ready = __ballot_sync(0xffffffffu, vi != QEMPTY);
-          const int n = ready == 0xffffffffu ? 32 : __ffs(~ready) - 1;     // written entries, in order
-          if (n > 0) {
-            __threadfence_block();
-            uint4 v = Vec<DT>::neg_inf();
-            if (lane < n) {
-              v = sm.qdata[p][t][slot];
-              sm.qidx[p][t][slot] = QEMPTY;
-            }
-            __syncwarp();
-            __threadfence_block();
-            head += n;
-            if (lane == 0) asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(smem_u32(&sm.qhead[p][t])), "r"(head) : "memory");
-            staged = filter_vector<DT>(v, vi, lane < n, A.V, tau, base, hist, stg, staged, lane);
-            if (advance_tau(tau, base, hist, k) && lane == 0)
-              sts_volatile_f32(&sm.tau[p][t], code_value(tau.code));
-            if (staged > SCAP - 32 * N) {
-              // the buffer is filling up: drop what tau has ruled out; if ties keep it
-              // full, sort it into the list and go on with the exact k-th key
-              staged = compact_keys(stg, staged, tau, lane);
-              if (staged > SCAP / 2) tau.key = merge_all<KL>(L, stg, staged, k, lane);
-            }
-            continue;
+        const int slot = (head_r + off) & (MQ - 1);
+        uint32_t vi = QEMPTY;
+        if (ring < NC) vi = lds_volatile_u32(&sm.qidx[p][t][ring][slot]);
+        bool ok = vi != QEMPTY;
+        const bool ok0 = __shfl_sync(0xffffffffu, ok, ring);        // the ring's head entry
+        ok = ok && ok0;                                              // entries leave a ring in order
+        if (__any_sync(0xffffffffu, ok)) {
+          __threadfence_block();
+          uint4 v = Vec<DT>::neg_inf();
+          if (ok) {
+            v = sm.qdata[p][t][ring][slot];
+            sm.qidx[p][t][ring][slot] = QEMPTY;
           }
+          const bool ok1 = __shfl_sync(0xffffffffu, ok, ring + 16);
+          const int took = (ok0 ? 1 : 0) + (ok1 ? 1 : 0);
+          head_r += took;
+          __syncwarp();
+          __threadfence_block();
+          if (lane < 16 && took > 0)
+            asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(smem_u32(&sm.qhead[p][t][ring])), "r"(head_r) : "memory");
+          // admission by the vector's maximum alone: count it, keep the vector
+          const uint32_t ob = f32_order_bits(Vec<DT>::vmax(v));
+          const bool in = ok && vector_alive(ob, vi, N, tau);
+          if (in) {
+            const uint32_t code = ob >> 16;
+            atomicAdd(&hist[code - base < (uint32_t)(NB - 1) ? code - base : (uint32_t)(NB - 1)], 1u);
+          }
+          const uint32_t bin_ = __ballot_sync(0xffffffffu, in);
+          if (in) {
+            const int o = nsv + __popc(bin_ & ((1u << lane) - 1u));
+            svd[o] = v;
+            svi[o] = vi;
+          }
+          nsv += __popc(bin_);
+          tau.cnt += __popc(bin_);
+          __syncwarp();
+          if (advance_tau(tau, base, hist, k) && lane == 0)
+            sts_volatile_f32(&sm.tau[p][t], code_value(tau.code));
+          if (nsv > SVCAP - 32) {
+            // the buffer is filling up: drop what tau has ruled out; if ties keep it
+            // full, sort the kept entries into the list and go on with the exact k-th key
+            nsv = compact_survivors<DT>(svd, svi, nsv, tau, lane);
+            if (nsv > SVCAP / 2) survivors_to_list<DT, KL>(L, svd, svi, nsv, A.V, tau, stg, k, lane);
+          }
+          continue;
         }
-        if (done && tailv == head) break;
-      } else if (done) {
-        break;
       }
+      if (done) break;
       if ((idle++ & 63u) == 0u) {
         if (*(volatile int*)&sm.abort) return;
         const long long now = clock64();
@@ -823,14 +907,16 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
     if (TOPK) {
       const char* ra = (const char*)A.za + row * A.ld * Vec<DT>::ESIZE;
       const char* rp = (const char*)A.zp + row * A.ld * Vec<DT>::ESIZE;
-      if (tail > 0) {
-        uint4 v = Vec<DT>::neg_inf();
-        if (lane == 0) v = load_tail_vector<DT>(rmine, nvec * N, tail);
-        staged = filter_vector<DT>(v, (uint32_t)nvec, lane == 0, A.V, tau, base, hist, stg, staged, lane);
-        advance_tau(tau, base, hist, k);
+      if (tail > 0) {                 // the ragged end of the row joins the kept vectors
+        if (lane == 0) {
+          svd[nsv] = load_tail_vector<DT>(rmine, nvec * N, tail);
+          svi[nsv] = (uint32_t)nvec;
+        }
+        nsv += 1;
+        __syncwarp();
       }
-      staged = compact_keys(stg, staged, tau, lane);
-      merge_all<KL>(L, stg, staged, k, lane);
+      nsv = compact_survivors<DT>(svd, svi, nsv, tau, lane);
+      survivors_to_list<DT, KL>(L, svd, svi, nsv, A.V, tau, stg, k, lane);
       // the record: this tensor's list, best first, every entry with both logits
 #pragma unroll
       for (int j = 0; j < KL; ++j) {
@@ -849,10 +935,8 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
         }
       }
       // hand the slot back clean (every ring entry was reset as it was drained)
-      if (lane == 0) {
-        sm.qtail[p][t] = 0; sm.qhead[p][t] = 0;
-        sts_volatile_f32(&sm.tau[p][t], JP_NEG_INF);
-      }
+      if (lane < NC) sm.qhead[p][t][lane] = 0;
+      if (lane == 0) sts_volatile_f32(&sm.tau[p][t], JP_NEG_INF);
     }
 
     if (lane == 0) {
@@ -868,8 +952,6 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
       const float f = 2.f * frexpf(S, &e);                // S = f * 2^(e-1)
       const double lse = ((double)M + (double)(e - 1)) * 0.6931471805599453 + (double)logf(f);
       const float lsef = (float)lse;
-      const int32_t x = A.tokens[row];
-      const float zx = Vec<DT>::load_scalar(rmine, x);
       const float lpx = (float)((double)zx - lse);
       if (t == 0) { A.rec.lse_a[rrow] = lsef; A.rec.lq[rrow] = lpx; A.rec.flag[rrow] = 1; }
       else        { A.rec.lse_p[rrow] = lsef; A.rec.lp[rrow] = lpx; }
@@ -886,14 +968,15 @@ __global__ void __launch_bounds__(NTHREADS, 1) stream_kernel(StreamArgs A) {
   StreamSmem& sm = *reinterpret_cast<StreamSmem*>(smem_raw);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-  for (int i = tid; i < 2 * 2 * QCAP; i += NTHREADS) (&sm.qidx[0][0][0])[i] = QEMPTY;
+  for (int i = tid; i < 2 * 2 * NC * MQ; i += NTHREADS) (&sm.qidx[0][0][0][0])[i] = QEMPTY;
+  for (int i = tid; i < 2 * 2 * NC; i += NTHREADS) (&sm.qhead[0][0][0])[i] = 0;
   if (tid == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], WPT); }
     for (int p = 0; p < 2; ++p) {
       mbar_init(&sm.row_done[p], NC);
       mbar_init(&sm.slot_free[p], 2);
-      mbar_init(&sm.bound_ready[p], NC);
-      for (int t = 0; t < 2; ++t) { sm.qtail[p][t] = 0; sm.qhead[p][t] = 0; sm.tau[p][t] = JP_NEG_INF; }
+      mbar_init(&sm.bound_ready[p], WPT);
+      for (int t = 0; t < 2; ++t) sm.tau[p][t] = JP_NEG_INF;
     }
     sm.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
