@@ -698,7 +698,7 @@ __device__ void consumer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_row
       const uint32_t v0 = tile * TV + wq * 32 + lane;
       const uint4* sa = &sm.ring[s][0][wq * 32 + lane];
       const uint4* sp = &sm.ring[s][1][wq * 32 + lane];
-      float tval_a = 0.f, tval_p = 0.f;
+      float tval_a = __int_as_float(0x7f800000), tval_p = __int_as_float(0x7f800000);
       if (TOPK) {
         if (first) {
           if (gq == 0) {
@@ -716,41 +716,65 @@ __device__ void consumer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_row
         tval_a = fmaxf(tau0_a, lds_volatile_f32(&sm.tau[p][0]));
         tval_p = fmaxf(tau0_p, lds_volatile_f32(&sm.tau[p][1]));
       }
+      // the rare path: some lane's vector may hold a top-k entry
+      auto push_pair = [&](const uint4& a4, const uint4& p4, float vm_a, float vm_p, uint32_t vi, bool in) -> bool {
+        const uint32_t ma = __ballot_sync(0xffffffffu, in && vm_a >= tval_a);
+        if (ma) {
+          q_a = push_candidates(sm.qdata[p][0][cw], sm.qidx[p][0][cw], &sm.qhead[p][0][cw], &sm.abort, ma, a4, vi, q_a,
+                                lane);
+          if (q_a.x < 0) return false;
+        }
+        const uint32_t mp = __ballot_sync(0xffffffffu, in && vm_p >= tval_p);
+        if (mp) {
+          q_p = push_candidates(sm.qdata[p][1][cw], sm.qidx[p][1][cw], &sm.qhead[p][1][cw], &sm.abort, mp, p4, vi, q_p,
+                                lane);
+          if (q_p.x < 0) return false;
+        }
+        return true;
+      };
+      if ((int64_t)(tile + 1) * TV <= nvec) {
+        // a full tile: passes of HV vectors per tensor, no bounds checks
 #pragma unroll 1
-      for (int h = 0; h < VPL / HV; ++h) {
-        uint4 va[HV], vp[HV];
-        bool in[HV];
+        for (int h = 0; h < VPL / HV; ++h, sa += HV * WPT * 32, sp += HV * WPT * 32) {
+          uint4 va[HV], vp[HV];
 #pragma unroll
-        for (int j = 0; j < HV; ++j) {
-          const int o = (h * HV + j) * WPT * 32;
-          in[j] = (int64_t)(v0 + o) < nvec;
-          va[j] = in[j] ? sa[o] : Vec<DT>::neg_inf();
-          vp[j] = in[j] ? sp[o] : Vec<DT>::neg_inf();
-        }
-        if (h == VPL / HV - 1) {
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&sm.empty[s]);     // the last vectors are in registers: stage free
-        }
-#pragma unroll
-        for (int j = 0; j < HV; ++j) {
-          const float vm_a = Vec<DT>::vmax(va[j]), vm_p = Vec<DT>::vmax(vp[j]);
-          accumulate<DT>(va[j], vm_a, oa);
-          accumulate<DT>(vp[j], vm_p, op);
-          if (TOPK) {
-            const uint32_t vi = v0 + (h * HV + j) * WPT * 32;
-            const uint32_t ma = __ballot_sync(0xffffffffu, in[j] && vm_a >= tval_a);
-            if (ma) {
-              q_a = push_candidates(sm.qdata[p][0][cw], sm.qidx[p][0][cw], &sm.qhead[p][0][cw], &sm.abort, ma, va[j],
-                                    vi, q_a, lane);
-              if (q_a.x < 0) return false;
-            }
-            const uint32_t mp = __ballot_sync(0xffffffffu, in[j] && vm_p >= tval_p);
-            if (mp) {
-              q_p = push_candidates(sm.qdata[p][1][cw], sm.qidx[p][1][cw], &sm.qhead[p][1][cw], &sm.abort, mp, vp[j],
-                                    vi, q_p, lane);
-              if (q_p.x < 0) return false;
-            }
+          for (int j = 0; j < HV; ++j) { va[j] = sa[j * WPT * 32]; vp[j] = sp[j * WPT * 32]; }
+          if (h == VPL / HV - 1) {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.empty[s]);   // the last vectors are in registers: stage free
           }
+          float vm_a[HV], vm_p[HV];
+          bool cand = false;
+#pragma unroll
+          for (int j = 0; j < HV; ++j) {
+            vm_a[j] = Vec<DT>::vmax(va[j]);
+            vm_p[j] = Vec<DT>::vmax(vp[j]);
+            accumulate<DT>(va[j], vm_a[j], oa);
+            accumulate<DT>(vp[j], vm_p[j], op);
+            cand |= (vm_a[j] >= tval_a) | (vm_p[j] >= tval_p);
+          }
+          if (TOPK && __any_sync(0xffffffffu, cand)) {
+#pragma unroll
+            for (int j = 0; j < HV; ++j)
+              if (!push_pair(va[j], vp[j], vm_a[j], vm_p[j], v0 + (h * HV + j) * WPT * 32, true)) return false;
+          }
+        }
+      } else {
+        // the row's last, partial tile: one vector per tensor at a time, bounds checked
+#pragma unroll 1
+        for (int j = 0; j < VPL; ++j) {
+          const uint32_t vi = v0 + j * WPT * 32;
+          const bool in = (int64_t)vi < nvec;
+          uint4 a4 = Vec<DT>::neg_inf(), p4 = Vec<DT>::neg_inf();
+          if (in) { a4 = sa[j * WPT * 32]; p4 = sp[j * WPT * 32]; }
+          if (j == VPL - 1) {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.empty[s]);
+          }
+          const float vm_a = Vec<DT>::vmax(a4), vm_p = Vec<DT>::vmax(p4);
+          accumulate<DT>(a4, vm_a, oa);
+          accumulate<DT>(p4, vm_p, op);
+          if (TOPK && !push_pair(a4, p4, vm_a, vm_p, vi, in)) return false;
         }
       }
       return true;
