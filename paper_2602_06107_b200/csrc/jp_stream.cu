@@ -61,13 +61,13 @@ constexpr int VPL = JP_VPL;               // 16-byte vectors per lane per tensor
 constexpr int TV = WPT * 32 * VPL;        // vectors per tensor per tile
 constexpr int HV = 2;                     // vectors per tensor a lane holds at a time
 static_assert(JP_VPL % HV == 0, "a tile is taken in passes of HV vectors");
-static_assert(NC <= 16, "one top-k warp polls two entries of up to 16 rings");
 static_assert(NC % NG == 0 && NG < JP_STAGES, "consumer groups must divide the warps and fit the ring");
 constexpr int STAGES = JP_STAGES;
-constexpr int MQ = 16;                    // candidate-vector ring entries per (slot, tensor, consumer warp); power of two
 constexpr int SCAP = 384;                 // buffered keys per top-k warp (used while sorting survivors into the list)
 constexpr int SVCAP = 192;                // candidate vectors a top-k warp keeps until the row ends
-constexpr int NB = 512;                   // histogram bins (16-bit order codes above the row's first bound)
+constexpr int NB = 512;                   // histogram bins: 16-bit order codes below the first tile's maximum
+constexpr int TP = TV / HV;               // passes per tensor per tile = pass maxima a top-k warp scans per tile
+static_assert(TP == 512, "a top-k lane scans 16 pass maxima per tile (4 x 16 bytes)");
 constexpr int NTOPK = 4;                  // top-k warps: (tensor, slot)
 constexpr int NWARPS = 1 + NC + NTOPK;
 constexpr int NTHREADS = NWARPS * 32;
@@ -76,17 +76,15 @@ constexpr long long kSpinLimit = 4000000000ll;   // clock cycles a wait may last
 
 struct __align__(128) StreamSmem {
   uint4 ring[STAGES][2][TV];              // [stage][tensor][vector]
-  uint4 qdata[2][2][NC][MQ];              // [slot][tensor][consumer warp] candidate vectors ...
   uint4 svdata[2][2][SVCAP];              // [slot][tensor] candidate vectors still alive under tau ...
+  float passmax[STAGES][2][TP];           // [stage][tensor] maximum of each consumer pass (HV vectors) of the tile
   unsigned long long skeys[2][2][SCAP];   // [slot][tensor] keys waiting to be sorted into the list
-  uint32_t qidx[2][2][NC][MQ];            // ... their vector index (QEMPTY = not written yet)
   uint32_t svidx[2][2][SVCAP];            // ... and the kept vectors' indices
-  uint32_t hist[2][2][NB];                // [slot][tensor] candidate vectors seen per order code of their maximum
-  unsigned long long full[STAGES], empty[STAGES];
-  unsigned long long row_done[2], slot_free[2], bound_ready[2];
-  int qhead[2][2][NC];                    // per ring: entries drained so far (top-k warp)
-  float tau[2][2];                        // published threshold (a logit value)
-  float warp_bound[2][2][NC];
+  uint32_t hist[2][2][NB];                // [slot][tensor] passes seen per order code of their maximum
+  unsigned long long full[STAGES];        // producer -> consumers: the tile's bytes have landed
+  unsigned long long seen[2][STAGES];     // [slot] consumers -> that slot's top-k warps: tile consumed, pass maxima written
+  unsigned long long empty[STAGES];       // -> producer: the stage may be refilled
+  unsigned long long row_done[2], slot_free[2];
   float part_mL[2][2][NC];
   float part_s[2][2][NC];
   int abort;
@@ -319,30 +317,6 @@ __device__ __forceinline__ uint4 load_tail_vector(const char* row, int64_t first
   return v;
 }
 
-// r-th largest (1-based) of the warp's 32 * NV values (NV per lane); -inf when
-// fewer than r of them are numbers above -inf.
-template <int NV>
-__device__ __forceinline__ float warp_rth_largest(const float (&v)[NV], int r, int lane) {
-  uint32_t ob[NV];
-#pragma unroll
-  for (int j = 0; j < NV; ++j) ob[j] = f32_order_bits(v[j]);
-  uint32_t mx = 0u;
-  for (int i = 0; i < r; ++i) {
-    uint32_t lm = ob[0];
-#pragma unroll
-    for (int j = 1; j < NV; ++j) lm = lm > ob[j] ? lm : ob[j];
-    mx = __reduce_max_sync(0xffffffffu, lm);
-    const uint32_t holders = __ballot_sync(0xffffffffu, lm == mx);
-    if (lane == __ffs(holders) - 1) {            // retire one copy of the maximum
-      bool gone = false;
-#pragma unroll
-      for (int j = 0; j < NV; ++j)
-        if (!gone && ob[j] == mx) { ob[j] = 0u; gone = true; }
-    }
-  }
-  return mx <= 0x007fffffu ? JP_NEG_INF : order_bits_f32(mx);
-}
-
 // ---- the sorted list of a top-k warp ---------------------------------------
 // 32*KPL keys, sorted descending, position p = lane*KPL + j in register j of a lane.
 __device__ __forceinline__ unsigned long long u64max(unsigned long long a, unsigned long long b) { return a > b ? a : b; }
@@ -465,19 +439,38 @@ __device__ __forceinline__ bool vector_alive(uint32_t ob, uint32_t vi, int n_per
   return (((unsigned long long)ob << 32) | (unsigned long long)(uint32_t)(~(vi * (uint32_t)n_per_vec))) > tau.key;
 }
 
-// Raises tau.code while at least k counted vectors stay at or above it.
-__device__ __forceinline__ bool advance_tau(Tau& tau, uint32_t base, const uint32_t* hist, int k) {
-  bool moved = false;
-  for (;;) {
-    const uint32_t bin = tau.code - base;
-    if (bin >= (uint32_t)(NB - 1)) break;
-    const int h = (int)lds_volatile_u32(&hist[bin]);
-    if (tau.cnt - h < k) break;
-    tau.cnt -= h;
-    tau.code += 1u;
-    moved = true;
+// The highest histogram bin with at least k counted passes at or above it (0 if
+// fewer than k passes were counted).  Lane l sums bins 16 l .. 16 l + 15, a shuffle
+// suffix scan finds the lane in which the count crosses k, and that lane walks its
+// 16 bins from the top.
+__device__ __forceinline__ int find_tau_bin(const uint32_t* hist, int k, int lane) {
+  const uint4* h4 = reinterpret_cast<const uint4*>(hist) + lane * 4;
+  uint32_t b[16];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const uint4 v = h4[q];
+    b[4 * q] = v.x; b[4 * q + 1] = v.y; b[4 * q + 2] = v.z; b[4 * q + 3] = v.w;
   }
-  return moved;
+  int mine = 0;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) mine += (int)b[i];
+  int suf = mine;                                   // passes in this lane's bins and all higher lanes'
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int o = __shfl_down_sync(0xffffffffu, suf, off);
+    if (lane + off < 32) suf += o;
+  }
+  const uint32_t ge = __ballot_sync(0xffffffffu, suf >= k);
+  if (ge == 0u) return 0;
+  const int L = 31 - __clz(ge);                     // the highest lane whose suffix reaches k
+  int run = suf - mine, bin = 0;
+  bool found = false;
+#pragma unroll
+  for (int i = 15; i >= 0; --i) {
+    run += (int)b[i];
+    if (!found && run >= k) { bin = i; found = true; }
+  }
+  return __shfl_sync(0xffffffffu, lane * 16 + bin, L);
 }
 
 // Drops the kept candidate vectors that tau has ruled out since they were kept.
@@ -567,64 +560,6 @@ __device__ __forceinline__ void raise_timeout(StreamSmem& sm, Scalars* sc) {
   atomicExch(&sc->status, (int)JP_ERR_TIMEOUT);
 }
 
-// A consumer warp hands the vectors that may hold a top-k entry (`cand` lanes) to
-// the slot's top-k warp through the warp's own small ring: no atomics, the tail
-// lives in a register.  The ring's head (entries the top-k warp has drained) is
-// re-read only when the ring looks full; that wait is bounded.  Each entry is
-// published by writing its index after its data.  Kept out of line: the streaming
-// loop only pays a ballot and a branch for a vector that is no candidate.
-// state.x = entries pushed so far, state.y = last head seen; returns the new state
-// (x < 0: the wait for room ran out).
-__device__ __noinline__ int2 push_candidates(uint4* qdata, uint32_t* qidx, const int* qhead, volatile int* abort,
-                                             uint32_t m, uint4 v, uint32_t vi, int2 state, int lane) {
-  int tail = state.x, head_known = state.y;
-  while (m) {
-    int room = MQ - (tail - head_known);
-    if (room <= 0) {
-      int spins = 0;
-      do {
-        head_known = (int)lds_volatile_u32(qhead);
-        room = MQ - (tail - head_known);
-      } while (room <= 0 && ++spins < (1 << 22) && !*abort);
-      if (room <= 0) { *abort = 1; return make_int2(-1, head_known); }
-    }
-    const int rank = __popc(m & ((1u << lane) - 1u));
-    const bool mine = ((m >> lane) & 1u) && rank < room;
-    if (mine) {
-      const int slot = (tail + rank) & (MQ - 1);
-      qdata[slot] = v;
-      __threadfence_block();
-      asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(smem_u32(&qidx[slot])), "r"(vi) : "memory");
-    }
-    const uint32_t took = __ballot_sync(0xffffffffu, mine);
-    m &= ~took;
-    tail += __popc(took);
-  }
-  return make_int2(tail, head_known);
-}
-
-// First tile of a row, first consumer group: no threshold exists yet.  Every warp
-// of the group takes the r-th largest of its vector maxima over the tile,
-// r = ceil(k / warps in the group); the smallest of these over the group has at
-// least k row entries at or above it (distinct vectors, r per warp), so it bounds
-// the k-th best logit of the row from below.  The vectors are only looked at here;
-// the streaming pass that follows reads them again from the stage.
-template <int DT>
-__device__ __noinline__ void first_tile_bound(const uint4* sa, const uint4* sp, uint32_t v0, int64_t nvec, int r,
-                                              float* bound_a, float* bound_p, int lane) {
-  float vm_a[VPL], vm_p[VPL];
-#pragma unroll
-  for (int j = 0; j < VPL; ++j) {
-    const bool in = (int64_t)(v0 + j * WPT * 32) < nvec;
-    vm_a[j] = in ? Vec<DT>::vmax(sa[j * WPT * 32]) : JP_NEG_INF;
-    vm_p[j] = in ? Vec<DT>::vmax(sp[j * WPT * 32]) : JP_NEG_INF;
-  }
-  const float ba = warp_rth_largest<VPL>(vm_a, r, lane);
-  const float bp = warp_rth_largest<VPL>(vm_p, r, lane);
-  if (lane == 0) { *bound_a = ba; *bound_p = bp; }
-  __syncwarp();
-}
-
 // ---- producer ---------------------------------------------------------------
 template <int DT>
 __device__ void producer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows) {
@@ -672,7 +607,6 @@ __device__ void consumer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_row
   const int64_t nvec = A.V / N;
   const int tail = (int)(A.V - nvec * N);
   const uint32_t ntiles = nvec > 0 ? (uint32_t)((nvec + TV - 1) / TV) : 1u;
-  const int r = (A.k + WPT - 1) / WPT;
   const int gq = cw / WPT;              // this warp's group: it takes tiles gq, gq + NG, ...
   const int wq = cw % WPT;              // its place among the warps that share a tile
   uint32_t g0 = 0;                      // ring position of the current row's tile 0
@@ -680,110 +614,79 @@ __device__ void consumer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_row
   for (int64_t it = blockIdx.x; it < n_rows; it += gridDim.x, ++lr, g0 += ntiles) {
     const int p = lr & 1;
     const uint32_t ph = (uint32_t)((lr >> 1) & 1);
-    // the slot's queue, tau and partial sums are free once both of its top-k warps
-    // have finished the row that used it before
+    // the slot's partial sums are free once both of its top-k warps have finished
+    // the row that used it before
     if (!mbar_wait(&sm.slot_free[p], ph ^ 1u, &sm.abort)) { raise_timeout(sm, A.sc); return; }
 
     Online oa{JP_NEG_INF, 0.f, 0ull}, op{JP_NEG_INF, 0.f, 0ull};
-    float tau0_a = JP_NEG_INF, tau0_p = JP_NEG_INF;
-    int2 q_a = make_int2(0, 0), q_p = make_int2(0, 0);  // this warp's rings: entries pushed, last head seen
 
-    // One tile of both rows; first = this warp's first tile of the row.  The tile is
-    // taken in passes of HV vectors per tensor: a short loop body keeps the streaming
-    // code small enough for the instruction caches and the live registers few.
-    auto consume_tile = [&](uint32_t tile, bool first) -> bool {
+    // One tile of both rows, taken in passes of HV vectors per tensor: a short loop
+    // body keeps the streaming code small for the instruction caches and the live
+    // registers few.  The only thing a consumer does for the top-k is to leave the
+    // maximum of every pass in shared memory; the top-k warps scan those.
+    auto consume_tile = [&](uint32_t tile) -> bool {
       const uint32_t g = g0 + tile;
       const uint32_t s = g % STAGES;
       if (!mbar_wait(&sm.full[s], (g / STAGES) & 1u, &sm.abort)) return false;
-      const uint32_t v0 = tile * TV + wq * 32 + lane;
       const uint4* sa = &sm.ring[s][0][wq * 32 + lane];
       const uint4* sp = &sm.ring[s][1][wq * 32 + lane];
-      float tval_a = __int_as_float(0x7f800000), tval_p = __int_as_float(0x7f800000);
-      if (TOPK) {
-        if (first) {
-          if (gq == 0) {
-            first_tile_bound<DT>(sa, sp, v0, nvec, r, &sm.warp_bound[p][0][wq], &sm.warp_bound[p][1][wq], lane);
-            if (lane == 0) mbar_arrive(&sm.bound_ready[p]);
-          }
-          if (!mbar_wait(&sm.bound_ready[p], ph, &sm.abort)) return false;
-          tau0_a = sm.warp_bound[p][0][0]; tau0_p = sm.warp_bound[p][1][0];
-#pragma unroll
-          for (int w = 1; w < WPT; ++w) {
-            tau0_a = fminf(tau0_a, sm.warp_bound[p][0][w]);
-            tau0_p = fminf(tau0_p, sm.warp_bound[p][1][w]);
-          }
-        }
-        tval_a = fmaxf(tau0_a, lds_volatile_f32(&sm.tau[p][0]));
-        tval_p = fmaxf(tau0_p, lds_volatile_f32(&sm.tau[p][1]));
-      }
-      // the rare path: some lane's vector may hold a top-k entry
-      auto push_pair = [&](const uint4& a4, const uint4& p4, float vm_a, float vm_p, uint32_t vi, bool in) -> bool {
-        const uint32_t ma = __ballot_sync(0xffffffffu, in && vm_a >= tval_a);
-        if (ma) {
-          q_a = push_candidates(sm.qdata[p][0][cw], sm.qidx[p][0][cw], &sm.qhead[p][0][cw], &sm.abort, ma, a4, vi, q_a,
-                                lane);
-          if (q_a.x < 0) return false;
-        }
-        const uint32_t mp = __ballot_sync(0xffffffffu, in && vm_p >= tval_p);
-        if (mp) {
-          q_p = push_candidates(sm.qdata[p][1][cw], sm.qidx[p][1][cw], &sm.qhead[p][1][cw], &sm.abort, mp, p4, vi, q_p,
-                                lane);
-          if (q_p.x < 0) return false;
-        }
-        return true;
-      };
+      float* pma = &sm.passmax[s][0][wq * 32 + lane];
+      float* pmp = &sm.passmax[s][1][wq * 32 + lane];
       if ((int64_t)(tile + 1) * TV <= nvec) {
-        // a full tile: passes of HV vectors per tensor, no bounds checks
+        // a full tile: no bounds checks
 #pragma unroll 1
-        for (int h = 0; h < VPL / HV; ++h, sa += HV * WPT * 32, sp += HV * WPT * 32) {
+        for (int h = 0; h < VPL / HV; ++h, sa += HV * WPT * 32, sp += HV * WPT * 32, pma += WPT * 32, pmp += WPT * 32) {
           uint4 va[HV], vp[HV];
 #pragma unroll
           for (int j = 0; j < HV; ++j) { va[j] = sa[j * WPT * 32]; vp[j] = sp[j * WPT * 32]; }
-          if (h == VPL / HV - 1) {
+          if (!TOPK && h == VPL / HV - 1) {
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm.empty[s]);   // the last vectors are in registers: stage free
           }
-          float vm_a[HV], vm_p[HV];
-          bool cand = false;
+          float ma = JP_NEG_INF, mp = JP_NEG_INF;
 #pragma unroll
           for (int j = 0; j < HV; ++j) {
-            vm_a[j] = Vec<DT>::vmax(va[j]);
-            vm_p[j] = Vec<DT>::vmax(vp[j]);
-            accumulate<DT>(va[j], vm_a[j], oa);
-            accumulate<DT>(vp[j], vm_p[j], op);
-            cand |= (vm_a[j] >= tval_a) | (vm_p[j] >= tval_p);
+            const float vm_a = Vec<DT>::vmax(va[j]), vm_p = Vec<DT>::vmax(vp[j]);
+            accumulate<DT>(va[j], vm_a, oa);
+            accumulate<DT>(vp[j], vm_p, op);
+            ma = fmaxf(ma, vm_a);
+            mp = fmaxf(mp, vm_p);
           }
-          if (TOPK && __any_sync(0xffffffffu, cand)) {
-#pragma unroll
-            for (int j = 0; j < HV; ++j)
-              if (!push_pair(va[j], vp[j], vm_a[j], vm_p[j], v0 + (h * HV + j) * WPT * 32, true)) return false;
-          }
+          if (TOPK) { *pma = ma; *pmp = mp; }
         }
       } else {
-        // the row's last, partial tile: one vector per tensor at a time, bounds checked
+        // the row's last, partial tile: bounds checked
+        const uint32_t v0 = tile * TV + wq * 32 + lane;
 #pragma unroll 1
-        for (int j = 0; j < VPL; ++j) {
-          const uint32_t vi = v0 + j * WPT * 32;
-          const bool in = (int64_t)vi < nvec;
-          uint4 a4 = Vec<DT>::neg_inf(), p4 = Vec<DT>::neg_inf();
-          if (in) { a4 = sa[j * WPT * 32]; p4 = sp[j * WPT * 32]; }
-          if (j == VPL - 1) {
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sm.empty[s]);
+        for (int h = 0; h < VPL / HV; ++h, pma += WPT * 32, pmp += WPT * 32) {
+          float ma = JP_NEG_INF, mp = JP_NEG_INF;
+#pragma unroll 1
+          for (int j = 0; j < HV; ++j) {
+            const int o = (h * HV + j) * WPT * 32;
+            uint4 a4 = Vec<DT>::neg_inf(), p4 = Vec<DT>::neg_inf();
+            if ((int64_t)(v0 + o) < nvec) { a4 = sa[o]; p4 = sp[o]; }
+            const float vm_a = Vec<DT>::vmax(a4), vm_p = Vec<DT>::vmax(p4);
+            accumulate<DT>(a4, vm_a, oa);
+            accumulate<DT>(p4, vm_p, op);
+            ma = fmaxf(ma, vm_a);
+            mp = fmaxf(mp, vm_p);
           }
-          const float vm_a = Vec<DT>::vmax(a4), vm_p = Vec<DT>::vmax(p4);
-          accumulate<DT>(a4, vm_a, oa);
-          accumulate<DT>(p4, vm_p, op);
-          if (TOPK && !push_pair(a4, p4, vm_a, vm_p, vi, in)) return false;
+          if (TOPK) { *pma = ma; *pmp = mp; }
         }
+        if (!TOPK) {
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&sm.empty[s]);
+        }
+      }
+      if (TOPK) {
+        // the top-k warps of this row's slot take it from here; they free the stage
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.seen[p][s]);
       }
       return true;
     };
-    bool first = true;
-    for (uint32_t tile = gq; tile < ntiles; tile += NG) {
-      if (!consume_tile(tile, first)) { raise_timeout(sm, A.sc); return; }
-      first = false;
-    }
+    for (uint32_t tile = gq; tile < ntiles; tile += NG)
+      if (!consume_tile(tile)) { raise_timeout(sm, A.sc); return; }
 
     if (tail > 0 && cw == 0 && lane == 0) {     // ragged end of the row: scalar loads
       const int64_t row = A.list[it];
@@ -819,6 +722,13 @@ __device__ void consumer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_row
 }
 
 // ---- top-k warps ---------------------------------------------------------------
+// One warp per (tensor t, row slot p).  For every tile of its row it waits until
+// the consumers are through with the stage, scans the 512 pass maxima they left
+// (16 per lane), counts in the histogram those at or above the running threshold
+// and copies the vectors behind them that are still alive from the stage into the
+// survivor buffer; then it frees the stage.  The threshold is the low edge of the
+// highest histogram bin with k counted passes at or above it: k different passes
+// hold k different entries of the row, so the k-th best logit is not below it.
 template <int DT, int KPL>
 __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, int t, int p, int lane) {
   constexpr int N = Vec<DT>::N;
@@ -826,12 +736,21 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
   constexpr int KL = KPL > 0 ? KPL : 1;
   const int64_t nvec = A.V / N;
   const int tail = (int)(A.V - nvec * N);
+  const uint32_t ntiles = nvec > 0 ? (uint32_t)((nvec + TV - 1) / TV) : 1u;
   const int k = A.k;
   unsigned long long* stg = sm.skeys[p][t];
   uint32_t* hist = sm.hist[p][t];
+  uint4* svd = sm.svdata[p][t];
+  uint32_t* svi = sm.svidx[p][t];
+  // A slot's `seen` barriers complete once per tile of that slot's rows, and this
+  // warp waits for every one of them in turn, so one phase bit per stage is enough.
+  // (A barrier shared by both slots would not do: a parity wait cannot tell "not yet
+  // reached" from "done" when the waiter skips phases.)
+  uint32_t seen_phase = 0u;
   int lr = p;
   for (int64_t it = (int64_t)blockIdx.x + (int64_t)p * gridDim.x; it < n_rows; it += 2ll * gridDim.x, lr += 2) {
     const uint32_t ph = (uint32_t)((lr >> 1) & 1);
+    const uint32_t g0 = (uint32_t)lr * ntiles;        // ring position of this row's tile 0
     const int64_t row = A.list[it];
     const int64_t rrow = A.record_offset + row;
     const char* rmine = (const char*)(t == 0 ? A.za : A.zp) + row * A.ld * Vec<DT>::ESIZE;
@@ -840,93 +759,114 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
     for (int j = 0; j < KL; ++j) L[j] = 0ull;
     Tau tau{0u, 0, 0ull};
     uint32_t base = 0u;
-    uint4* svd = sm.svdata[p][t];
-    uint32_t* svi = sm.svidx[p][t];
+    float tau_val = JP_NEG_INF;
     int nsv = 0;                                      // candidate vectors kept so far
 
     // the sampled token's logit is needed only at the end of the row: fetch it now
     float zx = 0.f;
     if (lane == 0) zx = Vec<DT>::load_scalar(rmine, A.tokens[row]);
-    const int ring = lane & 15, off = lane >> 4;      // this lane polls entry `off` past the head of ring `ring`
-    int head_r = 0;
 
     if (TOPK) {
-      for (int i = lane; i < NB; i += 32) hist[i] = 0u;
-      // the first consumer group's bound on the k-th best logit starts the histogram
-      if (!mbar_wait(&sm.bound_ready[p], ph, &sm.abort)) { raise_timeout(sm, A.sc); return; }
-      float tau0 = sm.warp_bound[p][t][0];
+      for (uint32_t tile = 0; tile < ntiles; ++tile) {
+        const uint32_t g = g0 + tile;
+        const uint32_t s = g % STAGES;
+        if (!mbar_wait(&sm.seen[p][s], (seen_phase >> s) & 1u, &sm.abort)) { raise_timeout(sm, A.sc); return; }
+        seen_phase ^= 1u << s;
+        const float* pm = sm.passmax[s][t];
+        const uint4* data = sm.ring[s][t];
+        // this lane's 16 pass maxima: entries q * 128 + lane * 4 + c
+        float v[16];
 #pragma unroll
-      for (int w = 1; w < WPT; ++w) tau0 = fminf(tau0, sm.warp_bound[p][t][w]);
-      base = order_code(tau0);
-      tau.code = base;
-      __syncwarp();
+        for (int q = 0; q < 4; ++q) {
+          const float4 f = reinterpret_cast<const float4*>(pm)[q * 32 + lane];
+          v[4 * q] = f.x; v[4 * q + 1] = f.y; v[4 * q + 2] = f.z; v[4 * q + 3] = f.w;
+        }
+        uint32_t hit = 0u;
+        if (tile == 0) {
+          // a new row: the histogram covers the NB order codes below this tile's maximum
+          // (everything lower shares bin 0, which stands for "no threshold"); every pass
+          // of the tile is counted, then the threshold is read off the histogram
+          float mx = v[0];
+#pragma unroll
+          for (int i = 1; i < 16; ++i) mx = fmaxf(mx, v[i]);
+          uint32_t top = __reduce_max_sync(0xffffffffu, order_code(mx));
+          base = top > (uint32_t)(NB - 1) ? top - (uint32_t)(NB - 1) : 0u;
+          for (int i = lane; i < NB; i += 32) hist[i] = 0u;
+          __syncwarp();
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const uint32_t code = order_code(v[i]);
+            atomicAdd(&hist[code > base ? code - base : 0u], 1u);
+          }
+          __syncwarp();
+          const int bin = find_tau_bin(hist, k, lane);
+          tau.code = bin > 0 ? base + (uint32_t)bin : 0u;
+          tau_val = bin > 0 ? code_value(tau.code) : JP_NEG_INF;
+#pragma unroll
+          for (int i = 0; i < 16; ++i) hit |= (v[i] >= tau_val ? 1u : 0u) << i;
+        } else {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) hit |= (v[i] >= tau_val ? 1u : 0u) << i;
+          if (__any_sync(0xffffffffu, hit != 0u)) {
+            // count the passes at or above the threshold (those are all there are: it only rises)
+            uint32_t hcount = hit;
+            while (__any_sync(0xffffffffu, hcount != 0u)) {
+              if (hcount) {
+                const int i = __ffs(hcount) - 1;
+                hcount &= hcount - 1u;
+                const uint32_t code = order_code(pm[(i >> 2) * 128 + lane * 4 + (i & 3)]);
+                const uint32_t bin = code > base ? code - base : 0u;
+                atomicAdd(&hist[bin < (uint32_t)(NB - 1) ? bin : (uint32_t)(NB - 1)], 1u);
+              }
+            }
+            __syncwarp();
+            const int bin = find_tau_bin(hist, k, lane);
+            tau.code = bin > 0 ? base + (uint32_t)bin : 0u;
+            tau_val = bin > 0 ? code_value(tau.code) : JP_NEG_INF;
+          }
+        }
+        // the vectors behind the hits: keep those that can still hold one of the k best
+        while (__any_sync(0xffffffffu, hit != 0u)) {
+          int e = 0;
+          const bool have = hit != 0u;
+          if (have) {
+            const int i = __ffs(hit) - 1;
+            hit &= hit - 1u;
+            e = (i >> 2) * 128 + lane * 4 + (i & 3);          // pass entry: pass h = e / (WPT*32), lane slot e % (WPT*32)
+          }
+#pragma unroll
+          for (int j = 0; j < HV; ++j) {
+            const uint32_t pos = (uint32_t)((e / (WPT * 32)) * HV + j) * (WPT * 32) + (uint32_t)(e % (WPT * 32));
+            const uint32_t vi = tile * TV + pos;
+            uint4 vec = Vec<DT>::neg_inf();
+            bool in = false;
+            if (have && (int64_t)vi < nvec) {
+              vec = data[pos];
+              in = vector_alive(f32_order_bits(Vec<DT>::vmax(vec)), vi, N, tau);
+            }
+            const uint32_t m = __ballot_sync(0xffffffffu, in);
+            if (in) {
+              const int o = nsv + __popc(m & ((1u << lane) - 1u));
+              svd[o] = vec;
+              svi[o] = vi;
+            }
+            nsv += __popc(m);
+            __syncwarp();
+            if (nsv > SVCAP - 32) {
+              // the buffer is filling up: drop what the threshold has ruled out; if ties keep
+              // it full, sort the kept entries into the list and go on with the exact k-th key
+              nsv = compact_survivors<DT>(svd, svi, nsv, tau, lane);
+              if (nsv > SVCAP / 2) survivors_to_list<DT, KL>(L, svd, svi, nsv, A.V, tau, stg, k, lane);
+            }
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.empty[s]);       // both tensors' warps done: the stage may be refilled
+      }
     }
 
-    long long t0 = 0;
-    uint32_t idle = 0;
-    for (;;) {
-      // probe the end of the row first: if the consumers are done, every entry they
-      // pushed is visible to the poll that follows
-      int done = 0;
-      if (lane == 0) done = mbar_try_wait(&sm.row_done[p], ph) ? 1 : 0;
-      done = __shfl_sync(0xffffffffu, done, 0);
-      if (TOPK) {
-        const int slot = (head_r + off) & (MQ - 1);
-        uint32_t vi = QEMPTY;
-        if (ring < NC) vi = lds_volatile_u32(&sm.qidx[p][t][ring][slot]);
-        bool ok = vi != QEMPTY;
-        const bool ok0 = __shfl_sync(0xffffffffu, ok, ring);        // the ring's head entry
-        ok = ok && ok0;                                              // entries leave a ring in order
-        if (__any_sync(0xffffffffu, ok)) {
-          __threadfence_block();
-          uint4 v = Vec<DT>::neg_inf();
-          if (ok) {
-            v = sm.qdata[p][t][ring][slot];
-            sm.qidx[p][t][ring][slot] = QEMPTY;
-          }
-          const bool ok1 = __shfl_sync(0xffffffffu, ok, ring + 16);
-          const int took = (ok0 ? 1 : 0) + (ok1 ? 1 : 0);
-          head_r += took;
-          __syncwarp();
-          __threadfence_block();
-          if (lane < 16 && took > 0)
-            asm volatile("st.volatile.shared.u32 [%0], %1;" ::"r"(smem_u32(&sm.qhead[p][t][ring])), "r"(head_r) : "memory");
-          // admission by the vector's maximum alone: count it, keep the vector
-          const uint32_t ob = f32_order_bits(Vec<DT>::vmax(v));
-          const bool in = ok && vector_alive(ob, vi, N, tau);
-          if (in) {
-            const uint32_t code = ob >> 16;
-            atomicAdd(&hist[code - base < (uint32_t)(NB - 1) ? code - base : (uint32_t)(NB - 1)], 1u);
-          }
-          const uint32_t bin_ = __ballot_sync(0xffffffffu, in);
-          if (in) {
-            const int o = nsv + __popc(bin_ & ((1u << lane) - 1u));
-            svd[o] = v;
-            svi[o] = vi;
-          }
-          nsv += __popc(bin_);
-          tau.cnt += __popc(bin_);
-          __syncwarp();
-          if (advance_tau(tau, base, hist, k) && lane == 0)
-            sts_volatile_f32(&sm.tau[p][t], code_value(tau.code));
-          if (nsv > SVCAP - 32) {
-            // the buffer is filling up: drop what tau has ruled out; if ties keep it
-            // full, sort the kept entries into the list and go on with the exact k-th key
-            nsv = compact_survivors<DT>(svd, svi, nsv, tau, lane);
-            if (nsv > SVCAP / 2) survivors_to_list<DT, KL>(L, svd, svi, nsv, A.V, tau, stg, k, lane);
-          }
-          continue;
-        }
-      }
-      if (done) break;
-      if ((idle++ & 63u) == 0u) {
-        if (*(volatile int*)&sm.abort) return;
-        const long long now = clock64();
-        if (idle == 1u) t0 = now;
-        else if (now - t0 > kSpinLimit) { raise_timeout(sm, A.sc); return; }
-      }
-      __nanosleep(JP_TOPK_SLEEP_NS);
-    }
+    // the consumers' per-warp (max, sum) pairs of this row
+    if (!mbar_wait(&sm.row_done[p], ph, &sm.abort)) { raise_timeout(sm, A.sc); return; }
 
     if (TOPK) {
       const char* ra = (const char*)A.za + row * A.ld * Vec<DT>::ESIZE;
@@ -958,9 +898,6 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
           }
         }
       }
-      // hand the slot back clean (every ring entry was reset as it was drained)
-      if (lane < NC) sm.qhead[p][t][lane] = 0;
-      if (lane == 0) sts_volatile_f32(&sm.tau[p][t], JP_NEG_INF);
     }
 
     if (lane == 0) {
@@ -992,15 +929,16 @@ __global__ void __launch_bounds__(NTHREADS, 1) stream_kernel(StreamArgs A) {
   StreamSmem& sm = *reinterpret_cast<StreamSmem*>(smem_raw);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-  for (int i = tid; i < 2 * 2 * NC * MQ; i += NTHREADS) (&sm.qidx[0][0][0][0])[i] = QEMPTY;
-  for (int i = tid; i < 2 * 2 * NC; i += NTHREADS) (&sm.qhead[0][0][0])[i] = 0;
   if (tid == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(&sm.full[s], 1); mbar_init(&sm.empty[s], WPT); }
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(&sm.full[s], 1);
+      mbar_init(&sm.seen[0][s], WPT);
+      mbar_init(&sm.seen[1][s], WPT);
+      mbar_init(&sm.empty[s], KPL > 0 ? 2 : WPT);     // with top-k the two top-k warps of the row free the stage
+    }
     for (int p = 0; p < 2; ++p) {
       mbar_init(&sm.row_done[p], NC);
       mbar_init(&sm.slot_free[p], 2);
-      mbar_init(&sm.bound_ready[p], WPT);
-      for (int t = 0; t < 2; ++t) sm.tau[p][t] = JP_NEG_INF;
     }
     sm.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
