@@ -49,7 +49,7 @@ namespace jp {
 #define JP_TOPK_SLEEP_NS 300
 #endif
 #ifndef JP_STAGES
-#define JP_STAGES 5
+#define JP_STAGES 4
 #endif
 #ifndef JP_NG
 #define JP_NG 2
@@ -64,11 +64,12 @@ static_assert(JP_VPL % HV == 0, "a tile is taken in passes of HV vectors");
 static_assert(NC % NG == 0 && NG < JP_STAGES, "consumer groups must divide the warps and fit the ring");
 constexpr int STAGES = JP_STAGES;
 constexpr int SCAP = 384;                 // buffered keys per top-k warp (used while sorting survivors into the list)
-constexpr int SVCAP = 192;                // candidate vectors a top-k warp keeps until the row ends
-constexpr int NB = 512;                   // histogram bins: 16-bit order codes below the first tile's maximum
+constexpr int SVCAP = 256;                // candidate vectors a top-k warp keeps until the row ends
+constexpr int NB = 256;                   // histogram bins: 16-bit order codes below the warp's first tile's maximum
 constexpr int TP = TV / HV;               // passes per tensor per tile = pass maxima a top-k warp scans per tile
 static_assert(TP == 512, "a top-k lane scans 16 pass maxima per tile (4 x 16 bytes)");
-constexpr int NTOPK = 4;                  // top-k warps: (tensor, slot)
+constexpr int NTOPK = 8;                  // top-k warps: (tensor, slot, tile parity)
+constexpr int XK = 128;                   // keys a parity-0 warp can hand over (a full list of JP_MAX_TOPK)
 constexpr int NWARPS = 1 + NC + NTOPK;
 constexpr int NTHREADS = NWARPS * 32;
 constexpr uint32_t QEMPTY = 0xffffffffu;
@@ -76,15 +77,20 @@ constexpr long long kSpinLimit = 4000000000ll;   // clock cycles a wait may last
 
 struct __align__(128) StreamSmem {
   uint4 ring[STAGES][2][TV];              // [stage][tensor][vector]
-  uint4 svdata[2][2][SVCAP];              // [slot][tensor] candidate vectors still alive under tau ...
+  uint4 svdata[2][2][2][SVCAP];           // [slot][tensor][tile parity] candidate vectors still alive under tau ...
   float passmax[STAGES][2][TP];           // [stage][tensor] maximum of each consumer pass (HV vectors) of the tile
-  unsigned long long skeys[2][2][SCAP];   // [slot][tensor] keys waiting to be sorted into the list
-  uint32_t svidx[2][2][SVCAP];            // ... and the kept vectors' indices
-  uint32_t hist[2][2][NB];                // [slot][tensor] passes seen per order code of their maximum
+  unsigned long long skeys[2][2][SCAP];   // [slot][tensor] keys waiting to be sorted into the list (final step)
+  unsigned long long xkeys[2][2][XK];     // [slot][tensor] the parity-0 warp's list, if it had to sort early
+  uint32_t svidx[2][2][2][SVCAP];         // ... and the kept vectors' indices
+  uint32_t hist[2][2][2][NB];             // [slot][tensor][tile parity] passes seen per order code of their maximum
   unsigned long long full[STAGES];        // producer -> consumers: the tile's bytes have landed
-  unsigned long long seen[2][STAGES];     // [slot] consumers -> that slot's top-k warps: tile consumed, pass maxima written
+  unsigned long long seen[2][2][STAGES];  // [slot][tile parity] consumers -> top-k warps: tile consumed, pass maxima written
   unsigned long long empty[STAGES];       // -> producer: the stage may be refilled
   unsigned long long row_done[2], slot_free[2];
+  unsigned long long scan_done[2][2];     // [slot][tensor] parity-0 warp -> parity-1 warp: my part of the row is in shared memory
+  unsigned long long final_done[2][2];    // [slot][tensor] parity-1 warp -> parity-0 warp: I have read it
+  int stg_lock[2][2];                     // [slot][tensor] skeys is shared by the two parity warps while they scan
+  int xstate[2][2][4];                    // [slot][tensor] parity-0 hand-over: kept vectors, tau code, keys in xkeys
   float part_mL[2][2][NC];
   float part_s[2][2][NC];
   int abort;
@@ -440,20 +446,21 @@ __device__ __forceinline__ bool vector_alive(uint32_t ob, uint32_t vi, int n_per
 }
 
 // The highest histogram bin with at least k counted passes at or above it (0 if
-// fewer than k passes were counted).  Lane l sums bins 16 l .. 16 l + 15, a shuffle
+// fewer than k passes were counted).  Lane l sums bins 8 l .. 8 l + 7, a shuffle
 // suffix scan finds the lane in which the count crosses k, and that lane walks its
-// 16 bins from the top.
+// bins from the top.
 __device__ __forceinline__ int find_tau_bin(const uint32_t* hist, int k, int lane) {
-  const uint4* h4 = reinterpret_cast<const uint4*>(hist) + lane * 4;
-  uint32_t b[16];
+  static_assert(NB == 256, "8 bins per lane");
+  const uint4* h4 = reinterpret_cast<const uint4*>(hist) + lane * 2;
+  uint32_t b[8];
 #pragma unroll
-  for (int q = 0; q < 4; ++q) {
+  for (int q = 0; q < 2; ++q) {
     const uint4 v = h4[q];
     b[4 * q] = v.x; b[4 * q + 1] = v.y; b[4 * q + 2] = v.z; b[4 * q + 3] = v.w;
   }
   int mine = 0;
 #pragma unroll
-  for (int i = 0; i < 16; ++i) mine += (int)b[i];
+  for (int i = 0; i < 8; ++i) mine += (int)b[i];
   int suf = mine;                                   // passes in this lane's bins and all higher lanes'
 #pragma unroll
   for (int off = 1; off < 32; off <<= 1) {
@@ -466,11 +473,11 @@ __device__ __forceinline__ int find_tau_bin(const uint32_t* hist, int k, int lan
   int run = suf - mine, bin = 0;
   bool found = false;
 #pragma unroll
-  for (int i = 15; i >= 0; --i) {
+  for (int i = 7; i >= 0; --i) {
     run += (int)b[i];
     if (!found && run >= k) { bin = i; found = true; }
   }
-  return __shfl_sync(0xffffffffu, lane * 16 + bin, L);
+  return __shfl_sync(0xffffffffu, lane * 8 + bin, L);
 }
 
 // Drops the kept candidate vectors that tau has ruled out since they were kept.
@@ -681,7 +688,7 @@ __device__ void consumer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_row
       if (TOPK) {
         // the top-k warps of this row's slot take it from here; they free the stage
         __syncwarp();
-        if (lane == 0) mbar_arrive(&sm.seen[p][s]);
+        if (lane == 0) mbar_arrive(&sm.seen[p][tile & 1u][s]);
       }
       return true;
     };
@@ -730,7 +737,7 @@ __device__ void consumer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_row
 // highest histogram bin with k counted passes at or above it: k different passes
 // hold k different entries of the row, so the k-th best logit is not below it.
 template <int DT, int KPL>
-__device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, int t, int p, int lane) {
+__device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, int t, int p, int par, int lane) {
   constexpr int N = Vec<DT>::N;
   constexpr bool TOPK = KPL > 0;
   constexpr int KL = KPL > 0 ? KPL : 1;
@@ -739,13 +746,18 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
   const uint32_t ntiles = nvec > 0 ? (uint32_t)((nvec + TV - 1) / TV) : 1u;
   const int k = A.k;
   unsigned long long* stg = sm.skeys[p][t];
-  uint32_t* hist = sm.hist[p][t];
-  uint4* svd = sm.svdata[p][t];
-  uint32_t* svi = sm.svidx[p][t];
-  // A slot's `seen` barriers complete once per tile of that slot's rows, and this
-  // warp waits for every one of them in turn, so one phase bit per stage is enough.
-  // (A barrier shared by both slots would not do: a parity wait cannot tell "not yet
-  // reached" from "done" when the waiter skips phases.)
+  uint32_t* hist = sm.hist[p][t][par];
+  uint4* svd = sm.svdata[p][t][par];
+  uint32_t* svi = sm.svidx[p][t][par];
+  // The tiles of a row are shared out by parity between two warps, each with a
+  // histogram, a threshold and a survivor buffer of its own (the k-th best pass of
+  // half the tiles is still a lower bound of the row's k-th best logit).  The
+  // parity-0 warp hands its survivors over in shared memory at the end of the row;
+  // the parity-1 warp sorts both sets into the list and writes the record.
+  // A (slot, parity) `seen` barrier completes once per tile of that slot's rows with
+  // that parity, and this warp waits for every one of them in turn, so one phase bit
+  // per stage is enough.  (A barrier shared by warps that skip phases would not do: a
+  // parity wait cannot tell "not yet reached" from "done".)
   uint32_t seen_phase = 0u;
   int lr = p;
   for (int64_t it = (int64_t)blockIdx.x + (int64_t)p * gridDim.x; it < n_rows; it += 2ll * gridDim.x, lr += 2) {
@@ -767,10 +779,12 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
     if (lane == 0) zx = Vec<DT>::load_scalar(rmine, A.tokens[row]);
 
     if (TOPK) {
-      for (uint32_t tile = 0; tile < ntiles; ++tile) {
+      // the parity-1 warp must have read what this warp handed over two rows ago
+      if (par == 0 && !mbar_wait(&sm.final_done[p][t], ph ^ 1u, &sm.abort)) { raise_timeout(sm, A.sc); return; }
+      for (uint32_t tile = (uint32_t)par; tile < ntiles; tile += 2) {
         const uint32_t g = g0 + tile;
         const uint32_t s = g % STAGES;
-        if (!mbar_wait(&sm.seen[p][s], (seen_phase >> s) & 1u, &sm.abort)) { raise_timeout(sm, A.sc); return; }
+        if (!mbar_wait(&sm.seen[p][par][s], (seen_phase >> s) & 1u, &sm.abort)) { raise_timeout(sm, A.sc); return; }
         seen_phase ^= 1u << s;
         const float* pm = sm.passmax[s][t];
         const uint4* data = sm.ring[s][t];
@@ -782,8 +796,8 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
           v[4 * q] = f.x; v[4 * q + 1] = f.y; v[4 * q + 2] = f.z; v[4 * q + 3] = f.w;
         }
         uint32_t hit = 0u;
-        if (tile == 0) {
-          // a new row: the histogram covers the NB order codes below this tile's maximum
+        if (tile == (uint32_t)par) {
+          // this warp's first tile of a new row: the histogram covers the NB order codes below this tile's maximum
           // (everything lower shares bin 0, which stands for "no threshold"); every pass
           // of the tile is counted, then the threshold is read off the histogram
           float mx = v[0];
@@ -856,7 +870,20 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
               // the buffer is filling up: drop what the threshold has ruled out; if ties keep
               // it full, sort the kept entries into the list and go on with the exact k-th key
               nsv = compact_survivors<DT>(svd, svi, nsv, tau, lane);
-              if (nsv > SVCAP / 2) survivors_to_list<DT, KL>(L, svd, svi, nsv, A.V, tau, stg, k, lane);
+              if (nsv > SVCAP / 2) {
+                // the key buffer is shared with the other parity's warp: take it (bounded wait)
+                int got = 0;
+                if (lane == 0) {
+                  for (int spins = 0; spins < (1 << 24) && !got; ++spins) got = atomicCAS(&sm.stg_lock[p][t], 0, 1) == 0;
+                }
+                got = __shfl_sync(0xffffffffu, got, 0);
+                if (!got) { raise_timeout(sm, A.sc); return; }
+                __threadfence_block();
+                survivors_to_list<DT, KL>(L, svd, svi, nsv, A.V, tau, stg, k, lane);
+                __syncwarp();
+                __threadfence_block();
+                if (lane == 0) atomicExch(&sm.stg_lock[p][t], 0);
+              }
             }
           }
         }
@@ -865,12 +892,33 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
       }
     }
 
+    if (par == 0) {
+      // hand this half of the row over: the survivors stay where they are; a list that
+      // had to be sorted early goes to xkeys
+      int nkeys = 0;
+      if (tau.key != 0ull) {
+#pragma unroll
+        for (int j = 0; j < KL; ++j) sm.xkeys[p][t][lane * KL + j] = L[j];
+        nkeys = 32 * KL;
+      }
+      if (lane == 0) { sm.xstate[p][t][0] = nsv; sm.xstate[p][t][1] = (int)tau.code; sm.xstate[p][t][2] = nkeys; }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sm.scan_done[p][t]);
+      continue;
+    }
+
     // the consumers' per-warp (max, sum) pairs of this row
     if (!mbar_wait(&sm.row_done[p], ph, &sm.abort)) { raise_timeout(sm, A.sc); return; }
 
     if (TOPK) {
       const char* ra = (const char*)A.za + row * A.ld * Vec<DT>::ESIZE;
       const char* rp = (const char*)A.zp + row * A.ld * Vec<DT>::ESIZE;
+      // the other half of the row; both thresholds are lower bounds of the row's k-th best
+      if (!mbar_wait(&sm.scan_done[p][t], ph, &sm.abort)) { raise_timeout(sm, A.sc); return; }
+      int n0 = sm.xstate[p][t][0];
+      const uint32_t code0 = (uint32_t)sm.xstate[p][t][1];
+      const int nk0 = sm.xstate[p][t][2];
+      if (code0 > tau.code) tau.code = code0;
       if (tail > 0) {                 // the ragged end of the row joins the kept vectors
         if (lane == 0) {
           svd[nsv] = load_tail_vector<DT>(rmine, nvec * N, tail);
@@ -881,6 +929,21 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
       }
       nsv = compact_survivors<DT>(svd, svi, nsv, tau, lane);
       survivors_to_list<DT, KL>(L, svd, svi, nsv, A.V, tau, stg, k, lane);
+      n0 = compact_survivors<DT>(sm.svdata[p][t][0], sm.svidx[p][t][0], n0, tau, lane);
+      survivors_to_list<DT, KL>(L, sm.svdata[p][t][0], sm.svidx[p][t][0], n0, A.V, tau, stg, k, lane);
+      if (nk0 > 0) {
+        int staged = 0;
+        for (int b = 0; b < nk0; b += 32) {
+          const unsigned long long key = sm.xkeys[p][t][b + lane];
+          const bool keep = key > tau.key;
+          const uint32_t m = __ballot_sync(0xffffffffu, keep);
+          if (keep) stg[staged + __popc(m & ((1u << lane) - 1u))] = key;
+          staged += __popc(m);
+        }
+        tau.key = merge_all<KL>(L, stg, staged, k, lane);
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sm.final_done[p][t]);     // the parity-0 warp may reuse its buffers
       // the record: this tensor's list, best first, every entry with both logits
 #pragma unroll
       for (int j = 0; j < KL; ++j) {
@@ -932,13 +995,13 @@ __global__ void __launch_bounds__(NTHREADS, 1) stream_kernel(StreamArgs A) {
   if (tid == 0) {
     for (int s = 0; s < STAGES; ++s) {
       mbar_init(&sm.full[s], 1);
-      mbar_init(&sm.seen[0][s], WPT);
-      mbar_init(&sm.seen[1][s], WPT);
+      for (int q = 0; q < 4; ++q) mbar_init(&sm.seen[q >> 1][q & 1][s], WPT);
       mbar_init(&sm.empty[s], KPL > 0 ? 2 : WPT);     // with top-k the two top-k warps of the row free the stage
     }
     for (int p = 0; p < 2; ++p) {
       mbar_init(&sm.row_done[p], NC);
       mbar_init(&sm.slot_free[p], 2);
+      for (int t = 0; t < 2; ++t) { mbar_init(&sm.scan_done[p][t], 1); mbar_init(&sm.final_done[p][t], 1); sm.stg_lock[p][t] = 0; }
     }
     sm.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -952,7 +1015,8 @@ __global__ void __launch_bounds__(NTHREADS, 1) stream_kernel(StreamArgs A) {
     consumer_loop<DT, (KPL > 0)>(A, sm, n_rows, warp - 1, lane);
   } else {
     const int tw = warp - 1 - NC;
-    topk_loop<DT, KPL>(A, sm, n_rows, tw & 1, tw >> 1, lane);
+    // without top-k there is nothing to share out: the parity-0 warps leave
+    if (KPL > 0 || (tw >> 2) == 1) topk_loop<DT, KPL>(A, sm, n_rows, tw & 1, (tw >> 1) & 1, tw >> 2, lane);
   }
 }
 
