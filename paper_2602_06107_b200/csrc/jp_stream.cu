@@ -49,7 +49,7 @@ namespace jp {
 #define JP_TOPK_SLEEP_NS 300
 #endif
 #ifndef JP_STAGES
-#define JP_STAGES 4
+#define JP_STAGES 5
 #endif
 #ifndef JP_NG
 #define JP_NG 2
@@ -64,7 +64,7 @@ static_assert(JP_VPL % HV == 0, "a tile is taken in passes of HV vectors");
 static_assert(NC % NG == 0 && NG < JP_STAGES, "consumer groups must divide the warps and fit the ring");
 constexpr int STAGES = JP_STAGES;
 constexpr int SCAP = 384;                 // buffered keys per top-k warp (used while sorting survivors into the list)
-constexpr int SVCAP = 256;                // candidate vectors a top-k warp keeps until the row ends
+constexpr int SVCAP = 320;                // candidate passes a top-k warp keeps until the row ends
 constexpr int NB = 256;                   // histogram bins: 16-bit order codes below the warp's first tile's maximum
 constexpr int TP = TV / HV;               // passes per tensor per tile = pass maxima a top-k warp scans per tile
 static_assert(TP == 512, "a top-k lane scans 16 pass maxima per tile (4 x 16 bytes)");
@@ -77,11 +77,11 @@ constexpr long long kSpinLimit = 4000000000ll;   // clock cycles a wait may last
 
 struct __align__(128) StreamSmem {
   uint4 ring[STAGES][2][TV];              // [stage][tensor][vector]
-  uint4 svdata[2][2][2][SVCAP];           // [slot][tensor][tile parity] candidate vectors still alive under tau ...
   float passmax[STAGES][2][TP];           // [stage][tensor] maximum of each consumer pass (HV vectors) of the tile
   unsigned long long skeys[2][2][SCAP];   // [slot][tensor] keys waiting to be sorted into the list (final step)
   unsigned long long xkeys[2][2][XK];     // [slot][tensor] the parity-0 warp's list, if it had to sort early
-  uint32_t svidx[2][2][2][SVCAP];         // ... and the kept vectors' indices
+  uint32_t svpass[2][2][2][SVCAP];        // [slot][tensor][tile parity] candidate passes still alive under tau: tile * TP + entry ...
+  float svmax[2][2][2][SVCAP];            // ... and their maxima
   uint32_t hist[2][2][2][NB];             // [slot][tensor][tile parity] passes seen per order code of their maximum
   unsigned long long full[STAGES];        // producer -> consumers: the tile's bytes have landed
   unsigned long long seen[2][2][STAGES];  // [slot][tile parity] consumers -> top-k warps: tile consumed, pass maxima written
@@ -437,12 +437,19 @@ __device__ __forceinline__ uint32_t order_code(float v) { return f32_order_bits(
 // low edge of a code's bin, as a logit
 __device__ __forceinline__ float code_value(uint32_t code) { return order_bits_f32(code << 16); }
 
-// Can the vector with index vi and maximum order bits `ob` still hold one of the k best?
-__device__ __forceinline__ bool vector_alive(uint32_t ob, uint32_t vi, int n_per_vec, const Tau& tau) {
+// First vector index of pass `id` (= tile * TP + entry) and the step to its next vector.
+__device__ __forceinline__ uint32_t pass_first_vector(uint32_t id) {
+  const uint32_t tile = id / TP, e = id % TP;
+  return tile * TV + (e / (WPT * 32)) * HV * (WPT * 32) + e % (WPT * 32);
+}
+
+// Can the pass with maximum order bits `ob` still hold one of the k best?
+__device__ __forceinline__ bool pass_alive(uint32_t ob, uint32_t id, int n_per_vec, const Tau& tau) {
   if ((ob >> 16) < tau.code) return false;
   if (tau.key == 0ull) return true;
-  // its best possible entry: the maximum at the vector's first index
-  return (((unsigned long long)ob << 32) | (unsigned long long)(uint32_t)(~(vi * (uint32_t)n_per_vec))) > tau.key;
+  // its best possible entry: the maximum at the first index of the pass's first vector
+  const uint32_t idx = pass_first_vector(id) * (uint32_t)n_per_vec;
+  return (((unsigned long long)ob << 32) | (unsigned long long)(uint32_t)(~idx)) > tau.key;
 }
 
 // The highest histogram bin with at least k counted passes at or above it (0 if
@@ -480,28 +487,27 @@ __device__ __forceinline__ int find_tau_bin(const uint32_t* hist, int k, int lan
   return __shfl_sync(0xffffffffu, lane * 8 + bin, L);
 }
 
-// Drops the kept candidate vectors that tau has ruled out since they were kept.
-template <int DT>
-__device__ __noinline__ int compact_survivors(uint4* svd, uint32_t* svi, int nsv, Tau tau, int lane) {
+// Drops the kept candidate passes that tau has ruled out since they were kept.
+__device__ __noinline__ int compact_survivors(uint32_t* svp, float* svm, int nsv, Tau tau, int n_per_vec, int lane) {
   int out = 0;
   for (int b = 0; b < nsv; b += 32) {
     const int i = b + lane;
-    uint4 v = Vec<DT>::neg_inf();
-    uint32_t vi = 0u;
+    uint32_t id = 0u;
+    float m = 0.f;
     bool keep = false;
     if (i < nsv) {
-      v = svd[i];
-      vi = svi[i];
-      keep = vector_alive(f32_order_bits(Vec<DT>::vmax(v)), vi, Vec<DT>::N, tau);
+      id = svp[i];
+      m = svm[i];
+      keep = pass_alive(f32_order_bits(m), id, n_per_vec, tau);
     }
-    const uint32_t m = __ballot_sync(0xffffffffu, keep);
+    const uint32_t bm = __ballot_sync(0xffffffffu, keep);
     __syncwarp();
     if (keep) {
-      const int o = out + __popc(m & ((1u << lane) - 1u));
-      svd[o] = v;
-      svi[o] = vi;
+      const int o = out + __popc(bm & ((1u << lane) - 1u));
+      svp[o] = id;
+      svm[o] = m;
     }
-    out += __popc(m);
+    out += __popc(bm);
     __syncwarp();
   }
   return out;
@@ -543,20 +549,31 @@ __device__ __noinline__ unsigned long long merge_all(unsigned long long (&L)[KPL
   return kth_key<KPL>(L, k);
 }
 
-// Sorts the entries of every kept vector into the list (exact from here on:
-// tau.key becomes the list's k-th key) and empties the survivor buffer.
+// Sorts the entries of every kept pass into the list (exact from here on: tau.key
+// becomes the list's k-th key) and empties the survivor buffer.  The vectors of a
+// pass are read back from memory (they left the ring long ago; a few hundred
+// 16-byte reads per row, mostly L2 hits).
 template <int DT, int KPL>
-__device__ __noinline__ void survivors_to_list(unsigned long long (&L)[KPL], const uint4* svd, const uint32_t* svi,
-                                               int& nsv, int64_t V, Tau& tau, unsigned long long* stg, int k,
-                                               int lane) {
+__device__ __noinline__ void survivors_to_list(unsigned long long (&L)[KPL], const uint32_t* svp, int& nsv,
+                                               const char* row, int64_t nvec, int64_t V, Tau& tau,
+                                               unsigned long long* stg, int k, int lane) {
   int staged = 0;
   for (int b = 0; b < nsv; b += 32) {
     const int i = b + lane;
-    uint4 v = Vec<DT>::neg_inf();
-    uint32_t vi = 0u;
-    if (i < nsv) { v = svd[i]; vi = svi[i]; }
-    staged = stage_entries<DT>(v, vi, i < nsv, V, tau, stg, staged, lane);
-    if (staged > SCAP - 32 * Vec<DT>::N) tau.key = merge_all<KPL>(L, stg, staged, k, lane);
+    const uint32_t v0 = i < nsv ? pass_first_vector(svp[i]) : 0u;
+    uint4 v[HV];
+    bool in[HV];
+#pragma unroll
+    for (int j = 0; j < HV; ++j) {
+      const uint32_t vi = v0 + j * (WPT * 32);
+      in[j] = i < nsv && (int64_t)vi < nvec;
+      v[j] = in[j] ? ldg_stream((const uint4*)row + vi) : Vec<DT>::neg_inf();
+    }
+#pragma unroll
+    for (int j = 0; j < HV; ++j) {
+      staged = stage_entries<DT>(v[j], v0 + j * (WPT * 32), in[j], V, tau, stg, staged, lane);
+      if (staged > SCAP - 32 * Vec<DT>::N) tau.key = merge_all<KPL>(L, stg, staged, k, lane);
+    }
   }
   tau.key = merge_all<KPL>(L, stg, staged, k, lane);
   nsv = 0;
@@ -747,8 +764,8 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
   const int k = A.k;
   unsigned long long* stg = sm.skeys[p][t];
   uint32_t* hist = sm.hist[p][t][par];
-  uint4* svd = sm.svdata[p][t][par];
-  uint32_t* svi = sm.svidx[p][t][par];
+  uint32_t* svp = sm.svpass[p][t][par];
+  float* svm = sm.svmax[p][t][par];
   // The tiles of a row are shared out by parity between two warps, each with a
   // histogram, a threshold and a survivor buffer of its own (the k-th best pass of
   // half the tiles is still a lower bound of the row's k-th best logit).  The
@@ -787,7 +804,6 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
         if (!mbar_wait(&sm.seen[p][par][s], (seen_phase >> s) & 1u, &sm.abort)) { raise_timeout(sm, A.sc); return; }
         seen_phase ^= 1u << s;
         const float* pm = sm.passmax[s][t];
-        const uint4* data = sm.ring[s][t];
         // this lane's 16 pass maxima: entries q * 128 + lane * 4 + c
         float v[16];
 #pragma unroll
@@ -839,51 +855,45 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
             tau_val = bin > 0 ? code_value(tau.code) : JP_NEG_INF;
           }
         }
-        // the vectors behind the hits: keep those that can still hold one of the k best
+        // keep the passes behind the hits that can still hold one of the k best: only
+        // their place and their maximum; their vectors are read back when the row ends
         while (__any_sync(0xffffffffu, hit != 0u)) {
-          int e = 0;
           const bool have = hit != 0u;
+          uint32_t id = 0u;
+          float m = JP_NEG_INF;
           if (have) {
             const int i = __ffs(hit) - 1;
             hit &= hit - 1u;
-            e = (i >> 2) * 128 + lane * 4 + (i & 3);          // pass entry: pass h = e / (WPT*32), lane slot e % (WPT*32)
+            const int e = (i >> 2) * 128 + lane * 4 + (i & 3);
+            id = tile * TP + (uint32_t)e;
+            m = pm[e];
           }
-#pragma unroll
-          for (int j = 0; j < HV; ++j) {
-            const uint32_t pos = (uint32_t)((e / (WPT * 32)) * HV + j) * (WPT * 32) + (uint32_t)(e % (WPT * 32));
-            const uint32_t vi = tile * TV + pos;
-            uint4 vec = Vec<DT>::neg_inf();
-            bool in = false;
-            if (have && (int64_t)vi < nvec) {
-              vec = data[pos];
-              in = vector_alive(f32_order_bits(Vec<DT>::vmax(vec)), vi, N, tau);
-            }
-            const uint32_t m = __ballot_sync(0xffffffffu, in);
-            if (in) {
-              const int o = nsv + __popc(m & ((1u << lane) - 1u));
-              svd[o] = vec;
-              svi[o] = vi;
-            }
-            nsv += __popc(m);
-            __syncwarp();
-            if (nsv > SVCAP - 32) {
-              // the buffer is filling up: drop what the threshold has ruled out; if ties keep
-              // it full, sort the kept entries into the list and go on with the exact k-th key
-              nsv = compact_survivors<DT>(svd, svi, nsv, tau, lane);
-              if (nsv > SVCAP / 2) {
-                // the key buffer is shared with the other parity's warp: take it (bounded wait)
-                int got = 0;
-                if (lane == 0) {
-                  for (int spins = 0; spins < (1 << 24) && !got; ++spins) got = atomicCAS(&sm.stg_lock[p][t], 0, 1) == 0;
-                }
-                got = __shfl_sync(0xffffffffu, got, 0);
-                if (!got) { raise_timeout(sm, A.sc); return; }
-                __threadfence_block();
-                survivors_to_list<DT, KL>(L, svd, svi, nsv, A.V, tau, stg, k, lane);
-                __syncwarp();
-                __threadfence_block();
-                if (lane == 0) atomicExch(&sm.stg_lock[p][t], 0);
+          const bool in = have && pass_alive(f32_order_bits(m), id, N, tau);
+          const uint32_t bm = __ballot_sync(0xffffffffu, in);
+          if (in) {
+            const int o = nsv + __popc(bm & ((1u << lane) - 1u));
+            svp[o] = id;
+            svm[o] = m;
+          }
+          nsv += __popc(bm);
+          __syncwarp();
+          if (nsv > SVCAP - 32) {
+            // the buffer is filling up: drop what the threshold has ruled out; if ties keep
+            // it full, sort the kept entries into the list and go on with the exact k-th key
+            nsv = compact_survivors(svp, svm, nsv, tau, N, lane);
+            if (nsv > SVCAP / 2) {
+              // the key buffer is shared with the other parity's warp: take it (bounded wait)
+              int got = 0;
+              if (lane == 0) {
+                for (int spins = 0; spins < (1 << 24) && !got; ++spins) got = atomicCAS(&sm.stg_lock[p][t], 0, 1) == 0;
               }
+              got = __shfl_sync(0xffffffffu, got, 0);
+              if (!got) { raise_timeout(sm, A.sc); return; }
+              __threadfence_block();
+              survivors_to_list<DT, KL>(L, svp, nsv, rmine, nvec, A.V, tau, stg, k, lane);
+              __syncwarp();
+              __threadfence_block();
+              if (lane == 0) atomicExch(&sm.stg_lock[p][t], 0);
             }
           }
         }
@@ -919,18 +929,16 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
       const uint32_t code0 = (uint32_t)sm.xstate[p][t][1];
       const int nk0 = sm.xstate[p][t][2];
       if (code0 > tau.code) tau.code = code0;
-      if (tail > 0) {                 // the ragged end of the row joins the kept vectors
-        if (lane == 0) {
-          svd[nsv] = load_tail_vector<DT>(rmine, nvec * N, tail);
-          svi[nsv] = (uint32_t)nvec;
-        }
-        nsv += 1;
-        __syncwarp();
+      nsv = compact_survivors(svp, svm, nsv, tau, N, lane);
+      survivors_to_list<DT, KL>(L, svp, nsv, rmine, nvec, A.V, tau, stg, k, lane);
+      n0 = compact_survivors(sm.svpass[p][t][0], sm.svmax[p][t][0], n0, tau, N, lane);
+      survivors_to_list<DT, KL>(L, sm.svpass[p][t][0], n0, rmine, nvec, A.V, tau, stg, k, lane);
+      if (tail > 0) {                 // the ragged end of the row
+        uint4 v = Vec<DT>::neg_inf();
+        if (lane == 0) v = load_tail_vector<DT>(rmine, nvec * N, tail);
+        int staged = stage_entries<DT>(v, (uint32_t)nvec, lane == 0, A.V, tau, stg, 0, lane);
+        tau.key = merge_all<KL>(L, stg, staged, k, lane);
       }
-      nsv = compact_survivors<DT>(svd, svi, nsv, tau, lane);
-      survivors_to_list<DT, KL>(L, svd, svi, nsv, A.V, tau, stg, k, lane);
-      n0 = compact_survivors<DT>(sm.svdata[p][t][0], sm.svidx[p][t][0], n0, tau, lane);
-      survivors_to_list<DT, KL>(L, sm.svdata[p][t][0], sm.svidx[p][t][0], n0, A.V, tau, stg, k, lane);
       if (nk0 > 0) {
         int staged = 0;
         for (int b = 0; b < nk0; b += 32) {
