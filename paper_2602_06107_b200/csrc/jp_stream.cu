@@ -63,13 +63,12 @@ constexpr int HV = 2;                     // vectors per tensor a lane holds at 
 static_assert(JP_VPL % HV == 0, "a tile is taken in passes of HV vectors");
 static_assert(NC % NG == 0 && NG < JP_STAGES, "consumer groups must divide the warps and fit the ring");
 constexpr int STAGES = JP_STAGES;
-constexpr int SCAP = 384;                 // buffered keys per top-k warp (used while sorting survivors into the list)
-constexpr int SVCAP = 320;                // candidate passes a top-k warp keeps until the row ends
+constexpr int SCAP = 288;                 // buffered keys per top-k warp (used while sorting survivors into the list)
+constexpr int SVCAP = 288;                // candidate passes a top-k warp keeps until the row ends
 constexpr int NB = 256;                   // histogram bins: 16-bit order codes below the warp's first tile's maximum
 constexpr int TP = TV / HV;               // passes per tensor per tile = pass maxima a top-k warp scans per tile
 static_assert(TP == 512, "a top-k lane scans 16 pass maxima per tile (4 x 16 bytes)");
 constexpr int NTOPK = 8;                  // top-k warps: (tensor, slot, tile parity)
-constexpr int XK = 128;                   // keys a parity-0 warp can hand over (a full list of JP_MAX_TOPK)
 constexpr int NWARPS = 1 + NC + NTOPK;
 constexpr int NTHREADS = NWARPS * 32;
 constexpr uint32_t QEMPTY = 0xffffffffu;
@@ -78,8 +77,7 @@ constexpr long long kSpinLimit = 4000000000ll;   // clock cycles a wait may last
 struct __align__(128) StreamSmem {
   uint4 ring[STAGES][2][TV];              // [stage][tensor][vector]
   float passmax[STAGES][2][TP];           // [stage][tensor] maximum of each consumer pass (HV vectors) of the tile
-  unsigned long long skeys[2][2][SCAP];   // [slot][tensor] keys waiting to be sorted into the list (final step)
-  unsigned long long xkeys[2][2][XK];     // [slot][tensor] the parity-0 warp's list, if it had to sort early
+  unsigned long long skeys[2][2][2][SCAP];  // [slot][tensor][tile parity] keys waiting to be sorted into the list; the parity-0 warp leaves its finished list here
   uint32_t svpass[2][2][2][SVCAP];        // [slot][tensor][tile parity] candidate passes still alive under tau: tile * TP + entry ...
   float svmax[2][2][2][SVCAP];            // ... and their maxima
   uint32_t hist[2][2][2][NB];             // [slot][tensor][tile parity] passes seen per order code of their maximum
@@ -89,7 +87,6 @@ struct __align__(128) StreamSmem {
   unsigned long long row_done[2], slot_free[2];
   unsigned long long scan_done[2][2];     // [slot][tensor] parity-0 warp -> parity-1 warp: my part of the row is in shared memory
   unsigned long long final_done[2][2];    // [slot][tensor] parity-1 warp -> parity-0 warp: I have read it
-  int stg_lock[2][2];                     // [slot][tensor] skeys is shared by the two parity warps while they scan
   int xstate[2][2][4];                    // [slot][tensor] parity-0 hand-over: kept vectors, tau code, keys in xkeys
   float part_mL[2][2][NC];
   float part_s[2][2][NC];
@@ -437,6 +434,18 @@ __device__ __forceinline__ uint32_t order_code(float v) { return f32_order_bits(
 // low edge of a code's bin, as a logit
 __device__ __forceinline__ float code_value(uint32_t code) { return order_bits_f32(code << 16); }
 
+// v[i] for a run-time i in 0..15 without indexing the register array (a select tree).
+__device__ __forceinline__ float select16(const float (&v)[16], int i) {
+  float a[8], b[4], c[2];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) a[j] = (i & 1) ? v[2 * j + 1] : v[2 * j];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) b[j] = (i & 2) ? a[2 * j + 1] : a[2 * j];
+#pragma unroll
+  for (int j = 0; j < 2; ++j) c[j] = (i & 4) ? b[2 * j + 1] : b[2 * j];
+  return (i & 8) ? c[1] : c[0];
+}
+
 // First vector index of pass `id` (= tile * TP + entry) and the step to its next vector.
 __device__ __forceinline__ uint32_t pass_first_vector(uint32_t id) {
   const uint32_t tile = id / TP, e = id % TP;
@@ -762,7 +771,7 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
   const int tail = (int)(A.V - nvec * N);
   const uint32_t ntiles = nvec > 0 ? (uint32_t)((nvec + TV - 1) / TV) : 1u;
   const int k = A.k;
-  unsigned long long* stg = sm.skeys[p][t];
+  unsigned long long* stg = sm.skeys[p][t][par];
   uint32_t* hist = sm.hist[p][t][par];
   uint32_t* svp = sm.svpass[p][t][par];
   float* svm = sm.svmax[p][t][par];
@@ -811,6 +820,10 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
           const float4 f = reinterpret_cast<const float4*>(pm)[q * 32 + lane];
           v[4 * q] = f.x; v[4 * q + 1] = f.y; v[4 * q + 2] = f.z; v[4 * q + 3] = f.w;
         }
+        // everything this warp needs of the tile is in registers: the stage (logits and
+        // pass maxima) may be refilled once the other tensor's warp says the same
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.empty[s]);
         uint32_t hit = 0u;
         if (tile == (uint32_t)par) {
           // this warp's first tile of a new row: the histogram covers the NB order codes below this tile's maximum
@@ -844,7 +857,7 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
               if (hcount) {
                 const int i = __ffs(hcount) - 1;
                 hcount &= hcount - 1u;
-                const uint32_t code = order_code(pm[(i >> 2) * 128 + lane * 4 + (i & 3)]);
+                const uint32_t code = order_code(select16(v, i));
                 const uint32_t bin = code > base ? code - base : 0u;
                 atomicAdd(&hist[bin < (uint32_t)(NB - 1) ? bin : (uint32_t)(NB - 1)], 1u);
               }
@@ -866,7 +879,7 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
             hit &= hit - 1u;
             const int e = (i >> 2) * 128 + lane * 4 + (i & 3);
             id = tile * TP + (uint32_t)e;
-            m = pm[e];
+            m = select16(v, i);
           }
           const bool in = have && pass_alive(f32_order_bits(m), id, N, tau);
           const uint32_t bm = __ballot_sync(0xffffffffu, in);
@@ -882,38 +895,25 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
             // it full, sort the kept entries into the list and go on with the exact k-th key
             nsv = compact_survivors(svp, svm, nsv, tau, N, lane);
             if (nsv > SVCAP / 2) {
-              // the key buffer is shared with the other parity's warp: take it (bounded wait)
-              int got = 0;
-              if (lane == 0) {
-                for (int spins = 0; spins < (1 << 24) && !got; ++spins) got = atomicCAS(&sm.stg_lock[p][t], 0, 1) == 0;
-              }
-              got = __shfl_sync(0xffffffffu, got, 0);
-              if (!got) { raise_timeout(sm, A.sc); return; }
-              __threadfence_block();
               survivors_to_list<DT, KL>(L, svp, nsv, rmine, nvec, A.V, tau, stg, k, lane);
-              __syncwarp();
-              __threadfence_block();
-              if (lane == 0) atomicExch(&sm.stg_lock[p][t], 0);
             }
           }
         }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sm.empty[s]);       // both tensors' warps done: the stage may be refilled
       }
     }
 
     if (par == 0) {
-      // hand this half of the row over: the survivors stay where they are; a list that
-      // had to be sorted early goes to xkeys
-      int nkeys = 0;
-      if (tau.key != 0ull) {
+      // this half of the row: sort the survivors into the list and leave the list in
+      // this warp's key buffer for the parity-1 warp
+      if (TOPK) {
+        nsv = compact_survivors(svp, svm, nsv, tau, N, lane);
+        survivors_to_list<DT, KL>(L, svp, nsv, rmine, nvec, A.V, tau, stg, k, lane);
 #pragma unroll
-        for (int j = 0; j < KL; ++j) sm.xkeys[p][t][lane * KL + j] = L[j];
-        nkeys = 32 * KL;
+        for (int j = 0; j < KL; ++j) stg[lane * KL + j] = L[j];
+        if (lane == 0) { sm.xstate[p][t][0] = 0; sm.xstate[p][t][1] = (int)tau.code; sm.xstate[p][t][2] = 32 * KL; }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.scan_done[p][t]);
       }
-      if (lane == 0) { sm.xstate[p][t][0] = nsv; sm.xstate[p][t][1] = (int)tau.code; sm.xstate[p][t][2] = nkeys; }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&sm.scan_done[p][t]);
       continue;
     }
 
@@ -923,16 +923,12 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
     if (TOPK) {
       const char* ra = (const char*)A.za + row * A.ld * Vec<DT>::ESIZE;
       const char* rp = (const char*)A.zp + row * A.ld * Vec<DT>::ESIZE;
-      // the other half of the row; both thresholds are lower bounds of the row's k-th best
-      if (!mbar_wait(&sm.scan_done[p][t], ph, &sm.abort)) { raise_timeout(sm, A.sc); return; }
-      int n0 = sm.xstate[p][t][0];
-      const uint32_t code0 = (uint32_t)sm.xstate[p][t][1];
-      const int nk0 = sm.xstate[p][t][2];
-      if (code0 > tau.code) tau.code = code0;
+      // this warp's half of the row into its list ...
       nsv = compact_survivors(svp, svm, nsv, tau, N, lane);
       survivors_to_list<DT, KL>(L, svp, nsv, rmine, nvec, A.V, tau, stg, k, lane);
-      n0 = compact_survivors(sm.svpass[p][t][0], sm.svmax[p][t][0], n0, tau, N, lane);
-      survivors_to_list<DT, KL>(L, sm.svpass[p][t][0], n0, rmine, nvec, A.V, tau, stg, k, lane);
+      // ... then the other half's list
+      if (!mbar_wait(&sm.scan_done[p][t], ph, &sm.abort)) { raise_timeout(sm, A.sc); return; }
+      const int nk0 = sm.xstate[p][t][2];
       if (tail > 0) {                 // the ragged end of the row
         uint4 v = Vec<DT>::neg_inf();
         if (lane == 0) v = load_tail_vector<DT>(rmine, nvec * N, tail);
@@ -942,7 +938,7 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
       if (nk0 > 0) {
         int staged = 0;
         for (int b = 0; b < nk0; b += 32) {
-          const unsigned long long key = sm.xkeys[p][t][b + lane];
+          const unsigned long long key = sm.skeys[p][t][0][b + lane];
           const bool keep = key > tau.key;
           const uint32_t m = __ballot_sync(0xffffffffu, keep);
           if (keep) stg[staged + __popc(m & ((1u << lane) - 1u))] = key;
@@ -1009,7 +1005,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) stream_kernel(StreamArgs A) {
     for (int p = 0; p < 2; ++p) {
       mbar_init(&sm.row_done[p], NC);
       mbar_init(&sm.slot_free[p], 2);
-      for (int t = 0; t < 2; ++t) { mbar_init(&sm.scan_done[p][t], 1); mbar_init(&sm.final_done[p][t], 1); sm.stg_lock[p][t] = 0; }
+      for (int t = 0; t < 2; ++t) { mbar_init(&sm.scan_done[p][t], 1); mbar_init(&sm.final_done[p][t], 1); }
     }
     sm.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
