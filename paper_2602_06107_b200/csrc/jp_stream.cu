@@ -599,35 +599,45 @@ __device__ void producer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_row
   constexpr int N = Vec<DT>::N;
   const int64_t nvec = A.V / N;
   const int ntiles = nvec > 0 ? (int)((nvec + TV - 1) / TV) : 1;
-  long long g = 0;
+  const uint32_t last_bytes = (uint32_t)((nvec - (int64_t)(ntiles - 1) * TV) * 16);   // 0 only when nvec == 0
+  const int64_t pitch = A.ld * Vec<DT>::ESIZE;
+  // This lane is the one latency-critical thread of the CTA: a freed stage waits for it.
+  // Stage and phase advance by increments, addresses by additions, and the next row's
+  // index is fetched one row ahead.
+  uint32_t s = 0, ph = 0, armed = 0;
   bool ok = true;
-  for (int64_t it = blockIdx.x; it < n_rows && ok; it += gridDim.x) {
-    const int64_t row = A.list[it];
-    const char* ra = (const char*)A.za + row * A.ld * Vec<DT>::ESIZE;
-    const char* rp = (const char*)A.zp + row * A.ld * Vec<DT>::ESIZE;
-    for (int tile = 0; tile < ntiles; ++tile, ++g) {
-      const int s = (int)(g % STAGES);
-      const uint32_t ph = (uint32_t)((g / STAGES) & 1);
+  int64_t it = blockIdx.x;
+  int64_t row = it < n_rows ? A.list[it] : 0;
+  while (it < n_rows && ok) {
+    const char* ra = (const char*)A.za + row * pitch;
+    const char* rp = (const char*)A.zp + row * pitch;
+    it += gridDim.x;
+    if (it < n_rows) row = A.list[it];
+    for (int tile = 0; tile < ntiles; ++tile, ra += TV * 16, rp += TV * 16) {
       if (!mbar_wait(&sm.empty[s], ph ^ 1u, &sm.abort)) { ok = false; break; }
-      const int64_t v0 = (int64_t)tile * TV;
-      const int64_t nv = nvec - v0 < TV ? nvec - v0 : TV;
-      const uint32_t bytes = (uint32_t)(nv > 0 ? nv * 16 : 0);
+      const uint32_t bytes = tile == ntiles - 1 ? last_bytes : (uint32_t)(TV * 16);
       if (bytes > 0) {
         mbar_arrive_expect_tx(&sm.full[s], 2u * bytes);
-        bulk_g2s(&sm.ring[s][0][0], ra + v0 * 16, bytes, &sm.full[s]);
-        bulk_g2s(&sm.ring[s][1][0], rp + v0 * 16, bytes, &sm.full[s]);
+        bulk_g2s(&sm.ring[s][0][0], ra, bytes, &sm.full[s]);
+        bulk_g2s(&sm.ring[s][1][0], rp, bytes, &sm.full[s]);
       } else {
         mbar_arrive(&sm.full[s]);
       }
+      ++armed;
+      if (++s == STAGES) { s = 0; ph ^= 1u; }
     }
   }
   if (!ok) {
-    // Leave no copy in flight: every stage this lane armed and nobody consumed
-    // completes once its bytes have landed.
+    // Leave no copy in flight: the stages this lane armed last and nobody consumed
+    // complete once their bytes have landed.
     raise_timeout(sm, A.sc);
-    for (long long h = g > STAGES ? g - STAGES : 0; h < g; ++h) {
+    const uint32_t n_back = armed < (uint32_t)STAGES ? armed : (uint32_t)STAGES;
+    for (uint32_t h = 0; h < n_back; ++h) {
+      // walk back from the stage armed last
+      if (s == 0) { s = STAGES; ph ^= 1u; }
+      --s;
       const long long t0 = clock64();
-      while (!mbar_try_wait(&sm.full[h % STAGES], (uint32_t)((h / STAGES) & 1)))
+      while (!mbar_try_wait(&sm.full[s], ph))
         if (clock64() - t0 > kSpinLimit) break;
     }
   }
