@@ -224,13 +224,32 @@ __global__ void __launch_bounds__(EPI_NT) epilogue_kernel(EpilogueArgs A) {
 // Every block folds the same partial sums in the same order, then writes its rows.
 __global__ void __launch_bounds__(EPI_NT) finalize_kernel(EpilogueArgs A) {
   __shared__ double s_kappa;
-  if (threadIdx.x == 0) {
-    long long nv = 0, na = 0;
-    double szk = 0.0, sa = 0.0;
-    for (int b = 0; b < A.n_part; ++b) {
-      nv += A.part->n_valid[b]; na += A.part->n_accept[b];
-      szk += A.part->sum_zk[b]; sa += A.part->sum_a[b];
+  __shared__ long long s_nv[EPI_NT], s_na[EPI_NT];
+  __shared__ double s_zk[EPI_NT], s_a[EPI_NT];
+  static_assert(kMaxPartials <= EPI_NT, "one thread per partial sum");
+  // every block folds the same partial sums in the same fixed tree (so all blocks get
+  // the same bits): thread i starts from partial i, halves are added pairwise
+  {
+    const int i = threadIdx.x;
+    const bool have = i < A.n_part;
+    s_nv[i] = have ? A.part->n_valid[i] : 0;
+    s_na[i] = have ? A.part->n_accept[i] : 0;
+    s_zk[i] = have ? A.part->sum_zk[i] : 0.0;
+    s_a[i] = have ? A.part->sum_a[i] : 0.0;
+  }
+  __syncthreads();
+  for (int half = EPI_NT / 2; half > 0; half >>= 1) {
+    if ((int)threadIdx.x < half) {
+      s_nv[threadIdx.x] += s_nv[threadIdx.x + half];
+      s_na[threadIdx.x] += s_na[threadIdx.x + half];
+      s_zk[threadIdx.x] += s_zk[threadIdx.x + half];
+      s_a[threadIdx.x] += s_a[threadIdx.x + half];
     }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    const long long nv = s_nv[0], na = s_na[0];
+    const double szk = s_zk[0], sa = s_a[0];
     double alpha = nv > 0 ? (double)na / (double)nv : 0.0;
     double mean_zk = nv > 0 ? szk / (double)nv : 0.0;
     double kappa = (nv > 0 && mean_zk > 0.0) ? alpha / mean_zk : 1.0;
