@@ -61,6 +61,7 @@ constexpr int VPL = JP_VPL;               // 16-byte vectors per lane per tensor
 constexpr int TV = WPT * 32 * VPL;        // vectors per tensor per tile
 constexpr int HV = 2;                     // vectors per tensor a lane holds at a time
 static_assert(JP_VPL % HV == 0, "a tile is taken in passes of HV vectors");
+static_assert(JP_NG == 2, "tiles go to consumer groups and top-k warps by parity; the producer keeps two phase masks");
 static_assert(NC % NG == 0 && NG < JP_STAGES, "consumer groups must divide the warps and fit the ring");
 constexpr int STAGES = JP_STAGES;
 constexpr int SCAP = 288;                 // buffered keys per top-k warp (used while sorting survivors into the list)
@@ -81,7 +82,9 @@ struct __align__(128) StreamSmem {
   uint32_t svpass[2][2][2][SVCAP];        // [slot][tensor][tile parity] candidate passes still alive under tau: tile * TP + entry ...
   float svmax[2][2][2][SVCAP];            // ... and their maxima
   uint32_t hist[2][2][2][NB];             // [slot][tensor][tile parity] passes seen per order code of their maximum
-  unsigned long long full[STAGES];        // producer -> consumers: the tile's bytes have landed
+  unsigned long long full[NG][STAGES];    // [consumer group] producer -> that group: the tile's bytes have landed.  One set per
+                                          // group, so that every waiter sees every phase of its barriers in turn: a group that
+                                          // skipped the other group's phases could take an unfinished earlier phase for its own
   unsigned long long seen[2][2][STAGES];  // [slot][tile parity] consumers -> top-k warps: tile consumed, pass maxima written
   unsigned long long empty[STAGES];       // -> producer: the stage may be refilled
   unsigned long long row_done[2], slot_free[2];
@@ -92,6 +95,8 @@ struct __align__(128) StreamSmem {
   float part_s[2][2][NC];
   int abort;
 };
+
+static_assert(sizeof(StreamSmem) <= 232448, "the CTA's shared memory exceeds the 227 KB an sm_100 CTA can have");
 
 // ---- mbarrier / bulk-copy wrappers ----------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -605,6 +610,7 @@ __device__ void producer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_row
   // Stage and phase advance by increments, addresses by additions, and the next row's
   // index is fetched one row ahead.
   uint32_t s = 0, ph = 0, armed = 0;
+  uint32_t fph0 = 0u, fph1 = 0u, last_grp = 0u, last_ph = 0u;   // per stage: phase bits of full[0], full[1]; group and phase armed last
   bool ok = true;
   int64_t it = blockIdx.x;
   int64_t row = it < n_rows ? A.list[it] : 0;
@@ -616,13 +622,18 @@ __device__ void producer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_row
     for (int tile = 0; tile < ntiles; ++tile, ra += TV * 16, rp += TV * 16) {
       if (!mbar_wait(&sm.empty[s], ph ^ 1u, &sm.abort)) { ok = false; break; }
       const uint32_t bytes = tile == ntiles - 1 ? last_bytes : (uint32_t)(TV * 16);
+      const int grp = tile % NG;
       if (bytes > 0) {
-        mbar_arrive_expect_tx(&sm.full[s], 2u * bytes);
-        bulk_g2s(&sm.ring[s][0][0], ra, bytes, &sm.full[s]);
-        bulk_g2s(&sm.ring[s][1][0], rp, bytes, &sm.full[s]);
+        mbar_arrive_expect_tx(&sm.full[grp][s], 2u * bytes);
+        bulk_g2s(&sm.ring[s][0][0], ra, bytes, &sm.full[grp][s]);
+        bulk_g2s(&sm.ring[s][1][0], rp, bytes, &sm.full[grp][s]);
       } else {
-        mbar_arrive(&sm.full[s]);
+        mbar_arrive(&sm.full[grp][s]);
       }
+      // remember what was armed last on this stage (for the clean-up after a time-out)
+      last_grp = (last_grp & ~(1u << s)) | ((uint32_t)grp << s);
+      if (grp) { last_ph = (last_ph & ~(1u << s)) | (((fph1 >> s) & 1u) << s); fph1 ^= 1u << s; }
+      else     { last_ph = (last_ph & ~(1u << s)) | (((fph0 >> s) & 1u) << s); fph0 ^= 1u << s; }
       ++armed;
       if (++s == STAGES) { s = 0; ph ^= 1u; }
     }
@@ -632,12 +643,9 @@ __device__ void producer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_row
     // complete once their bytes have landed.
     raise_timeout(sm, A.sc);
     const uint32_t n_back = armed < (uint32_t)STAGES ? armed : (uint32_t)STAGES;
-    for (uint32_t h = 0; h < n_back; ++h) {
-      // walk back from the stage armed last
-      if (s == 0) { s = STAGES; ph ^= 1u; }
-      --s;
+    for (uint32_t st = 0; st < n_back; ++st) {          // stages 0 .. n_back-1 are the ones ever armed
       const long long t0 = clock64();
-      while (!mbar_try_wait(&sm.full[s], ph))
+      while (!mbar_try_wait(&sm.full[(last_grp >> st) & 1u][st], (last_ph >> st) & 1u))
         if (clock64() - t0 > kSpinLimit) break;
     }
   }
@@ -653,6 +661,7 @@ __device__ void consumer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_row
   const int gq = cw / WPT;              // this warp's group: it takes tiles gq, gq + NG, ...
   const int wq = cw % WPT;              // its place among the warps that share a tile
   uint32_t g0 = 0;                      // ring position of the current row's tile 0
+  uint32_t fphase = 0u;                 // per stage: phase bit of this group's full barrier
   int lr = 0;
   for (int64_t it = blockIdx.x; it < n_rows; it += gridDim.x, ++lr, g0 += ntiles) {
     const int p = lr & 1;
@@ -670,7 +679,8 @@ __device__ void consumer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_row
     auto consume_tile = [&](uint32_t tile) -> bool {
       const uint32_t g = g0 + tile;
       const uint32_t s = g % STAGES;
-      if (!mbar_wait(&sm.full[s], (g / STAGES) & 1u, &sm.abort)) return false;
+      if (!mbar_wait(&sm.full[gq][s], (fphase >> s) & 1u, &sm.abort)) return false;
+      fphase ^= 1u << s;
       const uint4* sa = &sm.ring[s][0][wq * 32 + lane];
       const uint4* sp = &sm.ring[s][1][wq * 32 + lane];
       float* pma = &sm.passmax[s][0][wq * 32 + lane];
@@ -1008,7 +1018,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) stream_kernel(StreamArgs A) {
 
   if (tid == 0) {
     for (int s = 0; s < STAGES; ++s) {
-      mbar_init(&sm.full[s], 1);
+      for (int q = 0; q < NG; ++q) mbar_init(&sm.full[q][s], 1);
       for (int q = 0; q < 4; ++q) mbar_init(&sm.seen[q >> 1][q & 1][s], WPT);
       mbar_init(&sm.empty[s], KPL > 0 ? 2 : WPT);     // with top-k the two top-k warps of the row free the stage
     }
