@@ -9,26 +9,32 @@
 //   producer warp   one lane issues 1-D bulk async copies (global -> shared,
 //                   completion counted on an mbarrier) of the next tile of both
 //                   rows into a ring of STAGES shared-memory stages;
-//   consumer warps  wait for a stage, pull their 16-byte vectors into registers,
-//                   release the stage, then update the online (max, sum) of both
-//                   rows and test each vector's maximum against the row's current
-//                   top-k threshold tau; a vector that may hold a top-k entry is
-//                   copied, with its index, into a small shared-memory ring queue;
-//   top-k warps     four of them, one per (tensor, row slot): they drain the
-//                   queue while the consumers keep streaming.  Every entry at or
-//                   above tau is counted in a histogram over the 16-bit order code
-//                   of its logit and its 64-bit key is appended to a buffer; the
-//                   histogram gives the running tau (the highest code with at least
-//                   k entries at or above it) without sorting anything.  At the end
-//                   of the row the buffered keys at or above the final tau are
-//                   sorted into the list (bitonic sort / merge across the lanes),
-//                   the warp finishes the log-sum-exp, gathers the sampled token's
-//                   logit and writes the row's record.
+//   consumer warps  two groups that take alternate tiles of a row: wait for a stage,
+//                   pull their 16-byte vectors into registers pass by pass, update
+//                   the online (max, sum) of both rows and leave the maximum of
+//                   every pass (two vectors) in shared memory beside the stage;
+//   top-k warps     eight of them, one per (tensor, row slot, tile parity).  Per
+//                   tile a warp loads the 512 pass maxima (16 per lane), frees the
+//                   stage and counts the passes at or above its running threshold
+//                   tau in a histogram over the 16-bit order code of the maximum;
+//                   tau is the highest code with at least k passes at or above it
+//                   (k different passes hold k different entries, so the k-th best
+//                   logit is not below it): nothing is sorted while streaming.  A
+//                   pass at or above tau is kept as (pass, maximum).  At the end of
+//                   the row the vectors of the kept passes are read back, their
+//                   entries at or above tau are sorted into the list (bitonic sort /
+//                   merge across the lanes), the two parity warps' lists are merged,
+//                   and the warp finishes the log-sum-exp, gathers the sampled
+//                   token's logit and writes the row's record.
 //
-// Rows alternate between two "slots" (queue, tau, partial sums, barriers), so the
-// consumers start the next row while the top-k warps finish the previous one.
-// The total order of the top-k is (logit desc, index asc), one 64-bit key; the
-// result does not depend on the order in which candidates arrive.
+// Rows alternate between two "slots" (histograms, survivors, partial sums,
+// barriers), so the consumers start the next row while the top-k warps finish
+// the previous one.  The total order of the top-k is (logit desc, index asc), one
+// 64-bit key; the result does not depend on the order in which candidates arrive.
+//
+// Every mbarrier is waited on phase by phase by the same warps, each keeping its
+// own phase bits: a parity wait cannot tell a phase not yet reached from one that
+// is done, so a waiter that skipped phases could run ahead of the data.
 //
 // Every wait is bounded: a wait that runs out raises the CTA's abort flag, the
 // status word gets JP_ERR_TIMEOUT and every warp leaves its loop.
