@@ -10,27 +10,29 @@
 //                   completion counted on an mbarrier) of the next tile of both
 //                   rows into a ring of STAGES shared-memory stages;
 //   consumer warps  two groups that take alternate tiles of a row: wait for a stage,
-//                   pull their 16-byte vectors into registers pass by pass, update
-//                   the online (max, sum) of both rows and leave the maximum of
-//                   every pass (two vectors) in shared memory beside the stage;
-//   top-k warps     eight of them, one per (tensor, row slot, tile parity).  Per
-//                   tile a warp loads the 512 pass maxima (16 per lane), frees the
-//                   stage and counts the passes at or above its running threshold
-//                   tau in a histogram over the 16-bit order code of the maximum;
-//                   tau is the highest code with at least k passes at or above it
-//                   (k different passes hold k different entries, so the k-th best
-//                   logit is not below it): nothing is sorted while streaming.  A
-//                   pass at or above tau is kept as (pass, maximum).  At the end of
-//                   the row the vectors of the kept passes are read back, their
-//                   entries at or above tau are sorted into the list (bitonic sort /
-//                   merge across the lanes), the two parity warps' lists are merged,
-//                   and the warp finishes the log-sum-exp, gathers the sampled
-//                   token's logit and writes the row's record.
+//                   pull their 16-byte vectors into registers pass by pass (a pass
+//                   is two vectors per tensor), free the stage, update the online
+//                   (max, sum) of both rows and compare the maximum of each pass with
+//                   the row's running threshold tau.  A pass at or above tau (rare) is
+//                   counted in a histogram and appended to the row's candidate buffer;
+//   top-k warps     eight of them, one per (row slot, tensor).  Before a row starts its
+//                   warp reads a sample (the first vectors) of the row and publishes
+//                   the k-th best vector maximum of the sample as the first tau: the
+//                   k-th best of any subset is a lower bound of the row's k-th best
+//                   logit.  While the row streams it raises tau to the highest histogram
+//                   bin with at least k counted passes at or above it (k different
+//                   passes hold k different entries).  When the row is done it reads the
+//                   vectors of the candidate passes back, sorts their entries at or above
+//                   tau into the list (bitonic sort / merge across the lanes), finishes
+//                   the log-sum-exp, gathers the sampled token's logit and writes the
+//                   row's record.  A row whose candidates did not fit the buffer is
+//                   scanned again from memory by its warp (exact, slow, rare).
 //
-// Rows alternate between two "slots" (histograms, survivors, partial sums,
-// barriers), so the consumers start the next row while the top-k warps finish
-// the previous one.  The total order of the top-k is (logit desc, index asc), one
-// 64-bit key; the result does not depend on the order in which candidates arrive.
+// Rows cycle through four "slots" (histogram, candidates, partial sums, barriers),
+// so the consumers never wait for the top-k warps unless those fall three rows
+// behind.  The total order of the top-k is (logit desc, index asc), one 64-bit key;
+// the result does not depend on the order in which candidates arrive or on when tau
+// was raised.
 //
 // Every mbarrier is waited on phase by phase by the same warps, each keeping its
 // own phase bits: a parity wait cannot tell a phase not yet reached from one that
@@ -51,14 +53,20 @@ namespace jp {
 #ifndef JP_VPL
 #define JP_VPL 4
 #endif
-#ifndef JP_TOPK_SLEEP_NS
-#define JP_TOPK_SLEEP_NS 300
-#endif
 #ifndef JP_STAGES
 #define JP_STAGES 5
 #endif
 #ifndef JP_NG
 #define JP_NG 2
+#endif
+#ifndef JP_CAP
+#define JP_CAP 1024
+#endif
+#ifndef JP_SAMPLE_VPL
+#define JP_SAMPLE_VPL 32
+#endif
+#ifndef JP_TAU_NS
+#define JP_TAU_NS 200
 #endif
 constexpr int NC = JP_NC;                 // consumer warps
 constexpr int NG = JP_NG;                 // consumer groups: group q takes tiles q, q + NG, ...
@@ -67,38 +75,38 @@ constexpr int VPL = JP_VPL;               // 16-byte vectors per lane per tensor
 constexpr int TV = WPT * 32 * VPL;        // vectors per tensor per tile
 constexpr int HV = 2;                     // vectors per tensor a lane holds at a time
 static_assert(JP_VPL % HV == 0, "a tile is taken in passes of HV vectors");
-static_assert(JP_NG == 2, "tiles go to consumer groups and top-k warps by parity; the producer keeps two phase masks");
+static_assert(JP_NG == 2, "tiles go to consumer groups by parity; the producer keeps two phase masks");
 static_assert(NC % NG == 0 && NG < JP_STAGES, "consumer groups must divide the warps and fit the ring");
 constexpr int STAGES = JP_STAGES;
-constexpr int SCAP = 288;                 // buffered keys per top-k warp (used while sorting survivors into the list)
-constexpr int SVCAP = 288;                // candidate passes a top-k warp keeps until the row ends
-constexpr int NB = 256;                   // histogram bins: 16-bit order codes below the warp's first tile's maximum
-constexpr int TP = TV / HV;               // passes per tensor per tile = pass maxima a top-k warp scans per tile
-static_assert(TP == 512, "a top-k lane scans 16 pass maxima per tile (4 x 16 bytes)");
-constexpr int NTOPK = 8;                  // top-k warps: (tensor, slot, tile parity)
+constexpr int NSLOT = 4;                  // rows in flight between the consumers and the top-k warps
+constexpr int SCAP = 288;                 // keys a top-k warp buffers before it sorts them into the list
+constexpr int CAP = JP_CAP;               // candidate passes a row may collect before it falls back to a re-scan
+constexpr int NB = 256;                   // histogram bins
+constexpr int TP = TV / HV;               // passes per tensor per tile
+constexpr int SAMPLE = 32 * JP_SAMPLE_VPL;  // vectors of a row its top-k warp looks at before the row starts
+static_assert(SAMPLE <= CAP, "the sample's vector maxima are parked in the candidate buffer");
+constexpr int NTOPK = NSLOT * 2;          // top-k warps: (slot, tensor)
 constexpr int NWARPS = 1 + NC + NTOPK;
 constexpr int NTHREADS = NWARPS * 32;
-constexpr uint32_t QEMPTY = 0xffffffffu;
 constexpr long long kSpinLimit = 4000000000ll;   // clock cycles a wait may last (about 2 s)
 
 struct __align__(128) StreamSmem {
   uint4 ring[STAGES][2][TV];              // [stage][tensor][vector]
-  float passmax[STAGES][2][TP];           // [stage][tensor] maximum of each consumer pass (HV vectors) of the tile
-  unsigned long long skeys[2][2][2][SCAP];  // [slot][tensor][tile parity] keys waiting to be sorted into the list; the parity-0 warp leaves its finished list here
-  uint32_t svpass[2][2][2][SVCAP];        // [slot][tensor][tile parity] candidate passes still alive under tau: tile * TP + entry ...
-  float svmax[2][2][2][SVCAP];            // ... and their maxima
-  uint32_t hist[2][2][2][NB];             // [slot][tensor][tile parity] passes seen per order code of their maximum
+  unsigned long long skeys[NSLOT][2][SCAP];  // [slot][tensor] keys waiting to be sorted into the list
+  uint32_t cand[NSLOT][2][CAP];           // [slot][tensor] candidate passes: high bits of the maximum's order bits | pass id
+  uint32_t hist[NSLOT][2][NB];            // [slot][tensor] candidate passes per bin of their maximum
   unsigned long long full[NG][STAGES];    // [consumer group] producer -> that group: the tile's bytes have landed.  One set per
                                           // group, so that every waiter sees every phase of its barriers in turn: a group that
                                           // skipped the other group's phases could take an unfinished earlier phase for its own
-  unsigned long long seen[2][2][STAGES];  // [slot][tile parity] consumers -> top-k warps: tile consumed, pass maxima written
-  unsigned long long empty[STAGES];       // -> producer: the stage may be refilled
-  unsigned long long row_done[2], slot_free[2];
-  unsigned long long scan_done[2][2];     // [slot][tensor] parity-0 warp -> parity-1 warp: my part of the row is in shared memory
-  unsigned long long final_done[2][2];    // [slot][tensor] parity-1 warp -> parity-0 warp: I have read it
-  int xstate[2][2][4];                    // [slot][tensor] parity-0 hand-over: kept vectors, tau code, keys in xkeys
-  float part_mL[2][2][NC];
-  float part_s[2][2][NC];
+  unsigned long long empty[STAGES];       // consumers -> producer: the stage may be refilled
+  unsigned long long slot_ready[NSLOT];   // top-k warps -> consumers: the slot is set up for its next row
+  unsigned long long row_done[NSLOT];     // consumers -> top-k warps: the row has been streamed
+  float tau[NSLOT][2];                    // running threshold (only rises while a row streams)
+  uint32_t ncand[NSLOT][2];               // candidate passes appended so far (may pass CAP: then the row is re-scanned)
+  uint32_t bin_base[NSLOT][2];            // bin of a maximum = (order bits >> bin_shift) - bin_base, clipped to [0, NB-1]
+  uint32_t bin_shift[NSLOT][2];
+  float part_mL[NSLOT][2][NC];
+  float part_s[NSLOT][2][NC];
   int abort;
 };
 
@@ -174,6 +182,14 @@ __device__ __forceinline__ uint32_t lds_volatile_u32(const void* p) {
 }
 __device__ __forceinline__ void sts_volatile_f32(float* p, float v) {
   asm volatile("st.volatile.shared.f32 [%0], %1;" ::"r"(smem_u32(p)), "f"(v) : "memory");
+}
+__device__ __forceinline__ uint4 lds_volatile_v4(const void* p) {
+  uint4 v;
+  asm volatile("ld.volatile.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "r"(smem_u32(p))
+               : "memory");
+  return v;
 }
 
 // ---- packed fp32x2 arithmetic (two lanes of one 64-bit register pair) ------
@@ -429,66 +445,29 @@ __device__ __forceinline__ unsigned long long kth_key(const unsigned long long (
   return __shfl_sync(0xffffffffu, v, (k - 1) / KPL);
 }
 
-// The running threshold of one (row, tensor).  `code` is the highest 16-bit order
-// code with at least k of the candidate vectors seen so far having their maximum
-// at or above it: k different vectors hold k different entries, so the k-th best
-// logit of the row is at or above the low edge of that code's bin.  `cnt` counts
-// the vectors at or above it.  `key` is the exact k-th best key of the sorted
-// list once candidates have been sorted into it (0 before).
-struct Tau {
-  uint32_t code;
-  int cnt;
-  unsigned long long key;
-};
-
-__device__ __forceinline__ uint32_t order_code(float v) { return f32_order_bits(v) >> 16; }
-// low edge of a code's bin, as a logit
-__device__ __forceinline__ float code_value(uint32_t code) { return order_bits_f32(code << 16); }
-
-// v[i] for a run-time i in 0..15 without indexing the register array (a select tree).
-__device__ __forceinline__ float select16(const float (&v)[16], int i) {
-  float a[8], b[4], c[2];
-#pragma unroll
-  for (int j = 0; j < 8; ++j) a[j] = (i & 1) ? v[2 * j + 1] : v[2 * j];
-#pragma unroll
-  for (int j = 0; j < 4; ++j) b[j] = (i & 2) ? a[2 * j + 1] : a[2 * j];
-#pragma unroll
-  for (int j = 0; j < 2; ++j) c[j] = (i & 4) ? b[2 * j + 1] : b[2 * j];
-  return (i & 8) ? c[1] : c[0];
-}
-
-// First vector index of pass `id` (= tile * TP + entry) and the step to its next vector.
+// First vector index of pass `id` (= tile * TP + entry); its HV vectors are WPT * 32 apart.
 __device__ __forceinline__ uint32_t pass_first_vector(uint32_t id) {
   const uint32_t tile = id / TP, e = id % TP;
   return tile * TV + (e / (WPT * 32)) * HV * (WPT * 32) + e % (WPT * 32);
 }
 
-// Can the pass with maximum order bits `ob` still hold one of the k best?
-__device__ __forceinline__ bool pass_alive(uint32_t ob, uint32_t id, int n_per_vec, const Tau& tau) {
-  if ((ob >> 16) < tau.code) return false;
-  if (tau.key == 0ull) return true;
-  // its best possible entry: the maximum at the first index of the pass's first vector
-  const uint32_t idx = pass_first_vector(id) * (uint32_t)n_per_vec;
-  return (((unsigned long long)ob << 32) | (unsigned long long)(uint32_t)(~idx)) > tau.key;
-}
-
-// The highest histogram bin with at least k counted passes at or above it (0 if
-// fewer than k passes were counted).  Lane l sums bins 8 l .. 8 l + 7, a shuffle
-// suffix scan finds the lane in which the count crosses k, and that lane walks its
-// bins from the top.
+// The highest histogram bin with at least k counted entries at or above it (0 if
+// fewer than k were counted, or if the k-th lies in bin 0).  Lane l sums bins
+// 8 l .. 8 l + 7, a shuffle suffix scan finds the lane in which the count crosses
+// k, and that lane walks its bins from the top.  The histogram may be growing
+// while it is read: a count read early is only smaller, and so is the result.
 __device__ __forceinline__ int find_tau_bin(const uint32_t* hist, int k, int lane) {
   static_assert(NB == 256, "8 bins per lane");
-  const uint4* h4 = reinterpret_cast<const uint4*>(hist) + lane * 2;
   uint32_t b[8];
 #pragma unroll
   for (int q = 0; q < 2; ++q) {
-    const uint4 v = h4[q];
+    const uint4 v = lds_volatile_v4(hist + lane * 8 + q * 4);
     b[4 * q] = v.x; b[4 * q + 1] = v.y; b[4 * q + 2] = v.z; b[4 * q + 3] = v.w;
   }
   int mine = 0;
 #pragma unroll
   for (int i = 0; i < 8; ++i) mine += (int)b[i];
-  int suf = mine;                                   // passes in this lane's bins and all higher lanes'
+  int suf = mine;                                   // entries in this lane's bins and all higher lanes'
 #pragma unroll
   for (int off = 1; off < 32; off <<= 1) {
     const int o = __shfl_down_sync(0xffffffffu, suf, off);
@@ -507,37 +486,39 @@ __device__ __forceinline__ int find_tau_bin(const uint32_t* hist, int k, int lan
   return __shfl_sync(0xffffffffu, lane * 8 + bin, L);
 }
 
-// Drops the kept candidate passes that tau has ruled out since they were kept.
-__device__ __noinline__ int compact_survivors(uint32_t* svp, float* svm, int nsv, Tau tau, int n_per_vec, int lane) {
-  int out = 0;
-  for (int b = 0; b < nsv; b += 32) {
-    const int i = b + lane;
-    uint32_t id = 0u;
-    float m = 0.f;
-    bool keep = false;
-    if (i < nsv) {
-      id = svp[i];
-      m = svm[i];
-      keep = pass_alive(f32_order_bits(m), id, n_per_vec, tau);
-    }
-    const uint32_t bm = __ballot_sync(0xffffffffu, keep);
-    __syncwarp();
-    if (keep) {
-      const int o = out + __popc(bm & ((1u << lane) - 1u));
-      svp[o] = id;
-      svm[o] = m;
-    }
-    out += __popc(bm);
-    __syncwarp();
+// Low edge, as a logit, of histogram bin `bin` >= 1 under (base, shift).
+__device__ __forceinline__ float bin_edge(uint32_t base, uint32_t shift, int bin) {
+  const uint32_t top = 0xffffffffu >> shift;
+  const uint32_t code = base + (uint32_t)bin < top ? base + (uint32_t)bin : top;
+  return order_bits_f32(code << shift);
+}
+
+// What a consumer lane does with a pass whose maximum reached the row's threshold:
+// count it in the histogram its top-k warp reads tau from and append it to the
+// candidates (the high bits of the maximum's order bits over the pass id).  Out of
+// line: it runs for a fraction of a percent of the passes.
+__device__ __noinline__ void record_hits(StreamSmem& sm, int p, uint32_t id, uint32_t idmask, float ma, float mp,
+                                         float ta, float tp) {
+#pragma unroll 1
+  for (int t = 0; t < 2; ++t) {
+    const float m = t == 0 ? ma : mp;
+    if (!(m >= (t == 0 ? ta : tp))) continue;
+    const uint32_t ob = f32_order_bits(m);
+    const uint32_t c = ob >> sm.bin_shift[p][t], base = sm.bin_base[p][t];
+    const uint32_t bin = c > base ? (c - base < (uint32_t)(NB - 1) ? c - base : (uint32_t)(NB - 1)) : 0u;
+    atomicAdd(&sm.hist[p][t][bin], 1u);
+    const uint32_t o = atomicAdd(&sm.ncand[p][t], 1u);
+    if (o < (uint32_t)CAP) sm.cand[p][t][o] = (ob & ~idmask) | id;
   }
-  return out;
 }
 
 // Appends to the key buffer the keys of one vector's entries (one vector per lane)
-// that can still be among the k best.  Returns the new number of buffered keys.
+// that can still be among the k best: at or above the threshold (as order bits) and
+// above the list's current k-th key.  Returns the new number of buffered keys.
 template <int DT>
-__device__ __forceinline__ int stage_entries(const uint4& v, uint32_t vi, bool have, int64_t V, const Tau& tau,
-                                             unsigned long long* stg, int staged, int lane) {
+__device__ __forceinline__ int stage_entries(const uint4& v, uint32_t vi, bool have, int64_t V, uint32_t tau_ob,
+                                             unsigned long long kth, unsigned long long* stg, int staged,
+                                             int lane) {
   constexpr int N = Vec<DT>::N;
   const uint32_t lt = (1u << lane) - 1u;
 #pragma unroll
@@ -545,7 +526,7 @@ __device__ __forceinline__ int stage_entries(const uint4& v, uint32_t vi, bool h
     const uint32_t idx = vi * N + e;
     const uint32_t ob = f32_order_bits(Vec<DT>::get(v, e));
     const unsigned long long key = ((unsigned long long)ob << 32) | (unsigned long long)(uint32_t)(~idx);
-    const bool keep = have && (int64_t)idx < V && (ob >> 16) >= tau.code && key > tau.key;
+    const bool keep = have && (int64_t)idx < V && ob >= tau_ob && key > kth;
     const uint32_t bk = __ballot_sync(0xffffffffu, keep);
     if (keep) stg[staged + __popc(bk & lt)] = key;
     staged += __popc(bk);
@@ -569,34 +550,134 @@ __device__ __noinline__ unsigned long long merge_all(unsigned long long (&L)[KPL
   return kth_key<KPL>(L, k);
 }
 
-// Sorts the entries of every kept pass into the list (exact from here on: tau.key
-// becomes the list's k-th key) and empties the survivor buffer.  The vectors of a
-// pass are read back from memory (they left the ring long ago; a few hundred
-// 16-byte reads per row, mostly L2 hits).
-template <int DT, int KPL>
-__device__ __noinline__ void survivors_to_list(unsigned long long (&L)[KPL], const uint32_t* svp, int& nsv,
-                                               const char* row, int64_t nvec, int64_t V, Tau& tau,
-                                               unsigned long long* stg, int k, int lane) {
-  int staged = 0;
-  for (int b = 0; b < nsv; b += 32) {
+// Drops the candidates whose maximum is below the row's final threshold; returns
+// how many are left (packed at the front of the buffer).
+__device__ __noinline__ int compact_candidates(uint32_t* cand, int n, uint32_t tau_ob, uint32_t idmask, int lane) {
+  int out = 0;
+  for (int b = 0; b < n; b += 32) {
     const int i = b + lane;
-    const uint32_t v0 = i < nsv ? pass_first_vector(svp[i]) : 0u;
+    const uint32_t c = i < n ? cand[i] : 0u;
+    // the stored high bits with the low ones filled in bound the maximum from above
+    const bool keep = i < n && (c | idmask) >= tau_ob;
+    const uint32_t bm = __ballot_sync(0xffffffffu, keep);
+    __syncwarp();
+    if (keep) cand[out + __popc(bm & ((1u << lane) - 1u))] = c;
+    out += __popc(bm);
+    __syncwarp();
+  }
+  return out;
+}
+
+// Sorts the entries of the candidate passes into the list.  The vectors of a pass
+// are read back from memory (they left the ring long ago; a few hundred 16-byte
+// reads per row, mostly L2 hits).  Returns the list's k-th key.
+template <int DT, int KPL>
+__device__ __noinline__ unsigned long long candidates_to_list(unsigned long long (&L)[KPL], const uint32_t* cand,
+                                                              int n, uint32_t idmask, const char* row, int64_t nvec,
+                                                              int64_t V, uint32_t tau_ob, unsigned long long* stg,
+                                                              int k, int lane) {
+  int staged = 0;
+  unsigned long long kth = 0ull;
+  for (int b = 0; b < n; b += 32) {
+    const int i = b + lane;
+    const uint32_t v0 = i < n ? pass_first_vector(cand[i] & idmask) : 0u;
     uint4 v[HV];
     bool in[HV];
 #pragma unroll
     for (int j = 0; j < HV; ++j) {
       const uint32_t vi = v0 + j * (WPT * 32);
-      in[j] = i < nsv && (int64_t)vi < nvec;
+      in[j] = i < n && (int64_t)vi < nvec;
       v[j] = in[j] ? ldg_stream((const uint4*)row + vi) : Vec<DT>::neg_inf();
     }
 #pragma unroll
     for (int j = 0; j < HV; ++j) {
-      staged = stage_entries<DT>(v[j], v0 + j * (WPT * 32), in[j], V, tau, stg, staged, lane);
-      if (staged > SCAP - 32 * Vec<DT>::N) tau.key = merge_all<KPL>(L, stg, staged, k, lane);
+      staged = stage_entries<DT>(v[j], v0 + j * (WPT * 32), in[j], V, tau_ob, kth, stg, staged, lane);
+      if (staged > SCAP - 32 * Vec<DT>::N) kth = merge_all<KPL>(L, stg, staged, k, lane);
     }
   }
-  tau.key = merge_all<KPL>(L, stg, staged, k, lane);
-  nsv = 0;
+  return merge_all<KPL>(L, stg, staged, k, lane);
+}
+
+// The exact top-k of a whole row read again from memory by one warp: the way out
+// for a row whose candidates did not fit the buffer (long runs of ties at the top,
+// rows that keep rising, -inf padding above the k-th entry).  Returns the k-th key.
+template <int DT, int KPL>
+__device__ __noinline__ unsigned long long scan_row_exact(unsigned long long (&L)[KPL], const char* row,
+                                                          int64_t nvec, int64_t V, unsigned long long* stg, int k,
+                                                          int lane) {
+  int staged = 0;
+  unsigned long long kth = 0ull;
+  for (int64_t b = 0; b < nvec; b += 32) {
+    const int64_t vi = b + lane;
+    const bool in = vi < nvec;
+    const uint4 v = in ? ldg_stream((const uint4*)row + vi) : Vec<DT>::neg_inf();
+    // skip the 32 vectors at once when none reaches the value of the current k-th key
+    const uint32_t ob = f32_order_bits(Vec<DT>::vmax(v));
+    if (!__any_sync(0xffffffffu, in && ob >= (uint32_t)(kth >> 32))) continue;
+    staged = stage_entries<DT>(v, (uint32_t)vi, in, V, 0u, kth, stg, staged, lane);
+    if (staged > SCAP - 32 * Vec<DT>::N) kth = merge_all<KPL>(L, stg, staged, k, lane);
+  }
+  return merge_all<KPL>(L, stg, staged, k, lane);
+}
+
+// Before a row starts: the k-th best vector maximum of the row's first SAMPLE
+// vectors, as the low edge of its histogram bin (-inf if the sample has fewer than
+// k vectors), and the bin geometry (base, shift) for the row's candidate histogram.
+// The window of NB codes is anchored at the sample's maximum; the shift starts at 16
+// (bf16 resolution) and grows until the k-th best falls inside the window, so a
+// sample that spans many binades, or zero, gets coarser bins rather than none.
+template <int DT>
+__device__ __noinline__ float sample_threshold(const char* row, int64_t nvec, int k, uint32_t* hist, float* park,
+                                               uint32_t& base, uint32_t& shift, int lane) {
+  const int ns = (int)(nvec < (int64_t)SAMPLE ? nvec : (int64_t)SAMPLE);
+  base = 0xffffffffu;                       // nothing above it: every maximum counts in bin 0 = "no threshold"
+  shift = 16u;
+  if (ns < k) return JP_NEG_INF;
+  float mx = JP_NEG_INF;
+#pragma unroll 1
+  for (int c = 0; c < ns; c += 8 * 32) {
+    uint4 v[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int vi = c + j * 32 + lane;
+      v[j] = vi < ns ? ldg_stream((const uint4*)row + vi) : Vec<DT>::neg_inf();
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int vi = c + j * 32 + lane;
+      const float m = Vec<DT>::vmax(v[j]);
+      if (vi < ns) park[vi] = m;
+      mx = fmaxf(mx, m);
+    }
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+  const uint32_t ob_max = f32_order_bits(mx);
+  __syncwarp();
+  float tau0 = JP_NEG_INF;
+  for (uint32_t sh = 16u; sh < 32u; ++sh) {
+    const uint32_t cmax = ob_max >> sh;
+    const uint32_t b0 = cmax > (uint32_t)(NB - 1) ? cmax - (uint32_t)(NB - 1) : 0u;
+    for (int i = lane; i < NB; i += 32) hist[i] = 0u;
+    __syncwarp();
+    for (int i = lane; i < ns; i += 32) {
+      const uint32_t c = f32_order_bits(park[i]) >> sh;
+      atomicAdd(&hist[c > b0 ? c - b0 : 0u], 1u);        // c <= cmax, so the bin is at most NB - 1
+    }
+    __syncwarp();
+    const int bin = find_tau_bin(hist, k, lane);
+    if (bin > 0) {
+      const uint32_t code0 = b0 + (uint32_t)bin;
+      tau0 = order_bits_f32(code0 << sh);
+      base = code0 - 1u;                                 // the threshold's own code is bin 1; cmax is at most bin NB - 1
+      shift = sh;
+      break;
+    }
+    if (b0 == 0u) break;                                 // the window reaches the bottom of the order: no threshold
+  }
+  __syncwarp();
+  if (!(tau0 == tau0)) tau0 = JP_NEG_INF;                // the low edge of -inf's own bin is not a number
+  return tau0;
 }
 
 __device__ __forceinline__ void raise_timeout(StreamSmem& sm, Scalars* sc) {
@@ -664,24 +745,24 @@ __device__ void consumer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_row
   const int64_t nvec = A.V / N;
   const int tail = (int)(A.V - nvec * N);
   const uint32_t ntiles = nvec > 0 ? (uint32_t)((nvec + TV - 1) / TV) : 1u;
+  const uint32_t idmask = 0xffffffffu >> __clz(ntiles * (uint32_t)TP - 1u);   // covers every pass id of a row
   const int gq = cw / WPT;              // this warp's group: it takes tiles gq, gq + NG, ...
   const int wq = cw % WPT;              // its place among the warps that share a tile
   uint32_t g0 = 0;                      // ring position of the current row's tile 0
   uint32_t fphase = 0u;                 // per stage: phase bit of this group's full barrier
   int lr = 0;
   for (int64_t it = blockIdx.x; it < n_rows; it += gridDim.x, ++lr, g0 += ntiles) {
-    const int p = lr & 1;
-    const uint32_t ph = (uint32_t)((lr >> 1) & 1);
-    // the slot's partial sums are free once both of its top-k warps have finished
-    // the row that used it before
-    if (!mbar_wait(&sm.slot_free[p], ph ^ 1u, &sm.abort)) { raise_timeout(sm, A.sc); return; }
+    const int p = lr % NSLOT;
+    const uint32_t ph = (uint32_t)((lr / NSLOT) & 1);
+    // the slot's top-k warps have finished the row that used it before and set it up for this one
+    if (!mbar_wait(&sm.slot_ready[p], ph, &sm.abort)) { raise_timeout(sm, A.sc); return; }
 
     Online oa{JP_NEG_INF, 0.f, 0ull}, op{JP_NEG_INF, 0.f, 0ull};
 
     // One tile of both rows, taken in passes of HV vectors per tensor: a short loop
     // body keeps the streaming code small for the instruction caches and the live
-    // registers few.  The only thing a consumer does for the top-k is to leave the
-    // maximum of every pass in shared memory; the top-k warps scan those.
+    // registers few.  All a consumer does for the top-k is to compare the maximum of
+    // every pass with the row's threshold.
     auto consume_tile = [&](uint32_t tile) -> bool {
       const uint32_t g = g0 + tile;
       const uint32_t s = g % STAGES;
@@ -689,16 +770,17 @@ __device__ void consumer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_row
       fphase ^= 1u << s;
       const uint4* sa = &sm.ring[s][0][wq * 32 + lane];
       const uint4* sp = &sm.ring[s][1][wq * 32 + lane];
-      float* pma = &sm.passmax[s][0][wq * 32 + lane];
-      float* pmp = &sm.passmax[s][1][wq * 32 + lane];
+      float ta = 0.f, tp = 0.f;
+      if (TOPK) { ta = lds_volatile_f32(&sm.tau[p][0]); tp = lds_volatile_f32(&sm.tau[p][1]); }
+      uint32_t id = tile * (uint32_t)TP + (uint32_t)(wq * 32 + lane);
       if ((int64_t)(tile + 1) * TV <= nvec) {
         // a full tile: no bounds checks
 #pragma unroll 1
-        for (int h = 0; h < VPL / HV; ++h, sa += HV * WPT * 32, sp += HV * WPT * 32, pma += WPT * 32, pmp += WPT * 32) {
+        for (int h = 0; h < VPL / HV; ++h, sa += HV * WPT * 32, sp += HV * WPT * 32, id += WPT * 32) {
           uint4 va[HV], vp[HV];
 #pragma unroll
           for (int j = 0; j < HV; ++j) { va[j] = sa[j * WPT * 32]; vp[j] = sp[j * WPT * 32]; }
-          if (!TOPK && h == VPL / HV - 1) {
+          if (h == VPL / HV - 1) {
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm.empty[s]);   // the last vectors are in registers: stage free
           }
@@ -711,13 +793,13 @@ __device__ void consumer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_row
             ma = fmaxf(ma, vm_a);
             mp = fmaxf(mp, vm_p);
           }
-          if (TOPK) { *pma = ma; *pmp = mp; }
+          if (TOPK && (ma >= ta || mp >= tp)) record_hits(sm, p, id, idmask, ma, mp, ta, tp);
         }
       } else {
         // the row's last, partial tile: bounds checked
         const uint32_t v0 = tile * TV + wq * 32 + lane;
 #pragma unroll 1
-        for (int h = 0; h < VPL / HV; ++h, pma += WPT * 32, pmp += WPT * 32) {
+        for (int h = 0; h < VPL / HV; ++h, id += WPT * 32) {
           float ma = JP_NEG_INF, mp = JP_NEG_INF;
 #pragma unroll 1
           for (int j = 0; j < HV; ++j) {
@@ -730,17 +812,12 @@ __device__ void consumer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_row
             ma = fmaxf(ma, vm_a);
             mp = fmaxf(mp, vm_p);
           }
-          if (TOPK) { *pma = ma; *pmp = mp; }
+          // a pass with no vector inside the row holds nothing
+          if (TOPK && (int64_t)(v0 + h * HV * WPT * 32) < nvec && (ma >= ta || mp >= tp))
+            record_hits(sm, p, id, idmask, ma, mp, ta, tp);
         }
-        if (!TOPK) {
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&sm.empty[s]);
-        }
-      }
-      if (TOPK) {
-        // the top-k warps of this row's slot take it from here; they free the stage
         __syncwarp();
-        if (lane == 0) mbar_arrive(&sm.seen[p][tile & 1u][s]);
+        if (lane == 0) mbar_arrive(&sm.empty[s]);
       }
       return true;
     };
@@ -781,199 +858,98 @@ __device__ void consumer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_row
 }
 
 // ---- top-k warps ---------------------------------------------------------------
-// One warp per (tensor t, row slot p).  For every tile of its row it waits until
-// the consumers are through with the stage, scans the 512 pass maxima they left
-// (16 per lane), counts in the histogram those at or above the running threshold
-// and copies the vectors behind them that are still alive from the stage into the
-// survivor buffer; then it frees the stage.  The threshold is the low edge of the
-// highest histogram bin with k counted passes at or above it: k different passes
-// hold k different entries of the row, so the k-th best logit is not below it.
+// One warp per (row slot p, tensor t); it owns rows p, p + NSLOT, ... of the CTA.
 template <int DT, int KPL>
-__device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, int t, int p, int par, int lane) {
+__device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, int t, int p, int lane) {
   constexpr int N = Vec<DT>::N;
   constexpr bool TOPK = KPL > 0;
   constexpr int KL = KPL > 0 ? KPL : 1;
   const int64_t nvec = A.V / N;
   const int tail = (int)(A.V - nvec * N);
   const uint32_t ntiles = nvec > 0 ? (uint32_t)((nvec + TV - 1) / TV) : 1u;
+  const uint32_t idmask = 0xffffffffu >> __clz(ntiles * (uint32_t)TP - 1u);
   const int k = A.k;
-  unsigned long long* stg = sm.skeys[p][t][par];
-  uint32_t* hist = sm.hist[p][t][par];
-  uint32_t* svp = sm.svpass[p][t][par];
-  float* svm = sm.svmax[p][t][par];
-  // The tiles of a row are shared out by parity between two warps, each with a
-  // histogram, a threshold and a survivor buffer of its own (the k-th best pass of
-  // half the tiles is still a lower bound of the row's k-th best logit).  The
-  // parity-0 warp hands its survivors over in shared memory at the end of the row;
-  // the parity-1 warp sorts both sets into the list and writes the record.
-  // A (slot, parity) `seen` barrier completes once per tile of that slot's rows with
-  // that parity, and this warp waits for every one of them in turn, so one phase bit
-  // per stage is enough.  (A barrier shared by warps that skip phases would not do: a
-  // parity wait cannot tell "not yet reached" from "done".)
-  uint32_t seen_phase = 0u;
+  unsigned long long* stg = sm.skeys[p][t];
+  uint32_t* hist = sm.hist[p][t];
+  uint32_t* cand = sm.cand[p][t];
   int lr = p;
-  for (int64_t it = (int64_t)blockIdx.x + (int64_t)p * gridDim.x; it < n_rows; it += 2ll * gridDim.x, lr += 2) {
-    const uint32_t ph = (uint32_t)((lr >> 1) & 1);
-    const uint32_t g0 = (uint32_t)lr * ntiles;        // ring position of this row's tile 0
+  for (int64_t it = (int64_t)blockIdx.x + (int64_t)p * gridDim.x; it < n_rows;
+       it += (int64_t)NSLOT * gridDim.x, lr += NSLOT) {
+    const uint32_t ph = (uint32_t)((lr / NSLOT) & 1);
     const int64_t row = A.list[it];
     const int64_t rrow = A.record_offset + row;
     const char* rmine = (const char*)(t == 0 ? A.za : A.zp) + row * A.ld * Vec<DT>::ESIZE;
-    unsigned long long L[KL];
-#pragma unroll
-    for (int j = 0; j < KL; ++j) L[j] = 0ull;
-    Tau tau{0u, 0, 0ull};
-    uint32_t base = 0u;
-    float tau_val = JP_NEG_INF;
-    int nsv = 0;                                      // candidate vectors kept so far
 
     // the sampled token's logit is needed only at the end of the row: fetch it now
     float zx = 0.f;
     if (lane == 0) zx = Vec<DT>::load_scalar(rmine, A.tokens[row]);
 
+    // set the slot up for this row: first threshold from a sample, empty histogram and buffer
+    float cur = JP_NEG_INF;
+    uint32_t base = 0xffffffffu, shift = 16u;
     if (TOPK) {
-      // the parity-1 warp must have read what this warp handed over two rows ago
-      if (par == 0 && !mbar_wait(&sm.final_done[p][t], ph ^ 1u, &sm.abort)) { raise_timeout(sm, A.sc); return; }
-      for (uint32_t tile = (uint32_t)par; tile < ntiles; tile += 2) {
-        const uint32_t g = g0 + tile;
-        const uint32_t s = g % STAGES;
-        if (!mbar_wait(&sm.seen[p][par][s], (seen_phase >> s) & 1u, &sm.abort)) { raise_timeout(sm, A.sc); return; }
-        seen_phase ^= 1u << s;
-        const float* pm = sm.passmax[s][t];
-        // this lane's 16 pass maxima: entries q * 128 + lane * 4 + c
-        float v[16];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          const float4 f = reinterpret_cast<const float4*>(pm)[q * 32 + lane];
-          v[4 * q] = f.x; v[4 * q + 1] = f.y; v[4 * q + 2] = f.z; v[4 * q + 3] = f.w;
-        }
-        // everything this warp needs of the tile is in registers: the stage (logits and
-        // pass maxima) may be refilled once the other tensor's warp says the same
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sm.empty[s]);
-        uint32_t hit = 0u;
-        if (tile == (uint32_t)par) {
-          // this warp's first tile of a new row: the histogram covers the NB order codes below this tile's maximum
-          // (everything lower shares bin 0, which stands for "no threshold"); every pass
-          // of the tile is counted, then the threshold is read off the histogram
-          float mx = v[0];
-#pragma unroll
-          for (int i = 1; i < 16; ++i) mx = fmaxf(mx, v[i]);
-          uint32_t top = __reduce_max_sync(0xffffffffu, order_code(mx));
-          base = top > (uint32_t)(NB - 1) ? top - (uint32_t)(NB - 1) : 0u;
-          for (int i = lane; i < NB; i += 32) hist[i] = 0u;
-          __syncwarp();
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const uint32_t code = order_code(v[i]);
-            atomicAdd(&hist[code > base ? code - base : 0u], 1u);
-          }
-          __syncwarp();
+      cur = sample_threshold<DT>(rmine, nvec, k, hist, reinterpret_cast<float*>(cand), base, shift, lane);
+      for (int i = lane; i < NB; i += 32) hist[i] = 0u;
+      if (lane == 0) {
+        sm.ncand[p][t] = 0u;
+        sm.bin_base[p][t] = base;
+        sm.bin_shift[p][t] = shift;
+        sm.tau[p][t] = cur;
+      }
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(&sm.slot_ready[p]);
+
+    // while the row streams: raise tau to the highest bin with k candidates at or above it
+    {
+      long long t0 = 0;
+      for (uint32_t i = 0; !mbar_try_wait_for(&sm.row_done[p], ph, (uint32_t)JP_TAU_NS); ++i) {
+        if (TOPK) {
           const int bin = find_tau_bin(hist, k, lane);
-          tau.code = bin > 0 ? base + (uint32_t)bin : 0u;
-          tau_val = bin > 0 ? code_value(tau.code) : JP_NEG_INF;
-#pragma unroll
-          for (int i = 0; i < 16; ++i) hit |= (v[i] >= tau_val ? 1u : 0u) << i;
-        } else {
-#pragma unroll
-          for (int i = 0; i < 16; ++i) hit |= (v[i] >= tau_val ? 1u : 0u) << i;
-          if (__any_sync(0xffffffffu, hit != 0u)) {
-            // count the passes at or above the threshold (those are all there are: it only rises)
-            uint32_t hcount = hit;
-            while (__any_sync(0xffffffffu, hcount != 0u)) {
-              if (hcount) {
-                const int i = __ffs(hcount) - 1;
-                hcount &= hcount - 1u;
-                const uint32_t code = order_code(select16(v, i));
-                const uint32_t bin = code > base ? code - base : 0u;
-                atomicAdd(&hist[bin < (uint32_t)(NB - 1) ? bin : (uint32_t)(NB - 1)], 1u);
-              }
-            }
-            __syncwarp();
-            const int bin = find_tau_bin(hist, k, lane);
-            tau.code = bin > 0 ? base + (uint32_t)bin : 0u;
-            tau_val = bin > 0 ? code_value(tau.code) : JP_NEG_INF;
-          }
-        }
-        // keep the passes behind the hits that can still hold one of the k best: only
-        // their place and their maximum; their vectors are read back when the row ends
-        while (__any_sync(0xffffffffu, hit != 0u)) {
-          const bool have = hit != 0u;
-          uint32_t id = 0u;
-          float m = JP_NEG_INF;
-          if (have) {
-            const int i = __ffs(hit) - 1;
-            hit &= hit - 1u;
-            const int e = (i >> 2) * 128 + lane * 4 + (i & 3);
-            id = tile * TP + (uint32_t)e;
-            m = select16(v, i);
-          }
-          const bool in = have && pass_alive(f32_order_bits(m), id, N, tau);
-          const uint32_t bm = __ballot_sync(0xffffffffu, in);
-          if (in) {
-            const int o = nsv + __popc(bm & ((1u << lane) - 1u));
-            svp[o] = id;
-            svm[o] = m;
-          }
-          nsv += __popc(bm);
-          __syncwarp();
-          if (nsv > SVCAP - 32) {
-            // the buffer is filling up: drop what the threshold has ruled out; if ties keep
-            // it full, sort the kept entries into the list and go on with the exact k-th key
-            nsv = compact_survivors(svp, svm, nsv, tau, N, lane);
-            if (nsv > SVCAP / 2) {
-              survivors_to_list<DT, KL>(L, svp, nsv, rmine, nvec, A.V, tau, stg, k, lane);
+          if (bin > 0) {
+            const float val = bin_edge(base, shift, bin);
+            if (val > cur) {
+              cur = val;
+              if (lane == 0) sts_volatile_f32(&sm.tau[p][t], cur);
             }
           }
         }
+        if ((i & 63u) == 0u) {
+          const long long now = clock64();
+          if (i == 0u) t0 = now;
+          const int give_up = *(volatile int*)&sm.abort || now - t0 > kSpinLimit;
+          if (__any_sync(0xffffffffu, give_up)) { raise_timeout(sm, A.sc); return; }
+        }
       }
     }
-
-    if (par == 0) {
-      // this half of the row: sort the survivors into the list and leave the list in
-      // this warp's key buffer for the parity-1 warp
-      if (TOPK) {
-        nsv = compact_survivors(svp, svm, nsv, tau, N, lane);
-        survivors_to_list<DT, KL>(L, svp, nsv, rmine, nvec, A.V, tau, stg, k, lane);
-#pragma unroll
-        for (int j = 0; j < KL; ++j) stg[lane * KL + j] = L[j];
-        if (lane == 0) { sm.xstate[p][t][0] = 0; sm.xstate[p][t][1] = (int)tau.code; sm.xstate[p][t][2] = 32 * KL; }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sm.scan_done[p][t]);
-      }
-      continue;
-    }
-
-    // the consumers' per-warp (max, sum) pairs of this row
-    if (!mbar_wait(&sm.row_done[p], ph, &sm.abort)) { raise_timeout(sm, A.sc); return; }
 
     if (TOPK) {
       const char* ra = (const char*)A.za + row * A.ld * Vec<DT>::ESIZE;
       const char* rp = (const char*)A.zp + row * A.ld * Vec<DT>::ESIZE;
-      // this warp's half of the row into its list ...
-      nsv = compact_survivors(svp, svm, nsv, tau, N, lane);
-      survivors_to_list<DT, KL>(L, svp, nsv, rmine, nvec, A.V, tau, stg, k, lane);
-      // ... then the other half's list
-      if (!mbar_wait(&sm.scan_done[p][t], ph, &sm.abort)) { raise_timeout(sm, A.sc); return; }
-      const int nk0 = sm.xstate[p][t][2];
+      unsigned long long L[KL];
+#pragma unroll
+      for (int j = 0; j < KL; ++j) L[j] = 0ull;
+      unsigned long long kth;
+      uint32_t tau_ob = 0u;
+      const uint32_t total = lds_volatile_u32(&sm.ncand[p][t]);
+      if (total > (uint32_t)CAP) {
+        kth = scan_row_exact<DT, KL>(L, rmine, nvec, A.V, stg, k, lane);
+      } else {
+        const int bin = find_tau_bin(hist, k, lane);
+        if (bin > 0) {
+          const float val = bin_edge(base, shift, bin);
+          if (val > cur) cur = val;
+        }
+        tau_ob = f32_order_bits(cur);
+        const int n = compact_candidates(cand, (int)total, tau_ob, idmask, lane);
+        kth = candidates_to_list<DT, KL>(L, cand, n, idmask, rmine, nvec, A.V, tau_ob, stg, k, lane);
+      }
       if (tail > 0) {                 // the ragged end of the row
         uint4 v = Vec<DT>::neg_inf();
         if (lane == 0) v = load_tail_vector<DT>(rmine, nvec * N, tail);
-        int staged = stage_entries<DT>(v, (uint32_t)nvec, lane == 0, A.V, tau, stg, 0, lane);
-        tau.key = merge_all<KL>(L, stg, staged, k, lane);
+        int staged = stage_entries<DT>(v, (uint32_t)nvec, lane == 0, A.V, tau_ob, kth, stg, 0, lane);
+        kth = merge_all<KL>(L, stg, staged, k, lane);
       }
-      if (nk0 > 0) {
-        int staged = 0;
-        for (int b = 0; b < nk0; b += 32) {
-          const unsigned long long key = sm.skeys[p][t][0][b + lane];
-          const bool keep = key > tau.key;
-          const uint32_t m = __ballot_sync(0xffffffffu, keep);
-          if (keep) stg[staged + __popc(m & ((1u << lane) - 1u))] = key;
-          staged += __popc(m);
-        }
-        tau.key = merge_all<KL>(L, stg, staged, k, lane);
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&sm.final_done[p][t]);     // the parity-0 warp may reuse its buffers
       // the record: this tensor's list, best first, every entry with both logits
 #pragma unroll
       for (int j = 0; j < KL; ++j) {
@@ -1012,7 +988,6 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
       if (!isfinite(lsef)) atomicAdd(&A.sc->n_nonfinite, 1ull);
     }
     __syncwarp();
-    if (lane == 0) mbar_arrive(&sm.slot_free[p]);
   }
 }
 
@@ -1025,13 +1000,11 @@ __global__ void __launch_bounds__(NTHREADS, 1) stream_kernel(StreamArgs A) {
   if (tid == 0) {
     for (int s = 0; s < STAGES; ++s) {
       for (int q = 0; q < NG; ++q) mbar_init(&sm.full[q][s], 1);
-      for (int q = 0; q < 4; ++q) mbar_init(&sm.seen[q >> 1][q & 1][s], WPT);
-      mbar_init(&sm.empty[s], KPL > 0 ? 2 : WPT);     // with top-k the two top-k warps of the row free the stage
+      mbar_init(&sm.empty[s], WPT);
     }
-    for (int p = 0; p < 2; ++p) {
+    for (int p = 0; p < NSLOT; ++p) {
       mbar_init(&sm.row_done[p], NC);
-      mbar_init(&sm.slot_free[p], 2);
-      for (int t = 0; t < 2; ++t) { mbar_init(&sm.scan_done[p][t], 1); mbar_init(&sm.final_done[p][t], 1); }
+      mbar_init(&sm.slot_ready[p], 2);
     }
     sm.abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -1045,8 +1018,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) stream_kernel(StreamArgs A) {
     consumer_loop<DT, (KPL > 0)>(A, sm, n_rows, warp - 1, lane);
   } else {
     const int tw = warp - 1 - NC;
-    // without top-k there is nothing to share out: the parity-0 warps leave
-    if (KPL > 0 || (tw >> 2) == 1) topk_loop<DT, KPL>(A, sm, n_rows, tw & 1, (tw >> 1) & 1, tw >> 2, lane);
+    topk_loop<DT, KPL>(A, sm, n_rows, tw & 1, tw >> 1, lane);
   }
 }
 
