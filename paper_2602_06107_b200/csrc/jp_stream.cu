@@ -770,7 +770,7 @@ __device__ void consumer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_row
       fphase ^= 1u << s;
       const uint4* sa = &sm.ring[s][0][wq * 32 + lane];
       const uint4* sp = &sm.ring[s][1][wq * 32 + lane];
-      float ta = __int_as_float(0x7f800000), tp = ta;      // without top-k: nothing reaches +inf
+      float ta = 0.f, tp = 0.f;
       if (TOPK) { ta = lds_volatile_f32(&sm.tau[p][0]); tp = lds_volatile_f32(&sm.tau[p][1]); }
       uint32_t id = tile * (uint32_t)TP + (uint32_t)(wq * 32 + lane);
       if ((int64_t)(tile + 1) * TV <= nvec) {
@@ -780,31 +780,22 @@ __device__ void consumer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_row
           uint4 va[HV], vp[HV];
 #pragma unroll
           for (int j = 0; j < HV; ++j) { va[j] = sa[j * WPT * 32]; vp[j] = sp[j * WPT * 32]; }
-          float ma = JP_NEG_INF, mp = JP_NEG_INF, vm_a[HV], vm_p[HV];
+          float ma = JP_NEG_INF, mp = JP_NEG_INF;
 #pragma unroll
           for (int j = 0; j < HV; ++j) {
-            vm_a[j] = Vec<DT>::vmax(va[j]);
-            vm_p[j] = Vec<DT>::vmax(vp[j]);
-            ma = fmaxf(ma, vm_a[j]);
-            mp = fmaxf(mp, vm_p[j]);
+            const float vm_a = Vec<DT>::vmax(va[j]), vm_p = Vec<DT>::vmax(vp[j]);
+            accumulate<DT>(va[j], vm_a, oa);
+            accumulate<DT>(vp[j], vm_p, op);
+            ma = fmaxf(ma, vm_a);
+            mp = fmaxf(mp, vm_p);
           }
-          const bool hit = ma >= ta || mp >= tp;
-          if (h == VPL / HV - 1) {
-            // The tile's last vectors are in registers: the stage may be refilled.  The arrival
-            // must not overtake the loads (a load still queued behind a burst of shared-memory
-            // atomics was once seen to return the next tile's bytes), so it hangs on a vote that
-            // needs every lane's loaded data: the lane that arrives is chosen by the vote.
-            const uint32_t hits = __ballot_sync(0xffffffffu, hit);
-            const int leader = hits ? __ffs(hits) - 1 : 0;
-            if (lane == leader) mbar_arrive(&sm.empty[s]);
-          }
-#pragma unroll
-          for (int j = 0; j < HV; ++j) {
-            accumulate<DT>(va[j], vm_a[j], oa);
-            accumulate<DT>(vp[j], vm_p[j], op);
-          }
-          if (TOPK && hit) record_hits(sm, p, id, idmask, ma, mp, ta, tp);
+          if (TOPK && (ma >= ta || mp >= tp)) record_hits(sm, p, id, idmask, ma, mp, ta, tp);
         }
+        // Free the stage only now that arithmetic has consumed every loaded vector.  An arrival
+        // issued right after the last loads can overtake them: a load still queued behind a burst
+        // of shared-memory atomics was seen to return the next tile's bytes.
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.empty[s]);
       } else {
         // the row's last, partial tile: bounds checked
         const uint32_t v0 = tile * TV + wq * 32 + lane;
