@@ -93,8 +93,8 @@ constexpr long long kSpinLimit = 4000000000ll;   // clock cycles a wait may last
 struct __align__(128) StreamSmem {
   uint4 ring[STAGES][2][TV];              // [stage][tensor][vector]
   unsigned long long skeys[NSLOT][2][SCAP];  // [slot][tensor] keys waiting to be sorted into the list
-  uint32_t cand[NSLOT][2][CAP];           // [slot][tensor] candidate passes: high bits of the maximum's order bits | pass id
-  uint32_t hist[NSLOT][2][NB];            // [slot][tensor] candidate passes per bin of their maximum
+  uint32_t cand[NSLOT][2][CAP];           // [slot][tensor] candidate passes: high bits of the maximum's order bits | pass id; 0 = not written yet
+  uint32_t hist[NSLOT][2][NB];            // [slot][tensor] candidate passes per bin of their maximum (kept by the top-k warp)
   unsigned long long full[NG][STAGES];    // [consumer group] producer -> that group: the tile's bytes have landed.  One set per
                                           // group, so that every waiter sees every phase of its barriers in turn: a group that
                                           // skipped the other group's phases could take an unfinished earlier phase for its own
@@ -103,8 +103,6 @@ struct __align__(128) StreamSmem {
   unsigned long long row_done[NSLOT];     // consumers -> top-k warps: the row has been streamed
   float tau[NSLOT][2];                    // running threshold (only rises while a row streams)
   uint32_t ncand[NSLOT][2];               // candidate passes appended so far (may pass CAP: then the row is re-scanned)
-  uint32_t bin_base[NSLOT][2];            // bin of a maximum = (order bits >> bin_shift) - bin_base, clipped to [0, NB-1]
-  uint32_t bin_shift[NSLOT][2];
   float part_mL[NSLOT][2][NC];
   float part_s[NSLOT][2][NC];
   int abort;
@@ -493,23 +491,38 @@ __device__ __forceinline__ float bin_edge(uint32_t base, uint32_t shift, int bin
   return order_bits_f32(code << shift);
 }
 
-// What a consumer lane does with a pass whose maximum reached the row's threshold:
-// count it in the histogram its top-k warp reads tau from and append it to the
-// candidates (the high bits of the maximum's order bits over the pass id).  Out of
-// line: it runs for a fraction of a percent of the passes.
-__device__ __noinline__ void record_hits(StreamSmem& sm, int p, uint32_t id, uint32_t idmask, float ma, float mp,
-                                         float ta, float tp) {
-#pragma unroll 1
-  for (int t = 0; t < 2; ++t) {
-    const float m = t == 0 ? ma : mp;
-    if (!(m >= (t == 0 ? ta : tp))) continue;
-    const uint32_t ob = f32_order_bits(m);
-    const uint32_t c = ob >> sm.bin_shift[p][t], base = sm.bin_base[p][t];
-    const uint32_t bin = c > base ? (c - base < (uint32_t)(NB - 1) ? c - base : (uint32_t)(NB - 1)) : 0u;
-    atomicAdd(&sm.hist[p][t][bin], 1u);
-    const uint32_t o = atomicAdd(&sm.ncand[p][t], 1u);
-    if (o < (uint32_t)CAP) sm.cand[p][t][o] = (ob & ~idmask) | id;
+// What a consumer lane does with a pass whose maximum reached the row's threshold
+// (a fraction of a percent of the passes): append it to the row's candidates as the
+// high bits of the maximum's order bits over the pass id.  The slot's top-k warp
+// counts the candidates into its histogram as they appear.
+__device__ __forceinline__ void record_hit(uint32_t* ncand, uint32_t* cand, uint32_t id, uint32_t idmask, float m) {
+  const uint32_t o = atomicAdd(ncand, 1u);
+  if (o < (uint32_t)CAP) cand[o] = (f32_order_bits(m) & ~idmask) | id;
+}
+
+// Top-k warp: counts the candidates [seen, n) that have been written so far into
+// the histogram and returns the new `seen`.  A consumer bumps the counter before
+// it writes the entry, so an entry may still read 0 (the buffer is zeroed before
+// the row starts and no entry of a finite maximum is 0): counting stops there
+// unless `all` says that the row is done and everything has been written.
+__device__ __forceinline__ uint32_t count_candidates(const uint32_t* cand, uint32_t seen, uint32_t n, uint32_t* hist,
+                                                     uint32_t base, uint32_t shift, bool all, int lane) {
+  while (seen < n) {
+    const uint32_t i = seen + (uint32_t)lane;
+    const uint32_t e = i < n ? lds_volatile_u32(cand + i) : 0u;
+    const bool there = i < n && (all || e != 0u);
+    const uint32_t missing = ~__ballot_sync(0xffffffffu, there);
+    const uint32_t run = missing ? (uint32_t)(__ffs(missing) - 1) : 32u;   // leading lanes whose entry is there
+    if ((uint32_t)lane < run) {
+      const uint32_t c = e >> shift;                       // shift >= id bits: the pass id falls away
+      const uint32_t bin = c > base ? (c - base < (uint32_t)(NB - 1) ? c - base : (uint32_t)(NB - 1)) : 0u;
+      atomicAdd(&hist[bin], 1u);
+    }
+    seen += run;
+    if (run < 32u) break;
   }
+  __syncwarp();
+  return seen;
 }
 
 // Appends to the key buffer the keys of one vector's entries (one vector per lane)
@@ -624,14 +637,14 @@ __device__ __noinline__ unsigned long long scan_row_exact(unsigned long long (&L
 // vectors, as the low edge of its histogram bin (-inf if the sample has fewer than
 // k vectors), and the bin geometry (base, shift) for the row's candidate histogram.
 // The window of NB codes is anchored at the sample's maximum; the shift starts at 16
-// (bf16 resolution) and grows until the k-th best falls inside the window, so a
+// (bf16 resolution; more for rows so long that a pass id needs more than 16 bits) and grows until the k-th best falls inside the window, so a
 // sample that spans many binades, or zero, gets coarser bins rather than none.
 template <int DT>
 __device__ __noinline__ float sample_threshold(const char* row, int64_t nvec, int k, uint32_t* hist, float* park,
-                                               uint32_t& base, uint32_t& shift, int lane) {
+                                               uint32_t& base, uint32_t& shift, uint32_t min_shift, int lane) {
   const int ns = (int)(nvec < (int64_t)SAMPLE ? nvec : (int64_t)SAMPLE);
   base = 0xffffffffu;                       // nothing above it: every maximum counts in bin 0 = "no threshold"
-  shift = 16u;
+  shift = min_shift > 16u ? min_shift : 16u;  // a candidate keeps only the order bits above its pass id
   if (ns < k) return JP_NEG_INF;
   float mx = JP_NEG_INF;
 #pragma unroll 1
@@ -655,7 +668,7 @@ __device__ __noinline__ float sample_threshold(const char* row, int64_t nvec, in
   const uint32_t ob_max = f32_order_bits(mx);
   __syncwarp();
   float tau0 = JP_NEG_INF;
-  for (uint32_t sh = 16u; sh < 32u; ++sh) {
+  for (uint32_t sh = shift; sh < 32u; ++sh) {
     const uint32_t cmax = ob_max >> sh;
     const uint32_t b0 = cmax > (uint32_t)(NB - 1) ? cmax - (uint32_t)(NB - 1) : 0u;
     for (int i = lane; i < NB; i += 32) hist[i] = 0u;
@@ -789,7 +802,10 @@ __device__ void consumer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_row
             ma = fmaxf(ma, vm_a);
             mp = fmaxf(mp, vm_p);
           }
-          if (TOPK && (ma >= ta || mp >= tp)) record_hits(sm, p, id, idmask, ma, mp, ta, tp);
+          if (TOPK) {
+            if (ma >= ta) record_hit(&sm.ncand[p][0], sm.cand[p][0], id, idmask, ma);
+            if (mp >= tp) record_hit(&sm.ncand[p][1], sm.cand[p][1], id, idmask, mp);
+          }
         }
         // Free the stage only now that arithmetic has consumed every loaded vector.  An arrival
         // issued right after the last loads can overtake them: a load still queued behind a burst
@@ -814,8 +830,10 @@ __device__ void consumer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_row
             mp = fmaxf(mp, vm_p);
           }
           // a pass with no vector inside the row holds nothing
-          if (TOPK && (int64_t)(v0 + h * HV * WPT * 32) < nvec && (ma >= ta || mp >= tp))
-            record_hits(sm, p, id, idmask, ma, mp, ta, tp);
+          if (TOPK && (int64_t)(v0 + h * HV * WPT * 32) < nvec) {
+            if (ma >= ta) record_hit(&sm.ncand[p][0], sm.cand[p][0], id, idmask, ma);
+            if (mp >= tp) record_hit(&sm.ncand[p][1], sm.cand[p][1], id, idmask, mp);
+          }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&sm.empty[s]);
@@ -868,7 +886,8 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
   const int64_t nvec = A.V / N;
   const int tail = (int)(A.V - nvec * N);
   const uint32_t ntiles = nvec > 0 ? (uint32_t)((nvec + TV - 1) / TV) : 1u;
-  const uint32_t idmask = 0xffffffffu >> __clz(ntiles * (uint32_t)TP - 1u);
+  const uint32_t idbits = 32u - (uint32_t)__clz(ntiles * (uint32_t)TP - 1u);
+  const uint32_t idmask = 0xffffffffu >> (32u - idbits);
   const int k = A.k;
   unsigned long long* stg = sm.skeys[p][t];
   uint32_t* hist = sm.hist[p][t];
@@ -889,15 +908,15 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
     float cur = JP_NEG_INF;
     uint32_t base = 0xffffffffu, shift = 16u;
     if (TOPK) {
-      cur = sample_threshold<DT>(rmine, nvec, k, hist, reinterpret_cast<float*>(cand), base, shift, lane);
+      cur = sample_threshold<DT>(rmine, nvec, k, hist, reinterpret_cast<float*>(cand), base, shift, idbits, lane);
       for (int i = lane; i < NB; i += 32) hist[i] = 0u;
+      for (int i = lane; i < CAP / 4; i += 32) reinterpret_cast<uint4*>(cand)[i] = make_uint4(0u, 0u, 0u, 0u);
       if (lane == 0) {
         sm.ncand[p][t] = 0u;
-        sm.bin_base[p][t] = base;
-        sm.bin_shift[p][t] = shift;
         sm.tau[p][t] = cur;
       }
     }
+    uint32_t seen = 0u;                       // candidates counted into the histogram so far
     __syncwarp();
     if (lane == 0) mbar_arrive(&sm.slot_ready[p]);
 
@@ -906,12 +925,17 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
       long long t0 = 0;
       for (uint32_t i = 0; !mbar_try_wait_for(&sm.row_done[p], ph, (uint32_t)JP_TAU_NS); ++i) {
         if (TOPK) {
-          const int bin = find_tau_bin(hist, k, lane);
-          if (bin > 0) {
-            const float val = bin_edge(base, shift, bin);
-            if (val > cur) {
-              cur = val;
-              if (lane == 0) sts_volatile_f32(&sm.tau[p][t], cur);
+          const uint32_t nc = lds_volatile_u32(&sm.ncand[p][t]);
+          const uint32_t n = nc < (uint32_t)CAP ? nc : (uint32_t)CAP;
+          if (n > seen) {
+            seen = count_candidates(cand, seen, n, hist, base, shift, false, lane);
+            const int bin = find_tau_bin(hist, k, lane);
+            if (bin > 0) {
+              const float val = bin_edge(base, shift, bin);
+              if (val > cur) {
+                cur = val;
+                if (lane == 0) sts_volatile_f32(&sm.tau[p][t], cur);
+              }
             }
           }
         }
@@ -936,6 +960,7 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
       if (total > (uint32_t)CAP) {
         kth = scan_row_exact<DT, KL>(L, rmine, nvec, A.V, stg, k, lane);
       } else {
+        count_candidates(cand, seen, total, hist, base, shift, true, lane);
         const int bin = find_tau_bin(hist, k, lane);
         if (bin > 0) {
           const float val = bin_edge(base, shift, bin);
