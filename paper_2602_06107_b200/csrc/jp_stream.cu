@@ -53,14 +53,8 @@ namespace jp {
 #ifndef JP_VPL
 #define JP_VPL 4
 #endif
-#ifndef JP_STAGES
-#define JP_STAGES 5
-#endif
 #ifndef JP_NG
 #define JP_NG 2
-#endif
-#ifndef JP_CAP
-#define JP_CAP 1024
 #endif
 #ifndef JP_SAMPLE_VPL
 #define JP_SAMPLE_VPL 32
@@ -76,21 +70,26 @@ constexpr int TV = WPT * 32 * VPL;        // vectors per tensor per tile
 constexpr int HV = 2;                     // vectors per tensor a lane holds at a time
 static_assert(JP_VPL % HV == 0, "a tile is taken in passes of HV vectors");
 static_assert(JP_NG == 2, "tiles go to consumer groups by parity; the producer keeps two phase masks");
-static_assert(NC % NG == 0 && NG < JP_STAGES, "consumer groups must divide the warps and fit the ring");
-constexpr int STAGES = JP_STAGES;
+static_assert(NC % NG == 0, "consumer groups must divide the warps");
 constexpr int NSLOT = 4;                  // rows in flight between the consumers and the top-k warps
 constexpr int SCAP = 288;                 // keys a top-k warp buffers before it sorts them into the list
-constexpr int CAP = JP_CAP;               // candidate passes a row may collect before it falls back to a re-scan
 constexpr int NB = 256;                   // histogram bins
 constexpr int TP = TV / HV;               // passes per tensor per tile
 constexpr int SAMPLE = 32 * JP_SAMPLE_VPL;  // vectors of a row its top-k warp looks at before the row starts
-static_assert(SAMPLE <= CAP, "the sample's vector maxima are parked in the candidate buffer");
 constexpr int NTOPK = NSLOT * 2;          // top-k warps: (slot, tensor)
 constexpr int NWARPS = 1 + NC + NTOPK;
 constexpr int NTHREADS = NWARPS * 32;
 constexpr long long kSpinLimit = 4000000000ll;   // clock cycles a wait may last (about 2 s)
 
-struct __align__(128) StreamSmem {
+// NSTAGES: depth of the ring.  NCAND: candidate passes a row may collect before it
+// falls back to a re-scan.  The kernel for k <= 64 takes 5 stages and 1024 candidates;
+// for k <= 128 (about k (1 + ln(passes / k)) candidates per row) 4 stages and 2048.
+template <int NSTAGES, int NCAND>
+struct __align__(128) StreamSmemT {
+  static constexpr int STAGES = NSTAGES;
+  static constexpr int CAP = NCAND;
+  static_assert(NG < NSTAGES, "every consumer group needs a stage of its own and one must be in flight");
+  static_assert(SAMPLE <= NCAND, "the sample's vector maxima are parked in the candidate buffer");
   uint4 ring[STAGES][2][TV];              // [stage][tensor][vector]
   unsigned long long skeys[NSLOT][2][SCAP];  // [slot][tensor] keys waiting to be sorted into the list
   uint32_t cand[NSLOT][2][CAP];           // [slot][tensor] candidate passes: high bits of the maximum's order bits | pass id; 0 = not written yet
@@ -108,7 +107,10 @@ struct __align__(128) StreamSmem {
   int abort;
 };
 
-static_assert(sizeof(StreamSmem) <= 232448, "the CTA's shared memory exceeds the 227 KB an sm_100 CTA can have");
+template <int KPL>
+using StreamSmemFor = StreamSmemT<(KPL == 4 ? 4 : 5), (KPL == 4 ? 2048 : 1024)>;
+static_assert(sizeof(StreamSmemFor<1>) <= 232448 && sizeof(StreamSmemFor<4>) <= 232448,
+              "the CTA's shared memory exceeds the 227 KB an sm_100 CTA can have");
 
 // ---- mbarrier / bulk-copy wrappers ----------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -495,6 +497,7 @@ __device__ __forceinline__ float bin_edge(uint32_t base, uint32_t shift, int bin
 // (a fraction of a percent of the passes): append it to the row's candidates as the
 // high bits of the maximum's order bits over the pass id.  The slot's top-k warp
 // counts the candidates into its histogram as they appear.
+template <int CAP>
 __device__ __forceinline__ void record_hit(uint32_t* ncand, uint32_t* cand, uint32_t id, uint32_t idmask, float m) {
   const uint32_t o = atomicAdd(ncand, 1u);
   if (o < (uint32_t)CAP) cand[o] = (f32_order_bits(m) & ~idmask) | id;
@@ -693,15 +696,17 @@ __device__ __noinline__ float sample_threshold(const char* row, int64_t nvec, in
   return tau0;
 }
 
-__device__ __forceinline__ void raise_timeout(StreamSmem& sm, Scalars* sc) {
+template <class SM>
+__device__ __forceinline__ void raise_timeout(SM& sm, Scalars* sc) {
   sm.abort = 1;
   atomicExch(&sc->status, (int)JP_ERR_TIMEOUT);
 }
 
 // ---- producer ---------------------------------------------------------------
-template <int DT>
-__device__ void producer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows) {
+template <int DT, class SM>
+__device__ void producer_loop(const StreamArgs& A, SM& sm, int64_t n_rows) {
   constexpr int N = Vec<DT>::N;
+  constexpr int STAGES = SM::STAGES;
   const int64_t nvec = A.V / N;
   const int ntiles = nvec > 0 ? (int)((nvec + TV - 1) / TV) : 1;
   const uint32_t last_bytes = (uint32_t)((nvec - (int64_t)(ntiles - 1) * TV) * 16);   // 0 only when nvec == 0
@@ -752,9 +757,10 @@ __device__ void producer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_row
 }
 
 // ---- consumers ----------------------------------------------------------------
-template <int DT, bool TOPK>
-__device__ void consumer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, int cw, int lane) {
+template <int DT, bool TOPK, class SM>
+__device__ void consumer_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int cw, int lane) {
   constexpr int N = Vec<DT>::N;
+  constexpr int STAGES = SM::STAGES, CAP = SM::CAP;
   const int64_t nvec = A.V / N;
   const int tail = (int)(A.V - nvec * N);
   const uint32_t ntiles = nvec > 0 ? (uint32_t)((nvec + TV - 1) / TV) : 1u;
@@ -803,8 +809,8 @@ __device__ void consumer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_row
             mp = fmaxf(mp, vm_p);
           }
           if (TOPK) {
-            if (ma >= ta) record_hit(&sm.ncand[p][0], sm.cand[p][0], id, idmask, ma);
-            if (mp >= tp) record_hit(&sm.ncand[p][1], sm.cand[p][1], id, idmask, mp);
+            if (ma >= ta) record_hit<CAP>(&sm.ncand[p][0], sm.cand[p][0], id, idmask, ma);
+            if (mp >= tp) record_hit<CAP>(&sm.ncand[p][1], sm.cand[p][1], id, idmask, mp);
           }
         }
         // Free the stage only now that arithmetic has consumed every loaded vector.  An arrival
@@ -831,8 +837,8 @@ __device__ void consumer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_row
           }
           // a pass with no vector inside the row holds nothing
           if (TOPK && (int64_t)(v0 + h * HV * WPT * 32) < nvec) {
-            if (ma >= ta) record_hit(&sm.ncand[p][0], sm.cand[p][0], id, idmask, ma);
-            if (mp >= tp) record_hit(&sm.ncand[p][1], sm.cand[p][1], id, idmask, mp);
+            if (ma >= ta) record_hit<CAP>(&sm.ncand[p][0], sm.cand[p][0], id, idmask, ma);
+            if (mp >= tp) record_hit<CAP>(&sm.ncand[p][1], sm.cand[p][1], id, idmask, mp);
           }
         }
         __syncwarp();
@@ -878,9 +884,10 @@ __device__ void consumer_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_row
 
 // ---- top-k warps ---------------------------------------------------------------
 // One warp per (row slot p, tensor t); it owns rows p, p + NSLOT, ... of the CTA.
-template <int DT, int KPL>
-__device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, int t, int p, int lane) {
+template <int DT, int KPL, class SM>
+__device__ void topk_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int t, int p, int lane) {
   constexpr int N = Vec<DT>::N;
+  constexpr int CAP = SM::CAP;
   constexpr bool TOPK = KPL > 0;
   constexpr int KL = KPL > 0 ? KPL : 1;
   const int64_t nvec = A.V / N;
@@ -1020,7 +1027,9 @@ __device__ void topk_loop(const StreamArgs& A, StreamSmem& sm, int64_t n_rows, i
 template <int DT, int KPL>
 __global__ void __launch_bounds__(NTHREADS, 1) stream_kernel(StreamArgs A) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
-  StreamSmem& sm = *reinterpret_cast<StreamSmem*>(smem_raw);
+  using SM = StreamSmemFor<KPL>;
+  constexpr int STAGES = SM::STAGES;
+  SM& sm = *reinterpret_cast<SM*>(smem_raw);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
   if (tid == 0) {
@@ -1039,12 +1048,12 @@ __global__ void __launch_bounds__(NTHREADS, 1) stream_kernel(StreamArgs A) {
   const int64_t n_rows = A.sc->n_list;
 
   if (warp == 0) {
-    if (lane == 0) producer_loop<DT>(A, sm, n_rows);
+    if (lane == 0) producer_loop<DT, SM>(A, sm, n_rows);
   } else if (warp <= NC) {
-    consumer_loop<DT, (KPL > 0)>(A, sm, n_rows, warp - 1, lane);
+    consumer_loop<DT, (KPL > 0), SM>(A, sm, n_rows, warp - 1, lane);
   } else {
     const int tw = warp - 1 - NC;
-    topk_loop<DT, KPL>(A, sm, n_rows, tw & 1, tw >> 1, lane);
+    topk_loop<DT, KPL, SM>(A, sm, n_rows, tw & 1, tw >> 1, lane);
   }
 }
 
@@ -1164,9 +1173,9 @@ template <int DT, int KPL>
 static cudaError_t launch_stream_variant(const StreamArgs& a, cudaStream_t s, int grid) {
   // per device, and cheap: set on every launch rather than cached per process
   cudaError_t e = cudaFuncSetAttribute(stream_kernel<DT, KPL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)sizeof(StreamSmem));
+                                       (int)sizeof(StreamSmemFor<KPL>));
   if (e != cudaSuccess) return e;
-  stream_kernel<DT, KPL><<<grid, NTHREADS, sizeof(StreamSmem), s>>>(a);
+  stream_kernel<DT, KPL><<<grid, NTHREADS, sizeof(StreamSmemFor<KPL>), s>>>(a);
   return cudaGetLastError();
 }
 
