@@ -77,16 +77,19 @@ template <> struct Vec<JP_BF16> {
     return __uint_as_float((e & 1) ? (w & 0xffff0000u) : (w << 16));
   }
   __device__ static __forceinline__ float vmax(const uint4& v) {
-#ifdef JP_VMAX_F32
-    float m0 = fmaxf(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xffff0000u));
-    float m1 = fmaxf(__uint_as_float(v.y << 16), __uint_as_float(v.y & 0xffff0000u));
-    float m2 = fmaxf(__uint_as_float(v.z << 16), __uint_as_float(v.z & 0xffff0000u));
-    float m3 = fmaxf(__uint_as_float(v.w << 16), __uint_as_float(v.w & 0xffff0000u));
-    return fmaxf(fmaxf(m0, m1), fmaxf(m2, m3));
-#endif
     __nv_bfloat162 a = __hmax2(*(const __nv_bfloat162*)&v.x, *(const __nv_bfloat162*)&v.y);
     __nv_bfloat162 b = __hmax2(*(const __nv_bfloat162*)&v.z, *(const __nv_bfloat162*)&v.w);
     a = __hmax2(a, b);
+    uint32_t w = *(uint32_t*)&a;
+    return fmaxf(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+  }
+  // maximum over two vectors: one packed tree, unpacked once
+  __device__ static __forceinline__ float vmax2(const uint4& u, const uint4& v) {
+    __nv_bfloat162 a = __hmax2(*(const __nv_bfloat162*)&u.x, *(const __nv_bfloat162*)&u.y);
+    __nv_bfloat162 b = __hmax2(*(const __nv_bfloat162*)&u.z, *(const __nv_bfloat162*)&u.w);
+    __nv_bfloat162 c = __hmax2(*(const __nv_bfloat162*)&v.x, *(const __nv_bfloat162*)&v.y);
+    __nv_bfloat162 d = __hmax2(*(const __nv_bfloat162*)&v.z, *(const __nv_bfloat162*)&v.w);
+    a = __hmax2(__hmax2(a, b), __hmax2(c, d));
     uint32_t w = *(uint32_t*)&a;
     return fmaxf(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
   }
@@ -118,6 +121,7 @@ template <> struct Vec<JP_F32> {
     return fmaxf(fmaxf(__uint_as_float(v.x), __uint_as_float(v.y)),
                  fmaxf(__uint_as_float(v.z), __uint_as_float(v.w)));
   }
+  __device__ static __forceinline__ float vmax2(const uint4& u, const uint4& v) { return fmaxf(vmax(u), vmax(v)); }
   __device__ static __forceinline__ float load_scalar(const void* row, int64_t i) {
     return ((const float*)row)[i];
   }

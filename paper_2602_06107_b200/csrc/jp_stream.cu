@@ -149,10 +149,10 @@ __device__ __forceinline__ bool mbar_try_wait_for(unsigned long long* bar, uint3
       : "memory");
   return ok != 0;
 }
-// Bounded wait; false = gave up (or another warp did).  The clock is read once in
-// 64 polls, each of which may itself suspend the thread for a while.
-__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity, volatile int* abort) {
-  if (mbar_try_wait(bar, parity)) return true;
+// Bounded wait; false = gave up (or another warp did).  The first poll is inline;
+// the loop is out of line (the streaming code stays small).  The clock is read once
+// in 64 polls, each of which may itself suspend the thread for a while.
+__device__ __noinline__ bool mbar_wait_slow(unsigned long long* bar, uint32_t parity, volatile int* abort) {
   long long t0 = 0;
   for (uint32_t i = 0;; ++i) {
     if (mbar_try_wait_for(bar, parity, 2000u)) return true;
@@ -163,6 +163,10 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t pari
       else if (now - t0 > kSpinLimit) { *abort = 1; return false; }
     }
   }
+}
+__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity, volatile int* abort) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort);
 }
 __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, unsigned long long* bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
@@ -273,9 +277,9 @@ __device__ __forceinline__ unsigned long long add_exp2_poly2(unsigned long long 
   return ffma2(p2, pack2(sc0, sc1), s2);
 }
 
-// One 16-byte vector into the online (max, sum).
-template <int DT>
-__device__ __forceinline__ void accumulate(const uint4& v, float vm, Online& o) {
+// Raises the running maximum to vm (if it is higher) and moves the sums to the new
+// reference exponent.
+__device__ __forceinline__ void raise_max(float vm, Online& o) {
   if (vm > o.m) {
     const float nmL = ceilf(__fmul_rn(vm, kLog2e));
     if (o.m == JP_NEG_INF) {
@@ -287,28 +291,12 @@ __device__ __forceinline__ void accumulate(const uint4& v, float vm, Online& o) 
     o.m = vm;
     o.mL = nmL;
   }
-#ifdef JP_SCALAR_ACC
-  {
-    float s0, s1;
-    unpack2(o.s2, s0, s1);
-    const float nm = -o.mL;
-    if (DT == JP_BF16) {
-      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        s0 += ex2_approx(fmaf(__uint_as_float(w[i] << 16), kLog2e, nm));
-        s1 += ex2_approx(fmaf(__uint_as_float(w[i] & 0xffff0000u), kLog2e, nm));
-      }
-    } else {
-      s0 += ex2_approx(fmaf(__uint_as_float(v.x), kLog2e, nm));
-      s1 += ex2_approx(fmaf(__uint_as_float(v.y), kLog2e, nm));
-      s0 += ex2_approx(fmaf(__uint_as_float(v.z), kLog2e, nm));
-      s1 += ex2_approx(fmaf(__uint_as_float(v.w), kLog2e, nm));
-    }
-    o.s2 = pack2(s0, s1);
-    return;
-  }
-#endif
+}
+
+// Adds the terms 2^(z log2 e - mL) of one 16-byte vector to the sums; the running
+// maximum already covers the vector.
+template <int DT>
+__device__ __forceinline__ void add_terms(const uint4& v, Online& o) {
   const unsigned long long L2 = pack2(kLog2e, kLog2e);
   const unsigned long long nm2 = pack2(-o.mL, -o.mL);
   if (DT == JP_BF16) {
@@ -335,6 +323,13 @@ __device__ __forceinline__ void accumulate(const uint4& v, float vm, Online& o) 
     o.s2 = fadd2(o.s2, pack2(ex2_approx(a0), ex2_approx(a1)));
     o.s2 = fadd2(o.s2, pack2(ex2_approx(b0), ex2_approx(b1)));
   }
+}
+
+// One 16-byte vector, whose maximum is vm, into the online (max, sum).
+template <int DT>
+__device__ __forceinline__ void accumulate(const uint4& v, float vm, Online& o) {
+  raise_max(vm, o);
+  add_terms<DT>(v, o);
 }
 
 // The ragged end of a row (fewer than one 16-byte vector) as a -inf padded vector.
@@ -767,10 +762,13 @@ __device__ void consumer_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int c
   const uint32_t idmask = 0xffffffffu >> __clz(ntiles * (uint32_t)TP - 1u);   // covers every pass id of a row
   const int gq = cw / WPT;              // this warp's group: it takes tiles gq, gq + NG, ...
   const int wq = cw % WPT;              // its place among the warps that share a tile
-  uint32_t g0 = 0;                      // ring position of the current row's tile 0
+  static_assert(HV == 2, "a pass takes its maximum over two vectors");
+  const uint32_t nfull = (uint32_t)(nvec / TV);            // tiles of a row that need no bounds checks
+  const uint32_t row_step = ntiles % (uint32_t)STAGES;     // how far a row moves the ring position of tile 0
+  uint32_t s_row = (uint32_t)gq % (uint32_t)STAGES;        // stage of this group's first tile of the current row
   uint32_t fphase = 0u;                 // per stage: phase bit of this group's full barrier
   int lr = 0;
-  for (int64_t it = blockIdx.x; it < n_rows; it += gridDim.x, ++lr, g0 += ntiles) {
+  for (int64_t it = blockIdx.x; it < n_rows; it += gridDim.x, ++lr) {
     const int p = lr % NSLOT;
     const uint32_t ph = (uint32_t)((lr / NSLOT) & 1);
     // the slot's top-k warps have finished the row that used it before and set it up for this one
@@ -782,9 +780,7 @@ __device__ void consumer_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int c
     // body keeps the streaming code small for the instruction caches and the live
     // registers few.  All a consumer does for the top-k is to compare the maximum of
     // every pass with the row's threshold.
-    auto consume_tile = [&](uint32_t tile) -> bool {
-      const uint32_t g = g0 + tile;
-      const uint32_t s = g % STAGES;
+    auto consume_tile = [&](uint32_t tile, uint32_t s) -> bool {
       if (!mbar_wait(&sm.full[gq][s], (fphase >> s) & 1u, &sm.abort)) return false;
       fphase ^= 1u << s;
       const uint4* sa = &sm.ring[s][0][wq * 32 + lane];
@@ -792,21 +788,21 @@ __device__ void consumer_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int c
       float ta = 0.f, tp = 0.f;
       if (TOPK) { ta = lds_volatile_f32(&sm.tau[p][0]); tp = lds_volatile_f32(&sm.tau[p][1]); }
       uint32_t id = tile * (uint32_t)TP + (uint32_t)(wq * 32 + lane);
-      if ((int64_t)(tile + 1) * TV <= nvec) {
+      if (tile < nfull) {
         // a full tile: no bounds checks
 #pragma unroll 1
         for (int h = 0; h < VPL / HV; ++h, sa += HV * WPT * 32, sp += HV * WPT * 32, id += WPT * 32) {
           uint4 va[HV], vp[HV];
 #pragma unroll
           for (int j = 0; j < HV; ++j) { va[j] = sa[j * WPT * 32]; vp[j] = sp[j * WPT * 32]; }
-          float ma = JP_NEG_INF, mp = JP_NEG_INF;
+          // one maximum and one check of the running maximum per tensor per pass
+          const float ma = Vec<DT>::vmax2(va[0], va[1]), mp = Vec<DT>::vmax2(vp[0], vp[1]);
+          raise_max(ma, oa);
+          raise_max(mp, op);
 #pragma unroll
           for (int j = 0; j < HV; ++j) {
-            const float vm_a = Vec<DT>::vmax(va[j]), vm_p = Vec<DT>::vmax(vp[j]);
-            accumulate<DT>(va[j], vm_a, oa);
-            accumulate<DT>(vp[j], vm_p, op);
-            ma = fmaxf(ma, vm_a);
-            mp = fmaxf(mp, vm_p);
+            add_terms<DT>(va[j], oa);
+            add_terms<DT>(vp[j], op);
           }
           if (TOPK) {
             if (ma >= ta) record_hit<CAP>(&sm.ncand[p][0], sm.cand[p][0], id, idmask, ma);
@@ -846,8 +842,16 @@ __device__ void consumer_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int c
       }
       return true;
     };
-    for (uint32_t tile = gq; tile < ntiles; tile += NG)
-      if (!consume_tile(tile)) { raise_timeout(sm, A.sc); return; }
+    {
+      uint32_t s = s_row;
+      for (uint32_t tile = gq; tile < ntiles; tile += NG) {
+        if (!consume_tile(tile, s)) { raise_timeout(sm, A.sc); return; }
+        s += NG;
+        if (s >= (uint32_t)STAGES) s -= (uint32_t)STAGES;
+      }
+      s_row += row_step;
+      if (s_row >= (uint32_t)STAGES) s_row -= (uint32_t)STAGES;
+    }
 
     if (tail > 0 && cw == 0 && lane == 0) {     // ragged end of the row: scalar loads
       const int64_t row = A.list[it];
