@@ -62,6 +62,9 @@ namespace jp {
 #ifndef JP_TAU_NS
 #define JP_TAU_NS 200
 #endif
+#ifndef JP_TAU_MIN_NEW
+#define JP_TAU_MIN_NEW 1
+#endif
 constexpr int NC = JP_NC;                 // consumer warps
 constexpr int NG = JP_NG;                 // consumer groups: group q takes tiles q, q + NG, ...
 constexpr int WPT = NC / NG;              // warps that share one tile
@@ -238,11 +241,17 @@ __device__ __forceinline__ void merge_scaled(float& mL, float& s, float mL2, flo
   mL = M;
 }
 
-// Online softmax state of one thread for one tensor: running max m, the integer
-// reference exponent mL = ceil(m * log2 e), and two partial sums (packed)
-// relative to 2^mL.  Every term is 2^(z log2 e - mL) <= 1.
+// Online softmax state of one thread for one tensor: an integer reference exponent
+// mL and two partial sums (packed) of the terms 2^(z log2 e - mL).  The reference is
+// set from the first maximum the thread meets and moves again only when a logit
+// climbs more than kHeadroom binades above it (`lim` is that limit as a logit;
+// -inf = nothing seen yet): terms stay below 2^kHeadroom, far from overflow, and
+// anything more than 126 - kHeadroom binades below the row's maximum is below 2^-62
+// of the sum.  Tracking the exact running maximum instead made a few lanes of almost
+// every pass take the rescaling branch on their own.
+constexpr float kHeadroom = 64.f;
 struct Online {
-  float m, mL;
+  float lim, mL;
   unsigned long long s2;
 };
 
@@ -277,24 +286,22 @@ __device__ __forceinline__ unsigned long long add_exp2_poly2(unsigned long long 
   return ffma2(p2, pack2(sc0, sc1), s2);
 }
 
-// Raises the running maximum to vm (if it is higher) and moves the sums to the new
-// reference exponent.
+// Makes sure the reference exponent covers a maximum vm: moves it (and the sums,
+// by an exact power of two) when vm is beyond the limit.
 __device__ __forceinline__ void raise_max(float vm, Online& o) {
-  if (vm > o.m) {
+  if (vm > o.lim) {
     const float nmL = ceilf(__fmul_rn(vm, kLog2e));
-    if (o.m == JP_NEG_INF) {
-      o.s2 = 0ull;
-    } else if (nmL != o.mL) {
+    if (o.lim != JP_NEG_INF) {
       const float f = exp2_int(o.mL - nmL);
       o.s2 = fmul2(o.s2, pack2(f, f));
     }
-    o.m = vm;
     o.mL = nmL;
+    o.lim = __fmul_rn(nmL + kHeadroom, kLn2);
   }
 }
 
-// Adds the terms 2^(z log2 e - mL) of one 16-byte vector to the sums; the running
-// maximum already covers the vector.
+// Adds the terms 2^(z log2 e - mL) of one 16-byte vector to the sums; the reference
+// exponent already covers the vector.
 template <int DT>
 __device__ __forceinline__ void add_terms(const uint4& v, Online& o) {
   const unsigned long long L2 = pack2(kLog2e, kLog2e);
@@ -795,7 +802,7 @@ __device__ void consumer_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int c
           uint4 va[HV], vp[HV];
 #pragma unroll
           for (int j = 0; j < HV; ++j) { va[j] = sa[j * WPT * 32]; vp[j] = sp[j * WPT * 32]; }
-          // one maximum and one check of the running maximum per tensor per pass
+          // one maximum and one check against the reference exponent per tensor per pass
           const float ma = Vec<DT>::vmax2(va[0], va[1]), mp = Vec<DT>::vmax2(vp[0], vp[1]);
           raise_max(ma, oa);
           raise_max(mp, op);
@@ -870,8 +877,8 @@ __device__ void consumer_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int c
       unpack2(oa.s2, s0, s1); s_a = s0 + s1;
       unpack2(op.s2, s0, s1); s_p = s0 + s1;
     }
-    if (oa.m == JP_NEG_INF) mL_a = JP_NEG_INF;   // a thread that saw nothing must not set the scale
-    if (op.m == JP_NEG_INF) mL_p = JP_NEG_INF;
+    if (oa.lim == JP_NEG_INF) mL_a = JP_NEG_INF;   // a thread that saw nothing must not set the scale
+    if (op.lim == JP_NEG_INF) mL_p = JP_NEG_INF;
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
       merge_scaled(mL_a, s_a, __shfl_xor_sync(0xffffffffu, mL_a, off), __shfl_xor_sync(0xffffffffu, s_a, off));
@@ -938,7 +945,7 @@ __device__ void topk_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int t, in
         if (TOPK) {
           const uint32_t nc = lds_volatile_u32(&sm.ncand[p][t]);
           const uint32_t n = nc < (uint32_t)CAP ? nc : (uint32_t)CAP;
-          if (n > seen) {
+          if (n >= seen + (uint32_t)JP_TAU_MIN_NEW) {
             seen = count_candidates(cand, seen, n, hist, base, shift, false, lane);
             const int bin = find_tau_bin(hist, k, lane);
             if (bin > 0) {
