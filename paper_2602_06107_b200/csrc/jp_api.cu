@@ -21,6 +21,7 @@ struct jp_ctx {
   Records rec{};
   Scalars* sc = nullptr;
   int32_t* list = nullptr;
+  uint32_t* spill = nullptr;
   Partials* part = nullptr;
   // state of the records
   bool have_records = false;
@@ -49,7 +50,7 @@ namespace {
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
-  size_t scalars, partials, idx, za, zp, f[7], flag, ratio, dval, list, total;
+  size_t scalars, partials, idx, za, zp, f[7], flag, ratio, dval, list, spill, total;
 };
 
 Layout layout_for(int64_t rows, int k) {
@@ -67,6 +68,7 @@ Layout layout_for(int64_t rows, int k) {
   L.ratio = take((size_t)rows * 8);
   L.dval = take((size_t)rows * 4);
   L.list = take((size_t)rows * 4);
+  L.spill = take(kSpillBytes);
   L.total = off;
   return L;
 }
@@ -122,6 +124,7 @@ jp_status ensure_workspace(jp_ctx* c, int64_t rows, int k) {
   c->rec.ratio = (double*)(b + L.ratio);
   c->rec.dval = (float*)(b + L.dval);
   c->list = (int32_t*)(b + L.list);
+  c->spill = (uint32_t*)(b + L.spill);
   return JP_OK;
 }
 
@@ -165,7 +168,7 @@ jp_status stream_rows(jp_ctx* c, const jp_obrs_desc* d, int64_t ld, int k_eff, i
   StreamArgs a{};
   a.za = za; a.zp = zp; a.tokens = tokens; a.mask = mask;
   a.T = d->T; a.V = d->V; a.ld = ld; a.dtype = d->dtype; a.k = k_eff;
-  a.record_offset = record_offset; a.rec = c->rec; a.sc = c->sc; a.list = c->list;
+  a.record_offset = record_offset; a.rec = c->rec; a.sc = c->sc; a.list = c->list; a.spill = c->spill;
   const int slot = (int)(c->ev_count % jp_ctx::kEvRing);
   if (c->timing) {
     if (!c->ev0[slot]) { cudaEventCreate(&c->ev0[slot]); cudaEventCreate(&c->ev1[slot]); }

@@ -59,7 +59,14 @@ struct StreamArgs {
   Records rec;
   Scalars* sc;
   int32_t* list;           // [T] scratch: the call's valid rows, in no particular order
+  uint32_t* spill;         // [kStreamMaxCtas][kStreamSlots][2][kSpillCap] candidate passes that did not fit a CTA's shared memory
 };
+
+// Geometry of the stream kernel's spill area (fixed: it depends on neither T nor V).
+constexpr int kStreamMaxCtas = 192;   // the grid is one CTA per SM, clamped to this
+constexpr int kStreamSlots = 4;       // rows a CTA has in flight
+constexpr int kSpillCap = 4096;       // spilled candidates per (CTA, row slot, tensor)
+constexpr size_t kSpillBytes = (size_t)kStreamMaxCtas * kStreamSlots * 2 * kSpillCap * sizeof(uint32_t);
 
 struct ExactZArgs {
   const void* za;

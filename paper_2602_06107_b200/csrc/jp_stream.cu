@@ -62,9 +62,6 @@ namespace jp {
 #ifndef JP_TAU_NS
 #define JP_TAU_NS 200
 #endif
-#ifndef JP_TAU_MIN_NEW
-#define JP_TAU_MIN_NEW 1
-#endif
 constexpr int NC = JP_NC;                 // consumer warps
 constexpr int NG = JP_NG;                 // consumer groups: group q takes tiles q, q + NG, ...
 constexpr int WPT = NC / NG;              // warps that share one tile
@@ -499,22 +496,48 @@ __device__ __forceinline__ float bin_edge(uint32_t base, uint32_t shift, int bin
 // (a fraction of a percent of the passes): append it to the row's candidates as the
 // high bits of the maximum's order bits over the pass id.  The slot's top-k warp
 // counts the candidates into its histogram as they appear.
+// Where the candidates of (row slot p, tensor t) of this CTA go when shared memory is full.
+__device__ __forceinline__ uint32_t* spill_area(const StreamArgs& A, int p, int t) {
+  static_assert(NSLOT == kStreamSlots, "the workspace is laid out for this many row slots");
+  return A.spill + (((size_t)blockIdx.x * NSLOT + (size_t)p) * 2 + (size_t)t) * (size_t)kSpillCap;
+}
+// No room in shared memory: the entry goes to the workspace (out of line: rows with
+// that many candidates are rare, and the streaming code stays small).
+__device__ __noinline__ void spill_hit(uint32_t* spill, int pt, uint32_t o, uint32_t e) {
+  if (o < (uint32_t)kSpillCap) spill[((size_t)blockIdx.x * (NSLOT * 2) + (size_t)pt) * (size_t)kSpillCap + o] = e;
+}
 template <int CAP>
-__device__ __forceinline__ void record_hit(uint32_t* ncand, uint32_t* cand, uint32_t id, uint32_t idmask, float m) {
+__device__ __forceinline__ void record_hit(uint32_t* ncand, uint32_t* cand, uint32_t* spill, int pt, uint32_t id,
+                                           uint32_t idmask, float m) {
   const uint32_t o = atomicAdd(ncand, 1u);
-  if (o < (uint32_t)CAP) cand[o] = (f32_order_bits(m) & ~idmask) | id;
+  const uint32_t e = (f32_order_bits(m) & ~idmask) | id;
+  if (o < (uint32_t)CAP) cand[o] = e;
+  else spill_hit(spill, pt, o - (uint32_t)CAP, e);
+}
+
+__device__ __forceinline__ uint32_t ldg_cg_u32(const uint32_t* p) {   // from L2: another warp of the CTA wrote it
+  uint32_t v;
+  asm volatile("ld.global.cg.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+// Candidate i of a row: the first `cap` are in shared memory, later ones in the
+// workspace (read from L2: a consumer warp of this CTA wrote them).
+__device__ __forceinline__ uint32_t cand_load(const uint32_t* cand, const uint32_t* spill, uint32_t cap, uint32_t i) {
+  return i < cap ? lds_volatile_u32(cand + i) : ldg_cg_u32(spill + (i - cap));
 }
 
 // Top-k warp: counts the candidates [seen, n) that have been written so far into
 // the histogram and returns the new `seen`.  A consumer bumps the counter before
 // it writes the entry, so an entry may still read 0 (the buffer is zeroed before
 // the row starts and no entry of a finite maximum is 0): counting stops there
-// unless `all` says that the row is done and everything has been written.
-__device__ __forceinline__ uint32_t count_candidates(const uint32_t* cand, uint32_t seen, uint32_t n, uint32_t* hist,
-                                                     uint32_t base, uint32_t shift, bool all, int lane) {
+// unless `all` says that the row is done and everything has been written (only
+// then may n reach beyond the shared-memory buffer).
+__device__ __forceinline__ uint32_t count_candidates(const uint32_t* cand, const uint32_t* spill, uint32_t cap,
+                                                     uint32_t seen, uint32_t n, uint32_t* hist, uint32_t base,
+                                                     uint32_t shift, bool all, int lane) {
   while (seen < n) {
     const uint32_t i = seen + (uint32_t)lane;
-    const uint32_t e = i < n ? lds_volatile_u32(cand + i) : 0u;
+    const uint32_t e = i < n ? cand_load(cand, spill, cap, i) : 0u;
     const bool there = i < n && (all || e != 0u);
     const uint32_t missing = ~__ballot_sync(0xffffffffu, there);
     const uint32_t run = missing ? (uint32_t)(__ffs(missing) - 1) : 32u;   // leading lanes whose entry is there
@@ -568,18 +591,21 @@ __device__ __noinline__ unsigned long long merge_all(unsigned long long (&L)[KPL
   return kth_key<KPL>(L, k);
 }
 
-// Drops the candidates whose maximum is below the row's final threshold; returns
-// how many are left (packed at the front of the buffer).
-__device__ __noinline__ int compact_candidates(uint32_t* cand, int n, uint32_t tau_ob, uint32_t idmask, int lane) {
+// Drops the candidates whose maximum is below the row's final threshold; those left
+// are packed at the front of the shared-memory buffer.  Returns how many, or -1 if
+// they do not fit there (only with spilled candidates and long runs of ties).
+__device__ __noinline__ int compact_candidates(uint32_t* cand, const uint32_t* spill, int cap, int n, uint32_t tau_ob,
+                                               uint32_t idmask, int lane) {
   int out = 0;
   for (int b = 0; b < n; b += 32) {
     const int i = b + lane;
-    const uint32_t c = i < n ? cand[i] : 0u;
+    const uint32_t c = i < n ? cand_load(cand, spill, (uint32_t)cap, (uint32_t)i) : 0u;
     // the stored high bits with the low ones filled in bound the maximum from above
     const bool keep = i < n && (c | idmask) >= tau_ob;
     const uint32_t bm = __ballot_sync(0xffffffffu, keep);
     __syncwarp();
-    if (keep) cand[out + __popc(bm & ((1u << lane) - 1u))] = c;
+    if (out + __popc(bm) > cap) return -1;
+    if (keep) cand[out + __popc(bm & ((1u << lane) - 1u))] = c;     // out <= b: never ahead of the reads
     out += __popc(bm);
     __syncwarp();
   }
@@ -588,14 +614,14 @@ __device__ __noinline__ int compact_candidates(uint32_t* cand, int n, uint32_t t
 
 // Sorts the entries of the candidate passes into the list.  The vectors of a pass
 // are read back from memory (they left the ring long ago; a few hundred 16-byte
-// reads per row, mostly L2 hits).  Returns the list's k-th key.
+// reads per row, mostly L2 hits).  `kth` is the list's k-th key so far (0 for an
+// empty list); returns the new one.
 template <int DT, int KPL>
 __device__ __noinline__ unsigned long long candidates_to_list(unsigned long long (&L)[KPL], const uint32_t* cand,
                                                               int n, uint32_t idmask, const char* row, int64_t nvec,
-                                                              int64_t V, uint32_t tau_ob, unsigned long long* stg,
-                                                              int k, int lane) {
+                                                              int64_t V, uint32_t tau_ob, unsigned long long kth,
+                                                              unsigned long long* stg, int k, int lane) {
   int staged = 0;
-  unsigned long long kth = 0ull;
   for (int b = 0; b < n; b += 32) {
     const int i = b + lane;
     const uint32_t v0 = i < n ? pass_first_vector(cand[i] & idmask) : 0u;
@@ -812,8 +838,8 @@ __device__ void consumer_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int c
             add_terms<DT>(vp[j], op);
           }
           if (TOPK) {
-            if (ma >= ta) record_hit<CAP>(&sm.ncand[p][0], sm.cand[p][0], id, idmask, ma);
-            if (mp >= tp) record_hit<CAP>(&sm.ncand[p][1], sm.cand[p][1], id, idmask, mp);
+            if (ma >= ta) record_hit<CAP>(&sm.ncand[p][0], sm.cand[p][0], A.spill, 2 * p, id, idmask, ma);
+            if (mp >= tp) record_hit<CAP>(&sm.ncand[p][1], sm.cand[p][1], A.spill, 2 * p + 1, id, idmask, mp);
           }
         }
         // Free the stage only now that arithmetic has consumed every loaded vector.  An arrival
@@ -840,8 +866,8 @@ __device__ void consumer_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int c
           }
           // a pass with no vector inside the row holds nothing
           if (TOPK && (int64_t)(v0 + h * HV * WPT * 32) < nvec) {
-            if (ma >= ta) record_hit<CAP>(&sm.ncand[p][0], sm.cand[p][0], id, idmask, ma);
-            if (mp >= tp) record_hit<CAP>(&sm.ncand[p][1], sm.cand[p][1], id, idmask, mp);
+            if (ma >= ta) record_hit<CAP>(&sm.ncand[p][0], sm.cand[p][0], A.spill, 2 * p, id, idmask, ma);
+            if (mp >= tp) record_hit<CAP>(&sm.ncand[p][1], sm.cand[p][1], A.spill, 2 * p + 1, id, idmask, mp);
           }
         }
         __syncwarp();
@@ -945,8 +971,8 @@ __device__ void topk_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int t, in
         if (TOPK) {
           const uint32_t nc = lds_volatile_u32(&sm.ncand[p][t]);
           const uint32_t n = nc < (uint32_t)CAP ? nc : (uint32_t)CAP;
-          if (n >= seen + (uint32_t)JP_TAU_MIN_NEW) {
-            seen = count_candidates(cand, seen, n, hist, base, shift, false, lane);
+          if (n > seen) {
+            seen = count_candidates(cand, nullptr, (uint32_t)CAP, seen, n, hist, base, shift, false, lane);
             const int bin = find_tau_bin(hist, k, lane);
             if (bin > 0) {
               const float val = bin_edge(base, shift, bin);
@@ -975,18 +1001,27 @@ __device__ void topk_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int t, in
       unsigned long long kth;
       uint32_t tau_ob = 0u;
       const uint32_t total = lds_volatile_u32(&sm.ncand[p][t]);
-      if (total > (uint32_t)CAP) {
-        kth = scan_row_exact<DT, KL>(L, rmine, nvec, A.V, stg, k, lane);
-      } else {
-        count_candidates(cand, seen, total, hist, base, shift, true, lane);
+      int n = -1;
+      if (total <= (uint32_t)(CAP + kSpillCap)) {
+        // (candidates beyond the shared-memory buffer are in the workspace: rare)
+        const uint32_t* spill = spill_area(A, p, t);
+        count_candidates(cand, spill, (uint32_t)CAP, seen, total, hist, base, shift, true, lane);
         const int bin = find_tau_bin(hist, k, lane);
         if (bin > 0) {
           const float val = bin_edge(base, shift, bin);
           if (val > cur) cur = val;
         }
         tau_ob = f32_order_bits(cur);
-        const int n = compact_candidates(cand, (int)total, tau_ob, idmask, lane);
-        kth = candidates_to_list<DT, KL>(L, cand, n, idmask, rmine, nvec, A.V, tau_ob, stg, k, lane);
+        n = compact_candidates(cand, spill, CAP, (int)total, tau_ob, idmask, lane);
+      }
+      if (n >= 0) {
+        kth = candidates_to_list<DT, KL>(L, cand, n, idmask, rmine, nvec, A.V, tau_ob, 0ull, stg, k, lane);
+      } else {
+        // more candidates than shared memory and the spill area hold, or than fit after
+        // the threshold has thinned them out (rows that keep rising, long runs of ties at
+        // the top): read the row again
+        tau_ob = 0u;
+        kth = scan_row_exact<DT, KL>(L, rmine, nvec, A.V, stg, k, lane);
       }
       if (tail > 0) {                 // the ragged end of the row
         uint4 v = Vec<DT>::neg_inf();
@@ -1195,7 +1230,8 @@ cudaError_t launch_stream(const StreamArgs& a, cudaStream_t s, int sms) {
   prep_rows_kernel<<<(unsigned)((a.T + 255) / 256), 256, 0, s>>>(a);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  const int grid = (int)(a.T < sms ? a.T : sms);
+  int grid = (int)(a.T < sms ? a.T : sms);
+  if (grid > kStreamMaxCtas) grid = kStreamMaxCtas;      // the spill area is laid out for that many CTAs
   const int kpl = a.k <= 0 ? 0 : a.k <= 32 ? 1 : a.k <= 64 ? 2 : 4;
   if (a.dtype == JP_BF16) {
     switch (kpl) {
