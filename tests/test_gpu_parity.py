@@ -175,6 +175,35 @@ def test_adversarial_tie_rows(ctx):
         close(out["z_approx"].cpu().numpy()[ok], ref["zk"][ok])
 
 
+def test_rows_with_more_candidates_than_shared_memory_holds(ctx):
+    """Rows built so that far more passes reach the running threshold than the CTA's
+    buffer takes: a ramp over a fifth of the row (a few thousand candidates: they go
+    to the workspace), a ramp over the whole row and a constant row (more than the
+    workspace area takes as well: the row is read again), beside an ordinary row."""
+    V = 151936
+    for dt, k in ((torch.float32, 32), (torch.bfloat16, 64), (torch.float32, 128)):
+        rows = torch.full((6, V), -5.0, dtype=torch.float32)
+        n5 = V // 5
+        rows[0, :n5] = torch.linspace(0.0, 8.0, n5)
+        rows[1, :] = torch.linspace(-4.0, 9.0, V)
+        rows[2, :] = 0.75
+        rows[3, :] = torch.randn(V, generator=torch.Generator().manual_seed(5)) * 2.5
+        rows[4, V - n5:] = torch.linspace(0.0, 8.0, n5)          # the ramp at the end of the row
+        rows[5, :] = torch.linspace(9.0, -4.0, V)                # descending: the first passes win
+        za = rows.to(dt).cuda()
+        zp = rows.flip(0).to(dt).cuda().contiguous()
+        tok = torch.tensor([7, V - 1, 100, 5, V - 3, 0], dtype=torch.int32, device="cuda")
+        out = runner.forward(ctx, za, zp, tok, None, lam=1.5, k=k, seed=3)
+        ref = oracle.forward(to_numpy_bits(za), to_numpy_bits(zp), tok.cpu().numpy(), None, lam=1.5, k=k, seed=3)
+        assert out["stats"]["status"] == 0
+        assert np.array_equal(out["topk_idx_actor"].cpu().numpy(), ref["topk_idx_a"])
+        assert np.array_equal(out["topk_idx_policy"].cpu().numpy(), ref["topk_idx_p"])
+        close(out["lse_actor"].cpu().numpy(), ref["lse_a"])
+        close(out["lse_policy"].cpu().numpy(), ref["lse_p"])
+        close(out["logp_actor"].cpu().numpy(), ref["lq64"])
+        close(out["z_approx"].cpu().numpy(), ref["zk"])
+
+
 def test_small_vocab_just_above_k(ctx):
     for V, k, dt in ((136, 128, "bf16"), (132, 128, "f32"), (24, 5, "bf16"), (8, 3, "f32")):
         r = LogitRecipe(T=33, V=V, dtype=dt, sigma0=2.0, peaks=2, sigma=0.6, seed=V)
