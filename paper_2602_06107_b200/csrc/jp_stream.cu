@@ -1,32 +1,36 @@
 // Row-streaming kernels: each valid row of the actor and policy logits is read
-// from HBM once; the pass yields both log-sum-exps (online max / rescaled sum),
-// the sampled token's logits and the two top-k lists (Section 4.4.1: V_k is the
-// union of top-k(p_inf) and top-k(p_new)), each candidate carrying both logits.
-// A second kernel sums the exact normaliser Z over the vocabulary (Eq. obrs_dist).
+// from HBM once; the pass yields both log-sum-exps (online reference exponent /
+// rescaled sum), the sampled token's logits and the two top-k lists (Section 4.4.1:
+// V_k is the union of top-k(p_inf) and top-k(p_new)), each candidate carrying both
+// logits.  A second kernel sums the exact normaliser Z over the vocabulary
+// (Eq. obrs_dist).
 //
 // Shape of the stream kernel (one persistent CTA per SM, one row pair at a time):
 //
 //   producer warp   one lane issues 1-D bulk async copies (global -> shared,
 //                   completion counted on an mbarrier) of the next tile of both
-//                   rows into a ring of STAGES shared-memory stages;
+//                   rows into a ring of shared-memory stages;
 //   consumer warps  two groups that take alternate tiles of a row: wait for a stage,
 //                   pull their 16-byte vectors into registers pass by pass (a pass
-//                   is two vectors per tensor), free the stage, update the online
-//                   (max, sum) of both rows and compare the maximum of each pass with
-//                   the row's running threshold tau.  A pass at or above tau (rare) is
-//                   counted in a histogram and appended to the row's candidate buffer;
+//                   is two vectors per tensor), add the terms to the online sums of
+//                   both rows, compare the maximum of each pass with the row's running
+//                   threshold tau, and free the stage once arithmetic has consumed the
+//                   tile.  A pass at or above tau (a fraction of a percent) is appended
+//                   to the row's candidate buffer: one atomic and one store;
 //   top-k warps     eight of them, one per (row slot, tensor).  Before a row starts its
 //                   warp reads a sample (the first vectors) of the row and publishes
 //                   the k-th best vector maximum of the sample as the first tau: the
 //                   k-th best of any subset is a lower bound of the row's k-th best
-//                   logit.  While the row streams it raises tau to the highest histogram
-//                   bin with at least k counted passes at or above it (k different
-//                   passes hold k different entries).  When the row is done it reads the
-//                   vectors of the candidate passes back, sorts their entries at or above
-//                   tau into the list (bitonic sort / merge across the lanes), finishes
-//                   the log-sum-exp, gathers the sampled token's logit and writes the
-//                   row's record.  A row whose candidates did not fit the buffer is
-//                   scanned again from memory by its warp (exact, slow, rare).
+//                   logit.  While the row streams it counts the candidates into a
+//                   histogram as they appear and raises tau to the highest bin with at
+//                   least k of them at or above it (k different passes hold k different
+//                   entries).  When the row is done it drops the candidates that tau
+//                   has overtaken, reads the vectors of the others back, sorts their
+//                   entries at or above tau into the list (bitonic sort / merge across
+//                   the lanes), finishes the log-sum-exp, gathers the sampled token's
+//                   logit and writes the row's record.  Candidates beyond the buffer
+//                   go to a spill area in the workspace; a row with more than that
+//                   holds too is read again by its warp (exact, slow, adversarial).
 //
 // Rows cycle through four "slots" (histogram, candidates, partial sums, barriers),
 // so the consumers never wait for the top-k warps unless those fall three rows
