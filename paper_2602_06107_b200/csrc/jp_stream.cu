@@ -582,7 +582,7 @@ __device__ __forceinline__ int stage_entries(const uint4& v, uint32_t vi, bool h
 
 // Folds every buffered key into the sorted list; returns the list's k-th key.
 template <int KPL>
-__device__ __noinline__ unsigned long long merge_all(unsigned long long (&L)[KPL], const unsigned long long* stg,
+__device__ __forceinline__ unsigned long long merge_all(unsigned long long (&L)[KPL], const unsigned long long* stg,
                                                      int& staged, int k, int lane) {
   constexpr int SORT_MIN = 6 * KPL;       // below this, single inserts are cheaper than a sort + merge
   __syncwarp();
@@ -621,7 +621,7 @@ __device__ __noinline__ int compact_candidates(uint32_t* cand, const uint32_t* s
 // reads per row, mostly L2 hits).  `kth` is the list's k-th key so far (0 for an
 // empty list); returns the new one.
 template <int DT, int KPL>
-__device__ __noinline__ unsigned long long candidates_to_list(unsigned long long (&L)[KPL], const uint32_t* cand,
+__device__ __forceinline__ unsigned long long candidates_to_list(unsigned long long (&L)[KPL], const uint32_t* cand,
                                                               int n, uint32_t idmask, const char* row, int64_t nvec,
                                                               int64_t V, uint32_t tau_ob, unsigned long long kth,
                                                               unsigned long long* stg, int k, int lane) {
@@ -648,11 +648,14 @@ __device__ __noinline__ unsigned long long candidates_to_list(unsigned long long
 
 // The exact top-k of a whole row read again from memory by one warp: the way out
 // for a row whose candidates did not fit the buffer (long runs of ties at the top,
-// rows that keep rising, -inf padding above the k-th entry).  Returns the k-th key.
+// rows that keep rising, -inf padding above the k-th entry).  Leaves the list in the
+// key buffer.
 template <int DT, int KPL>
-__device__ __noinline__ unsigned long long scan_row_exact(unsigned long long (&L)[KPL], const char* row,
-                                                          int64_t nvec, int64_t V, unsigned long long* stg, int k,
-                                                          int lane) {
+__device__ __noinline__ void scan_row_exact(const char* row, int64_t nvec, int64_t V, unsigned long long* stg, int k,
+                                            int lane) {
+  unsigned long long L[KPL];
+#pragma unroll
+  for (int j = 0; j < KPL; ++j) L[j] = 0ull;
   int staged = 0;
   unsigned long long kth = 0ull;
   for (int64_t b = 0; b < nvec; b += 32) {
@@ -665,7 +668,12 @@ __device__ __noinline__ unsigned long long scan_row_exact(unsigned long long (&L
     staged = stage_entries<DT>(v, (uint32_t)vi, in, V, 0u, kth, stg, staged, lane);
     if (staged > SCAP - 32 * Vec<DT>::N) kth = merge_all<KPL>(L, stg, staged, k, lane);
   }
-  return merge_all<KPL>(L, stg, staged, k, lane);
+  merge_all<KPL>(L, stg, staged, k, lane);
+  // hand the list back through the key buffer (position lane * KPL + j), so that the
+  // caller's list can stay in registers
+#pragma unroll
+  for (int j = 0; j < KPL; ++j) stg[lane * KPL + j] = L[j];
+  __syncwarp();
 }
 
 // Before a row starts: the k-th best vector maximum of the row's first SAMPLE
@@ -1025,7 +1033,11 @@ __device__ void topk_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int t, in
         // the threshold has thinned them out (rows that keep rising, long runs of ties at
         // the top): read the row again
         tau_ob = 0u;
-        kth = scan_row_exact<DT, KL>(L, rmine, nvec, A.V, stg, k, lane);
+        scan_row_exact<DT, KL>(rmine, nvec, A.V, stg, k, lane);
+#pragma unroll
+        for (int j = 0; j < KL; ++j) L[j] = stg[lane * KL + j];
+        __syncwarp();
+        kth = kth_key<KL>(L, k);
       }
       if (tail > 0) {                 // the ragged end of the row
         uint4 v = Vec<DT>::neg_inf();
