@@ -595,6 +595,42 @@ __device__ __forceinline__ unsigned long long merge_all(unsigned long long (&L)[
   return kth_key<KPL>(L, k);
 }
 
+// Staging for the end of a row, where almost no entry passes: a lane first marks its
+// entries at or above the threshold (as a logit), and keys are built only for the
+// marked ones, one round per marked entry of the busiest lane; the buffer is folded
+// into the list only when the next round might not fit.
+template <int DT, int KPL>
+__device__ __forceinline__ int stage_above(unsigned long long (&L)[KPL], const uint4& v, uint32_t vi, bool have,
+                                           int64_t V, float tau_val, unsigned long long& kth,
+                                           unsigned long long* stg, int staged, int k, int lane) {
+  constexpr int N = Vec<DT>::N;
+  const uint32_t lt = (1u << lane) - 1u;
+  uint32_t marks = 0u;
+#pragma unroll
+  for (int e = 0; e < N; ++e) marks |= (have && Vec<DT>::get(v, e) >= tau_val ? 1u : 0u) << e;
+  while (__any_sync(0xffffffffu, marks != 0u)) {
+    if (staged > SCAP - 32) kth = merge_all<KPL>(L, stg, staged, k, lane);
+    bool keep = false;
+    unsigned long long key = 0ull;
+    if (marks) {
+      const int e = __ffs(marks) - 1;
+      marks &= marks - 1u;
+      float x = Vec<DT>::get(v, 0);
+#pragma unroll
+      for (int q = 1; q < N; ++q)
+        if (q == e) x = Vec<DT>::get(v, q);
+      const uint32_t idx = vi * N + (uint32_t)e;
+      key = make_key(x, idx);
+      keep = (int64_t)idx < V && key > kth;
+    }
+    const uint32_t bk = __ballot_sync(0xffffffffu, keep);
+    if (keep) stg[staged + __popc(bk & lt)] = key;
+    staged += __popc(bk);
+  }
+  __syncwarp();
+  return staged;
+}
+
 // Drops the candidates whose maximum is below the row's final threshold; those left
 // are packed at the front of the shared-memory buffer.  Returns how many, or -1 if
 // they do not fit there (only with spilled candidates and long runs of ties).
@@ -623,7 +659,7 @@ __device__ __noinline__ int compact_candidates(uint32_t* cand, const uint32_t* s
 template <int DT, int KPL>
 __device__ __forceinline__ unsigned long long candidates_to_list(unsigned long long (&L)[KPL], const uint32_t* cand,
                                                               int n, uint32_t idmask, const char* row, int64_t nvec,
-                                                              int64_t V, uint32_t tau_ob, unsigned long long kth,
+                                                              int64_t V, float tau_val, unsigned long long kth,
                                                               unsigned long long* stg, int k, int lane) {
   int staged = 0;
   for (int b = 0; b < n; b += 32) {
@@ -639,8 +675,7 @@ __device__ __forceinline__ unsigned long long candidates_to_list(unsigned long l
     }
 #pragma unroll
     for (int j = 0; j < HV; ++j) {
-      staged = stage_entries<DT>(v[j], v0 + j * (WPT * 32), in[j], V, tau_ob, kth, stg, staged, lane);
-      if (staged > SCAP - 32 * Vec<DT>::N) kth = merge_all<KPL>(L, stg, staged, k, lane);
+      staged = stage_above<DT, KPL>(L, v[j], v0 + j * (WPT * 32), in[j], V, tau_val, kth, stg, staged, k, lane);
     }
   }
   return merge_all<KPL>(L, stg, staged, k, lane);
@@ -689,6 +724,9 @@ __device__ __noinline__ float sample_threshold(const char* row, int64_t nvec, in
   base = 0xffffffffu;                       // nothing above it: every maximum counts in bin 0 = "no threshold"
   shift = min_shift > 16u ? min_shift : 16u;  // a candidate keeps only the order bits above its pass id
   if (ns < k) return JP_NEG_INF;
+  // ask L2 for the whole sample first: the loads below go eight at a time
+  for (int line = lane; line * 8 < ns; line += 32)
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(row + (size_t)line * 128));
   float mx = JP_NEG_INF;
 #pragma unroll 1
   for (int c = 0; c < ns; c += 8 * 32) {
@@ -1027,7 +1065,7 @@ __device__ void topk_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int t, in
         n = compact_candidates(cand, spill, CAP, (int)total, tau_ob, idmask, lane);
       }
       if (n >= 0) {
-        kth = candidates_to_list<DT, KL>(L, cand, n, idmask, rmine, nvec, A.V, tau_ob, 0ull, stg, k, lane);
+        kth = candidates_to_list<DT, KL>(L, cand, n, idmask, rmine, nvec, A.V, cur, 0ull, stg, k, lane);
       } else {
         // more candidates than shared memory and the spill area hold, or than fit after
         // the threshold has thinned them out (rows that keep rising, long runs of ties at
