@@ -172,11 +172,21 @@ __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t pari
   if (mbar_try_wait(bar, parity)) return true;
   return mbar_wait_slow(bar, parity, abort);
 }
-__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, unsigned long long* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                   smem_u32(dst)),
-               "l"(src), "r"(bytes), "r"(smem_u32(bar))
-               : "memory");
+// The copy carries an L2 policy: the streamed tiles are marked "evict first", so that
+// they do not push out the few lines that are read twice (a row's sample, read by its
+// top-k warp shortly before the row streams).
+__device__ __forceinline__ unsigned long long l2_evict_first_policy() {
+  unsigned long long pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, unsigned long long* bar,
+                                         unsigned long long policy) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
+          smem_u32(dst)),
+      "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(policy)
+      : "memory");
 }
 __device__ __forceinline__ float lds_volatile_f32(const float* p) {
   float v;
@@ -792,6 +802,7 @@ __device__ void producer_loop(const StreamArgs& A, SM& sm, int64_t n_rows) {
   // This lane is the one latency-critical thread of the CTA: a freed stage waits for it.
   // Stage and phase advance by increments, addresses by additions, and the next row's
   // index is fetched one row ahead.
+  const unsigned long long policy = l2_evict_first_policy();
   uint32_t s = 0, ph = 0, armed = 0;
   uint32_t fph0 = 0u, fph1 = 0u, last_grp = 0u, last_ph = 0u;   // per stage: phase bits of full[0], full[1]; group and phase armed last
   bool ok = true;
@@ -808,8 +819,8 @@ __device__ void producer_loop(const StreamArgs& A, SM& sm, int64_t n_rows) {
       const int grp = tile % NG;
       if (bytes > 0) {
         mbar_arrive_expect_tx(&sm.full[grp][s], 2u * bytes);
-        bulk_g2s(&sm.ring[s][0][0], ra, bytes, &sm.full[grp][s]);
-        bulk_g2s(&sm.ring[s][1][0], rp, bytes, &sm.full[grp][s]);
+        bulk_g2s(&sm.ring[s][0][0], ra, bytes, &sm.full[grp][s], policy);
+        bulk_g2s(&sm.ring[s][1][0], rp, bytes, &sm.full[grp][s], policy);
       } else {
         mbar_arrive(&sm.full[grp][s]);
       }
@@ -987,9 +998,19 @@ __device__ void topk_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int t, in
   uint32_t* hist = sm.hist[p][t];
   uint32_t* cand = sm.cand[p][t];
   int lr = p;
+  uint32_t watched = 0u;                     // phases of the watched slot's row_done seen so far
   for (int64_t it = (int64_t)blockIdx.x + (int64_t)p * gridDim.x; it < n_rows;
        it += (int64_t)NSLOT * gridDim.x, lr += NSLOT) {
     const uint32_t ph = (uint32_t)((lr / NSLOT) & 1);
+    if (TOPK && lr >= 2) {
+      // Do not look at the row before the consumers are one row away from it (the row two
+      // before it is done): the sample then still sits in L2 when the row streams, instead
+      // of being read from HBM twice.  The watched barrier is another slot's; its phases
+      // are waited for one by one, none skipped.
+      const uint32_t need = (uint32_t)(lr - 2) / NSLOT;
+      for (; watched <= need; ++watched)
+        if (!mbar_wait(&sm.row_done[(p + 2) % NSLOT], watched & 1u, &sm.abort)) { raise_timeout(sm, A.sc); return; }
+    }
     const int64_t row = A.list[it];
     const int64_t rrow = A.record_offset + row;
     const char* rmine = (const char*)(t == 0 ? A.za : A.zp) + row * A.ld * Vec<DT>::ESIZE;
