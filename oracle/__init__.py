@@ -176,8 +176,28 @@ def batch_weights(lq, lp, acc, a, zk, lam, c1=0.0, mask=None, bad=None):
     return w, w64, stats
 
 
+def ppo_terms(lq, lp, acc, weight, adv=None, mask=None, logp_ref=None, logq_ref=None, logp_inf=None,
+              clip=False, eps_lo=0.0, eps_hi=0.0, c2=0.0, tis_cap=0.0):
+    """Per-token PPO / Jackpot terms (Algorithm 1 steps 1, 3, 4; Eq. ppo_rollout): a dict of
+    rho, r_theta, slope_theta, obj_theta, F, r_omega, slope_omega, obj_omega, plus the raw [T, 8]."""
+    T = len(lq)
+    f32 = lambda a: None if a is None else np.ascontiguousarray(a, np.float32)
+    out = np.zeros((T, 8))
+    lib().jo_ppo_terms(ctypes.c_int64(T), _p(f32(lq), ctypes.c_float), _p(f32(lp), ctypes.c_float),
+                       _p(mask, ctypes.c_uint8), _p(np.ascontiguousarray(acc, np.uint8), ctypes.c_uint8),
+                       _p(f32(weight), ctypes.c_float), _p(f32(adv), ctypes.c_float),
+                       _p(f32(logp_ref), ctypes.c_float), _p(f32(logq_ref), ctypes.c_float),
+                       _p(f32(logp_inf), ctypes.c_float), ctypes.c_int(1 if clip else 0),
+                       ctypes.c_double(eps_lo), ctypes.c_double(eps_hi), ctypes.c_double(c2),
+                       ctypes.c_double(tis_cap), _p(out, ctypes.c_double))
+    names = ("rho", "r_theta", "slope_theta", "obj_theta", "F", "r_omega", "slope_omega", "obj_omega")
+    d = {n: out[:, i].copy() for i, n in enumerate(names)}
+    d["raw"] = out
+    return d
+
+
 def grad_rows(rows, za, zp, tokens, acc, weight, lse_a, lse_p, n_valid, mask=None, adv=None,
-              grad_out=1.0, lambda_distill=0.0):
+              grad_out=1.0, lambda_distill=0.0, ppo=None):
     T, V = _check2d(za)
     rows = np.ascontiguousarray(rows, dtype=np.int64)
     tokens = np.ascontiguousarray(tokens, dtype=np.int32)
@@ -190,11 +210,13 @@ def grad_rows(rows, za, zp, tokens, acc, weight, lse_a, lse_p, n_valid, mask=Non
                        _p(np.ascontiguousarray(weight, np.float32), ctypes.c_float),
                        _p(adv32, ctypes.c_float), _p(lse_a, ctypes.c_double), _p(lse_p, ctypes.c_double),
                        ctypes.c_double(n_valid), ctypes.c_double(grad_out), ctypes.c_double(lambda_distill),
+                       _p(None if ppo is None else np.ascontiguousarray(ppo["raw"], np.float64), ctypes.c_double),
                        _p(da, ctypes.c_double), _p(dp, ctypes.c_double))
     return da, dp
 
 
-def loss(za64, zp64, tokens, acc, weight64, adv64, logp_ref, logq_ref, pfix, lambda_distill, mask=None):
+def loss(za64, zp64, tokens, acc, weight64, adv64, logp_ref, logq_ref, pfix, lambda_distill, mask=None,
+         f_actor=None, clip=False, eps_lo=0.0, eps_hi=0.0):
     T, V = za64.shape
     tokens = np.ascontiguousarray(tokens, dtype=np.int32)
     args = [np.ascontiguousarray(x, np.float64) for x in (za64, zp64)]
@@ -207,7 +229,10 @@ def loss(za64, zp64, tokens, acc, weight64, adv64, logp_ref, logq_ref, pfix, lam
                                _p(np.ascontiguousarray(logp_ref, np.float64), ctypes.c_double),
                                _p(np.ascontiguousarray(logq_ref, np.float64), ctypes.c_double),
                                _p(np.ascontiguousarray(pfix, np.float64), ctypes.c_double),
-                               ctypes.c_double(lambda_distill)))
+                               ctypes.c_double(lambda_distill),
+                               _p(None if f_actor is None else np.ascontiguousarray(f_actor, np.float64),
+                                  ctypes.c_double),
+                               ctypes.c_int(1 if clip else 0), ctypes.c_double(eps_lo), ctypes.c_double(eps_hi)))
 
 
 def kl_rows(za, zp, lse_a, lse_p, mask=None):

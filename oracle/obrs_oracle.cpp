@@ -315,6 +315,58 @@ void jo_batch_weights(int64_t T, const float* lq, const float* lp, const uint8_t
   stats8[7] = 0.0;
 }
 
+// Algorithm 1, steps 1, 3 and 4, and Eq. ppo_rollout, per proposed token, away from
+// the first update after a rollout (where every ratio is 1):
+//   policy:  r_theta = p_new(a)/p_ref(a),
+//            rho     = min(w_OBRS, c1) * min(p_ref(a)/p_new(a), c2)     (w already carries c1)
+//            obj     = Mask * rho * min(r_theta A, clip(r_theta, 1-eps_lo, 1+eps_hi) A)
+//   rollout: r_omega = p_omega(a)/p_omega_ref(a),  F = min(p_omega_ref(a)/p_inf(a), tis_cap)
+//            obj     = F * min(r_omega A, clip(r_omega, 1-eps_lo, 1+eps_hi) A)
+// `slope` is d obj / d r (rho and F sit under stop-gradient): the coefficient A when the
+// unclipped branch of the min is the active one, else 0.  A missing log-prob array
+// means that ratio is 1; c2 <= 0 / tis_cap <= 0 mean no cap; clip == 0 means no clipping.
+// out8 per token: rho, r_theta, slope_theta, obj_theta, F, r_omega, slope_omega, obj_omega.
+void jo_ppo_terms(int64_t T, const float* lq, const float* lp, const uint8_t* mask,
+                  const uint8_t* accept, const float* weight, const float* adv,
+                  const float* logp_ref, const float* logq_ref, const float* logp_inf, int clip,
+                  double eps_lo, double eps_hi, double c2, double tis_cap, double* out8) {
+  for (int64_t t = 0; t < T; ++t) {
+    double* o = out8 + 8 * t;
+    for (int i = 0; i < 8; ++i) o[i] = 0.0;
+    if (!row_valid(mask, t)) continue;
+    const double A = adv ? (double)adv[t] : 1.0;
+    auto surrogate = [&](double r, double* slope) {
+      double unclipped = r * A;
+      if (!clip) { *slope = A; return unclipped; }
+      double rc = std::min(std::max(r, 1.0 - eps_lo), 1.0 + eps_hi);
+      double clipped = rc * A;
+      if (unclipped <= clipped) { *slope = A; return unclipped; }   // min picks the live branch
+      *slope = 0.0;
+      return clipped;
+    };
+    // policy side
+    double r_theta = logp_ref ? std::exp((double)lp[t] - (double)logp_ref[t]) : 1.0;
+    double inv = 1.0 / r_theta;
+    if (c2 > 0.0) inv = std::min(inv, c2);
+    double rho = (double)weight[t] * inv;
+    double slope_t = 0.0;
+    double s_t = surrogate(r_theta, &slope_t);
+    double m = accept[t] ? 1.0 : 0.0;
+    o[0] = rho; o[1] = r_theta; o[2] = m * rho * slope_t; o[3] = m * rho * s_t;
+    // rollout side
+    double lq_ref = logq_ref ? (double)logq_ref[t] : (double)lq[t];
+    double r_omega = std::exp((double)lq[t] - lq_ref);
+    double F = 1.0;
+    if (logp_inf) {
+      F = std::exp(lq_ref - (double)logp_inf[t]);
+      if (tis_cap > 0.0) F = std::min(F, tis_cap);
+    }
+    double slope_o = 0.0;
+    double s_o = surrogate(r_omega, &slope_o);
+    o[4] = F; o[5] = r_omega; o[6] = F * slope_o; o[7] = F * s_o;
+  }
+}
+
 // Step 9: gradient with respect to both logit tensors of the loss to minimise
 //   J = -L^{PPO-OBRS}(theta) - L^{PPO}(omega) + lambda_distill L^{distill}(omega)
 // (Eq. sys_joint_obj with "update using the gradient of -L"), expectations over
@@ -322,13 +374,14 @@ void jo_batch_weights(int64_t T, const float* lq, const float* lp, const uint8_t
 // ratios r_theta = r_omega = 1 and F = 1 at the evaluation point:
 //   dJ/dzp[t,v] = -(g/N) Mask_t w_t A_t (1[v=x_t] - p_t(v))
 //   dJ/dza[t,v] = -(g/N) A_t (1[v=x_t] - q_t(v)) + (g lambda_distill/N)(q_t(v) - p_t(v))
-// Mask_t, w_t and the p inside the KL sit under stop-gradient.
+// Mask_t, w_t and the p inside the KL sit under stop-gradient.  With `ppo8` (the
+// output of jo_ppo_terms) the two PPO coefficients take their general form instead.
 // rows[0..n_rows) selects which rows are written, each as V doubles.
 void jo_grad_rows(int64_t n_rows, const int64_t* rows, int64_t V, int64_t ld, int dtype,
                   const void* za, const void* zp, const int32_t* tokens, const uint8_t* mask,
                   const uint8_t* accept, const float* weight, const float* adv,
                   const double* lse_a, const double* lse_p, double n_valid, double grad_out,
-                  double lambda_distill, double* d_actor, double* d_policy) {
+                  double lambda_distill, const double* ppo8, double* d_actor, double* d_policy) {
 #pragma omp parallel for schedule(dynamic, 1)
   for (int64_t i = 0; i < n_rows; ++i) {
     int64_t t = rows[i];
@@ -341,6 +394,11 @@ void jo_grad_rows(int64_t n_rows, const int64_t* rows, int64_t V, int64_t ld, in
     double A = adv ? (double)adv[t] : 1.0;
     double coef_p = -(grad_out / n_valid) * (accept[t] ? 1.0 : 0.0) * (double)weight[t] * A;
     double coef_a = -(grad_out / n_valid) * A;
+    if (ppo8) {
+      // general form: d obj / d logit = (d obj / d r) * r * (1[v=x] - prob(v)), both sides
+      coef_p = -(grad_out / n_valid) * ppo8[8 * t + 2] * ppo8[8 * t + 1];
+      coef_a = -(grad_out / n_valid) * ppo8[8 * t + 6] * ppo8[8 * t + 5];
+    }
     double coef_d = grad_out * lambda_distill / n_valid;
     for (int64_t v = 0; v < V; ++v) {
       double q = std::exp(logit_at(za, dtype, t * ld + v) - lse_a[t]);
@@ -355,13 +413,17 @@ void jo_grad_rows(int64_t n_rows, const int64_t* rows, int64_t V, int64_t ld, in
 // The scalar J itself, as a function of live double logits, with every
 // stop-gradient quantity passed in as a constant: used only to differentiate
 // numerically against jo_grad_rows.
-//   J = -(1/N) sum_t Mask_t w_t A_t p_zp(x_t)/p_ref_t - (1/N) sum_t A_t q_za(x_t)/q_ref_t
-//       + lambda_distill (1/N) sum_t KL(pfix_t || q_za(.))
+//   J = -(1/N) sum_t Mask_t w_t S(p_zp(x_t)/p_ref_t) - (1/N) sum_t f_t S(q_za(x_t)/q_ref_t)
+//       + lambda_distill (1/N) sum_t KL(pfix_t || q_za(.)),
+//   S(r) = min(r A_t, clip(r, 1-eps_lo, 1+eps_hi) A_t)   (S(r) = r A_t when clip == 0);
+// w_t stands for the whole stop-gradient weight of the policy term (rho of Algorithm 1),
+// f_t for F of Eq. ppo_rollout (NULL: 1).
 // za, zp: [T,V] doubles; logp_ref, logq_ref: [T]; pfix: [T,V] probabilities.
 double jo_loss(int64_t T, int64_t V, const double* za, const double* zp, const int32_t* tokens,
                const uint8_t* mask, const uint8_t* accept, const double* weight,
                const double* adv, const double* logp_ref, const double* logq_ref,
-               const double* pfix, double lambda_distill) {
+               const double* pfix, double lambda_distill, const double* f_actor, int clip,
+               double eps_lo, double eps_hi) {
   int64_t N = 0;
   for (int64_t t = 0; t < T; ++t) N += row_valid(mask, t) ? 1 : 0;
   if (N == 0) return 0.0;
@@ -379,8 +441,13 @@ double jo_loss(int64_t T, int64_t V, const double* za, const double* zp, const i
     double A = adv ? adv[t] : 1.0;
     double r_theta = std::exp(rp[x] - lsp - logp_ref[t]);
     double r_omega = std::exp(ra[x] - lsa - logq_ref[t]);
-    J -= (accept[t] ? 1.0 : 0.0) * weight[t] * A * r_theta;
-    J -= A * r_omega;
+    auto surrogate = [&](double r) {
+      if (!clip) return r * A;
+      double rc = std::min(std::max(r, 1.0 - eps_lo), 1.0 + eps_hi);
+      return std::min(r * A, rc * A);
+    };
+    J -= (accept[t] ? 1.0 : 0.0) * weight[t] * surrogate(r_theta);
+    J -= (f_actor ? f_actor[t] : 1.0) * surrogate(r_omega);
     double kl = 0.0;
     for (int64_t v = 0; v < V; ++v) {
       double pf = pfix[t * V + v];

@@ -453,3 +453,99 @@ def test_loss_function_value_by_hand():
                     np.log(p[rows, tok]), np.log(q[rows, tok]), p, 0.4)
     by_hand = (-(acc * w * adv).sum() - adv.sum() + 0.4 * (p * np.log(p / q)).sum()) / T
     assert J == pytest.approx(by_hand, rel=1e-12)
+
+
+# ---- Algorithm 1 steps 1, 3, 4 and Eq. ppo_rollout away from the first update ----------------
+
+def test_ppo_terms_reduce_to_the_first_update_case():
+    # no reference log-probs: every ratio is 1, rho is the OBRS weight, F is 1
+    lq = np.array([-1.0, -2.0, -0.5], np.float32)
+    lp = np.array([-1.5, -1.0, -0.7], np.float32)
+    acc = np.array([1, 0, 1], np.uint8)
+    w = np.array([1.2, 0.8, 2.0], np.float32)
+    adv = np.array([0.5, -1.0, 2.0], np.float32)
+    t = oracle.ppo_terms(lq, lp, acc, w, adv, clip=True, eps_lo=0.2, eps_hi=0.3, c2=5.0, tis_cap=2.0)
+    assert np.allclose(t["rho"], w) and np.all(t["r_theta"] == 1) and np.all(t["r_omega"] == 1) and np.all(t["F"] == 1)
+    assert np.allclose(t["slope_theta"], acc * w * adv) and np.allclose(t["slope_omega"], adv)
+    assert np.allclose(t["obj_theta"], acc * w * adv) and np.allclose(t["obj_omega"], adv)
+
+
+def test_ppo_terms_by_hand():
+    # token 0: ratio above the clip with a positive advantage -> clipped, no gradient
+    # token 1: ratio below the clip with a negative advantage -> clipped, no gradient
+    # token 2: ratio above the clip with a negative advantage -> the min keeps the live branch
+    # token 3: inside the clip range
+    r = np.array([1.5, 0.6, 1.5, 1.1])
+    lp = np.log(np.array([0.3, 0.2, 0.3, 0.22])).astype(np.float32)
+    logp_ref = (lp.astype(np.float64) - np.log(r)).astype(np.float32)
+    lq = np.log(np.array([0.25, 0.25, 0.25, 0.25])).astype(np.float32)
+    acc = np.ones(4, np.uint8)
+    w = np.array([2.0, 2.0, 2.0, 2.0], np.float32)
+    adv = np.array([1.0, -1.0, -1.0, 1.0], np.float32)
+    t = oracle.ppo_terms(lq, lp, acc, w, adv, logp_ref=logp_ref, clip=True, eps_lo=0.2, eps_hi=0.28, c2=0.8)
+    r32 = np.exp(lp.astype(np.float64) - logp_ref.astype(np.float64))
+    rho = 2.0 * np.minimum(1.0 / r32, 0.8)
+    assert np.allclose(t["r_theta"], r32, rtol=1e-12) and np.allclose(t["rho"], rho, rtol=1e-12)
+    assert t["slope_theta"][0] == 0 and t["obj_theta"][0] == pytest.approx(rho[0] * 1.28)
+    assert t["slope_theta"][1] == 0 and t["obj_theta"][1] == pytest.approx(rho[1] * -0.8)
+    assert t["slope_theta"][2] == pytest.approx(rho[2] * -1.0) and t["obj_theta"][2] == pytest.approx(rho[2] * -r32[2])
+    assert t["slope_theta"][3] == pytest.approx(rho[3]) and t["obj_theta"][3] == pytest.approx(rho[3] * r32[3])
+    # rollout side: F = min(p_omega_ref / p_inf, cap), ratio against p_omega_ref
+    logq_ref = np.log(np.array([0.2, 0.3, 0.25, 0.25])).astype(np.float32)
+    logp_inf = np.log(np.array([0.05, 0.3, 0.5, 0.25])).astype(np.float32)
+    t = oracle.ppo_terms(lq, lp, acc, w, adv, logq_ref=logq_ref, logp_inf=logp_inf, clip=False, tis_cap=2.0)
+    F = np.minimum(np.exp(logq_ref.astype(np.float64) - logp_inf.astype(np.float64)), 2.0)
+    r_om = np.exp(lq.astype(np.float64) - logq_ref.astype(np.float64))
+    assert F[0] == 2.0 and np.allclose(t["F"], F) and np.allclose(t["r_omega"], r_om)
+    assert np.allclose(t["slope_omega"], F * adv) and np.allclose(t["obj_omega"], F * r_om * adv)
+    # a rejected token carries no policy term; a masked one nothing at all
+    t = oracle.ppo_terms(lq, lp, np.array([0, 1, 1, 1], np.uint8), w, adv, mask=np.array([1, 0, 1, 1], np.uint8))
+    assert t["obj_theta"][0] == 0 and t["slope_theta"][0] == 0 and np.all(t["raw"][1] == 0)
+
+
+def test_general_gradients_by_central_differences():
+    T, V = 5, 12
+    za, zp, tok = _rand_rows(T, V, seed=28, sigma=0.8)
+    rng = np.random.default_rng(28)
+    adv = np.array([0.8, -0.6, 1.1, -1.2, 0.4], np.float32)
+    fwd = oracle.forward(za, zp, tok, None, lam=0.9, k=4, seed=6)
+    acc = np.array([1, 1, 0, 1, 1], np.uint8)
+    p, q = _pq(za, zp)
+    rows = np.arange(T)
+    # reference log-probs that put tokens on both sides of the clip range (and none on a kink)
+    ratio_t = np.array([1.35, 0.7, 1.1, 1.4, 0.95])
+    ratio_o = np.array([0.9, 1.3, 0.6, 0.75, 1.05])
+    logp_ref = (np.log(p[rows, tok]) - np.log(ratio_t)).astype(np.float32)
+    logq_ref = (np.log(q[rows, tok]) - np.log(ratio_o)).astype(np.float32)
+    logp_inf = (logq_ref + rng.normal(0, 0.5, T)).astype(np.float32)
+    kw = dict(clip=True, eps_lo=0.2, eps_hi=0.25)
+    terms = oracle.ppo_terms(fwd["lq"], fwd["lp"], acc, fwd["w"], adv, logp_ref=logp_ref, logq_ref=logq_ref,
+                             logp_inf=logp_inf, c2=0.9, tis_cap=1.5, **kw)
+    lam_d, g_out = 0.3, 0.7
+    da, dp = oracle.grad_rows(rows, za, zp, tok, acc, fwd["w"], fwd["lse_a"], fwd["lse_p"], T, adv=adv,
+                              grad_out=g_out, lambda_distill=lam_d, ppo=terms)
+    consts = dict(tokens=tok, acc=acc, weight64=terms["rho"], adv64=adv.astype(np.float64),
+                  logp_ref=logp_ref.astype(np.float64), logq_ref=logq_ref.astype(np.float64), pfix=p,
+                  lambda_distill=lam_d, f_actor=terms["F"], **kw)
+    za64, zp64 = za.astype(np.float64), zp.astype(np.float64)
+    h = 1e-6
+    for which, grad in (("a", da), ("p", dp)):
+        for t in range(T):
+            for v in range(V):
+                zp_p, zp_m, za_p, za_m = zp64.copy(), zp64.copy(), za64.copy(), za64.copy()
+                if which == "a":
+                    za_p[t, v] += h
+                    za_m[t, v] -= h
+                else:
+                    zp_p[t, v] += h
+                    zp_m[t, v] -= h
+                fd = g_out * (oracle.loss(za_p, zp_p, **consts) - oracle.loss(za_m, zp_m, **consts)) / (2 * h)
+                assert grad[t, v] == pytest.approx(fd, rel=2e-4, abs=1e-8), (which, t, v)
+    # clipped tokens: the policy gradient of token 0 (ratio 1.35, A > 0) and token 1 (0.7, A < 0) is zero,
+    # token 3 (1.4, A < 0) is live; the rejected token 2 has none
+    assert np.all(dp[0] == 0) and np.all(dp[1] == 0) and np.all(dp[2] == 0) and np.any(dp[3] != 0)
+    # without the optional inputs the general path gives the first-update gradients
+    base = oracle.ppo_terms(fwd["lq"], fwd["lp"], acc, fwd["w"], adv)
+    da1, dp1 = oracle.grad_rows(rows, za, zp, tok, acc, fwd["w"], fwd["lse_a"], fwd["lse_p"], T, adv=adv, ppo=base)
+    da0, dp0 = oracle.grad_rows(rows, za, zp, tok, acc, fwd["w"], fwd["lse_a"], fwd["lse_p"], T, adv=adv)
+    assert np.allclose(da1, da0, rtol=1e-12, atol=0) and np.allclose(dp1, dp0, rtol=1e-12, atol=0)
