@@ -138,8 +138,17 @@ jp_status jp_obrs_forward(jp_ctx* ctx, const jp_obrs_desc* desc, const void* act
  * distill_loss combined as Eq. sys_joint_obj; the PPO terms are maximised and
  * the distillation term minimised, so the loss is
  *   J = -L^{PPO-OBRS}(theta) - L^{PPO}(omega) + lambda_distill L^{distill}(omega),
- * a mean over the batch's N valid proposed tokens, evaluated where the ratios
- * r_theta = r_omega = 1 and F = 1). */
+ * a mean over the batch's N valid proposed tokens.  With the optional fields all
+ * zero the loss is evaluated where the ratios r_theta = r_omega = 1 and F = 1 (the
+ * first update after a rollout).  With them (Algorithm 1 steps 1, 3 and 4 for the
+ * policy, Eq. ppo_rollout for the rollout model), per proposed token a_t:
+ *   r_theta = p_new(a_t)/p_ref(a_t),  rho = weight_t * min(p_ref(a_t)/p_new(a_t), c2)
+ *   policy term  Mask_t SG(rho) min(r_theta A_t, clip(r_theta, 1-eps_lo, 1+eps_hi) A_t)
+ *   r_omega = p_omega(a_t)/p_omega_ref(a_t),  F = min(p_omega_ref(a_t)/p_inf(a_t), tis_cap)
+ *   rollout term SG(F) min(r_omega A_t, clip(r_omega, 1-eps_lo, 1+eps_hi) A_t)
+ * (weight_t is the forward's output and already carries the c1 clip; p_new(a_t) and
+ * p_omega(a_t) are the forward's log-probs, kept in the context's records.)  A token
+ * whose min sits on its clipped branch gets no gradient from that term. */
 typedef struct {
   const float* advantages;  /* [T] A_t; NULL means 1                                   */
   float lambda_distill;     /* >= 0                                                    */
@@ -148,11 +157,27 @@ typedef struct {
                                last forward / jp_batch_finalize                        */
   int64_t record_offset;    /* index of row 0 in the context's records (the chunk's
                                token_offset for chunked batches, else 0)               */
+  /* optional, device pointers, all may be NULL / 0 (see above) */
+  const float* logp_ref;        /* [T] log p_ref(a_t), the policy before this update; NULL: r_theta = 1 */
+  const float* logp_actor_ref;  /* [T] log p_omega,ref(a_t), the rollout model before this update
+                                   (training engine); NULL: r_omega = 1                          */
+  const float* logp_inf;        /* [T] log p_inf(a_t) as the rollout engine reported it; NULL: F = 1 */
+  float eps_lo, eps_hi;         /* PPO clip range [1 - eps_lo, 1 + eps_hi]; both 0: no clipping   */
+  float c2;                     /* cap on p_ref/p_new in rho; <= 0: none                          */
+  float tis_cap;                /* cap of the truncated importance weight F; <= 0: none           */
+  float* out_obj_policy;        /* [T] the policy term per token (0 for masked / rejected rows)   */
+  float* out_obj_actor;         /* [T] the rollout term per token                                 */
+  float* out_kl;                /* [T] KL(p_new(.|s_t) || p_omega(.|s_t)), the distillation term   */
+  double* out_loss;             /* [4] J, L^{PPO-OBRS}, L^{PPO}, L^{distill}: this call's rows summed
+                                   in a fixed order and divided by N (chunked batches: add the
+                                   chunks' values); needs the three per-token outputs above       */
 } jp_obrs_bwd_desc;
 
 /* Writes dJ/d(actor logits) and dJ/d(policy logits), both [T, ld] bf16:
  *   d_policy[t,v] = -(g/N) accept_t w_t A_t (1[v = x_t] - p_t(v))
  *   d_actor[t,v]  = -(g/N) A_t (1[v = x_t] - q_t(v)) + (g lambda_distill/N)(q_t(v) - p_t(v))
+ * (first-update form; in general w_t A_t becomes rho_t A_t r_theta on the live branch of
+ * the min and 0 on the clipped one, and A_t becomes F_t A_t r_omega likewise).
  * accept / weight are the forward's outputs.  The log-sum-exps come from the
  * context's records of the matching forward (JP_ERR_STATE if there are none).
  * For bf16 logits d_actor_logits may alias actor_logits and d_policy_logits may

@@ -66,6 +66,10 @@ class jp_obrs_bwd_desc(ctypes.Structure):
         ("advantages", ctypes.c_void_p), ("lambda_distill", ctypes.c_float),
         ("grad_out", ctypes.c_float), ("n_valid", ctypes.c_int64),
         ("record_offset", ctypes.c_int64),
+        ("logp_ref", ctypes.c_void_p), ("logp_actor_ref", ctypes.c_void_p), ("logp_inf", ctypes.c_void_p),
+        ("eps_lo", ctypes.c_float), ("eps_hi", ctypes.c_float), ("c2", ctypes.c_float), ("tis_cap", ctypes.c_float),
+        ("out_obj_policy", ctypes.c_void_p), ("out_obj_actor", ctypes.c_void_p), ("out_kl", ctypes.c_void_p),
+        ("out_loss", ctypes.c_void_p),
     ]
 
 
@@ -252,13 +256,20 @@ def read_stats(buf: torch.Tensor) -> dict:
     return jp_stats.from_buffer_copy(raw).as_dict()
 
 
-def make_bwd_desc(advantages=None, lambda_distill=0.0, grad_out=1.0, n_valid=0, record_offset=0):
+def make_bwd_desc(advantages=None, lambda_distill=0.0, grad_out=1.0, n_valid=0, record_offset=0, *,
+                  logp_ref=None, logp_actor_ref=None, logp_inf=None, eps_lo=0.0, eps_hi=0.0, c2=0.0, tis_cap=0.0,
+                  out_obj_policy=None, out_obj_actor=None, out_kl=None, out_loss=None):
     b = jp_obrs_bwd_desc()
     b.advantages = advantages.data_ptr() if advantages is not None else None
     b.lambda_distill = lambda_distill
     b.grad_out = grad_out
     b.n_valid = n_valid
     b.record_offset = record_offset
+    for name, t in (("logp_ref", logp_ref), ("logp_actor_ref", logp_actor_ref), ("logp_inf", logp_inf),
+                    ("out_obj_policy", out_obj_policy), ("out_obj_actor", out_obj_actor), ("out_kl", out_kl),
+                    ("out_loss", out_loss)):
+        setattr(b, name, t.data_ptr() if t is not None else None)
+    b.eps_lo, b.eps_hi, b.c2, b.tis_cap = eps_lo, eps_hi, c2, tis_cap
     return b
 
 

@@ -457,6 +457,9 @@ jp_status jp_obrs_backward(jp_ctx* c, const jp_obrs_desc* d, const jp_obrs_bwd_d
   if (b->record_offset < 0 || b->record_offset + d->T > c->rec_rows)
     return fail(c, JP_ERR_INVALID_ARG, "rows fall outside the forward's records");
   if (b->lambda_distill < 0.f) return fail(c, JP_ERR_INVALID_ARG, "lambda_distill < 0");
+  if (b->eps_lo < 0.f || b->eps_hi < 0.f || b->eps_lo >= 1.f) return fail(c, JP_ERR_INVALID_ARG, "clip range: need 0 <= eps_lo < 1 and eps_hi >= 0");
+  if (b->out_loss && (!b->out_obj_policy || !b->out_obj_actor || !b->out_kl))
+    return fail(c, JP_ERR_INVALID_ARG, "out_loss needs out_obj_policy, out_obj_actor and out_kl");
   if (d->T == 0) return JP_OK;
   if (!za || !zp || !tokens || !accept || !weight || !d_actor || !d_policy)
     return fail(c, JP_ERR_INVALID_ARG, "a required pointer is NULL");
@@ -474,9 +477,15 @@ jp_status jp_obrs_backward(jp_ctx* c, const jp_obrs_desc* d, const jp_obrs_bwd_d
   g.T = d->T; g.V = d->V; g.ld = ld; g.dtype = d->dtype; g.record_offset = b->record_offset;
   g.lambda_distill = b->lambda_distill; g.grad_out = b->grad_out == 0.f ? 1.f : b->grad_out;
   g.n_valid = b->n_valid; g.rec = c->rec; g.sc = c->sc;
-  e = launch_grad(g, c->stream, c->sms);
+  g.logp_ref = b->logp_ref; g.logp_actor_ref = b->logp_actor_ref; g.logp_inf = b->logp_inf;
+  g.clip = (b->eps_lo > 0.f || b->eps_hi > 0.f) ? 1 : 0;
+  g.eps_lo = b->eps_lo; g.eps_hi = b->eps_hi; g.c2 = b->c2; g.tis_cap = b->tis_cap;
+  g.out_obj_policy = b->out_obj_policy; g.out_obj_actor = b->out_obj_actor; g.out_kl = b->out_kl;
+  g.out_loss = b->out_loss;
+  int n_launch = 0;
+  e = launch_grad(g, c->stream, c->sms, &n_launch);
   if (e != cudaSuccess) return cuda_fail(c, e, "gradient kernel launch");
-  c->launches += 1;
+  c->launches += n_launch;
   return JP_OK;
 }
 

@@ -116,6 +116,16 @@ struct GradArgs {
   int64_t n_valid;         // 0 = read sc->stats.n_valid on the device
   Records rec;
   Scalars* sc;
+  // beyond the first update (all optional)
+  const float* logp_ref;
+  const float* logp_actor_ref;
+  const float* logp_inf;
+  int32_t clip;            // 1 = PPO clipping on
+  float eps_lo, eps_hi, c2, tis_cap;
+  float* out_obj_policy;
+  float* out_obj_actor;
+  float* out_kl;
+  double* out_loss;
 };
 
 int stream_grid_size(int device);   // number of SMs
@@ -127,6 +137,6 @@ cudaError_t launch_budget_solve(const EpilogueArgs& a, double budget, cudaStream
 cudaError_t launch_epilogue(const EpilogueArgs& a, cudaStream_t s, int* n_launch);
 cudaError_t launch_reweight(int64_t T, const Records& rec, const Scalars* sc, double kappa, float c1,
                             float* out_weight, cudaStream_t s);
-cudaError_t launch_grad(const GradArgs& a, cudaStream_t s, int sms);
+cudaError_t launch_grad(const GradArgs& a, cudaStream_t s, int sms, int* n_launch);
 
 }  // namespace jp

@@ -74,13 +74,15 @@ def forward_chunked(ctx: B.Context, chunks, T_total, V, dtype_code, *, lam=None,
 
 
 def backward(ctx: B.Context, za, zp, tokens, mask, accept, weight, *, advantages=None, lambda_distill=0.0,
-             grad_out=1.0, n_valid=0, record_offset=0, d_actor=None, d_policy=None):
+             grad_out=1.0, n_valid=0, record_offset=0, d_actor=None, d_policy=None, **general):
+    """``general``: the optional fields of jp_obrs_bwd_desc (logp_ref, logp_actor_ref, logp_inf, eps_lo,
+    eps_hi, c2, tis_cap, out_obj_policy, out_obj_actor, out_kl, out_loss)."""
     T, V = za.shape
     if d_actor is None:
         d_actor = torch.empty((T, za.stride(0)), dtype=torch.bfloat16, device=za.device)[:, :V]
     if d_policy is None:
         d_policy = torch.empty((T, zp.stride(0)), dtype=torch.bfloat16, device=za.device)[:, :V]
     desc = B.make_desc(za)
-    bwd = B.make_bwd_desc(advantages, lambda_distill, grad_out, n_valid, record_offset)
+    bwd = B.make_bwd_desc(advantages, lambda_distill, grad_out, n_valid, record_offset, **general)
     B.jp_obrs_backward(ctx, desc, bwd, za, zp, tokens, mask, accept, weight, d_actor, d_policy)
     return d_actor, d_policy

@@ -154,3 +154,92 @@ def test_training_step_chunked_budget_then_backward(ctx):
     check_grads(da[sub], dp[sub], np.arange(len(rows)), za_s, zp_s, tok_s, None, out["accept"][sub].cpu().numpy(),
                 out["weight"][sub].cpu().numpy(), lg["lse_a"], lg["lse_p"], out["stats"]["n_valid"],
                 adv[sub].cpu().numpy(), 1.0)
+
+
+@pytest.mark.parametrize("dtype,V", [("bf16", 20000), ("f32", 4099 + 5)])
+def test_backward_general_form_matches_oracle(ctx, dtype, V):
+    """Away from the first update: PPO ratios against reference log-probs, asymmetric clip,
+    rho with c2, the truncated importance weight F, per-token terms, KL and the loss."""
+    T = 120
+    r = LogitRecipe(T=T, V=V, dtype=dtype, sigma0=2.5, peaks=4, sigma=1.0, seed=21)
+    za, zp, tok = make_logits(r, "cuda")
+    g = torch.Generator(device="cuda").manual_seed(7)
+    mask = (torch.arange(T, device="cuda") % 7 != 3).to(torch.uint8)
+    adv = torch.randn(T, generator=g, device="cuda")
+    out = runner.forward(ctx, za, zp, tok, mask, lam=1.3, k=16, seed=5, c1=3.0)
+    # reference log-probs scattered around the current ones so that tokens land on both
+    # sides of the clip range
+    logp_ref = out["logp_policy"] + 0.35 * torch.randn(T, generator=g, device="cuda")
+    logq_ref = out["logp_actor"] + 0.35 * torch.randn(T, generator=g, device="cuda")
+    logp_inf = logq_ref + 0.5 * torch.randn(T, generator=g, device="cuda")
+    eps_lo, eps_hi = float(np.float32(0.2)), float(np.float32(0.28))
+    c2, cap = float(np.float32(1.25)), float(np.float32(1.5))
+    lam_d, g_out = 0.6, 0.5
+    obj_p = torch.empty(T, device="cuda")
+    obj_a = torch.empty(T, device="cuda")
+    kl = torch.empty(T, device="cuda")
+    loss = torch.zeros(4, dtype=torch.float64, device="cuda")
+    da, dp = runner.backward(ctx, za, zp, tok, mask, out["accept"], out["weight"], advantages=adv,
+                             lambda_distill=lam_d, grad_out=g_out, logp_ref=logp_ref, logp_actor_ref=logq_ref,
+                             logp_inf=logp_inf, eps_lo=eps_lo, eps_hi=eps_hi, c2=c2, tis_cap=cap,
+                             out_obj_policy=obj_p, out_obj_actor=obj_a, out_kl=kl, out_loss=loss)
+    torch.cuda.synchronize()
+    za_np, zp_np = to_numpy_bits(za.contiguous()), to_numpy_bits(zp.contiguous())
+    m_np, acc, w = mask.cpu().numpy(), out["accept"].cpu().numpy(), out["weight"].cpu().numpy()
+    lq, lp = out["logp_actor"].cpu().numpy(), out["logp_policy"].cpu().numpy()
+    terms = oracle.ppo_terms(lq, lp, acc, w, adv.cpu().numpy(), mask=m_np, logp_ref=logp_ref.cpu().numpy(),
+                             logq_ref=logq_ref.cpu().numpy(), logp_inf=logp_inf.cpu().numpy(), clip=True,
+                             eps_lo=eps_lo, eps_hi=eps_hi, c2=c2, tis_cap=cap)
+    # the fixture must exercise every branch
+    valid = m_np != 0
+    assert (terms["slope_theta"][valid & (acc != 0)] == 0).any() and (terms["slope_theta"][valid] != 0).any()
+    assert (terms["slope_omega"][valid] == 0).any() and (terms["F"][valid] == cap).any()
+    # per-token terms (decisions taken in double on both sides; values rounded to fp32)
+    assert np.allclose(obj_p.cpu().numpy(), terms["obj_theta"], rtol=1e-5, atol=1e-7)
+    assert np.allclose(obj_a.cpu().numpy(), terms["obj_omega"], rtol=1e-5, atol=1e-7)
+    ref = oracle.forward(za_np, zp_np, tok.cpu().numpy(), m_np, lam=1.3, k=16, seed=5, c1=3.0)
+    kl_ref = oracle.kl_rows(za_np, zp_np, ref["lse_a"], ref["lse_p"], mask=m_np)
+    # KL = sum_v p (zp - za) - lse_p + lse_a in fp32: the two log-sum-exps (~10, half an ulp = 5e-7 each)
+    # cancel against the sum, so the error is absolute, a few 1e-6
+    assert np.allclose(kl.cpu().numpy(), kl_ref, rtol=1e-4, atol=5e-6)
+    N = out["stats"]["n_valid"]
+    l1, l2, l3 = terms["obj_theta"].sum() / N, terms["obj_omega"].sum() / N, kl_ref.sum() / N
+    got = loss.cpu().numpy()
+    assert np.allclose(got[1:], [l1, l2, l3], rtol=1e-4, atol=5e-6)
+    assert got[0] == pytest.approx(-l1 - l2 + lam_d * l3, rel=1e-4, abs=1e-5)
+    # gradients
+    rows = np.arange(0, T, 2)
+    ra, rp = oracle.grad_rows(rows, za_np, zp_np, tok.cpu().numpy(), acc, w, ref["lse_a"], ref["lse_p"], float(N),
+                              mask=m_np, adv=adv.cpu().numpy(), grad_out=g_out, lambda_distill=lam_d, ppo=terms)
+    ga = da[rows].float().cpu().numpy().astype(np.float64)
+    gp = dp[rows].float().cpu().numpy().astype(np.float64)
+    q = np.exp(_widen(za_np[rows]) - ref["lse_a"][rows][:, None])
+    p = np.exp(_widen(zp_np[rows]) - ref["lse_p"][rows][:, None])
+    hot = np.zeros_like(q)
+    hot[np.arange(len(rows)), tok.cpu().numpy()[rows]] = 1.0
+    scale = g_out / N
+    ca = np.abs(terms["slope_omega"] * terms["r_omega"])[rows][:, None]
+    cp = np.abs(terms["slope_theta"] * terms["r_theta"])[rows][:, None]
+    floor_a = 1e-4 * scale * (ca * np.maximum(q, hot) + lam_d * (q + p)) + 1e-30
+    floor_p = 1e-4 * scale * cp * np.maximum(p, hot) + 1e-30
+    assert not (np.abs(ga - ra) > 2e-2 * np.abs(ra) + floor_a).any()
+    assert not (np.abs(gp - rp) > 2e-2 * np.abs(rp) + floor_p).any()
+    clipped = (terms["slope_theta"][rows] == 0)
+    assert np.all(gp[clipped] == 0), "a clipped, rejected or masked token must not reach the policy gradient"
+
+
+def test_backward_general_form_defaults_equal_first_update(ctx):
+    r = LogitRecipe(T=64, V=8192, dtype="bf16", sigma0=2.5, peaks=4, sigma=1.0, seed=12)
+    za, zp, tok = make_logits(r, "cuda")
+    out = runner.forward(ctx, za, zp, tok, None, lam=1.0, k=8, seed=1)
+    adv = torch.randn(64, device="cuda")
+    da, dp = runner.backward(ctx, za, zp, tok, None, out["accept"], out["weight"], advantages=adv, lambda_distill=1.0)
+    # the reference log-probs equal to the current ones: every ratio is 1 and nothing is clipped
+    da1, dp1 = runner.backward(ctx, za, zp, tok, None, out["accept"], out["weight"], advantages=adv,
+                               lambda_distill=1.0, logp_ref=out["logp_policy"], logp_actor_ref=out["logp_actor"],
+                               logp_inf=out["logp_actor"], eps_lo=0.2, eps_hi=0.2, c2=10.0, tis_cap=10.0)
+    torch.cuda.synchronize()
+    assert torch.equal(da, da1) and torch.equal(dp, dp1)
+    with pytest.raises(B.JackpotError, match="out_loss needs"):
+        runner.backward(ctx, za, zp, tok, None, out["accept"], out["weight"],
+                        out_loss=torch.zeros(4, dtype=torch.float64, device="cuda"))
