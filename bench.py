@@ -305,6 +305,13 @@ def run_ours(args, rank, world, local_rank):
         "fwd_bwd": fb,
         "cpu_baseline": cpu_baseline,
     }
+    # this GPU's plain streaming rates, measured now with the library's probe kernel: the forward
+    # only reads its logits, so the read-only rate is the tighter reference beside the copy rate
+    try:
+        line["roofline"]["read_only_gbs_now"] = B.jp_probe_stream(za, None, reps=20)
+        line["roofline"]["copy_gbs_now"] = B.jp_probe_stream(za, zp, reps=10)
+    except Exception as exc:                                   # a measurement aid must not lose the line
+        line["roofline"]["probe_error"] = str(exc)
     # DRAM bytes per launch of the row stream, from an ncu capture of a smaller case
     # scaled by rows (traffic is proportional to the rows streamed); null unless the
     # capture was taken from the kernel source as it stands

@@ -212,6 +212,15 @@ jp_status jp_batch_finalize(jp_ctx* ctx, const jp_obrs_desc* desc_outputs, float
  * (c1 <= 0: no clip).  JP_ERR_STATE without records. */
 jp_status jp_obrs_apply_kappa(jp_ctx* ctx, double kappa, float c1, float* out_weight);
 
+/* Measurement aid (the paper has no counterpart): streams `bytes` of device memory
+ * at src through a plain kernel `reps` times on the given stream and returns the
+ * device time of one repetition in milliseconds.  dst == NULL: the buffer is only
+ * read; else it is copied to dst (bytes more are written).  Pointers 16-byte aligned;
+ * the call synchronises on the stream.  bench.py reports the read-only rate beside
+ * the copy rate, since the forward pass only reads its logits. */
+jp_status jp_probe_stream(const void* src, void* dst, int64_t bytes, int reps, void* cuda_stream,
+                          float* out_ms_per_rep);
+
 /* Same forward with every pointer in HOST memory (pinned memory makes the
  * copies asynchronous): the library stages the rows through device buffers it
  * owns, chunk by chunk with copies overlapping compute, writes the outputs back

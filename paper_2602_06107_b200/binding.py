@@ -24,7 +24,7 @@ JP_ERR_TOO_LARGE = -8
 EXPORTS = (
     "jp_create", "jp_destroy", "jp_set_stream", "jp_obrs_workspace_bytes", "jp_reserve",
     "jp_obrs_forward", "jp_obrs_backward", "jp_batch_begin", "jp_batch_chunk", "jp_batch_finalize",
-    "jp_obrs_forward_host", "jp_obrs_apply_kappa", "jp_budget_lambda_static", "jp_status_string", "jp_last_error", "jp_launch_count",
+    "jp_obrs_forward_host", "jp_obrs_apply_kappa", "jp_budget_lambda_static", "jp_probe_stream", "jp_status_string", "jp_last_error", "jp_launch_count",
     "jp_enable_kernel_timing", "jp_stream_kernel_times",
 )
 
@@ -100,6 +100,7 @@ def load():
                                      vp, vp, vp, vp, vp, vp, vp, vp]
     lib.jp_obrs_apply_kappa.argtypes = [vp, ctypes.c_double, f32, vp]
     lib.jp_budget_lambda_static.argtypes = [vp, vp, vp, i64, f32, vp, vp]
+    lib.jp_probe_stream.argtypes = [vp, vp, i64, ctypes.c_int, vp, ctypes.POINTER(ctypes.c_float)]
     lib.jp_batch_begin.argtypes = [vp, i64, i64, i32, ctypes.c_int, f32]
     lib.jp_batch_chunk.argtypes = [vp, ctypes.POINTER(jp_obrs_desc), vp, vp, vp, vp]
     lib.jp_batch_finalize.argtypes = [vp, ctypes.POINTER(jp_obrs_desc), f32, i32, u64, vp, vp, vp, vp, vp]
@@ -227,6 +228,20 @@ def jp_budget_lambda_static(logp_actor, logp_policy, mask, T: int, budget: float
         stream = torch.cuda.current_stream().cuda_stream
     return int(lib.jp_budget_lambda_static(_ptr(logp_actor), _ptr(logp_policy), _ptr(mask), T, budget,
                                            _ptr(out_lambda), ctypes.c_void_p(stream)))
+
+
+def jp_probe_stream(src, dst=None, reps: int = 10, stream=None) -> float:
+    """GB/s of a plain kernel that reads ``src`` (and writes it to ``dst`` if given): bytes moved / device time."""
+    lib = load()
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    nbytes = src.numel() * src.element_size()
+    ms = ctypes.c_float(0.0)
+    st = lib.jp_probe_stream(_ptr(src), _ptr(dst), nbytes, reps, ctypes.c_void_p(stream), ctypes.byref(ms))
+    if st != 0:
+        raise JackpotError(f"jp_probe_stream: {lib.jp_status_string(st).decode()}")
+    moved = nbytes * (2 if dst is not None else 1)
+    return moved / (ms.value * 1e-3) / 1e9
 
 
 def jp_batch_begin(ctx: Context, T_total: int, V: int, dtype: int, k: int, fixed_lambda_for_exact_mode=0.0):
