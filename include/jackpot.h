@@ -192,7 +192,10 @@ jp_status jp_obrs_backward(jp_ctx* ctx, const jp_obrs_desc* desc, const jp_obrs_
  * batch-wide).  begin -> chunk x n (rows stream once, records accumulate at
  * desc->token_offset .. +T) -> finalize (lambda, decisions, Z_approx, kappa,
  * weights for all T_total rows; outputs are [T_total]).  Rows no chunk covered
- * count as masked.  Exact mode (k >= V) needs a fixed lambda given at begin. */
+ * count as masked.  Exact mode (k >= V) needs a fixed lambda given at begin.
+ * desc_outputs of jp_batch_finalize carries c1, the optional per-token outputs and
+ * token_offset = the global row index of the batch's row 0 (0 unless this batch is
+ * one shard of a larger one: the accept draws are keyed on the global index). */
 jp_status jp_batch_begin(jp_ctx* ctx, int64_t T_total, int64_t V, int32_t dtype, int k,
                          float fixed_lambda_for_exact_mode);
 jp_status jp_batch_chunk(jp_ctx* ctx, const jp_obrs_desc* desc, const void* actor_logits,
@@ -201,6 +204,16 @@ jp_status jp_batch_finalize(jp_ctx* ctx, const jp_obrs_desc* desc_outputs, float
                             int32_t lambda_mode, uint64_t seed, uint8_t* out_accept,
                             float* out_weight, float* out_logp_actor, float* out_logp_policy,
                             jp_stats* out_stats);
+
+/* Between the last jp_batch_chunk and jp_batch_finalize: the log-probs of the
+ * sampled tokens that the streamed rows have left in the records, [T_total] fp32
+ * each (0 for rows that are masked, have a bad token id or were not streamed), and
+ * which rows are valid, [T_total] u8.  Any pointer may be NULL.  A batch spread over
+ * several devices in budget mode gathers these from all of them, solves one lambda
+ * over the whole batch (Theorem 3.4 applied to the batch's sampled tokens; see
+ * jp_budget_lambda_static) and finalizes every shard with that fixed lambda: the
+ * rows are still streamed once. */
+jp_status jp_batch_logprobs(jp_ctx* ctx, float* out_logp_actor, float* out_logp_policy, uint8_t* out_valid);
 
 /* Weights with a calibration factor supplied by the caller (Section 4.4.2: kappa
  * is a batch-wide scalar).  A batch whose rows are spread over several devices

@@ -24,7 +24,7 @@ JP_ERR_TOO_LARGE = -8
 EXPORTS = (
     "jp_create", "jp_destroy", "jp_set_stream", "jp_obrs_workspace_bytes", "jp_reserve",
     "jp_obrs_forward", "jp_obrs_backward", "jp_batch_begin", "jp_batch_chunk", "jp_batch_finalize",
-    "jp_obrs_forward_host", "jp_obrs_apply_kappa", "jp_budget_lambda_static", "jp_probe_stream", "jp_status_string", "jp_last_error", "jp_launch_count",
+    "jp_obrs_forward_host", "jp_obrs_apply_kappa", "jp_batch_logprobs", "jp_budget_lambda_static", "jp_probe_stream", "jp_status_string", "jp_last_error", "jp_launch_count",
     "jp_enable_kernel_timing", "jp_stream_kernel_times",
 )
 
@@ -99,6 +99,7 @@ def load():
     lib.jp_obrs_backward.argtypes = [vp, ctypes.POINTER(jp_obrs_desc), ctypes.POINTER(jp_obrs_bwd_desc),
                                      vp, vp, vp, vp, vp, vp, vp, vp]
     lib.jp_obrs_apply_kappa.argtypes = [vp, ctypes.c_double, f32, vp]
+    lib.jp_batch_logprobs.argtypes = [vp, vp, vp, vp]
     lib.jp_budget_lambda_static.argtypes = [vp, vp, vp, i64, f32, vp, vp]
     lib.jp_probe_stream.argtypes = [vp, vp, i64, ctypes.c_int, vp, ctypes.POINTER(ctypes.c_float)]
     lib.jp_batch_begin.argtypes = [vp, i64, i64, i32, ctypes.c_int, f32]
@@ -214,6 +215,10 @@ def jp_obrs_backward(ctx: Context, desc: jp_obrs_desc, bwd: jp_obrs_bwd_desc, ac
     ctx.check(ctx.lib.jp_obrs_backward(ctx.h, ctypes.byref(desc), ctypes.byref(bwd), _ptr(actor_logits),
                                        _ptr(policy_logits), _ptr(tokens), _ptr(mask), _ptr(accept),
                                        _ptr(weight), _ptr(d_actor_logits), _ptr(d_policy_logits)))
+
+
+def jp_batch_logprobs(ctx: Context, out_logp_actor, out_logp_policy, out_valid):
+    ctx.check(ctx.lib.jp_batch_logprobs(ctx.h, _ptr(out_logp_actor), _ptr(out_logp_policy), _ptr(out_valid)))
 
 
 def jp_obrs_apply_kappa(ctx: Context, kappa: float, c1: float, out_weight):

@@ -411,7 +411,9 @@ jp_status jp_batch_finalize(jp_ctx* c, const jp_obrs_desc* dout, float lambda_or
     return fail(c, JP_ERR_UNSUPPORTED, "exact mode in a chunked batch supports a fixed lambda only");
   cudaSetDevice(c->device);
   float c1 = dout ? dout->c1 : 0.f;
-  EpilogueArgs ea = epilogue_args(c, dout, c->rec_rows, c->rec_k, seed, c->batch_rng_base, c1, out_accept, out_weight,
+  // record row 0 of this batch may sit at a global row index of its own (one shard of a larger batch)
+  const int64_t rng_base = c->batch_rng_base + (dout ? dout->token_offset : 0);
+  EpilogueArgs ea = epilogue_args(c, dout, c->rec_rows, c->rec_k, seed, rng_base, c1, out_accept, out_weight,
                                   out_lq, out_lp, out_stats);
   ea.aux_zx = nullptr;
   int nl = 0;
@@ -428,6 +430,16 @@ jp_status jp_batch_finalize(jp_ctx* c, const jp_obrs_desc* dout, float lambda_or
   if (e != cudaSuccess) return cuda_fail(c, e, "epilogue launch");
   c->batch_open = false;
   c->have_records = true;
+  return JP_OK;
+}
+
+jp_status jp_batch_logprobs(jp_ctx* c, float* out_logp_actor, float* out_logp_policy, uint8_t* out_valid) {
+  if (!c) return JP_ERR_INVALID_ARG;
+  if (!c->batch_open) return fail(c, JP_ERR_STATE, "jp_batch_logprobs outside jp_batch_begin .. jp_batch_finalize");
+  cudaSetDevice(c->device);
+  cudaError_t e = launch_logprobs(c->rec_rows, c->rec, out_logp_actor, out_logp_policy, out_valid, c->stream);
+  if (e != cudaSuccess) return cuda_fail(c, e, "log-prob copy launch");
+  if (c->rec_rows > 0) c->launches += 1;
   return JP_OK;
 }
 

@@ -289,6 +289,18 @@ __global__ void __launch_bounds__(EPI_NT) finalize_kernel(EpilogueArgs A) {
 // The weights again, with a calibration factor the caller supplies: a batch that
 // is spread over several devices sums (N, accepted, sum of Z_approx) over all of
 // them (Section 4.4.2: kappa is batch-wide) and hands the resulting kappa back.
+// The log-probs of the sampled tokens as the records hold them so far (0 for rows
+// that are masked, bad or not streamed yet), plus the validity flags.
+__global__ void __launch_bounds__(EPI_NT) logprobs_kernel(int64_t T, Records rec, float* out_lq, float* out_lp,
+                                                          uint8_t* out_valid) {
+  const int64_t i = (int64_t)blockIdx.x * EPI_NT + threadIdx.x;
+  if (i >= T) return;
+  const bool v = rec.flag[i] != 0;
+  if (out_lq) out_lq[i] = v ? rec.lq[i] : 0.f;
+  if (out_lp) out_lp[i] = v ? rec.lp[i] : 0.f;
+  if (out_valid) out_valid[i] = v ? 1 : 0;
+}
+
 __global__ void __launch_bounds__(EPI_NT) reweight_kernel(int64_t T, Records rec, const Scalars* sc, double kappa,
                                                           float c1, float* out_weight) {
   const int64_t r = (int64_t)blockIdx.x * EPI_NT + threadIdx.x;
@@ -335,6 +347,13 @@ cudaError_t launch_epilogue(const EpilogueArgs& a, cudaStream_t s, int* n_launch
   unsigned blocks = (unsigned)((a.T + EPI_NT - 1) / EPI_NT);
   finalize_kernel<<<blocks < 1 ? 1 : blocks, EPI_NT, 0, s>>>(a);
   *n_launch += 2;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_logprobs(int64_t T, const Records& rec, float* out_lq, float* out_lp, uint8_t* out_valid,
+                            cudaStream_t s) {
+  if (T <= 0) return cudaSuccess;
+  logprobs_kernel<<<(unsigned)((T + EPI_NT - 1) / EPI_NT), EPI_NT, 0, s>>>(T, rec, out_lq, out_lp, out_valid);
   return cudaGetLastError();
 }
 

@@ -137,6 +137,8 @@ cudaError_t launch_budget_solve(const EpilogueArgs& a, double budget, cudaStream
 cudaError_t launch_epilogue(const EpilogueArgs& a, cudaStream_t s, int* n_launch);
 cudaError_t launch_reweight(int64_t T, const Records& rec, const Scalars* sc, double kappa, float c1,
                             float* out_weight, cudaStream_t s);
+cudaError_t launch_logprobs(int64_t T, const Records& rec, float* out_lq, float* out_lp, uint8_t* out_valid,
+                            cudaStream_t s);
 cudaError_t launch_grad(const GradArgs& a, cudaStream_t s, int sms, int* n_launch);
 
 }  // namespace jp

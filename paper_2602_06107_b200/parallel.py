@@ -53,3 +53,45 @@ def max_over_ranks(value: float, group=None, device=None) -> float:
     if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
         dist.all_reduce(t, op=dist.ReduceOp.MAX, group=group)
     return float(t.item())
+
+
+def gather_rows(x: torch.Tensor, group=None) -> torch.Tensor:
+    """All ranks' 1-D shards of a row-indexed array, concatenated in rank order (shards may differ in length)."""
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size(group) == 1:
+        return x
+    world = dist.get_world_size(group)
+    n = torch.tensor([x.numel()], dtype=torch.int64, device=x.device)
+    sizes = [torch.zeros_like(n) for _ in range(world)]
+    dist.all_gather(sizes, n, group=group)
+    sizes = [int(s.item()) for s in sizes]
+    pad = torch.zeros(max(sizes), dtype=x.dtype, device=x.device)
+    pad[: x.numel()] = x
+    parts = [torch.empty_like(pad) for _ in range(world)]
+    dist.all_gather(parts, pad, group=group)
+    return torch.cat([p[:s] for p, s in zip(parts, sizes)])
+
+
+def global_lambda_from_budget(logp_actor, logp_policy, valid, budget: float, solve, group=None) -> float:
+    """One lambda for a batch whose rows are spread over the ranks (budget mode).
+
+    Every rank passes its shard's log-probs of the sampled tokens and validity flags (from
+    jp_batch_logprobs); they are all-gathered (12 bytes a token: at most 1.5 MB for the largest
+    workload) and every rank solves the same system with `solve(logp_actor, logp_policy, valid,
+    budget) -> float`, on a GPU `solve_on_device` below.  The result is the same on all ranks
+    because the inputs are."""
+    lq = gather_rows(logp_actor, group)
+    lp = gather_rows(logp_policy, group)
+    v = gather_rows(valid, group)
+    return float(solve(lq, lp, v, budget))
+
+
+def solve_on_device(logp_actor, logp_policy, valid, budget: float) -> float:
+    """The library's batch-level budget solve on device arrays (jp_budget_lambda_static: no allocation
+    inside the library, at most JP_STATIC_MAX_ROWS rows)."""
+    from . import binding as B
+    out = torch.zeros(1, dtype=torch.float32, device=logp_actor.device)
+    st = B.jp_budget_lambda_static(logp_actor.contiguous(), logp_policy.contiguous(), valid.contiguous(),
+                                   logp_actor.numel(), budget, out)
+    if st != 0:
+        raise B.JackpotError(f"jp_budget_lambda_static: status {st}")
+    return float(out.item())

@@ -327,3 +327,53 @@ def test_row_shards_with_a_batch_wide_kappa_match_the_undivided_batch(ctx):
     with pytest.raises(B.JackpotError, match="sequence"):
         B.jp_obrs_apply_kappa(fresh, 1.0, 0.0, w)
     fresh.close()
+
+
+def test_row_shards_in_budget_mode_share_one_lambda(ctx):
+    """Two shards of one batch in budget mode: each streams its rows once (chunked API), the
+    log-probs are gathered, one lambda is solved for the whole batch and every shard is
+    finalized with it; decisions, lambda and (after the kappa exchange) weights equal those
+    of one budget-mode call over the whole batch."""
+    from paper_2602_06107_b200 import parallel
+    T, V, k, budget = 320, 6000, 12, 0.6
+    r = LogitRecipe(T=T, V=V, dtype="bf16", sigma0=2.5, peaks=4, sigma=1.2, seed=62)
+    za, zp, tok = make_logits(r, "cuda")
+    mask = (torch.arange(T, device="cuda") % 5 != 2).to(torch.uint8)
+    whole = runner.forward(ctx, za, zp, tok, mask, budget=budget, k=k, seed=3, c1=2.5)
+    ctxs = [B.Context(0), B.Context(0)]
+    shards = [parallel.shard_rows(T, 2, rank) for rank in range(2)]
+    lqs, lps, vs = [], [], []
+    for (lo, hi), c in zip(shards, ctxs):
+        n = hi - lo
+        B.jp_batch_begin(c, n, V, B.JP_BF16, k, 0.0)
+        B.jp_batch_chunk(c, B.make_desc(za[lo:hi], token_offset=0), za[lo:hi], zp[lo:hi], tok[lo:hi], mask[lo:hi])
+        lq, lp = torch.empty(n, device="cuda"), torch.empty(n, device="cuda")
+        v = torch.empty(n, dtype=torch.uint8, device="cuda")
+        B.jp_batch_logprobs(c, lq, lp, v)
+        lqs.append(lq); lps.append(lp); vs.append(v)
+    # what the all-gather would hand to every rank
+    lam = parallel.solve_on_device(torch.cat(lqs), torch.cat(lps), torch.cat(vs), budget)
+    close(lam, whole["stats"]["lambda_used"], rtol=1e-6)
+    outs, tot = [], torch.zeros(3, dtype=torch.float64)
+    for (lo, hi), c in zip(shards, ctxs):
+        n = hi - lo
+        o = runner._alloc_outputs(n, "cuda")
+        d = B.jp_obrs_desc()
+        d.c1 = 2.5
+        d.token_offset = lo
+        B.jp_batch_finalize(c, d, lam, B.JP_LAMBDA_FIXED, 3, o["accept"], o["weight"], o["logp_actor"],
+                            o["logp_policy"], o["stats_buf"])
+        torch.cuda.synchronize()
+        o["stats"] = B.read_stats(o["stats_buf"])
+        outs.append(o)
+        tot += parallel.batch_totals(o["stats"])
+    kappa = parallel.kappa_from_totals(tot)
+    for c, o in zip(ctxs, outs):
+        B.jp_obrs_apply_kappa(c, kappa, 2.5, o["weight"])
+    torch.cuda.synchronize()
+    if float(np.float32(lam)) == float(np.float32(whole["stats"]["lambda_used"])):
+        assert torch.equal(torch.cat([o["accept"] for o in outs]), whole["accept"])
+        close(kappa, whole["stats"]["kappa"], rtol=1e-9)
+        close(torch.cat([o["weight"] for o in outs]).cpu().numpy(), whole["weight"].cpu().numpy())
+    for c in ctxs:
+        c.close()

@@ -56,7 +56,12 @@ def _worker(rank, world, port, T, V, out_q):
                              lam=1.4, k=8, seed=3, token_offset=lo)
         kappa, tot = parallel.global_kappa(ref["stats"])
         slow = parallel.max_over_ranks(float(rank + 1))
-        out_q.put((rank, lo, hi, kappa, tot.tolist(), slow, ref["accept"].tolist(), ref["zk"].tolist()))
+        # budget mode: one lambda for the whole batch from the gathered log-probs of the shards
+        valid = torch.from_numpy((mask[lo:hi] != 0).astype(np.uint8))
+        lam_b = parallel.global_lambda_from_budget(
+            torch.from_numpy(ref["lq"]), torch.from_numpy(ref["lp"]), valid, 0.55,
+            lambda a, b, v, bud: oracle.lambda_from_budget(a.numpy(), b.numpy(), bud, v.numpy()))
+        out_q.put((rank, lo, hi, kappa, tot.tolist(), slow, ref["accept"].tolist(), ref["zk"].tolist(), lam_b))
     finally:
         dist.destroy_process_group()
 
@@ -85,3 +90,5 @@ def test_two_ranks_agree_with_the_undivided_batch():
     zk = np.concatenate([np.asarray(g[7]) for g in got])
     assert np.array_equal(acc, whole["accept"]), "decisions depend on the split"
     assert np.array_equal(zk, whole["zk"])
+    lam_whole = oracle.lambda_from_budget(whole["lq"], whole["lp"], 0.55, mask)
+    assert got[0][8] == got[1][8] == lam_whole, "the gathered solve must equal the undivided batch's"
