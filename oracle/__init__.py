@@ -235,6 +235,16 @@ def loss(za64, zp64, tokens, acc, weight64, adv64, logp_ref, logq_ref, pfix, lam
                                ctypes.c_int(1 if clip else 0), ctypes.c_double(eps_lo), ctypes.c_double(eps_hi)))
 
 
+def row_lambda(za, zp, budget, mask=None):
+    """Per-row lambda meeting an acceptance budget (Theorem 3.4), with KL(p||q) and KL(p||q~)."""
+    T, V = _check2d(za)
+    lam, kb, ka = np.zeros(T), np.zeros(T), np.zeros(T)
+    lib().jo_row_lambda(ctypes.c_int64(T), ctypes.c_int64(V), ctypes.c_int64(V), ctypes.c_int(_dtype_code(za)),
+                        _vp(za), _vp(zp), _p(mask, ctypes.c_uint8), ctypes.c_double(budget),
+                        _p(lam, ctypes.c_double), _p(kb, ctypes.c_double), _p(ka, ctypes.c_double))
+    return dict(lam=lam, kl_before=kb, kl_after=ka)
+
+
 def kl_rows(za, zp, lse_a, lse_p, mask=None):
     T, V = _check2d(za)
     kl = np.zeros(T)

@@ -458,6 +458,70 @@ double jo_loss(int64_t T, int64_t V, const double* za, const double* zp, const i
   return J / (double)N;
 }
 
+// Theorem 3.4, literally: for ONE pair of distributions (a row), the lambda at which the
+// OBRS rule a_v = min(1, p_v / (lambda q_v)) accepts exactly the budget,
+//   Z(lambda) = sum_v q_v a_v = sum_v min(q_v, p_v / lambda) = budget.
+// Z is continuous and non-increasing in lambda.  With the entries ordered by ratio
+// r_v = p_v / q_v ascending, on [r_(j), r_(j+1)] the j lowest ratios are accepted in part:
+//   Z(lambda) = sum_{i > j} q_(i) + (1 / lambda) sum_{i <= j} p_(i),
+// so lambda_j = P_j / (budget - Qtail_j); the j whose lambda_j lies in its own interval
+// is the answer.  budget == 1 gives min_v r_v (the largest lambda that accepts everything).
+// Also returns KL(p || q) and KL(p || q~), q~ = min(q, p/lambda) / Z (Figure 2b).
+void jo_row_lambda(int64_t T, int64_t V, int64_t ld, int dtype, const void* za, const void* zp,
+                   const uint8_t* mask, double budget, double* lambda, double* kl_before,
+                   double* kl_after) {
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int64_t t = 0; t < T; ++t) {
+    lambda[t] = 0.0;
+    if (kl_before) kl_before[t] = 0.0;
+    if (kl_after) kl_after[t] = 0.0;
+    if (!row_valid(mask, t)) continue;
+    const double lsa = row_lse(za, dtype, t * ld, V), lsp = row_lse(zp, dtype, t * ld, V);
+    std::vector<double> lq(V), lpv(V);
+    std::vector<int64_t> order(V);
+    for (int64_t v = 0; v < V; ++v) {
+      lq[v] = logit_at(za, dtype, t * ld + v) - lsa;
+      lpv[v] = logit_at(zp, dtype, t * ld + v) - lsp;
+      order[v] = v;
+    }
+    std::sort(order.begin(), order.end(), [&](int64_t a, int64_t b) {
+      double da = lpv[a] - lq[a], db = lpv[b] - lq[b];
+      return da < db || (da == db && a < b);
+    });
+    // suffix sums of q in ratio order
+    std::vector<double> qtail(V + 1, 0.0);
+    for (int64_t j = V - 1; j >= 0; --j) qtail[j] = qtail[j + 1] + std::exp(lq[order[j]]);
+    double lam = std::exp(lpv[order[0]] - lq[order[0]]);       // budget 1: everything accepted in full
+    if (budget < qtail[0]) {
+      double phead = 0.0;
+      for (int64_t j = 1; j <= V; ++j) {                       // the j lowest ratios are cut
+        phead += std::exp(lpv[order[j - 1]]);
+        double denom = budget - qtail[j];
+        if (denom <= 0.0) continue;
+        double cand = phead / denom;
+        double lo = std::exp(lpv[order[j - 1]] - lq[order[j - 1]]);
+        double hi = j < V ? std::exp(lpv[order[j]] - lq[order[j]]) : HUGE_VAL;
+        if (cand >= lo * (1.0 - 1e-15) && cand <= hi * (1.0 + 1e-15)) { lam = cand; break; }
+      }
+    }
+    lambda[t] = lam;
+    if (kl_before || kl_after) {
+      double kb = 0.0, ka = 0.0, Z = 0.0;
+      for (int64_t v = 0; v < V; ++v) {
+        double p = std::exp(lpv[v]), q = std::exp(lq[v]);
+        double kept = std::min(q, p / lam);
+        Z += kept;
+        if (p > 0.0) {
+          kb += p * (lpv[v] - lq[v]);
+          ka += p * (lpv[v] - std::log(kept));
+        }
+      }
+      if (kl_before) kl_before[t] = kb;
+      if (kl_after) kl_after[t] = ka + std::log(Z);
+    }
+  }
+}
+
 // Step 10 (diagnostic): KL(p_t || q_t) per row, the actor-policy gap of Figure 2.
 void jo_kl_rows(int64_t T, int64_t V, int64_t ld, int dtype, const void* za, const void* zp,
                 const uint8_t* mask, const double* lse_a, const double* lse_p, double* kl) {

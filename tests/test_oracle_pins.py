@@ -549,3 +549,53 @@ def test_general_gradients_by_central_differences():
     da1, dp1 = oracle.grad_rows(rows, za, zp, tok, acc, fwd["w"], fwd["lse_a"], fwd["lse_p"], T, adv=adv, ppo=base)
     da0, dp0 = oracle.grad_rows(rows, za, zp, tok, acc, fwd["w"], fwd["lse_a"], fwd["lse_p"], T, adv=adv)
     assert np.allclose(da1, da0, rtol=1e-12, atol=0) and np.allclose(dp1, dp0, rtol=1e-12, atol=0)
+
+
+# ---- Theorem 3.4 per distribution: the lambda that meets an acceptance budget ------------------
+
+def test_row_lambda_meets_the_budget_and_is_unique():
+    za, zp, _ = _rand_rows(40, 300, seed=31, sigma=1.2)
+    p, q = _pq(za, zp)
+    for b in (0.3, 0.6, 0.9, 0.999):
+        r = oracle.row_lambda(za, zp, b)
+        lam = r["lam"][:, None]
+        Z = np.minimum(q, p / lam).sum(1)                      # brute force from the definition
+        assert np.allclose(Z, b, rtol=1e-12, atol=0)
+        # Z is strictly decreasing around the solution (a unique root): a slightly smaller lambda accepts more
+        assert np.all(np.minimum(q, p / (lam * 0.999)).sum(1) > b) and np.all(np.minimum(q, p / (lam * 1.001)).sum(1) < b)
+    # the budget is monotone in lambda: a tighter budget needs a larger lambda
+    l3, l6, l9 = (oracle.row_lambda(za, zp, b)["lam"] for b in (0.3, 0.6, 0.9))
+    assert np.all(l3 > l6) and np.all(l6 > l9)
+    # budget 1: the largest lambda that still accepts everything is the smallest ratio
+    assert np.allclose(oracle.row_lambda(za, zp, 1.0)["lam"], (p / q).min(1), rtol=1e-12)
+
+
+def test_row_lambda_closed_forms():
+    # p == q: Z(lambda) = min(1, 1/lambda), so lambda = 1 / budget
+    za, _, _ = _rand_rows(5, 64, seed=32)
+    assert np.allclose(oracle.row_lambda(za, za, 0.4)["lam"], 2.5, rtol=1e-12)
+    # two outcomes, q = (1/2, 1/2), p = (0.9, 0.1): ratios 1.8 and 0.2
+    zq = np.log(np.array([[0.5, 0.5]])).astype(np.float64)
+    zpp = np.log(np.array([[0.9, 0.1]])).astype(np.float64)
+    za2, zp2 = zq.astype(np.float32), zpp.astype(np.float32)
+    p2, q2 = _pq(za2, zp2)
+    # budget 0.7: only the low-ratio outcome is cut: 0.5 + 0.1/lambda = 0.7 -> lambda = 0.5
+    assert oracle.row_lambda(za2, zp2, 0.7)["lam"][0] == pytest.approx(p2[0, 1] / (0.7 - q2[0, 0]), rel=1e-12)
+    assert oracle.row_lambda(za2, zp2, 0.7)["lam"][0] == pytest.approx(0.5, rel=1e-6)
+    # budget 0.25: both are cut: 1/lambda = 0.25 -> lambda = 4 (above the largest ratio: classical rejection sampling)
+    assert oracle.row_lambda(za2, zp2, 0.25)["lam"][0] == pytest.approx(4.0, rel=1e-6)
+
+
+def test_row_lambda_kl_before_and_after():
+    za, zp, _ = _rand_rows(30, 200, seed=33, sigma=1.5)
+    p, q = _pq(za, zp)
+    r = oracle.row_lambda(za, zp, 0.7)
+    kept = np.minimum(q, p / r["lam"][:, None])
+    qt = kept / kept.sum(1, keepdims=True)
+    assert np.allclose(r["kl_before"], (p * np.log(p / q)).sum(1), rtol=1e-10)
+    assert np.allclose(r["kl_after"], (p * np.log(p / qt)).sum(1), rtol=1e-10)
+    assert np.all(r["kl_after"] <= r["kl_before"] + 1e-12)      # Theorem 3.3: the kept distribution is closer to p
+    # masked rows give zeros
+    m = np.ones(30, np.uint8); m[3] = 0
+    rm = oracle.row_lambda(za, zp, 0.7, mask=m)
+    assert rm["lam"][3] == 0 and rm["kl_after"][3] == 0 and rm["lam"][4] == r["lam"][4]
