@@ -225,6 +225,21 @@ jp_status jp_batch_logprobs(jp_ctx* ctx, float* out_logp_actor, float* out_logp_
  * (c1 <= 0: no clip).  JP_ERR_STATE without records. */
 jp_status jp_obrs_apply_kappa(jp_ctx* ctx, double kappa, float c1, float* out_weight);
 
+/* Theorem 3.4 for single distributions: for every row t the lambda_t at which the
+ * OBRS rule accepts exactly `budget` of the proposal's mass,
+ *   sum_v min(q_t(v), p_t(v) / lambda_t) = budget,   q_t, p_t = softmax of the rows,
+ * [T] fp32 (budget in (0, 1]; budget == 1 gives the smallest ratio p/q, the largest
+ * lambda that still accepts everything).  Optionally KL(p_t || q_t), KL(p_t || q~_t)
+ * with q~ the accepted distribution (Theorem 3.3: never larger; Figure 2b), and the
+ * number of Newton steps taken, [T] each, NULL to skip.  Masked rows give 0.  Uses
+ * desc's T, V, ld, dtype only; independent of the forward pass and its records.
+ * This is the per-distribution budget of the theorem, not the batch-level lambda that
+ * jp_obrs_forward solves in JP_LAMBDA_FROM_BUDGET mode. */
+jp_status jp_obrs_row_lambda(jp_ctx* ctx, const jp_obrs_desc* desc, const void* actor_logits,
+                             const void* policy_logits, const uint8_t* mask, float budget,
+                             float* out_lambda, float* out_kl_before, float* out_kl_after,
+                             int32_t* out_iterations);
+
 /* Measurement aid (the paper has no counterpart): streams `bytes` of device memory
  * at src through a plain kernel `reps` times on the given stream and returns the
  * device time of one repetition in milliseconds.  dst == NULL: the buffer is only

@@ -24,7 +24,7 @@ JP_ERR_TOO_LARGE = -8
 EXPORTS = (
     "jp_create", "jp_destroy", "jp_set_stream", "jp_obrs_workspace_bytes", "jp_reserve",
     "jp_obrs_forward", "jp_obrs_backward", "jp_batch_begin", "jp_batch_chunk", "jp_batch_finalize",
-    "jp_obrs_forward_host", "jp_obrs_apply_kappa", "jp_batch_logprobs", "jp_budget_lambda_static", "jp_probe_stream", "jp_status_string", "jp_last_error", "jp_launch_count",
+    "jp_obrs_forward_host", "jp_obrs_apply_kappa", "jp_batch_logprobs", "jp_obrs_row_lambda", "jp_budget_lambda_static", "jp_probe_stream", "jp_status_string", "jp_last_error", "jp_launch_count",
     "jp_enable_kernel_timing", "jp_stream_kernel_times",
 )
 
@@ -100,6 +100,7 @@ def load():
                                      vp, vp, vp, vp, vp, vp, vp, vp]
     lib.jp_obrs_apply_kappa.argtypes = [vp, ctypes.c_double, f32, vp]
     lib.jp_batch_logprobs.argtypes = [vp, vp, vp, vp]
+    lib.jp_obrs_row_lambda.argtypes = [vp, ctypes.POINTER(jp_obrs_desc), vp, vp, vp, f32, vp, vp, vp, vp]
     lib.jp_budget_lambda_static.argtypes = [vp, vp, vp, i64, f32, vp, vp]
     lib.jp_probe_stream.argtypes = [vp, vp, i64, ctypes.c_int, vp, ctypes.POINTER(ctypes.c_float)]
     lib.jp_batch_begin.argtypes = [vp, i64, i64, i32, ctypes.c_int, f32]
@@ -215,6 +216,13 @@ def jp_obrs_backward(ctx: Context, desc: jp_obrs_desc, bwd: jp_obrs_bwd_desc, ac
     ctx.check(ctx.lib.jp_obrs_backward(ctx.h, ctypes.byref(desc), ctypes.byref(bwd), _ptr(actor_logits),
                                        _ptr(policy_logits), _ptr(tokens), _ptr(mask), _ptr(accept),
                                        _ptr(weight), _ptr(d_actor_logits), _ptr(d_policy_logits)))
+
+
+def jp_obrs_row_lambda(ctx: Context, desc, za, zp, mask, budget: float, out_lambda, out_kl_before=None,
+                       out_kl_after=None, out_iterations=None):
+    ctx.check(ctx.lib.jp_obrs_row_lambda(ctx.h, ctypes.byref(desc), _ptr(za), _ptr(zp), _ptr(mask), budget,
+                                         _ptr(out_lambda), _ptr(out_kl_before), _ptr(out_kl_after),
+                                         _ptr(out_iterations)))
 
 
 def jp_batch_logprobs(ctx: Context, out_logp_actor, out_logp_policy, out_valid):

@@ -433,6 +433,32 @@ jp_status jp_batch_finalize(jp_ctx* c, const jp_obrs_desc* dout, float lambda_or
   return JP_OK;
 }
 
+jp_status jp_obrs_row_lambda(jp_ctx* c, const jp_obrs_desc* d, const void* za, const void* zp, const uint8_t* mask,
+                             float budget, float* out_lambda, float* out_kl_before, float* out_kl_after,
+                             int32_t* out_iterations) {
+  if (!c) return JP_ERR_INVALID_ARG;
+  int64_t ld = 0;
+  jp_status st = check_shape(c, d, &ld);
+  if (st != JP_OK) return st;
+  if (!(budget > 0.f) || budget > 1.f) return fail(c, JP_ERR_INVALID_ARG, "budget must lie in (0, 1]");
+  if (d->T == 0) return JP_OK;
+  if (!za || !zp || !out_lambda) return fail(c, JP_ERR_INVALID_ARG, "a required pointer is NULL");
+  if (!aligned16(za) || !aligned16(zp)) return fail(c, JP_ERR_ALIGNMENT, "logit base pointers must be 16-byte aligned");
+  cudaSetDevice(c->device);
+  st = ensure_workspace(c, c->cap_rows > 0 ? c->cap_rows : 1, c->cap_k > 0 ? c->cap_k : 1);   // for the scalars
+  if (st != JP_OK) return st;
+  cudaError_t e = cudaMemsetAsync(&c->sc->row_counter2, 0, sizeof(int32_t), c->stream);
+  if (e != cudaSuccess) return cuda_fail(c, e, "cudaMemsetAsync");
+  RowLambdaArgs a{};
+  a.za = za; a.zp = zp; a.mask = mask; a.T = d->T; a.V = d->V; a.ld = ld; a.dtype = d->dtype; a.budget = budget;
+  a.sc = c->sc; a.out_lambda = out_lambda; a.out_kl_before = out_kl_before; a.out_kl_after = out_kl_after;
+  a.out_iters = out_iterations;
+  e = launch_row_lambda(a, c->stream, c->sms);
+  if (e != cudaSuccess) return cuda_fail(c, e, "row lambda kernel launch");
+  c->launches += 1;
+  return JP_OK;
+}
+
 jp_status jp_batch_logprobs(jp_ctx* c, float* out_logp_actor, float* out_logp_policy, uint8_t* out_valid) {
   if (!c) return JP_ERR_INVALID_ARG;
   if (!c->batch_open) return fail(c, JP_ERR_STATE, "jp_batch_logprobs outside jp_batch_begin .. jp_batch_finalize");

@@ -128,6 +128,20 @@ struct GradArgs {
   double* out_loss;
 };
 
+struct RowLambdaArgs {
+  const void* za;
+  const void* zp;
+  const uint8_t* mask;
+  int64_t T, V, ld;
+  int32_t dtype;
+  float budget;
+  Scalars* sc;
+  float* out_lambda;       // [T]
+  float* out_kl_before;    // [T] or null
+  float* out_kl_after;     // [T] or null
+  int32_t* out_iters;      // [T] or null
+};
+
 int stream_grid_size(int device);   // number of SMs
 cudaError_t launch_stream(const StreamArgs& a, cudaStream_t s, int sms);
 cudaError_t launch_exact_z(const ExactZArgs& a, cudaStream_t s, int sms);
@@ -139,6 +153,7 @@ cudaError_t launch_reweight(int64_t T, const Records& rec, const Scalars* sc, do
                             float* out_weight, cudaStream_t s);
 cudaError_t launch_logprobs(int64_t T, const Records& rec, float* out_lq, float* out_lp, uint8_t* out_valid,
                             cudaStream_t s);
+cudaError_t launch_row_lambda(const RowLambdaArgs& a, cudaStream_t s, int sms);
 cudaError_t launch_grad(const GradArgs& a, cudaStream_t s, int sms, int* n_launch);
 
 }  // namespace jp

@@ -10,7 +10,9 @@
 Only the library calls are timed (CUDA events on the context's stream); input generation is
 outside the timed regions.  One JSON line per measurement.
 
-    python -m paper_2602_06107_b200.measure_configs [cfg3_batch] [cfg4_sweep] [cfg5_train]
+  row_lambda  the per-distribution budget of Theorem 3.4 on the headline shape (4096 rows).
+
+    python -m paper_2602_06107_b200.measure_configs [cfg3_batch] [cfg4_sweep] [cfg5_train] [row_lambda]
 """
 from __future__ import annotations
 
@@ -161,14 +163,40 @@ def cfg5_train(ctx):
           kappa=st["kappa"], status=st["status"])
 
 
+def row_lambda(ctx):
+    """Theorem 3.4 per distribution on the headline shape: the lambda of every row for a budget,
+    with KL(p||q) before and KL(p||kept) after (the quantities of the paper's simulation figure)."""
+    cfg = CONFIGS["cfg2_qwen3"]
+    za, zp, _ = make_logits(cfg["recipe"], DEV)
+    T, V = za.shape
+    lam = torch.empty(T, device=DEV)
+    kb, ka = torch.empty(T, device=DEV), torch.empty(T, device=DEV)
+    it = torch.empty(T, dtype=torch.int32, device=DEV)
+    d = B.make_desc(za)
+    for budget in (0.5, 0.7, 0.9):
+        for _ in range(2):
+            B.jp_obrs_row_lambda(ctx, d, za, zp, None, budget, lam, kb, ka, it)
+        t = _Timer()
+        reps = 5
+        with t:
+            for _ in range(reps):
+                B.jp_obrs_row_lambda(ctx, d, za, zp, None, budget, lam, kb, ka, it)
+        ms = t.ms() / reps
+        steps = it.float().mean().item()
+        _emit(workload="row_lambda", rows=T, budget=budget, ms=ms, rows_per_s=T / (ms * 1e-3),
+              mean_newton_steps=steps, max_newton_steps=int(it.max().item()),
+              passes_over_the_rows=4.0 + steps, mean_lambda=lam.mean().item(), mean_kl_before=kb.mean().item(),
+              mean_kl_after=ka.mean().item())
+
+
 def main(argv):
     assert torch.cuda.is_available(), "needs a CUDA device"
     jp_build.build()
     torch.cuda.set_device(0)
-    which = [a for a in argv if not a.startswith("-")] or ["cfg3_batch", "cfg4_sweep", "cfg5_train"]
+    which = [a for a in argv if not a.startswith("-")] or ["cfg3_batch", "cfg4_sweep", "cfg5_train", "row_lambda"]
     ctx = B.Context(0)
     for name in which:
-        {"cfg3_batch": cfg3_batch, "cfg4_sweep": cfg4_sweep, "cfg5_train": cfg5_train}[name](ctx)
+        {"cfg3_batch": cfg3_batch, "cfg4_sweep": cfg4_sweep, "cfg5_train": cfg5_train, "row_lambda": row_lambda}[name](ctx)
         torch.cuda.empty_cache()
     ctx.close()
 
