@@ -77,6 +77,25 @@ def make_logits(r: LogitRecipe, device="cpu", block_rows: int = 256, rows=None):
     return za, zp, tok
 
 
+def make_dirichlet_logits(T: int, V: int, concentration: float, noise: float, seed: int, dtype="f32", device="cpu"):
+    """Simulated distribution pairs in the manner of the paper's numerical simulation: every row of the
+    policy is a draw from a symmetric Dirichlet (as log-probabilities, from Gamma draws), the actor is the
+    same row with Gaussian noise of scale ``noise`` added to the log-probabilities, which sets how far the
+    two distributions are apart.  The paper states no parameters for its figure; these are free."""
+    g = torch.Generator(device=device)
+    g.manual_seed(seed)
+    conc = torch.full((T, V), float(concentration), device=device)
+    gam = torch._standard_gamma(conc, generator=g).clamp_min_(1e-30)
+    logp = torch.log(gam)
+    logp = logp - torch.logsumexp(logp, dim=1, keepdim=True)
+    act = logp + noise * torch.randn((T, V), generator=g, device=device)
+    dt = torch_dtype(dtype)
+    zp, za = logp.to(dt), act.to(dt)
+    u = torch.rand((T, V), generator=g, device=device).clamp_(1e-30, 1.0 - 1e-7)
+    tok = (za.float() - torch.log(-torch.log(u))).argmax(dim=1).to(torch.int32)
+    return za, zp, tok
+
+
 def make_lengths_mask(n_resp: int, max_len: int, min_len: int, seed: int, device="cpu"):
     """Padded batch layout: ``n_resp`` responses with lengths U{min_len..max_len},
     each padded to ``max_len``; returns (mask[n_resp*max_len] uint8, lengths)."""

@@ -10,9 +10,11 @@
 Only the library calls are timed (CUDA events on the context's stream); input generation is
 outside the timed regions.  One JSON line per measurement.
 
-  row_lambda  the per-distribution budget of Theorem 3.4 on the headline shape (4096 rows).
+  row_lambda  the per-distribution budget of Theorem 3.4 on the headline shape (4096 rows);
+  simulation  Dirichlet pairs at growing distance: acceptance rate and divergence before / after
+              rejection (not run by default).
 
-    python -m paper_2602_06107_b200.measure_configs [cfg3_batch] [cfg4_sweep] [cfg5_train] [row_lambda]
+    python -m paper_2602_06107_b200.measure_configs [cfg3_batch] [cfg4_sweep] [cfg5_train] [row_lambda] [simulation]
 """
 from __future__ import annotations
 
@@ -189,6 +191,25 @@ def row_lambda(ctx):
               mean_kl_after=ka.mean().item())
 
 
+def simulation(ctx):
+    """The paper's numerical simulation, qualitatively: Dirichlet pairs at growing distance; acceptance
+    rate of OBRS at lambda = 1 (the exact normaliser Z) and the divergence to the target before and after
+    rejection at an acceptance budget of 0.9."""
+    from .inputs import make_dirichlet_logits
+    T, V = 2048, 32768
+    for noise in (0.1, 0.25, 0.5, 1.0, 1.5):
+        za, zp, tok = make_dirichlet_logits(T, V, 0.3, noise, seed=7, device=DEV)
+        ex = runner.forward(ctx, za, zp, tok, None, lam=1.0, k=V, seed=1)
+        kb, ka = torch.empty(T, device=DEV), torch.empty(T, device=DEV)
+        lam = torch.empty(T, device=DEV)
+        B.jp_obrs_row_lambda(ctx, B.make_desc(za), za, zp, None, 0.9, lam, kb, ka, None)
+        torch.cuda.synchronize()
+        _emit(workload="simulation", rows=T, V=V, noise=noise, mean_kl_p_q=kb.mean().item(),
+              acceptance_at_lambda_1=ex["z_approx"].mean().item(),
+              mean_kl_after_budget_0p9=ka.mean().item(), kl_reduction_factor=(kb.mean() / ka.mean()).item(),
+              mean_lambda_for_budget_0p9=lam.mean().item())
+
+
 def main(argv):
     assert torch.cuda.is_available(), "needs a CUDA device"
     jp_build.build()
@@ -196,7 +217,7 @@ def main(argv):
     which = [a for a in argv if not a.startswith("-")] or ["cfg3_batch", "cfg4_sweep", "cfg5_train", "row_lambda"]
     ctx = B.Context(0)
     for name in which:
-        {"cfg3_batch": cfg3_batch, "cfg4_sweep": cfg4_sweep, "cfg5_train": cfg5_train, "row_lambda": row_lambda}[name](ctx)
+        {"cfg3_batch": cfg3_batch, "cfg4_sweep": cfg4_sweep, "cfg5_train": cfg5_train, "row_lambda": row_lambda, "simulation": simulation}[name](ctx)
         torch.cuda.empty_cache()
     ctx.close()
 
