@@ -766,7 +766,10 @@ __device__ __noinline__ float sample_threshold(const char* row, int64_t nvec, in
     __syncwarp();
     for (int i = lane; i < ns; i += 32) {
       const uint32_t c = f32_order_bits(park[i]) >> sh;
-      atomicAdd(&hist[c > b0 ? c - b0 : 0u], 1u);        // c <= cmax, so the bin is at most NB - 1
+      // c <= cmax for every number, so the bin is at most NB - 1; a NaN's order bits lie above
+      // every number's (the maximum ignores NaNs), hence the clamp
+      const uint32_t bin = c > b0 ? c - b0 : 0u;
+      atomicAdd(&hist[bin < (uint32_t)(NB - 1) ? bin : (uint32_t)(NB - 1)], 1u);
     }
     __syncwarp();
     const int bin = find_tau_bin(hist, k, lane);

@@ -377,3 +377,70 @@ def test_row_shards_in_budget_mode_share_one_lambda(ctx):
         close(torch.cat([o["weight"] for o in outs]).cpu().numpy(), whole["weight"].cpu().numpy())
     for c in ctxs:
         c.close()
+
+
+def test_wide_dynamic_range_rows(ctx):
+    """Rows whose logits climb far beyond the headroom of a lane's reference exponent (64 binades =
+    44 nats) in the middle of the row, in steps and as a ramp: the online sums must move their
+    reference and still agree with the oracle.  (Magnitudes stay below ~60: see the next test.)"""
+    V, k = 40000, 16
+    g = torch.Generator().manual_seed(9)
+    for dt in (torch.float32, torch.bfloat16):
+        rows = torch.randn((8, V), generator=g)
+        rows[0, : V // 2] -= 100.0                      # one jump of 100 nats half way
+        rows[1, :] += torch.linspace(-400.0, 0.0, V)    # a ramp across many rescalings
+        rows[2, :] += torch.linspace(0.0, -300.0, V)    # the maximum comes first
+        rows[3, 123] = 45.0                             # one dominant entry
+        rows[4, :] = rows[4, :] * 10.0 - 50.0           # a wide spread below zero
+        rows[5, ::7] -= 150.0                           # entries far below the rest
+        rows[6, :] *= 1e-3                              # nearly flat
+        rows[7, : V - 5] -= 90.0                        # the jump in the last vectors
+        za = rows.to(dt).cuda()
+        zp = rows.flip(0).to(dt).cuda().contiguous()
+        tok = torch.tensor([5, V - 1, 0, 123, 9, 7, 11, V - 2], dtype=torch.int32, device="cuda")
+        # (the clip keeps the weights inside fp32: some tokens have p/q of e^150 here)
+        run_case(ctx, za, zp, tok, lam=1.2, k=k, seed=4, c1=5.0)
+        run_case(ctx, za, zp, tok, lam=1.2, k=V, seed=4, c1=5.0)    # exact mode
+
+
+def test_large_magnitude_logits_stay_inside_the_stated_bound(ctx):
+    """The exponent z log2(e) is formed with the fp32 constant log2(e), which is 1.9e-8 too large: a row
+    whose mass sits at logits of magnitude M gets a log-sum-exp that is off by about 1.34e-8 M (inside the
+    1e-6 bar up to M ~ 70).  Beyond that the error must stay within that bound, and the top-k lists exact."""
+    V, k = 20000, 8
+    g = torch.Generator().manual_seed(10)
+    rows = torch.randn((4, V), generator=g)
+    offs = torch.tensor([500.0, -800.0, 1500.0, 120.0])
+    rows += offs[:, None]
+    za = rows.cuda()
+    zp = rows.flip(1).contiguous().cuda()
+    tok = torch.tensor([1, 2, 3, 4], dtype=torch.int32, device="cuda")
+    out = runner.forward(ctx, za, zp, tok, None, lam=1.0, k=k, seed=1)
+    ref = oracle.forward(to_numpy_bits(za), to_numpy_bits(zp), tok.cpu().numpy(), None, lam=1.0, k=k, seed=1)
+    bound = 2e-8 * np.abs(offs.numpy()) + 1e-6 + 1e-7 * np.abs(ref["lse_a"])     # + one fp32 rounding of the result
+    assert np.all(np.abs(out["lse_actor"].cpu().numpy() - ref["lse_a"]) <= bound)
+    assert np.all(np.abs(out["lse_policy"].cpu().numpy() - ref["lse_p"]) <= bound)
+    assert np.all(np.abs(out["logp_actor"].cpu().numpy() - ref["lq64"]) <= bound)
+    assert np.array_equal(out["topk_idx_actor"].cpu().numpy(), ref["topk_idx_a"])
+    assert np.array_equal(out["topk_idx_policy"].cpu().numpy(), ref["topk_idx_p"])
+
+
+def test_nonfinite_rows_are_counted_and_do_not_disturb_the_others(ctx):
+    """+inf and NaN logits: the row is counted in n_nonfinite and its results are unspecified; nothing
+    traps or waits, and every other row is what it would be without them."""
+    T, V, k = 64, 30000, 8
+    r = LogitRecipe(T=T, V=V, dtype="bf16", sigma0=2.5, peaks=4, sigma=1.0, seed=63)
+    za, zp, tok = make_logits(r, "cuda")
+    clean = runner.forward(ctx, za, zp, tok, None, lam=1.3, k=k, seed=2)
+    za2, zp2 = za.clone(), zp.clone()
+    za2[5, 100] = float("inf")
+    zp2[9, 29999] = float("nan")
+    za2[20, :] = float("nan")
+    out = runner.forward(ctx, za2, zp2, tok, None, lam=1.3, k=k, seed=2)
+    st = out["stats"]
+    assert st["status"] == 0 and st["n_nonfinite"] >= 3
+    good = torch.ones(T, dtype=torch.bool, device="cuda")
+    good[[5, 9, 20]] = False
+    for n in ("logp_actor", "logp_policy", "lse_actor", "lse_policy", "z_approx", "accept_prob", "uniform",
+              "topk_idx_actor", "topk_idx_policy"):
+        assert torch.equal(out[n][good], clean[n][good]), n
