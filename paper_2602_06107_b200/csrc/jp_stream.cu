@@ -1137,7 +1137,10 @@ __device__ void topk_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int t, in
         if (sm.part_mL[p][t][w] != JP_NEG_INF) S += sm.part_s[p][t][w] * exp2_int(sm.part_mL[p][t][w] - M);
       int e;
       const float f = 2.f * frexpf(S, &e);                // S = f * 2^(e-1)
-      const double lse = ((double)M + (double)(e - 1)) * 0.6931471805599453 + (double)logf(f);
+      // The exponents were formed with the fp32 constant log2(e), which is short of log2(e) by a
+      // factor 1 - 1.335e-8: what was summed is exp(z (1 - eps)), whose log-sum-exp is lse - eps * (lse - H)
+      // with H the entropy of the row (at most ln V).  Scaling by 1 + eps leaves eps * H < 2e-7.
+      const double lse = (((double)M + (double)(e - 1)) * 0.6931471805599453 + (double)logf(f)) * (1.0 + 1.33497582e-8);
       const float lsef = (float)lse;
       const float lpx = (float)((double)zx - lse);
       if (t == 0) { A.rec.lse_a[rrow] = lsef; A.rec.lq[rrow] = lpx; A.rec.flag[rrow] = 1; }

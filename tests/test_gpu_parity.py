@@ -403,10 +403,12 @@ def test_wide_dynamic_range_rows(ctx):
         run_case(ctx, za, zp, tok, lam=1.2, k=V, seed=4, c1=5.0)    # exact mode
 
 
-def test_large_magnitude_logits_stay_inside_the_stated_bound(ctx):
-    """The exponent z log2(e) is formed with the fp32 constant log2(e), which is 1.9e-8 too large: a row
-    whose mass sits at logits of magnitude M gets a log-sum-exp that is off by about 1.34e-8 M (inside the
-    1e-6 bar up to M ~ 70).  Beyond that the error must stay within that bound, and the top-k lists exact."""
+def test_large_magnitude_logits(ctx):
+    """The exponent z log2(e) is formed with the fp32 constant log2(e), which is short by a factor
+    1 - 1.335e-8; the kernel scales the finished log-sum-exp back, which leaves an error below
+    1.335e-8 x (entropy of the row) < 2e-7.  So rows whose mass sits at logits of magnitude 100 to
+    1500 must still give log-probs inside the usual bar (the log-sum-exp itself is published in
+    fp32: half an ulp of its own magnitude), and exact top-k lists."""
     V, k = 20000, 8
     g = torch.Generator().manual_seed(10)
     rows = torch.randn((4, V), generator=g)
@@ -417,12 +419,13 @@ def test_large_magnitude_logits_stay_inside_the_stated_bound(ctx):
     tok = torch.tensor([1, 2, 3, 4], dtype=torch.int32, device="cuda")
     out = runner.forward(ctx, za, zp, tok, None, lam=1.0, k=k, seed=1)
     ref = oracle.forward(to_numpy_bits(za), to_numpy_bits(zp), tok.cpu().numpy(), None, lam=1.0, k=k, seed=1)
-    bound = 2e-8 * np.abs(offs.numpy()) + 1e-6 + 1e-7 * np.abs(ref["lse_a"])     # + one fp32 rounding of the result
-    assert np.all(np.abs(out["lse_actor"].cpu().numpy() - ref["lse_a"]) <= bound)
-    assert np.all(np.abs(out["lse_policy"].cpu().numpy() - ref["lse_p"]) <= bound)
-    assert np.all(np.abs(out["logp_actor"].cpu().numpy() - ref["lq64"]) <= bound)
+    close(out["logp_actor"].cpu().numpy(), ref["lq64"])
+    close(out["logp_policy"].cpu().numpy(), ref["lp64"])
+    assert np.all(np.abs(out["lse_actor"].cpu().numpy() - ref["lse_a"]) <= 1e-6 + 6e-8 * np.abs(ref["lse_a"]))
+    assert np.all(np.abs(out["lse_policy"].cpu().numpy() - ref["lse_p"]) <= 1e-6 + 6e-8 * np.abs(ref["lse_p"]))
     assert np.array_equal(out["topk_idx_actor"].cpu().numpy(), ref["topk_idx_a"])
     assert np.array_equal(out["topk_idx_policy"].cpu().numpy(), ref["topk_idx_p"])
+    close(out["z_approx"].cpu().numpy(), ref["zk"])
 
 
 def test_nonfinite_rows_are_counted_and_do_not_disturb_the_others(ctx):
