@@ -31,7 +31,6 @@ struct jp_ctx {
   int32_t rec_dtype = 0;
   bool batch_open = false;
   bool batch_exact = false;
-  int64_t batch_rng_base = 0;   // Philox counter of record row 0 in a chunked batch
   int64_t launches = 0;
   bool timing = false;
   static constexpr int kEvRing = 256;
@@ -377,7 +376,6 @@ jp_status jp_batch_begin(jp_ctx* c, int64_t T_total, int64_t V, int32_t dtype, i
   c->launches += 2;
   c->batch_open = true;
   c->batch_exact = exact;
-  c->batch_rng_base = 0;
   c->have_records = false;
   c->rec_rows = T_total; c->rec_V = V; c->rec_k = k_eff; c->rec_dtype = dtype;
   return JP_OK;
@@ -412,7 +410,7 @@ jp_status jp_batch_finalize(jp_ctx* c, const jp_obrs_desc* dout, float lambda_or
   cudaSetDevice(c->device);
   float c1 = dout ? dout->c1 : 0.f;
   // record row 0 of this batch may sit at a global row index of its own (one shard of a larger batch)
-  const int64_t rng_base = c->batch_rng_base + (dout ? dout->token_offset : 0);
+  const int64_t rng_base = dout ? dout->token_offset : 0;
   EpilogueArgs ea = epilogue_args(c, dout, c->rec_rows, c->rec_k, seed, rng_base, c1, out_accept, out_weight,
                                   out_lq, out_lp, out_stats);
   ea.aux_zx = nullptr;
@@ -586,7 +584,6 @@ jp_status jp_obrs_forward_host(jp_ctx* c, const jp_obrs_desc* d, const void* za,
 
   st = jp_batch_begin(c, d->T, d->V, d->dtype, k, exact ? lambda_or_budget : 0.f);
   if (st != JP_OK) return st;
-  c->batch_rng_base = d->token_offset;
   // order the copy stream after whatever the compute stream did before
   cudaEventRecord(c->compute_done[0], c->stream);
   cudaEventRecord(c->compute_done[1], c->stream);

@@ -447,3 +447,31 @@ def test_nonfinite_rows_are_counted_and_do_not_disturb_the_others(ctx):
     for n in ("logp_actor", "logp_policy", "lse_actor", "lse_policy", "z_approx", "accept_prob", "uniform",
               "topk_idx_actor", "topk_idx_policy"):
         assert torch.equal(out[n][good], clean[n][good]), n
+
+
+def test_host_buffer_entry_point_equals_the_device_path(ctx):
+    """jp_obrs_forward_host stages host rows through device slots chunk by chunk: with a mask, a
+    global row offset, several (uneven) chunks, pinned and pageable memory, fixed lambda and a
+    budget, it must return the bits of the device-resident call."""
+    T, V, k = 700, 12008, 16
+    r = LogitRecipe(T=T, V=V, dtype="bf16", sigma0=2.5, peaks=4, sigma=1.1, seed=64)
+    za, zp, tok = make_logits(r, "cuda")
+    mask = (torch.arange(T, device="cuda") % 9 != 4).to(torch.uint8)
+    for kw, lam_or_budget, mode in ((dict(lam=1.4), 1.4, B.JP_LAMBDA_FIXED), (dict(budget=0.55), 0.55, B.JP_LAMBDA_FROM_BUDGET)):
+        dev = runner.forward(ctx, za, zp, tok, mask, k=k, seed=6, c1=2.0, token_offset=1000, **kw)
+        for pinned in (True, False):
+            def host(t):
+                t = t.cpu()
+                return t.pin_memory() if pinned else t
+            hza, hzp, htok, hmask = host(za), host(zp), host(tok), host(mask)
+            hacc = host(torch.empty(T, dtype=torch.uint8))
+            hw, hlq, hlp = (host(torch.empty(T, dtype=torch.float32)) for _ in range(3))
+            hst = host(torch.zeros(B.STATS_BYTES, dtype=torch.uint8))
+            d = B.make_desc(hza, lambda_mode=mode, c1=2.0, token_offset=1000)
+            B.jp_obrs_forward_host(ctx, d, hza, hzp, htok, hmask, lam_or_budget, k, 6, hacc, hw, hlq, hlp, hst, 300)
+            assert torch.equal(hacc, dev["accept"].cpu())
+            assert torch.equal(hw, dev["weight"].cpu())
+            assert torch.equal(hlq, dev["logp_actor"].cpu()) and torch.equal(hlp, dev["logp_policy"].cpu())
+            st = B.read_stats(hst)
+            assert st["n_accept"] == dev["stats"]["n_accept"] and st["kappa"] == dev["stats"]["kappa"]
+            assert st["lambda_used"] == dev["stats"]["lambda_used"]
