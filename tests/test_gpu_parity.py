@@ -475,3 +475,52 @@ def test_host_buffer_entry_point_equals_the_device_path(ctx):
             st = B.read_stats(hst)
             assert st["n_accept"] == dev["stats"]["n_accept"] and st["kappa"] == dev["stats"]["kappa"]
             assert st["lambda_used"] == dev["stats"]["lambda_used"]
+
+
+def test_one_context_through_changing_shapes_equals_fresh_contexts(ctx):
+    """A context re-lays its workspace out as shapes, dtypes and k change from call to call; nothing
+    of an earlier call may leak into a later one."""
+    cases = [("bf16", 300, 20000, 64), ("f32", 200, 4099 + 5, 8), ("bf16", 310, 151936, 128), ("bf16", 300, 20000, 20000),
+             ("bf16", 64, 512, 4), ("bf16", 300, 20000, 64)]
+    names = ("accept", "weight", "logp_actor", "logp_policy", "z_approx", "topk_idx_actor", "topk_idx_policy")
+    for i, (dt, T, V, k) in enumerate(cases):
+        r = LogitRecipe(T=T, V=V, dtype=dt, sigma0=2.5, peaks=4, sigma=1.0, seed=70 + i)
+        za, zp, tok = make_logits(r, "cuda")
+        mask = (torch.arange(T, device="cuda") % 5 != 1).to(torch.uint8)
+        a = runner.forward(ctx, za, zp, tok, mask, lam=1.3, k=k, seed=i)
+        fresh = B.Context(0)
+        b = runner.forward(fresh, za, zp, tok, mask, lam=1.3, k=k, seed=i)
+        for n in names:
+            if k >= V and n.startswith("topk"):
+                continue
+            assert torch.equal(a[n], b[n]), (i, n)
+        assert a["stats"] == b["stats"], i
+        fresh.close()
+
+
+def test_forward_on_a_side_stream():
+    """The context enqueues on the stream it was given; results equal those of the default stream."""
+    r = LogitRecipe(T=200, V=30000, dtype="bf16", sigma0=2.5, peaks=4, sigma=1.0, seed=80)
+    za, zp, tok = make_logits(r, "cuda")
+    c0 = B.Context(0)
+    ref = runner.forward(c0, za, zp, tok, None, lam=1.2, k=16, seed=3)
+    c0.close()
+    side = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(side):
+        c1 = B.Context(0)                       # binds torch's current stream: the side stream
+        out = runner.forward(c1, za, zp, tok, None, lam=1.2, k=16, seed=3)
+        side.synchronize()
+        c1.close()
+    for n in ("accept", "weight", "logp_actor", "topk_idx_policy"):
+        assert torch.equal(out[n], ref[n]), n
+
+
+def test_stream_probe_reports_a_plausible_rate():
+    x = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    y = torch.empty_like(x)
+    rd = B.jp_probe_stream(x, None, reps=5)
+    cp = B.jp_probe_stream(x, y, reps=5)
+    assert 1000.0 < rd < 12000.0 and 1000.0 < cp < 12000.0
+    with pytest.raises(B.JackpotError):
+        B.jp_probe_stream(x[1:], None, reps=1)          # not 16-byte aligned
