@@ -35,36 +35,45 @@ def close(a, b, rtol=RTOL, atol=ATOL):
     assert not bad.any(), f"{bad.sum()} of {bad.size} differ; worst {np.abs(a - b).max():.3e}"
 
 
+def check_block(out, b0, za_b, zp_b, tok_b, mask_b, lam, k, seed):
+    """Oracle on one block of consecutive rows that starts at global row b0; the accept draw of
+    row t is keyed on its global index, which the oracle gets through token_offset."""
+    n = za_b.shape[0]
+    sl = slice(b0, b0 + n)
+    m = None if mask_b is None else mask_b.cpu().numpy()
+    ref = oracle.forward(to_numpy_bits(za_b), to_numpy_bits(zp_b), tok_b.cpu().numpy(), m, lam=lam, k=k,
+                         seed=seed, token_offset=b0)
+    valid = np.ones(n, bool) if m is None else m != 0
+    g = {n_: out[n_][sl].cpu().numpy() for n_ in ("logp_actor", "logp_policy", "lse_actor", "lse_policy",
+                                                  "accept_prob", "uniform", "z_approx", "accept", "weight",
+                                                  "topk_idx_actor", "topk_idx_policy")}
+    close(g["logp_actor"], ref["lq64"])
+    close(g["logp_policy"], ref["lp64"])
+    close(g["lse_actor"][valid], ref["lse_a"][valid])
+    close(g["lse_policy"][valid], ref["lse_p"][valid])
+    assert np.array_equal(g["topk_idx_actor"][valid], ref["topk_idx_a"][valid])
+    assert np.array_equal(g["topk_idx_policy"][valid], ref["topk_idx_p"][valid])
+    assert np.array_equal(g["uniform"], ref["u"])
+    close(g["accept_prob"], ref["a"])
+    close(g["z_approx"], ref["zk"])
+    diff = g["accept"] != ref["accept"]
+    near = np.abs(ref["u"].astype(np.float64) - ref["a"].astype(np.float64)) < 1e-6
+    assert not (diff & ~near).any()
+    # weight = min(kappa * Z_approx * max(lambda, p/q), c1) with the batch's kappa
+    d = (ref["lp"] - ref["lq"]).astype(np.float64)
+    w_ref = out["stats"]["kappa"] * ref["zk"] * np.maximum(lam, np.exp(d))
+    c1 = out.get("c1", 0.0)
+    if c1 > 0:
+        w_ref = np.minimum(w_ref, c1)
+    close(g["weight"][valid], w_ref[valid])
+    return int(diff.sum())
+
+
 def check_blocks(out, za, zp, tok, mask, lam, k, seed, blocks, block_rows=8):
-    """Oracle on blocks of consecutive rows; the accept draw of row t is keyed on
-    its global index, which the oracle gets through token_offset."""
     flips = 0
     for b0 in blocks:
         sl = slice(b0, b0 + block_rows)
-        m = None if mask is None else mask[sl].cpu().numpy()
-        ref = oracle.forward(to_numpy_bits(za[sl]), to_numpy_bits(zp[sl]), tok[sl].cpu().numpy(), m, lam=lam, k=k,
-                             seed=seed, token_offset=b0)
-        valid = np.ones(block_rows, bool) if m is None else m != 0
-        g = {n: out[n][sl].cpu().numpy() for n in ("logp_actor", "logp_policy", "lse_actor", "lse_policy",
-                                                   "accept_prob", "uniform", "z_approx", "accept", "weight",
-                                                   "topk_idx_actor", "topk_idx_policy")}
-        close(g["logp_actor"], ref["lq64"])
-        close(g["logp_policy"], ref["lp64"])
-        close(g["lse_actor"][valid], ref["lse_a"][valid])
-        close(g["lse_policy"][valid], ref["lse_p"][valid])
-        assert np.array_equal(g["topk_idx_actor"][valid], ref["topk_idx_a"][valid])
-        assert np.array_equal(g["topk_idx_policy"][valid], ref["topk_idx_p"][valid])
-        assert np.array_equal(g["uniform"], ref["u"])
-        close(g["accept_prob"], ref["a"])
-        close(g["z_approx"], ref["zk"])
-        diff = g["accept"] != ref["accept"]
-        near = np.abs(ref["u"].astype(np.float64) - ref["a"].astype(np.float64)) < 1e-6
-        assert not (diff & ~near).any()
-        flips += int(diff.sum())
-        # weight = kappa * Z_approx * max(lambda, p/q) with the batch's kappa
-        d = (ref["lp"] - ref["lq"]).astype(np.float64)
-        w_ref = out["stats"]["kappa"] * ref["zk"] * np.maximum(lam, np.exp(d))
-        close(g["weight"][valid], w_ref[valid])
+        flips += check_block(out, b0, za[sl], zp[sl], tok[sl], None if mask is None else mask[sl], lam, k, seed)
     return flips
 
 
@@ -154,3 +163,85 @@ def test_sweep_shape_top_k_against_exact(ctx, k):
     close(zx[sl], ref["z_exact"])
     close(zk[sl], ref["zk"])
     assert np.array_equal(out["topk_idx_actor"][sl].cpu().numpy(), ref["topk_idx_a"])
+
+
+def _recipe(r0, T, seed):
+    return LogitRecipe(T=T, V=r0.V, dtype=r0.dtype, sigma0=r0.sigma0, peaks=r0.peaks, peak_lo=r0.peak_lo,
+                       peak_hi=r0.peak_hi, sigma=r0.sigma, seed=seed)
+
+
+def test_padded_batch_all_rows_streamed(ctx):
+    """The padded-batch shape at its full 131,072 rows: chunks are made, handed to the library and
+    dropped one after the other (the whole batch is 80 GB of logits); blocks of rows kept from every
+    fourth chunk, among them rows on both sides of a response's end, go through the oracle."""
+    cfg = CONFIGS["cfg3_batch"]
+    r0, chunk = cfg["recipe"], cfg["chunk"]
+    T, V, k = r0.T, r0.V, cfg["k"]
+    mask, lengths = make_lengths_mask(cfg["n_resp"], cfg["max_len"], cfg["min_len"], seed=cfg["seed"], device="cuda")
+    ends = (torch.arange(cfg["n_resp"]) * cfg["max_len"] + lengths.cpu()).tolist()
+    kept = {}
+
+    def chunks():
+        for c, off in enumerate(range(0, T, chunk)):
+            za, zp, tok = make_logits(_recipe(r0, chunk, r0.seed + 17 * c), "cuda")
+            if c % 4 == 0:
+                starts = [off, off + chunk - 8]
+                starts += [min(int(e) - 4, off + chunk - 8) for e in ends if off + 8 <= e < off + chunk][:1]
+                for b0 in starts:
+                    sl = slice(b0 - off, b0 - off + 8)
+                    kept[b0] = (za[sl].clone(), zp[sl].clone(), tok[sl].clone())
+            yield off, za, zp, tok, mask[off:off + chunk]
+            torch.cuda.synchronize()          # the chunk's memory goes back to the pool only after its pass
+
+    out = runner.forward_chunked(ctx, chunks(), T, V, B.JP_BF16, budget=cfg["budget"], k=k, seed=cfg["seed"], aux=True)
+    batch_properties(out, mask)
+    st = out["stats"]
+    assert st["n_valid"] == int(lengths.sum().item())
+    assert abs(st["mean_accept_prob"] - cfg["budget"]) < 5e-6
+    assert abs(st["alpha_hat"] - cfg["budget"]) < 4 * np.sqrt(0.25 / st["n_valid"])
+    lam_ref = oracle.lambda_from_budget(out["logp_actor"].cpu().numpy(), out["logp_policy"].cpu().numpy(),
+                                        cfg["budget"], mask.cpu().numpy())
+    close(st["lambda_used"], np.float32(lam_ref))
+    lam = float(np.float32(st["lambda_used"]))
+    assert len(kept) >= 8
+    for b0, (za_b, zp_b, tok_b) in kept.items():
+        check_block(out, b0, za_b, zp_b, tok_b, mask[b0:b0 + 8], lam, k, cfg["seed"])
+
+
+def test_training_shape_all_rows_forward_and_backward(ctx):
+    """The training-step shape at its full 32,768 rows: chunked forward with a budget and a weight
+    clip, then one fused backward per chunk; sampled rows of the forward and of both gradients go
+    through the oracle."""
+    from test_gpu_backward import check_grads
+    cfg = CONFIGS["cfg5_train"]
+    r0, chunk, k = cfg["recipe"], cfg["chunk"], cfg["k"]
+    T, V = r0.T, r0.V
+    parts = [make_logits(_recipe(r0, chunk, r0.seed + 31 * c), "cuda") for c in range(T // chunk)]
+    out = runner.forward_chunked(ctx, [(c * chunk, za, zp, tok, None) for c, (za, zp, tok) in enumerate(parts)], T, V,
+                                 B.JP_BF16, budget=cfg["budget"], k=k, seed=cfg["seed"], c1=cfg["c1"], aux=True)
+    out["c1"] = cfg["c1"]
+    batch_properties(out, None)
+    st = out["stats"]
+    assert abs(st["mean_accept_prob"] - cfg["budget"]) < 5e-6
+    lam = float(np.float32(st["lambda_used"]))
+    assert np.all(out["weight"].cpu().numpy() <= np.float32(cfg["c1"]))
+    g = torch.Generator(device="cpu").manual_seed(cfg["seed"])
+    adv = torch.randn(T, generator=g).cuda()
+    for c, (za, zp, tok) in enumerate(parts):
+        off = c * chunk
+        for b0 in (off, off + chunk // 2 + 3, off + chunk - 8):
+            sl = slice(b0 - off, b0 - off + 8)
+            check_block(out, b0, za[sl], zp[sl], tok[sl], None, lam, k, cfg["seed"])
+    da, dp = torch.empty_like(parts[0][0]), torch.empty_like(parts[0][1])      # one chunk's gradients at a time
+    for c, (za, zp, tok) in enumerate(parts):
+        sl = slice(c * chunk, (c + 1) * chunk)
+        runner.backward(ctx, za, zp, tok, None, out["accept"][sl], out["weight"][sl], advantages=adv[sl],
+                        lambda_distill=cfg["lambda_distill"], record_offset=c * chunk, d_actor=da, d_policy=dp)
+        torch.cuda.synchronize()
+        rows = np.array([0, 1, chunk // 3, chunk - 1])
+        sub = torch.from_numpy(rows).cuda()
+        za_s, zp_s, tok_s = to_numpy_bits(za[sub]), to_numpy_bits(zp[sub]), tok[sub].cpu().numpy()
+        lg = oracle.lse_gather(za_s, zp_s, tok_s)
+        check_grads(da[sub], dp[sub], np.arange(len(rows)), za_s, zp_s, tok_s, None, out["accept"][sl][sub].cpu().numpy(),
+                    out["weight"][sl][sub].cpu().numpy(), lg["lse_a"], lg["lse_p"], st["n_valid"],
+                    adv[sl][sub].cpu().numpy(), cfg["lambda_distill"])
