@@ -225,6 +225,41 @@ jp_status jp_batch_logprobs(jp_ctx* ctx, float* out_logp_actor, float* out_logp_
  * (c1 <= 0: no clip).  JP_ERR_STATE without records. */
 jp_status jp_obrs_apply_kappa(jp_ctx* ctx, double kappa, float c1, float* out_weight);
 
+/* Vocabulary-parallel forward (Section 4.4 names the [tokens, vocabulary] logits as the
+ * memory bottleneck; here every device holds a slice of the vocabulary's columns of both
+ * tensors, as a vocabulary-parallel output layer leaves them).  Three steps per device:
+ *
+ *   jp_vshard_local   streams this device's columns once (the same row kernel as
+ *                     jp_obrs_forward) and packs, per row, the slice's log-sum-exp of both
+ *                     tensors, the sampled token's two logits if the slice holds it, and the
+ *                     slice's two top-k lists with both logits of every entry, into
+ *                     out_packed [T, jp_vshard_record_floats(k)] (device, 4-byte words);
+ *   (the caller gathers every shard's out_packed into gathered [n_shards, T, words], shard
+ *    order = ascending vocab_offset: an all-gather over the devices)
+ *   jp_vshard_merge   turns the gathered lines into the records of the whole vocabulary:
+ *                     lse = log sum_s exp(lse_s); log-probs of the sampled token from its
+ *                     owner's logits; each top-k list = the k best of the shards' k best
+ *                     under the same order (higher logit first, ties by lower index);
+ *   jp_batch_finalize then completes the forward from the records exactly as for a chunked
+ *                     batch: lambda (fixed or from a budget), acceptance (Eq. obrs_accept),
+ *                     the accept draws, Z_approx (Eq. z_approx), kappa and the weights.
+ *                     Every device ends with the same outputs for all T rows.
+ *
+ * desc describes the slice: T rows, V = the slice's width (> k), ld, dtype.  tokens are ids in
+ * [0, V_total) (others make the row invalid and are counted in n_bad_token); vocab_offset is
+ * the slice's first column.  The slices of the shards must tile [0, V_total) without overlap.
+ * 1 <= k <= JP_MAX_TOPK (no exact mode: JP_ERR_UNSUPPORTED); n_shards * k <= 2048
+ * (JP_ERR_TOO_LARGE).  A row is valid if every shard found it valid.  All pointers device
+ * memory owned by the caller; the calls enqueue on the context's stream and return.  The
+ * context's records afterwards describe the whole vocabulary, so jp_obrs_backward (which
+ * takes the logits of the whole row) does not apply to a slice. */
+size_t jp_vshard_record_floats(int k);
+jp_status jp_vshard_local(jp_ctx* ctx, const jp_obrs_desc* desc, const void* actor_logits,
+                          const void* policy_logits, const int32_t* tokens, const uint8_t* mask,
+                          int64_t vocab_offset, int64_t V_total, int k, float* out_packed);
+jp_status jp_vshard_merge(jp_ctx* ctx, int n_shards, int my_shard, const float* gathered, int64_t T,
+                          int64_t V_total, int k);
+
 /* Theorem 3.4 for single distributions: for every row t the lambda_t at which the
  * OBRS rule accepts exactly `budget` of the proposal's mass,
  *   sum_v min(q_t(v), p_t(v) / lambda_t) = budget,   q_t, p_t = softmax of the rows,

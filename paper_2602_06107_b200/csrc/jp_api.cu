@@ -22,6 +22,8 @@ struct jp_ctx {
   Scalars* sc = nullptr;
   int32_t* list = nullptr;
   uint32_t* spill = nullptr;
+  int32_t* vtok = nullptr;       // a vocabulary shard's view of the call: local token ids ...
+  uint8_t* vmask = nullptr;      // ... and row validity (2 = this shard holds the sampled token)
   Partials* part = nullptr;
   // state of the records
   bool have_records = false;
@@ -31,6 +33,9 @@ struct jp_ctx {
   int32_t rec_dtype = 0;
   bool batch_open = false;
   bool batch_exact = false;
+  bool vshard_local_done = false;   // jp_vshard_local has run: jp_vshard_merge may follow
+  int64_t vshard_T = 0;
+  int vshard_k = 0;
   int64_t launches = 0;
   bool timing = false;
   static constexpr int kEvRing = 256;
@@ -49,7 +54,7 @@ namespace {
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
-  size_t scalars, partials, idx, za, zp, f[7], flag, ratio, dval, list, spill, total;
+  size_t scalars, partials, idx, za, zp, f[9], flag, ratio, dval, list, spill, vtok, vmask, total;
 };
 
 Layout layout_for(int64_t rows, int k) {
@@ -62,12 +67,14 @@ Layout layout_for(int64_t rows, int k) {
   L.idx = take(cand * 4);
   L.za = take(cand * 4);
   L.zp = take(cand * 4);
-  for (int i = 0; i < 7; ++i) L.f[i] = take((size_t)rows * 4);
+  for (int i = 0; i < 9; ++i) L.f[i] = take((size_t)rows * 4);
   L.flag = take((size_t)rows);
   L.ratio = take((size_t)rows * 8);
   L.dval = take((size_t)rows * 4);
   L.list = take((size_t)rows * 4);
   L.spill = take(kSpillBytes);
+  L.vtok = take((size_t)rows * 4);
+  L.vmask = take((size_t)rows);
   L.total = off;
   return L;
 }
@@ -119,11 +126,15 @@ jp_status ensure_workspace(jp_ctx* c, int64_t rows, int k) {
   c->rec.zk = (float*)(b + L.f[4]);
   c->rec.zx = (float*)(b + L.f[5]);
   c->rec.a = (float*)(b + L.f[6]);
+  c->rec.lse_a_lo = (float*)(b + L.f[7]);
+  c->rec.lse_p_lo = (float*)(b + L.f[8]);
   c->rec.flag = (uint8_t*)(b + L.flag);
   c->rec.ratio = (double*)(b + L.ratio);
   c->rec.dval = (float*)(b + L.dval);
   c->list = (int32_t*)(b + L.list);
   c->spill = (uint32_t*)(b + L.spill);
+  c->vtok = (int32_t*)(b + L.vtok);
+  c->vmask = (uint8_t*)(b + L.vmask);
   return JP_OK;
 }
 
@@ -428,6 +439,66 @@ jp_status jp_batch_finalize(jp_ctx* c, const jp_obrs_desc* dout, float lambda_or
   if (e != cudaSuccess) return cuda_fail(c, e, "epilogue launch");
   c->batch_open = false;
   c->have_records = true;
+  return JP_OK;
+}
+
+size_t jp_vshard_record_floats(int k) { return k < 1 ? 0 : (size_t)vshard_words(k); }
+
+jp_status jp_vshard_local(jp_ctx* c, const jp_obrs_desc* d, const void* za, const void* zp, const int32_t* tokens,
+                          const uint8_t* mask, int64_t vocab_offset, int64_t V_total, int k, float* out_packed) {
+  if (!c) return JP_ERR_INVALID_ARG;
+  int64_t ld = 0;
+  jp_status st = check_shape(c, d, &ld);
+  if (st != JP_OK) return st;
+  if (c->batch_open) return fail(c, JP_ERR_STATE, "a chunked batch is open: finalize it first");
+  if (k < 1 || k > JP_MAX_TOPK) return fail(c, JP_ERR_UNSUPPORTED, "vocabulary shards support 1 <= k <= JP_MAX_TOPK (no exact mode)");
+  if ((int64_t)k >= d->V) return fail(c, JP_ERR_UNSUPPORTED, "a vocabulary shard must be wider than k columns");
+  if (vocab_offset < 0 || vocab_offset + d->V > V_total || V_total > (int64_t)0x7fffffff)
+    return fail(c, JP_ERR_INVALID_ARG, "shard columns fall outside [0, V_total)");
+  if (d->T > 0 && !out_packed) return fail(c, JP_ERR_INVALID_ARG, "out_packed is NULL");
+  cudaSetDevice(c->device);
+  if ((st = ensure_workspace(c, d->T > 0 ? d->T : 1, k)) != JP_OK) return st;
+  cudaError_t e = launch_reset(c->sc, 1.0f, c->stream);
+  if (e != cudaSuccess) return cuda_fail(c, e, "reset launch");
+  c->launches += 1;
+  c->have_records = false;
+  c->vshard_local_done = false;
+  if (d->T > 0) {
+    if (!tokens) return fail(c, JP_ERR_INVALID_ARG, "tokens pointer is NULL");
+    e = launch_vshard_localize(d->T, tokens, mask, vocab_offset, d->V, V_total, c->vtok, c->vmask, c->sc, c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e, "shard token launch");
+    c->launches += 1;
+    if ((st = stream_rows(c, d, ld, k, 0, za, zp, c->vtok, c->vmask, false, false)) != JP_OK) return st;
+    e = launch_vshard_export(d->T, k, c->rec, za, zp, ld, d->dtype, c->vtok, c->vmask, vocab_offset, out_packed,
+                             c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e, "shard export launch");
+    c->launches += 1;
+  }
+  c->vshard_local_done = true;
+  c->vshard_T = d->T;
+  c->vshard_k = k;
+  c->rec_dtype = d->dtype;
+  return JP_OK;
+}
+
+jp_status jp_vshard_merge(jp_ctx* c, int n_shards, int my_shard, const float* gathered, int64_t T, int64_t V_total,
+                          int k) {
+  if (!c) return JP_ERR_INVALID_ARG;
+  if (!c->vshard_local_done) return fail(c, JP_ERR_STATE, "jp_vshard_merge without jp_vshard_local");
+  if (T != c->vshard_T || k != c->vshard_k) return fail(c, JP_ERR_INVALID_ARG, "T / k differ from jp_vshard_local");
+  if (n_shards < 1 || my_shard < 0 || my_shard >= n_shards) return fail(c, JP_ERR_INVALID_ARG, "shard index out of range");
+  if ((int64_t)n_shards * k > kVshardMaxEntries)
+    return fail(c, JP_ERR_TOO_LARGE, "n_shards * k beyond the merge kernel's 2048 entries per list");
+  if (T > 0 && !gathered) return fail(c, JP_ERR_INVALID_ARG, "gathered is NULL");
+  cudaSetDevice(c->device);
+  cudaError_t e = launch_vshard_merge(n_shards, my_shard, gathered, T, k, c->rec, c->sc, c->stream);
+  if (e != cudaSuccess) return cuda_fail(c, e, "shard merge launch");
+  if (T > 0) c->launches += 1;
+  // the records now describe the whole vocabulary: jp_batch_finalize completes the forward
+  c->vshard_local_done = false;
+  c->batch_open = true;
+  c->batch_exact = false;
+  c->rec_rows = T; c->rec_V = V_total; c->rec_k = k;
   return JP_OK;
 }
 

@@ -15,6 +15,8 @@ struct Records {
   float* zp;        // [cap, 2k]  policy logit of every candidate
   float* lse_a;     // [cap]
   float* lse_p;     // [cap]
+  float* lse_a_lo;  // [cap] what fp32 rounding took from the log-sum-exp (lse = lse_a + lse_a_lo to ~2^-48)
+  float* lse_p_lo;  // [cap]
   float* lq;        // [cap] log p_inf(a_t)
   float* lp;        // [cap] log p_target(a_t)
   float* zk;        // [cap] Z_approx (or exact Z when k >= V)
@@ -154,6 +156,22 @@ cudaError_t launch_reweight(int64_t T, const Records& rec, const Scalars* sc, do
 cudaError_t launch_logprobs(int64_t T, const Records& rec, float* out_lq, float* out_lp, uint8_t* out_valid,
                             cudaStream_t s);
 cudaError_t launch_row_lambda(const RowLambdaArgs& a, cudaStream_t s, int sms);
+
+// Vocabulary shards (jp_vshard.cu).  Packed per-row record of one shard, in 4-byte words:
+// [0] flag  [1] owner of the sampled token  [2,3] lse actor (hi, lo)  [4,5] lse policy (hi, lo)
+// [6,7] the sampled token's two logits (owner only)  [8, 8+2k) global indices of the two lists
+// [8+2k, 8+4k) actor logits of the entries  [8+4k, 8+6k) policy logits of the entries.
+constexpr int kVshardHeader = 8;
+constexpr int kVshardMaxEntries = 2048;   // n_shards * k the merge kernel ranks in shared memory
+__host__ __device__ inline int64_t vshard_words(int k) { return kVshardHeader + 6 * (int64_t)k; }
+cudaError_t launch_vshard_localize(int64_t T, const int32_t* tokens, const uint8_t* mask, int64_t vocab_offset,
+                                   int64_t V_shard, int64_t V_total, int32_t* tok_local, uint8_t* mask_local,
+                                   Scalars* sc, cudaStream_t s);
+cudaError_t launch_vshard_export(int64_t T, int k, const Records& rec, const void* za, const void* zp, int64_t ld,
+                                 int32_t dtype, const int32_t* tok_local, const uint8_t* mask_local,
+                                 int64_t vocab_offset, float* out, cudaStream_t s);
+cudaError_t launch_vshard_merge(int n_shards, int my_shard, const float* gathered, int64_t T, int k,
+                                const Records& rec, Scalars* sc, cudaStream_t s);
 cudaError_t launch_grad(const GradArgs& a, cudaStream_t s, int sms, int* n_launch);
 
 }  // namespace jp

@@ -1142,8 +1142,9 @@ __device__ void topk_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int t, in
       const double lse = (((double)M + (double)(e - 1)) * 0.6931471805599453 + (double)logf(f)) * (1.0 + 1.33497582e-8);
       const float lsef = (float)lse;
       const float lpx = (float)((double)zx - lse);
-      if (t == 0) { A.rec.lse_a[rrow] = lsef; A.rec.lq[rrow] = lpx; A.rec.flag[rrow] = 1; }
-      else        { A.rec.lse_p[rrow] = lsef; A.rec.lp[rrow] = lpx; }
+      const float lo = (float)(lse - (double)lsef);
+      if (t == 0) { A.rec.lse_a[rrow] = lsef; A.rec.lse_a_lo[rrow] = lo; A.rec.lq[rrow] = lpx; A.rec.flag[rrow] = 1; }
+      else        { A.rec.lse_p[rrow] = lsef; A.rec.lse_p_lo[rrow] = lo; A.rec.lp[rrow] = lpx; }
       if (!isfinite(lsef)) atomicAdd(&A.sc->n_nonfinite, 1ull);
     }
     __syncwarp();
@@ -1201,6 +1202,7 @@ __global__ void __launch_bounds__(256) prep_rows_kernel(StreamArgs A) {
       const int64_t rrow = A.record_offset + row;
       A.rec.flag[rrow] = 0;
       A.rec.lse_a[rrow] = 0.f; A.rec.lse_p[rrow] = 0.f;
+      A.rec.lse_a_lo[rrow] = 0.f; A.rec.lse_p_lo[rrow] = 0.f;
       A.rec.lq[rrow] = 0.f; A.rec.lp[rrow] = 0.f;
     }
   }

@@ -1,0 +1,191 @@
+// Vocabulary-parallel form of the forward pass (Section 4.4: the full-vocabulary pass over
+// [tokens, vocabulary] logits is the memory bottleneck; here every device holds a slice of
+// the vocabulary's columns).  A shard streams its columns once with the ordinary row
+// kernel, which leaves per row the log-sum-exp of the slice and the slice's two top-k lists
+// with both logits of every entry.  Those records are packed, exchanged between the shards
+// by the caller, and merged here into the records of the whole vocabulary:
+//   lse        = log sum_s exp(lse_s)                       (both tensors)
+//   log-probs  = the owner shard's logits of the sampled token minus lse
+//   top-k(p)   = the k best of the union of the shards' k best (the k best of the whole
+//                vocabulary lie in it), same total order: higher logit first, equal
+//                logits by lower index
+// after which acceptance, Z_approx (Eq. z_approx over the union of the two lists), the
+// batch calibration and the weights run from the records exactly as on one device.
+#include "jp_common.cuh"
+#include "jp_internal.h"
+
+namespace jp {
+namespace {
+
+constexpr int VS_NT = 128;
+
+__global__ void __launch_bounds__(256) vshard_localize_kernel(int64_t T, const int32_t* tokens, const uint8_t* mask,
+                                                              int64_t vocab_offset, int64_t V_shard, int64_t V_total,
+                                                              int32_t* tok_local, uint8_t* mask_local, Scalars* sc) {
+  const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
+  if (i >= T) return;
+  bool valid = mask == nullptr || mask[i] != 0;
+  const int64_t x = tokens[i];
+  if (valid && (x < 0 || x >= V_total)) {
+    valid = false;
+    atomicAdd(&sc->n_bad_token, 1ull);
+  }
+  const int64_t loc = x - vocab_offset;
+  const bool owner = valid && loc >= 0 && loc < V_shard;
+  // a shard that does not hold the sampled token streams the row all the same (column 0
+  // stands in for the token; the log-prob it yields is never used)
+  tok_local[i] = owner ? (int32_t)loc : 0;
+  mask_local[i] = valid ? (owner ? 2 : 1) : 0;
+}
+
+// One warp per row: the shard's records of the row as one packed line.
+__global__ void __launch_bounds__(VS_NT) vshard_export_kernel(int64_t T, int k, Records rec, const void* za,
+                                                              const void* zp, int64_t ld, int32_t dtype,
+                                                              const int32_t* tok_local, const uint8_t* mask_local,
+                                                              int64_t vocab_offset, float* out) {
+  const int lane = threadIdx.x & 31;
+  const int64_t r = (int64_t)blockIdx.x * (VS_NT / 32) + (threadIdx.x >> 5);
+  if (r >= T) return;
+  float* o = out + r * vshard_words(k);
+  const bool flag = rec.flag[r] != 0;
+  if (lane == 0) {
+    const bool owner = flag && mask_local[r] == 2;
+    float xa = 0.f, xp = 0.f;
+    if (owner) {
+      const int64_t x = tok_local[r];
+      if (dtype == JP_BF16) {
+        xa = Vec<JP_BF16>::load_scalar((const char*)za + r * ld * Vec<JP_BF16>::ESIZE, x);
+        xp = Vec<JP_BF16>::load_scalar((const char*)zp + r * ld * Vec<JP_BF16>::ESIZE, x);
+      } else {
+        xa = Vec<JP_F32>::load_scalar((const char*)za + r * ld * Vec<JP_F32>::ESIZE, x);
+        xp = Vec<JP_F32>::load_scalar((const char*)zp + r * ld * Vec<JP_F32>::ESIZE, x);
+      }
+    }
+    o[0] = __int_as_float(flag ? 1 : 0);
+    o[1] = __int_as_float(owner ? 1 : 0);
+    o[2] = flag ? rec.lse_a[r] : 0.f;
+    o[3] = flag ? rec.lse_a_lo[r] : 0.f;
+    o[4] = flag ? rec.lse_p[r] : 0.f;
+    o[5] = flag ? rec.lse_p_lo[r] : 0.f;
+    o[6] = xa;
+    o[7] = xp;
+  }
+  for (int j = lane; j < 2 * k; j += 32) {
+    const int64_t e = r * (2 * k) + j;
+    const int32_t idx = flag ? rec.idx[e] : -1;
+    o[kVshardHeader + j] = __int_as_float(idx >= 0 ? (int32_t)(idx + vocab_offset) : -1);
+    o[kVshardHeader + 2 * k + j] = idx >= 0 ? rec.za[e] : 0.f;
+    o[kVshardHeader + 4 * k + j] = idx >= 0 ? rec.zp[e] : 0.f;
+  }
+}
+
+// One block per row.  Every entry of the shards' lists gets its rank among the entries of
+// its tensor by counting the keys above it (keys are distinct: the shards' columns are
+// disjoint); ranks below k are the merged list.
+__global__ void __launch_bounds__(VS_NT) vshard_merge_kernel(int n_shards, int my_shard, const float* g, int64_t T,
+                                                             int k, Records rec, Scalars* sc) {
+  extern __shared__ unsigned long long keys[];      // [2][n_shards * k]
+  const int64_t r = blockIdx.x;
+  const int tid = threadIdx.x;
+  const int n = n_shards * k;
+  const int64_t W = vshard_words(k);
+  auto line = [&](int s) { return g + ((int64_t)s * T + r) * W; };
+
+  for (int e = tid; e < 2 * n; e += VS_NT) {
+    const int t = e / n, x = e % n, s = x / k, j = x % k;
+    const float* o = line(s);
+    const int32_t idx = __float_as_int(o[kVshardHeader + t * k + j]);
+    const float v = o[kVshardHeader + (t == 0 ? 2 * k : 4 * k) + t * k + j];
+    keys[e] = idx >= 0 ? make_key(v, (uint32_t)idx) : 0ull;
+  }
+  for (int j = tid; j < 2 * k; j += VS_NT) {
+    const int64_t e = r * (2 * k) + j;
+    rec.idx[e] = -1; rec.za[e] = 0.f; rec.zp[e] = 0.f;
+  }
+  __syncthreads();
+
+  bool all = true;
+  for (int s = 0; s < n_shards; ++s) all = all && __float_as_int(line(s)[0]) != 0;
+
+  if (all) {
+    for (int e = tid; e < 2 * n; e += VS_NT) {
+      const unsigned long long key = keys[e];
+      if (key == 0ull) continue;
+      const int t = e / n, x = e % n, s = x / k, j = x % k;
+      const unsigned long long* kt = keys + t * n;
+      int above = 0;
+      for (int y = 0; y < n; ++y) above += kt[y] > key ? 1 : 0;
+      if (above < k) {
+        const float* o = line(s);
+        const int64_t dst = r * (2 * k) + (int64_t)t * k + above;
+        rec.idx[dst] = (int32_t)key_index(key);
+        rec.za[dst] = o[kVshardHeader + 2 * k + t * k + j];
+        rec.zp[dst] = o[kVshardHeader + 4 * k + t * k + j];
+      }
+    }
+  }
+
+  if (tid == 0) {
+    if (!all) {
+      rec.flag[r] = 0;
+      rec.lse_a[r] = 0.f; rec.lse_p[r] = 0.f; rec.lse_a_lo[r] = 0.f; rec.lse_p_lo[r] = 0.f;
+      rec.lq[r] = 0.f; rec.lp[r] = 0.f;
+    } else {
+      double ma = -INFINITY, mp = -INFINITY, xa = 0.0, xp = 0.0;
+      for (int s = 0; s < n_shards; ++s) {
+        const float* o = line(s);
+        ma = fmax(ma, (double)o[2] + (double)o[3]);
+        mp = fmax(mp, (double)o[4] + (double)o[5]);
+        if (__float_as_int(o[1]) != 0) { xa = (double)o[6]; xp = (double)o[7]; }
+      }
+      double sa = 0.0, sp = 0.0;
+      for (int s = 0; s < n_shards; ++s) {
+        const float* o = line(s);
+        sa += exp(((double)o[2] + (double)o[3]) - ma);
+        sp += exp(((double)o[4] + (double)o[5]) - mp);
+      }
+      const double la = ma + log(sa), lp = mp + log(sp);
+      const float laf = (float)la, lpf = (float)lp;
+      rec.lse_a[r] = laf; rec.lse_a_lo[r] = (float)(la - (double)laf);
+      rec.lse_p[r] = lpf; rec.lse_p_lo[r] = (float)(lp - (double)lpf);
+      rec.lq[r] = (float)(xa - la);
+      rec.lp[r] = (float)(xp - lp);
+      rec.flag[r] = 1;
+      // a row that only another shard found non-finite counts here as well
+      const float* mine = line(my_shard);
+      if ((!isfinite(laf) || !isfinite(lpf)) && isfinite(mine[2]) && isfinite(mine[4]))
+        atomicAdd(&sc->n_nonfinite, 1ull);
+    }
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_vshard_localize(int64_t T, const int32_t* tokens, const uint8_t* mask, int64_t vocab_offset,
+                                   int64_t V_shard, int64_t V_total, int32_t* tok_local, uint8_t* mask_local,
+                                   Scalars* sc, cudaStream_t s) {
+  if (T <= 0) return cudaSuccess;
+  vshard_localize_kernel<<<(unsigned)((T + 255) / 256), 256, 0, s>>>(T, tokens, mask, vocab_offset, V_shard, V_total,
+                                                                   tok_local, mask_local, sc);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_vshard_export(int64_t T, int k, const Records& rec, const void* za, const void* zp, int64_t ld,
+                                 int32_t dtype, const int32_t* tok_local, const uint8_t* mask_local,
+                                 int64_t vocab_offset, float* out, cudaStream_t s) {
+  if (T <= 0) return cudaSuccess;
+  const int wpb = VS_NT / 32;
+  vshard_export_kernel<<<(unsigned)((T + wpb - 1) / wpb), VS_NT, 0, s>>>(T, k, rec, za, zp, ld, dtype, tok_local,
+                                                                        mask_local, vocab_offset, out);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_vshard_merge(int n_shards, int my_shard, const float* gathered, int64_t T, int k,
+                                const Records& rec, Scalars* sc, cudaStream_t s) {
+  if (T <= 0) return cudaSuccess;
+  const size_t smem = (size_t)2 * n_shards * k * sizeof(unsigned long long);   // <= 32 KB by kVshardMaxEntries
+  vshard_merge_kernel<<<(unsigned)T, VS_NT, smem, s>>>(n_shards, my_shard, gathered, T, k, rec, sc);
+  return cudaGetLastError();
+}
+
+}  // namespace jp

@@ -95,3 +95,58 @@ def solve_on_device(logp_actor, logp_policy, valid, budget: float) -> float:
     if st != 0:
         raise B.JackpotError(f"jp_budget_lambda_static: status {st}")
     return float(out.item())
+
+
+# ---- vocabulary shards: every rank holds a slice of the vocabulary's columns of all rows ------------
+
+def shard_columns(V: int, world: int, rank: int, align: int = 8):
+    """Column range [lo, hi) of rank `rank`: balanced, every boundary but the last a multiple of
+    `align` elements (a slice of a row-major tensor must start on a 16-byte boundary: 8 bf16 / 4 fp32)."""
+    if world < 1 or not (0 <= rank < world) or V < 1 or align < 1:
+        raise ValueError("need world >= 1, 0 <= rank < world, V >= 1, align >= 1")
+    units = -(-V // align)
+    q, r = divmod(units, world)
+    lo_u = rank * q + min(rank, r)
+    hi_u = lo_u + q + (1 if rank < r else 0)
+    return min(lo_u * align, V), min(hi_u * align, V)
+
+
+def gather_shard_records(packed: torch.Tensor, group=None) -> torch.Tensor:
+    """[T, words] of every rank -> [world, T, words] in rank order (= ascending column offset)."""
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size(group) == 1:
+        return packed.unsqueeze(0).contiguous()
+    world = dist.get_world_size(group)
+    out = torch.empty((world * packed.shape[0],) + tuple(packed.shape[1:]), dtype=packed.dtype, device=packed.device)
+    dist.all_gather_into_tensor(out, packed.contiguous(), group=group)       # concatenated along the rows
+    return out.view((world,) + tuple(packed.shape))
+
+
+def forward_vocab_parallel(ctx, za, zp, tokens, mask, vocab_offset: int, V_total: int, *, lam=None, budget=None,
+                           k=20, seed=0, c1=0.0, aux=False, group=None, gather=gather_shard_records, shard_index=None):
+    """The forward over column slices: local pass, one all-gather of the packed records
+    (T x (8 + 6k) words per rank), merge, finalize.  Every rank returns the outputs of all T rows."""
+    from . import binding as B
+    from . import runner
+    assert (lam is None) != (budget is None)
+    T = za.shape[0]
+    if shard_index is None:
+        shard_index = dist.get_rank(group) if dist.is_available() and dist.is_initialized() else 0
+    packed = torch.empty((T, B.jp_vshard_record_floats(k)), dtype=torch.float32, device=za.device)
+    B.jp_vshard_local(ctx, B.make_desc(za), za, zp, tokens, mask, vocab_offset, V_total, k, packed)
+    gathered = gather(packed, group)
+    B.jp_vshard_merge(ctx, gathered.shape[0], shard_index, gathered, T, V_total, k)
+    out = runner._alloc_outputs(T, za.device)
+    d = B.jp_obrs_desc()
+    d.c1 = c1
+    auxd = {}
+    if aux:
+        auxd = runner._alloc_aux(T, k, V_total, za.device, False)
+        for n, t in auxd.items():
+            setattr(d, n, t.data_ptr())
+    mode = B.JP_LAMBDA_FIXED if budget is None else B.JP_LAMBDA_FROM_BUDGET
+    B.jp_batch_finalize(ctx, d, lam if budget is None else budget, mode, seed, out["accept"], out["weight"],
+                        out["logp_actor"], out["logp_policy"], out["stats_buf"])
+    out.update(auxd)
+    torch.cuda.synchronize()
+    out["stats"] = B.read_stats(out["stats_buf"])
+    return out

@@ -92,3 +92,58 @@ def test_two_ranks_agree_with_the_undivided_batch():
     assert np.array_equal(zk, whole["zk"])
     lam_whole = oracle.lambda_from_budget(whole["lq"], whole["lp"], 0.55, mask)
     assert got[0][8] == got[1][8] == lam_whole, "the gathered solve must equal the undivided batch's"
+
+
+def test_shard_columns_tiles_the_vocabulary_on_aligned_boundaries():
+    for V in (1, 7, 4099, 50001, 151936):
+        for world in (1, 2, 3, 8):
+            for align in (4, 8):
+                spans = [parallel.shard_columns(V, world, r, align) for r in range(world)]
+                assert spans[0][0] == 0 and spans[-1][1] == V
+                assert all(a[1] == b[0] for a, b in zip(spans, spans[1:]))
+                assert all(lo % align == 0 or lo == V for lo, _ in spans)
+                widths = [hi - lo for lo, hi in spans if hi > lo]
+                assert max(widths) - min(widths) < 2 * align or V < world * align
+    with pytest.raises(ValueError):
+        parallel.shard_columns(10, 2, 2)
+
+
+def _vocab_worker(rank, world, port, T, V, out_q):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        # every rank holds a slice of the columns; what it would publish per row is the slice's
+        # log-sum-exp (the oracle's, of the slice alone, standing in for the GPU pass of the shard)
+        r = LogitRecipe(T=T, V=V, dtype="bf16", sigma0=2.5, peaks=4, sigma=1.2, seed=10)
+        za, zp, tok = make_logits(r, "cpu", block_rows=T)
+        lo, hi = parallel.shard_columns(V, world, rank)
+        part = oracle.lse_gather(to_numpy_bits(za[:, lo:hi].contiguous()), to_numpy_bits(zp[:, lo:hi].contiguous()),
+                                 np.zeros(T, np.int32))
+        packed = torch.from_numpy(np.stack([part["lse_a"], part["lse_p"], np.full(T, float(rank))], 1))
+        gathered = parallel.gather_shard_records(packed)
+        out_q.put((rank, gathered.numpy()))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_ranks_gather_shard_records_in_column_order():
+    T, V, world = 12, 4096, 2
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_vocab_worker, args=(r, world, port, T, V, q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    res = dict(q.get(timeout=120) for _ in range(world))
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert np.array_equal(res[0], res[1]) and res[0].shape == (world, T, 3)
+    assert np.all(res[0][0, :, 2] == 0) and np.all(res[0][1, :, 2] == 1)
+    # the merge identity the device kernel uses: log sum_s exp(lse_s) is the row's log-sum-exp
+    r = LogitRecipe(T=T, V=V, dtype="bf16", sigma0=2.5, peaks=4, sigma=1.2, seed=10)
+    za, zp, tok = make_logits(r, "cpu", block_rows=T)
+    whole = oracle.lse_gather(to_numpy_bits(za), to_numpy_bits(zp), np.zeros(T, np.int32))
+    merged = np.logaddexp(res[0][0, :, 0], res[0][1, :, 0])
+    assert np.allclose(merged, whole["lse_a"], rtol=0, atol=1e-12)
