@@ -80,8 +80,8 @@ __global__ void __launch_bounds__(VS_NT) vshard_export_kernel(int64_t T, int k, 
 }
 
 // One block per row.  Every entry of the shards' lists gets its rank among the entries of
-// its tensor by counting the keys above it (keys are distinct: the shards' columns are
-// disjoint); ranks below k are the merged list.
+// its tensor by counting the keys above it in every shard's (sorted) list (keys are
+// distinct: the shards' columns are disjoint); ranks below k are the merged list.
 __global__ void __launch_bounds__(VS_NT) vshard_merge_kernel(int n_shards, int my_shard, const float* g, int64_t T,
                                                              int k, Records rec, Scalars* sc) {
   extern __shared__ unsigned long long keys[];      // [2][n_shards * k]
@@ -112,9 +112,19 @@ __global__ void __launch_bounds__(VS_NT) vshard_merge_kernel(int n_shards, int m
       const unsigned long long key = keys[e];
       if (key == 0ull) continue;
       const int t = e / n, x = e % n, s = x / k, j = x % k;
+      // every shard's list is sorted best first (empty slots, key 0, at its end): the keys above
+      // this one are a prefix of each list, found by bisection
       const unsigned long long* kt = keys + t * n;
       int above = 0;
-      for (int y = 0; y < n; ++y) above += kt[y] > key ? 1 : 0;
+      for (int s2 = 0; s2 < n_shards && above < k; ++s2) {
+        const unsigned long long* Ls = kt + s2 * k;
+        int lo = 0, hi = k;
+        while (lo < hi) {
+          const int mid = (lo + hi) >> 1;
+          if (Ls[mid] > key) lo = mid + 1; else hi = mid;
+        }
+        above += lo;
+      }
       if (above < k) {
         const float* o = line(s);
         const int64_t dst = r * (2 * k) + (int64_t)t * k + above;

@@ -12,9 +12,11 @@ outside the timed regions.  One JSON line per measurement.
 
   row_lambda  the per-distribution budget of Theorem 3.4 on the headline shape (4096 rows);
   simulation  Dirichlet pairs at growing distance: acceptance rate and divergence before / after
-              rejection (not run by default).
+              rejection (not run by default);
+  vocab_shards  the headline batch split by columns over 2, 4 and 8 shards: one shard's local pass,
+              the merge of all shards' records and the finalize, timed apart (not run by default).
 
-    python -m paper_2602_06107_b200.measure_configs [cfg3_batch] [cfg4_sweep] [cfg5_train] [row_lambda] [simulation]
+    python -m paper_2602_06107_b200.measure_configs [cfg3_batch] [cfg4_sweep] [cfg5_train] [row_lambda] [simulation] [vocab_shards]
 """
 from __future__ import annotations
 
@@ -210,6 +212,47 @@ def simulation(ctx):
               mean_lambda_for_budget_0p9=lam.mean().item())
 
 
+def vocab_shards(ctx):
+    """One rank's share of the vocabulary-parallel forward on the headline shape.  The shards run one
+    after the other here (a rank has one of them); every phase of shard 0 is timed on its own."""
+    from . import parallel
+    cfg = CONFIGS["cfg2_qwen3"]
+    za, zp, tok = make_logits(cfg["recipe"], DEV)
+    T, V = za.shape
+    k, lam = cfg["k"], cfg["lam"]
+    words = B.jp_vshard_record_floats(k)
+    for n in (2, 4, 8):
+        bounds = [parallel.shard_columns(V, n, s) for s in range(n)]
+        gathered = torch.empty((n, T, words), device=DEV)
+        for s, (lo, hi) in enumerate(bounds):
+            zs, ps = za[:, lo:hi], zp[:, lo:hi]
+            B.jp_vshard_local(ctx, B.make_desc(zs), zs, ps, tok, None, lo, V, k, gathered[s])
+        lo, hi = bounds[0]
+        zs, ps = za[:, lo:hi], zp[:, lo:hi]
+        d0 = B.make_desc(zs)
+        out = runner._alloc_outputs(T, DEV)
+        tl, tm, tf = _Timer(), _Timer(), _Timer()
+        reps = 20
+        for i in range(reps + 3):
+            if i == 3:
+                tl, tm, tf = _Timer(), _Timer(), _Timer()
+            with tl:
+                B.jp_vshard_local(ctx, d0, zs, ps, tok, None, lo, V, k, gathered[0])
+            with tm:
+                B.jp_vshard_merge(ctx, n, 0, gathered, T, V, k)
+            with tf:
+                B.jp_batch_finalize(ctx, B.jp_obrs_desc(), lam, B.JP_LAMBDA_FIXED, cfg["seed"], out["accept"],
+                                    out["weight"], out["logp_actor"], out["logp_policy"], out["stats_buf"])
+        ms_l, ms_m, ms_f = tl.ms() / reps, tm.ms() / reps, tf.ms() / reps
+        st = B.read_stats(out["stats_buf"])
+        gb = 2.0 * T * (hi - lo) * 2 / 1e9
+        _emit(workload="vocab_shards", rows=T, shards=n, shard_columns=hi - lo, k=k, local_ms=ms_l,
+              local_gb_per_s=gb / (ms_l * 1e-3), merge_ms=ms_m, finalize_ms=ms_f,
+              all_gather_bytes_per_rank=T * words * 4, rank_total_ms=ms_l + ms_m + ms_f,
+              tokens_per_s=T / ((ms_l + ms_m + ms_f) * 1e-3), n_accept=st["n_accept"], kappa=st["kappa"],
+              status=st["status"])
+
+
 def main(argv):
     assert torch.cuda.is_available(), "needs a CUDA device"
     jp_build.build()
@@ -217,7 +260,8 @@ def main(argv):
     which = [a for a in argv if not a.startswith("-")] or ["cfg3_batch", "cfg4_sweep", "cfg5_train", "row_lambda"]
     ctx = B.Context(0)
     for name in which:
-        {"cfg3_batch": cfg3_batch, "cfg4_sweep": cfg4_sweep, "cfg5_train": cfg5_train, "row_lambda": row_lambda, "simulation": simulation}[name](ctx)
+        {"cfg3_batch": cfg3_batch, "cfg4_sweep": cfg4_sweep, "cfg5_train": cfg5_train, "row_lambda": row_lambda, "simulation": simulation,
+         "vocab_shards": vocab_shards}[name](ctx)
         torch.cuda.empty_cache()
     ctx.close()
 
