@@ -251,14 +251,27 @@ jp_status jp_obrs_apply_kappa(jp_ctx* ctx, double kappa, float c1, float* out_we
  * 1 <= k <= JP_MAX_TOPK (no exact mode: JP_ERR_UNSUPPORTED); n_shards * k <= 2048
  * (JP_ERR_TOO_LARGE).  A row is valid if every shard found it valid.  All pointers device
  * memory owned by the caller; the calls enqueue on the context's stream and return.  The
- * context's records afterwards describe the whole vocabulary, so jp_obrs_backward (which
- * takes the logits of the whole row) does not apply to a slice. */
+ * context's records afterwards describe the whole vocabulary; the gradients of a slice come
+ * from jp_vshard_backward.
+ *
+ * jp_vshard_backward: jp_obrs_backward for the columns [vocab_offset, vocab_offset + desc->V)
+ * of rows whose records the merge and finalize left in this context.  The gradient of the
+ * joint objective (Eq. sys_joint_obj) with respect to a logit needs, beside the logit itself,
+ * only the row's two log-sum-exps and per-token scalars, all in the records, and the one-hot
+ * term falls on the slice that holds the sampled token; so every device writes the gradient
+ * of its own columns with no further exchange.  Arguments as for jp_obrs_backward with desc,
+ * logits and gradients describing the slice and tokens holding ids in [0, V_total);
+ * out_kl / out_loss need whole rows and are JP_ERR_UNSUPPORTED here. */
 size_t jp_vshard_record_floats(int k);
 jp_status jp_vshard_local(jp_ctx* ctx, const jp_obrs_desc* desc, const void* actor_logits,
                           const void* policy_logits, const int32_t* tokens, const uint8_t* mask,
                           int64_t vocab_offset, int64_t V_total, int k, float* out_packed);
 jp_status jp_vshard_merge(jp_ctx* ctx, int n_shards, int my_shard, const float* gathered, int64_t T,
                           int64_t V_total, int k);
+jp_status jp_vshard_backward(jp_ctx* ctx, const jp_obrs_desc* desc, const jp_obrs_bwd_desc* bwd,
+                             const void* actor_logits, const void* policy_logits, const int32_t* tokens,
+                             const uint8_t* mask, int64_t vocab_offset, const uint8_t* accept,
+                             const float* weight, void* d_actor_logits, void* d_policy_logits);
 
 /* Theorem 3.4 for single distributions: for every row t the lambda_t at which the
  * OBRS rule accepts exactly `budget` of the proposal's mass,

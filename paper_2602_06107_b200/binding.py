@@ -24,7 +24,7 @@ JP_ERR_TOO_LARGE = -8
 EXPORTS = (
     "jp_create", "jp_destroy", "jp_set_stream", "jp_obrs_workspace_bytes", "jp_reserve",
     "jp_obrs_forward", "jp_obrs_backward", "jp_batch_begin", "jp_batch_chunk", "jp_batch_finalize",
-    "jp_obrs_forward_host", "jp_obrs_apply_kappa", "jp_batch_logprobs", "jp_obrs_row_lambda", "jp_vshard_record_floats", "jp_vshard_local", "jp_vshard_merge", "jp_budget_lambda_static", "jp_probe_stream", "jp_status_string", "jp_last_error", "jp_launch_count",
+    "jp_obrs_forward_host", "jp_obrs_apply_kappa", "jp_batch_logprobs", "jp_obrs_row_lambda", "jp_vshard_record_floats", "jp_vshard_local", "jp_vshard_merge", "jp_vshard_backward", "jp_budget_lambda_static", "jp_probe_stream", "jp_status_string", "jp_last_error", "jp_launch_count",
     "jp_enable_kernel_timing", "jp_stream_kernel_times",
 )
 
@@ -105,6 +105,8 @@ def load():
     lib.jp_vshard_record_floats.restype = ctypes.c_size_t
     lib.jp_vshard_local.argtypes = [vp, ctypes.POINTER(jp_obrs_desc), vp, vp, vp, vp, i64, i64, ctypes.c_int, vp]
     lib.jp_vshard_merge.argtypes = [vp, ctypes.c_int, ctypes.c_int, vp, i64, i64, ctypes.c_int]
+    lib.jp_vshard_backward.argtypes = [vp, ctypes.POINTER(jp_obrs_desc), ctypes.POINTER(jp_obrs_bwd_desc),
+                                       vp, vp, vp, vp, i64, vp, vp, vp, vp]
     lib.jp_budget_lambda_static.argtypes = [vp, vp, vp, i64, f32, vp, vp]
     lib.jp_probe_stream.argtypes = [vp, vp, i64, ctypes.c_int, vp, ctypes.POINTER(ctypes.c_float)]
     lib.jp_batch_begin.argtypes = [vp, i64, i64, i32, ctypes.c_int, f32]
@@ -240,6 +242,13 @@ def jp_vshard_local(ctx: Context, desc, za, zp, tokens, mask, vocab_offset: int,
 
 def jp_vshard_merge(ctx: Context, n_shards: int, my_shard: int, gathered, T: int, V_total: int, k: int):
     ctx.check(ctx.lib.jp_vshard_merge(ctx.h, n_shards, my_shard, _ptr(gathered), T, V_total, k))
+
+
+def jp_vshard_backward(ctx: Context, desc, bwd, za, zp, tokens, mask, vocab_offset: int, accept, weight, d_actor,
+                       d_policy):
+    ctx.check(ctx.lib.jp_vshard_backward(ctx.h, ctypes.byref(desc), ctypes.byref(bwd), _ptr(za), _ptr(zp),
+                                         _ptr(tokens), _ptr(mask), vocab_offset, _ptr(accept), _ptr(weight),
+                                         _ptr(d_actor), _ptr(d_policy)))
 
 
 def jp_batch_logprobs(ctx: Context, out_logp_actor, out_logp_policy, out_valid):

@@ -465,7 +465,7 @@ jp_status jp_vshard_local(jp_ctx* c, const jp_obrs_desc* d, const void* za, cons
   c->vshard_local_done = false;
   if (d->T > 0) {
     if (!tokens) return fail(c, JP_ERR_INVALID_ARG, "tokens pointer is NULL");
-    e = launch_vshard_localize(d->T, tokens, mask, vocab_offset, d->V, V_total, c->vtok, c->vmask, c->sc, c->stream);
+    e = launch_vshard_localize(d->T, tokens, mask, vocab_offset, d->V, V_total, 0, c->vtok, c->vmask, c->sc, c->stream);
     if (e != cudaSuccess) return cuda_fail(c, e, "shard token launch");
     c->launches += 1;
     if ((st = stream_rows(c, d, ld, k, 0, za, zp, c->vtok, c->vmask, false, false)) != JP_OK) return st;
@@ -550,17 +550,26 @@ jp_status jp_obrs_apply_kappa(jp_ctx* c, double kappa, float c1, float* out_weig
   return JP_OK;
 }
 
-jp_status jp_obrs_backward(jp_ctx* c, const jp_obrs_desc* d, const jp_obrs_bwd_desc* b,
-                           const void* za, const void* zp, const int32_t* tokens,
-                           const uint8_t* mask, const uint8_t* accept, const float* weight,
-                           void* d_actor, void* d_policy) {
+}  // extern "C"
+
+namespace {
+// slice_offset < 0: the rows are whole; otherwise they are the columns [slice_offset, slice_offset + V)
+// of rows whose records describe rec_V columns.
+jp_status backward_impl(jp_ctx* c, const jp_obrs_desc* d, const jp_obrs_bwd_desc* b,
+                        const void* za, const void* zp, const int32_t* tokens,
+                        const uint8_t* mask, const uint8_t* accept, const float* weight,
+                        void* d_actor, void* d_policy, int64_t slice_offset) {
   if (!c) return JP_ERR_INVALID_ARG;
   int64_t ld = 0;
   jp_status st = check_shape(c, d, &ld);
   if (st != JP_OK) return st;
   if (!b) return fail(c, JP_ERR_INVALID_ARG, "bwd desc is NULL");
   if (!c->have_records) return fail(c, JP_ERR_STATE, "no forward records in this context: run the forward (or finalize the batch) first");
-  if (d->V != c->rec_V || d->dtype != c->rec_dtype) return fail(c, JP_ERR_STATE, "V / dtype differ from the forward that left the records");
+  const bool slice = slice_offset >= 0;
+  if (!slice && (d->V != c->rec_V || d->dtype != c->rec_dtype)) return fail(c, JP_ERR_STATE, "V / dtype differ from the forward that left the records");
+  if (slice && d->dtype != c->rec_dtype) return fail(c, JP_ERR_STATE, "dtype differs from the forward that left the records");
+  if (slice && slice_offset + d->V > c->rec_V) return fail(c, JP_ERR_INVALID_ARG, "slice columns fall outside the vocabulary of the records");
+  if (slice && (b->out_kl || b->out_loss)) return fail(c, JP_ERR_UNSUPPORTED, "the per-row KL and the loss value need whole rows");
   if (b->record_offset < 0 || b->record_offset + d->T > c->rec_rows)
     return fail(c, JP_ERR_INVALID_ARG, "rows fall outside the forward's records");
   if (b->lambda_distill < 0.f) return fail(c, JP_ERR_INVALID_ARG, "lambda_distill < 0");
@@ -578,6 +587,12 @@ jp_status jp_obrs_backward(jp_ctx* c, const jp_obrs_desc* d, const jp_obrs_bwd_d
   cudaSetDevice(c->device);
   cudaError_t e = cudaMemsetAsync(&c->sc->row_counter2, 0, sizeof(int32_t), c->stream);
   if (e != cudaSuccess) return cuda_fail(c, e, "cudaMemsetAsync");
+  if (slice) {
+    e = launch_vshard_localize(d->T, tokens, mask, slice_offset, d->V, c->rec_V, -1, c->vtok, nullptr, nullptr, c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e, "slice token launch");
+    c->launches += 1;
+    tokens = c->vtok;
+  }
   GradArgs g{};
   g.za = za; g.zp = zp; g.tokens = tokens; g.mask = mask; g.accept = accept; g.weight = weight;
   g.adv = b->advantages; g.d_actor = d_actor; g.d_policy = d_policy;
@@ -594,6 +609,25 @@ jp_status jp_obrs_backward(jp_ctx* c, const jp_obrs_desc* d, const jp_obrs_bwd_d
   if (e != cudaSuccess) return cuda_fail(c, e, "gradient kernel launch");
   c->launches += n_launch;
   return JP_OK;
+}
+}  // namespace
+
+extern "C" {
+
+jp_status jp_obrs_backward(jp_ctx* c, const jp_obrs_desc* d, const jp_obrs_bwd_desc* b,
+                           const void* za, const void* zp, const int32_t* tokens,
+                           const uint8_t* mask, const uint8_t* accept, const float* weight,
+                           void* d_actor, void* d_policy) {
+  return backward_impl(c, d, b, za, zp, tokens, mask, accept, weight, d_actor, d_policy, -1);
+}
+
+jp_status jp_vshard_backward(jp_ctx* c, const jp_obrs_desc* d, const jp_obrs_bwd_desc* b,
+                             const void* za, const void* zp, const int32_t* tokens,
+                             const uint8_t* mask, int64_t vocab_offset, const uint8_t* accept,
+                             const float* weight, void* d_actor, void* d_policy) {
+  if (!c) return JP_ERR_INVALID_ARG;
+  if (vocab_offset < 0) return fail(c, JP_ERR_INVALID_ARG, "vocab_offset < 0");
+  return backward_impl(c, d, b, za, zp, tokens, mask, accept, weight, d_actor, d_policy, vocab_offset);
 }
 
 jp_status jp_obrs_forward_host(jp_ctx* c, const jp_obrs_desc* d, const void* za, const void* zp,

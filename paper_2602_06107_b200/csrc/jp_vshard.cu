@@ -21,21 +21,23 @@ constexpr int VS_NT = 128;
 
 __global__ void __launch_bounds__(256) vshard_localize_kernel(int64_t T, const int32_t* tokens, const uint8_t* mask,
                                                               int64_t vocab_offset, int64_t V_shard, int64_t V_total,
-                                                              int32_t* tok_local, uint8_t* mask_local, Scalars* sc) {
+                                                              int32_t foreign, int32_t* tok_local,
+                                                              uint8_t* mask_local, Scalars* sc) {
   const int64_t i = (int64_t)blockIdx.x * 256 + threadIdx.x;
   if (i >= T) return;
   bool valid = mask == nullptr || mask[i] != 0;
   const int64_t x = tokens[i];
   if (valid && (x < 0 || x >= V_total)) {
     valid = false;
-    atomicAdd(&sc->n_bad_token, 1ull);
+    if (sc) atomicAdd(&sc->n_bad_token, 1ull);
   }
   const int64_t loc = x - vocab_offset;
   const bool owner = valid && loc >= 0 && loc < V_shard;
-  // a shard that does not hold the sampled token streams the row all the same (column 0
-  // stands in for the token; the log-prob it yields is never used)
-  tok_local[i] = owner ? (int32_t)loc : 0;
-  mask_local[i] = valid ? (owner ? 2 : 1) : 0;
+  // Forward (foreign = 0): a shard that does not hold the sampled token streams the row all
+  // the same; column 0 stands in for the token and the log-prob it yields is never used.
+  // Backward (foreign = -1): no column of such a shard carries the one-hot term.
+  tok_local[i] = owner ? (int32_t)loc : foreign;
+  if (mask_local) mask_local[i] = valid ? (owner ? 2 : 1) : 0;
 }
 
 // One warp per row: the shard's records of the row as one packed line.
@@ -172,11 +174,11 @@ __global__ void __launch_bounds__(VS_NT) vshard_merge_kernel(int n_shards, int m
 }  // namespace
 
 cudaError_t launch_vshard_localize(int64_t T, const int32_t* tokens, const uint8_t* mask, int64_t vocab_offset,
-                                   int64_t V_shard, int64_t V_total, int32_t* tok_local, uint8_t* mask_local,
-                                   Scalars* sc, cudaStream_t s) {
+                                   int64_t V_shard, int64_t V_total, int32_t foreign, int32_t* tok_local,
+                                   uint8_t* mask_local, Scalars* sc, cudaStream_t s) {
   if (T <= 0) return cudaSuccess;
   vshard_localize_kernel<<<(unsigned)((T + 255) / 256), 256, 0, s>>>(T, tokens, mask, vocab_offset, V_shard, V_total,
-                                                                   tok_local, mask_local, sc);
+                                                                   foreign, tok_local, mask_local, sc);
   return cudaGetLastError();
 }
 

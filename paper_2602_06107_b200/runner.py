@@ -74,9 +74,10 @@ def forward_chunked(ctx: B.Context, chunks, T_total, V, dtype_code, *, lam=None,
 
 
 def backward(ctx: B.Context, za, zp, tokens, mask, accept, weight, *, advantages=None, lambda_distill=0.0,
-             grad_out=1.0, n_valid=0, record_offset=0, d_actor=None, d_policy=None, **general):
+             grad_out=1.0, n_valid=0, record_offset=0, d_actor=None, d_policy=None, vocab_offset=None, **general):
     """``general``: the optional fields of jp_obrs_bwd_desc (logp_ref, logp_actor_ref, logp_inf, eps_lo,
-    eps_hi, c2, tis_cap, out_obj_policy, out_obj_actor, out_kl, out_loss)."""
+    eps_hi, c2, tis_cap, out_obj_policy, out_obj_actor, out_kl, out_loss).  ``vocab_offset``: the logits are
+    the columns from there on of rows whose records a vocabulary-parallel forward left (jp_vshard_backward)."""
     T, V = za.shape
     if d_actor is None:
         d_actor = torch.empty((T, za.stride(0)), dtype=torch.bfloat16, device=za.device)[:, :V]
@@ -84,5 +85,8 @@ def backward(ctx: B.Context, za, zp, tokens, mask, accept, weight, *, advantages
         d_policy = torch.empty((T, zp.stride(0)), dtype=torch.bfloat16, device=za.device)[:, :V]
     desc = B.make_desc(za)
     bwd = B.make_bwd_desc(advantages, lambda_distill, grad_out, n_valid, record_offset, **general)
-    B.jp_obrs_backward(ctx, desc, bwd, za, zp, tokens, mask, accept, weight, d_actor, d_policy)
+    if vocab_offset is None:
+        B.jp_obrs_backward(ctx, desc, bwd, za, zp, tokens, mask, accept, weight, d_actor, d_policy)
+    else:
+        B.jp_vshard_backward(ctx, desc, bwd, za, zp, tokens, mask, vocab_offset, accept, weight, d_actor, d_policy)
     return d_actor, d_policy

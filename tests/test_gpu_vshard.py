@@ -162,3 +162,52 @@ def test_shard_call_sequence_and_limits(ranks):
                         out["logp_actor"], out["logp_policy"], out["stats_buf"])
     torch.cuda.synchronize()
     assert B.read_stats(out["stats_buf"])["n_valid"] == 8
+
+
+@pytest.mark.parametrize("dtype,V,n", [("bf16", 20000, 3), ("f32", 4099, 2)])
+def test_slice_gradients_match_oracle_on_whole_rows(ranks, dtype, V, n):
+    """Every rank writes the gradient of its own columns from the merged records; side by side
+    the slices are the oracle's gradient of the whole rows (general form: ratios, clip, c2, F)."""
+    from test_gpu_backward import check_grads
+    T, k, lam, seed = 90, 16, 1.3, 5
+    align = 8                                    # gradients are bf16: slices start on 8 elements
+    ld = -(-V // align) * align
+    r = LogitRecipe(T=T, V=ld, dtype=dtype, sigma0=2.5, peaks=4, sigma=1.0, seed=41)
+    zaf, zpf, _ = make_logits(r, "cuda")
+    za, zp = zaf[:, :V], zpf[:, :V]
+    g = torch.Generator(device="cuda").manual_seed(6)
+    gum = -torch.log(-torch.log(torch.rand((T, V), generator=g, device="cuda").clamp_(1e-30, 1 - 1e-7)))
+    tok = (za.float() + gum).argmax(1).to(torch.int32)
+    tok[4], tok[5] = V - 1, 0
+    mask = (torch.arange(T, device="cuda") % 6 != 1).to(torch.uint8)
+    adv = torch.randn(T, generator=g, device="cuda")
+    bounds = [parallel.shard_columns(V, n, s, align) for s in range(n)]
+    outs = run_shards(ranks, za, zp, tok, mask, bounds, lam=lam, k=k, seed=seed, c1=3.0, finish=tuple(range(n)))
+    out = outs[0]
+    da = torch.full((T, ld), 7.0, dtype=torch.bfloat16, device="cuda")
+    dp = torch.full((T, ld), 7.0, dtype=torch.bfloat16, device="cuda")
+    for s, (lo, hi) in enumerate(bounds):
+        runner.backward(ranks[s], za[:, lo:hi], zp[:, lo:hi], tok, mask, out["accept"], out["weight"], advantages=adv,
+                        lambda_distill=1.0, grad_out=0.5, d_actor=da[:, lo:hi], d_policy=dp[:, lo:hi], vocab_offset=lo)
+    torch.cuda.synchronize()
+    assert torch.all(da[:, V:] == 7.0) and torch.all(dp[:, V:] == 7.0)
+    za_np, zp_np = to_numpy_bits(za.contiguous()), to_numpy_bits(zp.contiguous())
+    ref = oracle.forward(za_np, zp_np, tok.cpu().numpy(), mask.cpu().numpy(), lam=lam, k=k, seed=seed, c1=3.0)
+    rows = np.arange(0, T, 2)
+    check_grads(da[:, :V], dp[:, :V], rows, za_np, zp_np, tok.cpu().numpy(), mask.cpu().numpy(),
+                out["accept"].cpu().numpy(), out["weight"].cpu().numpy(), ref["lse_a"], ref["lse_p"],
+                out["stats"]["n_valid"], adv.cpu().numpy(), 1.0, g=0.5)
+    # and the same bits as the single-device backward of the whole rows
+    one = runner.forward(ranks[n], za, zp, tok, mask, lam=lam, k=k, seed=seed, c1=3.0)
+    da1, dp1 = runner.backward(ranks[n], za, zp, tok, mask, out["accept"], out["weight"], advantages=adv,
+                               lambda_distill=1.0, grad_out=0.5)
+    torch.cuda.synchronize()
+    same = (da[:, :V] == da1).float().mean().item(), (dp[:, :V] == dp1).float().mean().item()
+    print("share of gradient elements bit-identical to the single-device backward:", same)
+    assert min(same) > 0.999
+    # whole-row outputs are refused on a slice
+    lo, hi = bounds[0]
+    with pytest.raises(B.JackpotError, match="whole rows"):
+        runner.backward(ranks[0], za[:, lo:hi], zp[:, lo:hi], tok, mask, out["accept"], out["weight"],
+                        d_actor=da[:, lo:hi], d_policy=dp[:, lo:hi], vocab_offset=lo,
+                        out_kl=torch.empty(T, device="cuda"))
