@@ -261,11 +261,25 @@ jp_status jp_obrs_apply_kappa(jp_ctx* ctx, double kappa, float c1, float* out_we
  * term falls on the slice that holds the sampled token; so every device writes the gradient
  * of its own columns with no further exchange.  Arguments as for jp_obrs_backward with desc,
  * logits and gradients describing the slice and tokens holding ids in [0, V_total);
- * out_kl / out_loss need whole rows and are JP_ERR_UNSUPPORTED here. */
+ * out_kl / out_loss need whole rows and are JP_ERR_UNSUPPORTED here.
+ *
+ * jp_vshard_local_push is jp_vshard_local with the all-gather folded into the export kernel:
+ * gathered_of_shard is a HOST array of n_shards DEVICE pointers, entry p being shard p's gathered
+ * buffer [n_shards, T, words] as this device can address it (its own buffer, and the peers'
+ * through peer-mapped memory: CUDA IPC or symmetric memory, set up by the caller); the kernel
+ * stores this shard's lines at [my_shard] of every one of them with plain stores (no multicast,
+ * no bulk copies).  n_shards <= 16.  The caller makes sure every shard's push has completed
+ * (its stream reached the end of the call, then a barrier over the devices) before any shard
+ * runs jp_vshard_merge on its gathered buffer, and that no shard is still merging the previous
+ * batch from a buffer that is pushed to again. */
 size_t jp_vshard_record_floats(int k);
 jp_status jp_vshard_local(jp_ctx* ctx, const jp_obrs_desc* desc, const void* actor_logits,
                           const void* policy_logits, const int32_t* tokens, const uint8_t* mask,
                           int64_t vocab_offset, int64_t V_total, int k, float* out_packed);
+jp_status jp_vshard_local_push(jp_ctx* ctx, const jp_obrs_desc* desc, const void* actor_logits,
+                               const void* policy_logits, const int32_t* tokens, const uint8_t* mask,
+                               int64_t vocab_offset, int64_t V_total, int k, int n_shards, int my_shard,
+                               float* const* gathered_of_shard);
 jp_status jp_vshard_merge(jp_ctx* ctx, int n_shards, int my_shard, const float* gathered, int64_t T,
                           int64_t V_total, int k);
 jp_status jp_vshard_backward(jp_ctx* ctx, const jp_obrs_desc* desc, const jp_obrs_bwd_desc* bwd,

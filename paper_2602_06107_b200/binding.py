@@ -24,7 +24,7 @@ JP_ERR_TOO_LARGE = -8
 EXPORTS = (
     "jp_create", "jp_destroy", "jp_set_stream", "jp_obrs_workspace_bytes", "jp_reserve",
     "jp_obrs_forward", "jp_obrs_backward", "jp_batch_begin", "jp_batch_chunk", "jp_batch_finalize",
-    "jp_obrs_forward_host", "jp_obrs_apply_kappa", "jp_batch_logprobs", "jp_obrs_row_lambda", "jp_vshard_record_floats", "jp_vshard_local", "jp_vshard_merge", "jp_vshard_backward", "jp_budget_lambda_static", "jp_probe_stream", "jp_status_string", "jp_last_error", "jp_launch_count",
+    "jp_obrs_forward_host", "jp_obrs_apply_kappa", "jp_batch_logprobs", "jp_obrs_row_lambda", "jp_vshard_record_floats", "jp_vshard_local", "jp_vshard_local_push", "jp_vshard_merge", "jp_vshard_backward", "jp_budget_lambda_static", "jp_probe_stream", "jp_status_string", "jp_last_error", "jp_launch_count",
     "jp_enable_kernel_timing", "jp_stream_kernel_times",
 )
 
@@ -104,6 +104,8 @@ def load():
     lib.jp_vshard_record_floats.argtypes = [ctypes.c_int]
     lib.jp_vshard_record_floats.restype = ctypes.c_size_t
     lib.jp_vshard_local.argtypes = [vp, ctypes.POINTER(jp_obrs_desc), vp, vp, vp, vp, i64, i64, ctypes.c_int, vp]
+    lib.jp_vshard_local_push.argtypes = [vp, ctypes.POINTER(jp_obrs_desc), vp, vp, vp, vp, i64, i64, ctypes.c_int,
+                                         ctypes.c_int, ctypes.c_int, ctypes.POINTER(vp)]
     lib.jp_vshard_merge.argtypes = [vp, ctypes.c_int, ctypes.c_int, vp, i64, i64, ctypes.c_int]
     lib.jp_vshard_backward.argtypes = [vp, ctypes.POINTER(jp_obrs_desc), ctypes.POINTER(jp_obrs_bwd_desc),
                                        vp, vp, vp, vp, i64, vp, vp, vp, vp]
@@ -238,6 +240,15 @@ def jp_vshard_record_floats(k: int) -> int:
 def jp_vshard_local(ctx: Context, desc, za, zp, tokens, mask, vocab_offset: int, V_total: int, k: int, out_packed):
     ctx.check(ctx.lib.jp_vshard_local(ctx.h, ctypes.byref(desc), _ptr(za), _ptr(zp), _ptr(tokens), _ptr(mask),
                                       vocab_offset, V_total, k, _ptr(out_packed)))
+
+
+def jp_vshard_local_push(ctx: Context, desc, za, zp, tokens, mask, vocab_offset: int, V_total: int, k: int,
+                         my_shard: int, gathered_of_shard):
+    """``gathered_of_shard``: per shard, its gathered buffer as this device addresses it (tensor or raw pointer)."""
+    n = len(gathered_of_shard)
+    arr = (ctypes.c_void_p * n)(*[_ptr(g) for g in gathered_of_shard])
+    ctx.check(ctx.lib.jp_vshard_local_push(ctx.h, ctypes.byref(desc), _ptr(za), _ptr(zp), _ptr(tokens), _ptr(mask),
+                                           vocab_offset, V_total, k, n, my_shard, arr))
 
 
 def jp_vshard_merge(ctx: Context, n_shards: int, my_shard: int, gathered, T: int, V_total: int, k: int):

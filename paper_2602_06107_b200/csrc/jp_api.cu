@@ -444,8 +444,12 @@ jp_status jp_batch_finalize(jp_ctx* c, const jp_obrs_desc* dout, float lambda_or
 
 size_t jp_vshard_record_floats(int k) { return k < 1 ? 0 : (size_t)vshard_words(k); }
 
-jp_status jp_vshard_local(jp_ctx* c, const jp_obrs_desc* d, const void* za, const void* zp, const int32_t* tokens,
-                          const uint8_t* mask, int64_t vocab_offset, int64_t V_total, int k, float* out_packed) {
+}  // extern "C"
+
+namespace {
+jp_status vshard_local_impl(jp_ctx* c, const jp_obrs_desc* d, const void* za, const void* zp, const int32_t* tokens,
+                            const uint8_t* mask, int64_t vocab_offset, int64_t V_total, int k,
+                            const VshardDests& dests, int64_t line0) {
   if (!c) return JP_ERR_INVALID_ARG;
   int64_t ld = 0;
   jp_status st = check_shape(c, d, &ld);
@@ -455,7 +459,8 @@ jp_status jp_vshard_local(jp_ctx* c, const jp_obrs_desc* d, const void* za, cons
   if ((int64_t)k >= d->V) return fail(c, JP_ERR_UNSUPPORTED, "a vocabulary shard must be wider than k columns");
   if (vocab_offset < 0 || vocab_offset + d->V > V_total || V_total > (int64_t)0x7fffffff)
     return fail(c, JP_ERR_INVALID_ARG, "shard columns fall outside [0, V_total)");
-  if (d->T > 0 && !out_packed) return fail(c, JP_ERR_INVALID_ARG, "out_packed is NULL");
+  for (int p = 0; p < dests.n; ++p)
+    if (d->T > 0 && !dests.dst[p]) return fail(c, JP_ERR_INVALID_ARG, "a destination of the packed records is NULL");
   cudaSetDevice(c->device);
   if ((st = ensure_workspace(c, d->T > 0 ? d->T : 1, k)) != JP_OK) return st;
   cudaError_t e = launch_reset(c->sc, 1.0f, c->stream);
@@ -469,7 +474,7 @@ jp_status jp_vshard_local(jp_ctx* c, const jp_obrs_desc* d, const void* za, cons
     if (e != cudaSuccess) return cuda_fail(c, e, "shard token launch");
     c->launches += 1;
     if ((st = stream_rows(c, d, ld, k, 0, za, zp, c->vtok, c->vmask, false, false)) != JP_OK) return st;
-    e = launch_vshard_export(d->T, k, c->rec, za, zp, ld, d->dtype, c->vtok, c->vmask, vocab_offset, out_packed,
+    e = launch_vshard_export(d->T, k, c->rec, za, zp, ld, d->dtype, c->vtok, c->vmask, vocab_offset, dests, line0,
                              c->stream);
     if (e != cudaSuccess) return cuda_fail(c, e, "shard export launch");
     c->launches += 1;
@@ -479,6 +484,31 @@ jp_status jp_vshard_local(jp_ctx* c, const jp_obrs_desc* d, const void* za, cons
   c->vshard_k = k;
   c->rec_dtype = d->dtype;
   return JP_OK;
+}
+}  // namespace
+
+extern "C" {
+
+jp_status jp_vshard_local(jp_ctx* c, const jp_obrs_desc* d, const void* za, const void* zp, const int32_t* tokens,
+                          const uint8_t* mask, int64_t vocab_offset, int64_t V_total, int k, float* out_packed) {
+  VshardDests dests{};
+  dests.n = 1;
+  dests.dst[0] = out_packed;
+  return vshard_local_impl(c, d, za, zp, tokens, mask, vocab_offset, V_total, k, dests, 0);
+}
+
+jp_status jp_vshard_local_push(jp_ctx* c, const jp_obrs_desc* d, const void* za, const void* zp,
+                               const int32_t* tokens, const uint8_t* mask, int64_t vocab_offset, int64_t V_total,
+                               int k, int n_shards, int my_shard, float* const* gathered_of_shard) {
+  if (!c) return JP_ERR_INVALID_ARG;
+  if (!d) return fail(c, JP_ERR_INVALID_ARG, "desc is NULL");
+  if (n_shards < 1 || n_shards > kVshardMaxDests) return fail(c, JP_ERR_TOO_LARGE, "at most 16 shards can be pushed to");
+  if (my_shard < 0 || my_shard >= n_shards) return fail(c, JP_ERR_INVALID_ARG, "shard index out of range");
+  if (!gathered_of_shard) return fail(c, JP_ERR_INVALID_ARG, "gathered_of_shard is NULL");
+  VshardDests dests{};
+  dests.n = n_shards;
+  for (int p = 0; p < n_shards; ++p) dests.dst[p] = gathered_of_shard[p];
+  return vshard_local_impl(c, d, za, zp, tokens, mask, vocab_offset, V_total, k, dests, (int64_t)my_shard * d->T);
 }
 
 jp_status jp_vshard_merge(jp_ctx* c, int n_shards, int my_shard, const float* gathered, int64_t T, int64_t V_total,

@@ -163,13 +163,18 @@ cudaError_t launch_row_lambda(const RowLambdaArgs& a, cudaStream_t s, int sms);
 // [8+2k, 8+4k) actor logits of the entries  [8+4k, 8+6k) policy logits of the entries.
 constexpr int kVshardHeader = 8;
 constexpr int kVshardMaxEntries = 2048;   // n_shards * k the merge kernel ranks in shared memory
+constexpr int kVshardMaxDests = 16;       // shards a local pass can push its lines to
+struct VshardDests {
+  float* dst[kVshardMaxDests];
+  int n;
+};
 __host__ __device__ inline int64_t vshard_words(int k) { return kVshardHeader + 6 * (int64_t)k; }
 cudaError_t launch_vshard_localize(int64_t T, const int32_t* tokens, const uint8_t* mask, int64_t vocab_offset,
                                    int64_t V_shard, int64_t V_total, int32_t foreign, int32_t* tok_local,
                                    uint8_t* mask_local, Scalars* sc, cudaStream_t s);
 cudaError_t launch_vshard_export(int64_t T, int k, const Records& rec, const void* za, const void* zp, int64_t ld,
                                  int32_t dtype, const int32_t* tok_local, const uint8_t* mask_local,
-                                 int64_t vocab_offset, float* out, cudaStream_t s);
+                                 int64_t vocab_offset, const VshardDests& dests, int64_t line0, cudaStream_t s);
 cudaError_t launch_vshard_merge(int n_shards, int my_shard, const float* gathered, int64_t T, int k,
                                 const Records& rec, Scalars* sc, cudaStream_t s);
 cudaError_t launch_grad(const GradArgs& a, cudaStream_t s, int sms, int* n_launch);

@@ -40,15 +40,21 @@ __global__ void __launch_bounds__(256) vshard_localize_kernel(int64_t T, const i
   if (mask_local) mask_local[i] = valid ? (owner ? 2 : 1) : 0;
 }
 
-// One warp per row: the shard's records of the row as one packed line.
+// One warp per row: the shard's records of the row as one packed line, stored at line
+// line0 + r of every destination.  With one destination this is the local export; with one
+// per shard (each the same place in a peer's gathered buffer, reachable by plain stores:
+// peer-mapped device memory) the export is also the all-gather, pushed by the producer.
 __global__ void __launch_bounds__(VS_NT) vshard_export_kernel(int64_t T, int k, Records rec, const void* za,
                                                               const void* zp, int64_t ld, int32_t dtype,
                                                               const int32_t* tok_local, const uint8_t* mask_local,
-                                                              int64_t vocab_offset, float* out) {
+                                                              int64_t vocab_offset, VshardDests dests, int64_t line0) {
   const int lane = threadIdx.x & 31;
   const int64_t r = (int64_t)blockIdx.x * (VS_NT / 32) + (threadIdx.x >> 5);
   if (r >= T) return;
-  float* o = out + r * vshard_words(k);
+  const int64_t o = (line0 + r) * vshard_words(k);
+  auto put = [&](int64_t w, float v) {
+    for (int p = 0; p < dests.n; ++p) dests.dst[p][o + w] = v;
+  };
   const bool flag = rec.flag[r] != 0;
   if (lane == 0) {
     const bool owner = flag && mask_local[r] == 2;
@@ -63,21 +69,21 @@ __global__ void __launch_bounds__(VS_NT) vshard_export_kernel(int64_t T, int k, 
         xp = Vec<JP_F32>::load_scalar((const char*)zp + r * ld * Vec<JP_F32>::ESIZE, x);
       }
     }
-    o[0] = __int_as_float(flag ? 1 : 0);
-    o[1] = __int_as_float(owner ? 1 : 0);
-    o[2] = flag ? rec.lse_a[r] : 0.f;
-    o[3] = flag ? rec.lse_a_lo[r] : 0.f;
-    o[4] = flag ? rec.lse_p[r] : 0.f;
-    o[5] = flag ? rec.lse_p_lo[r] : 0.f;
-    o[6] = xa;
-    o[7] = xp;
+    put(0, __int_as_float(flag ? 1 : 0));
+    put(1, __int_as_float(owner ? 1 : 0));
+    put(2, flag ? rec.lse_a[r] : 0.f);
+    put(3, flag ? rec.lse_a_lo[r] : 0.f);
+    put(4, flag ? rec.lse_p[r] : 0.f);
+    put(5, flag ? rec.lse_p_lo[r] : 0.f);
+    put(6, xa);
+    put(7, xp);
   }
   for (int j = lane; j < 2 * k; j += 32) {
     const int64_t e = r * (2 * k) + j;
     const int32_t idx = flag ? rec.idx[e] : -1;
-    o[kVshardHeader + j] = __int_as_float(idx >= 0 ? (int32_t)(idx + vocab_offset) : -1);
-    o[kVshardHeader + 2 * k + j] = idx >= 0 ? rec.za[e] : 0.f;
-    o[kVshardHeader + 4 * k + j] = idx >= 0 ? rec.zp[e] : 0.f;
+    put(kVshardHeader + j, __int_as_float(idx >= 0 ? (int32_t)(idx + vocab_offset) : -1));
+    put(kVshardHeader + 2 * k + j, idx >= 0 ? rec.za[e] : 0.f);
+    put(kVshardHeader + 4 * k + j, idx >= 0 ? rec.zp[e] : 0.f);
   }
 }
 
@@ -184,11 +190,11 @@ cudaError_t launch_vshard_localize(int64_t T, const int32_t* tokens, const uint8
 
 cudaError_t launch_vshard_export(int64_t T, int k, const Records& rec, const void* za, const void* zp, int64_t ld,
                                  int32_t dtype, const int32_t* tok_local, const uint8_t* mask_local,
-                                 int64_t vocab_offset, float* out, cudaStream_t s) {
+                                 int64_t vocab_offset, const VshardDests& dests, int64_t line0, cudaStream_t s) {
   if (T <= 0) return cudaSuccess;
   const int wpb = VS_NT / 32;
   vshard_export_kernel<<<(unsigned)((T + wpb - 1) / wpb), VS_NT, 0, s>>>(T, k, rec, za, zp, ld, dtype, tok_local,
-                                                                        mask_local, vocab_offset, out);
+                                                                        mask_local, vocab_offset, dests, line0);
   return cudaGetLastError();
 }
 

@@ -122,18 +122,32 @@ def gather_shard_records(packed: torch.Tensor, group=None) -> torch.Tensor:
 
 
 def forward_vocab_parallel(ctx, za, zp, tokens, mask, vocab_offset: int, V_total: int, *, lam=None, budget=None,
-                           k=20, seed=0, c1=0.0, aux=False, group=None, gather=gather_shard_records, shard_index=None):
+                           k=20, seed=0, c1=0.0, aux=False, group=None, gather=gather_shard_records, shard_index=None, push_to=None,
+                           own_gathered=None):
     """The forward over column slices: local pass, one all-gather of the packed records
-    (T x (8 + 6k) words per rank), merge, finalize.  Every rank returns the outputs of all T rows."""
+    (T x (8 + 6k) words per rank), merge, finalize.  Every rank returns the outputs of all T rows.
+    ``push_to``: per shard, that shard's gathered buffer [world, T, words] as this device addresses it
+    (tensors, or raw peer-mapped pointers with this rank's own buffer in ``own_gathered``); the local
+    pass then pushes its lines there itself and no collective runs."""
     from . import binding as B
     from . import runner
     assert (lam is None) != (budget is None)
     T = za.shape[0]
     if shard_index is None:
         shard_index = dist.get_rank(group) if dist.is_available() and dist.is_initialized() else 0
-    packed = torch.empty((T, B.jp_vshard_record_floats(k)), dtype=torch.float32, device=za.device)
-    B.jp_vshard_local(ctx, B.make_desc(za), za, zp, tokens, mask, vocab_offset, V_total, k, packed)
-    gathered = gather(packed, group)
+    if push_to is not None:
+        # the export kernel stores this shard's lines into every shard's gathered buffer (peer-mapped
+        # memory); all that is left of the exchange is to wait until every shard has done so
+        gathered = push_to[shard_index] if isinstance(push_to[shard_index], torch.Tensor) else own_gathered
+        B.jp_vshard_local_push(ctx, B.make_desc(za), za, zp, tokens, mask, vocab_offset, V_total, k, shard_index,
+                               push_to)
+        torch.cuda.synchronize()
+        if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
+            dist.barrier(group)
+    else:
+        packed = torch.empty((T, B.jp_vshard_record_floats(k)), dtype=torch.float32, device=za.device)
+        B.jp_vshard_local(ctx, B.make_desc(za), za, zp, tokens, mask, vocab_offset, V_total, k, packed)
+        gathered = gather(packed, group)
     B.jp_vshard_merge(ctx, gathered.shape[0], shard_index, gathered, T, V_total, k)
     out = runner._alloc_outputs(T, za.device)
     d = B.jp_obrs_desc()

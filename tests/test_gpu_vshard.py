@@ -211,3 +211,33 @@ def test_slice_gradients_match_oracle_on_whole_rows(ranks, dtype, V, n):
         runner.backward(ranks[0], za[:, lo:hi], zp[:, lo:hi], tok, mask, out["accept"], out["weight"],
                         d_actor=da[:, lo:hi], d_policy=dp[:, lo:hi], vocab_offset=lo,
                         out_kl=torch.empty(T, device="cuda"))
+
+
+def test_pushed_lines_equal_the_gathered_ones(ranks):
+    """The export that stores into every shard's gathered buffer (here all of them on the one GPU,
+    standing in for peer-mapped memory) leaves in each what the all-gather leaves."""
+    T, V, n, k = 150, 24000, 4, 16
+    r = LogitRecipe(T=T, V=V, dtype="bf16", sigma0=3.0, peaks=6, sigma=1.0, seed=51)
+    za, zp, tok = make_logits(r, "cuda")
+    mask = (torch.arange(T, device="cuda") % 5 != 0).to(torch.uint8)
+    bounds = [parallel.shard_columns(V, n, s) for s in range(n)]
+    words = B.jp_vshard_record_floats(k)
+    stacked = torch.empty((n, T, words), device="cuda")
+    bufs = [torch.full((n, T, words), float("nan"), device="cuda") for _ in range(n)]
+    for s, (lo, hi) in enumerate(bounds):
+        zs, ps = za[:, lo:hi], zp[:, lo:hi]
+        B.jp_vshard_local(ranks[s], B.make_desc(zs), zs, ps, tok, mask, lo, V, k, stacked[s])
+        B.jp_vshard_local_push(ranks[s], B.make_desc(zs), zs, ps, tok, mask, lo, V, k, s, bufs)
+    torch.cuda.synchronize()
+    for b in bufs:
+        assert torch.equal(b.view(torch.int32), stacked.view(torch.int32))
+    # through the glue: push, then merge and finalize from the rank's own buffer
+    lo, hi = bounds[2]
+    out = parallel.forward_vocab_parallel(ranks[2], za[:, lo:hi], zp[:, lo:hi], tok, mask, lo, V, lam=1.5, k=k, seed=3,
+                                          aux=True, shard_index=2, push_to=bufs)
+    ref = oracle.forward(to_numpy_bits(za), to_numpy_bits(zp), tok.cpu().numpy(), mask.cpu().numpy(), lam=1.5, k=k,
+                         seed=3)
+    check_forward(out, ref, k, V, mask.cpu().numpy(), 0.0)
+    with pytest.raises(B.JackpotError, match="16"):
+        B.jp_vshard_local_push(ranks[0], B.make_desc(za[:, :hi]), za[:, :hi], zp[:, :hi], tok, mask, 0, V, k, 0,
+                               [bufs[0]] * 17)
