@@ -67,7 +67,7 @@ namespace jp {
 #define JP_TAU_NS 200
 #endif
 constexpr int NC = JP_NC;                 // consumer warps
-constexpr int NG = JP_NG;                 // consumer groups: group q takes tiles q, q + NG, ...
+constexpr int NG = JP_NG;                 // consumer groups: a row's tiles go to them in turn, starting with first_group(row)
 constexpr int WPT = NC / NG;              // warps that share one tile
 constexpr int VPL = JP_VPL;               // 16-byte vectors per lane per tensor per tile
 constexpr int TV = WPT * 32 * VPL;        // vectors per tensor per tile
@@ -108,6 +108,7 @@ struct __align__(128) StreamSmemT {
   uint32_t ncand[NSLOT][2];               // candidate passes appended so far (may pass CAP: then the row is re-scanned)
   float part_mL[NSLOT][2][NC];
   float part_s[NSLOT][2][NC];
+  uint32_t g0[NSLOT];                     // group that takes tile 0 of the slot's row
   int abort;
 };
 
@@ -787,6 +788,14 @@ __device__ __noinline__ float sample_threshold(const char* row, int64_t nvec, in
   return tau0;
 }
 
+// Which consumer group takes tile 0 of a row.  Tiles go to the groups in turn; starting every
+// row with the same group would leave that group one tile behind on every row with an odd
+// number of tiles.  The choice hangs on the row's index in the batch alone (a hash bit), never on where
+// the row sits in the CTA's walk, so that a row's sums are added in the same order in every run.
+__device__ __forceinline__ uint32_t first_group(int64_t row) {
+  return (uint32_t)(((uint32_t)row * 0x9E3779B1u) >> 16) % (uint32_t)NG;
+}
+
 template <class SM>
 __device__ __forceinline__ void raise_timeout(SM& sm, Scalars* sc) {
   sm.abort = 1;
@@ -814,12 +823,13 @@ __device__ void producer_loop(const StreamArgs& A, SM& sm, int64_t n_rows) {
   while (it < n_rows && ok) {
     const char* ra = (const char*)A.za + row * pitch;
     const char* rp = (const char*)A.zp + row * pitch;
+    const int g0 = (int)first_group(A.record_offset + row);
     it += gridDim.x;
     if (it < n_rows) row = A.list[it];
     for (int tile = 0; tile < ntiles; ++tile, ra += TV * 16, rp += TV * 16) {
       if (!mbar_wait(&sm.empty[s], ph ^ 1u, &sm.abort)) { ok = false; break; }
       const uint32_t bytes = tile == ntiles - 1 ? last_bytes : (uint32_t)(TV * 16);
-      const int grp = tile % NG;
+      const int grp = (tile + g0) % NG;
       if (bytes > 0) {
         mbar_arrive_expect_tx(&sm.full[grp][s], 2u * bytes);
         bulk_g2s(&sm.ring[s][0][0], ra, bytes, &sm.full[grp][s], policy);
@@ -862,7 +872,7 @@ __device__ void consumer_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int c
   static_assert(HV == 2, "a pass takes its maximum over two vectors");
   const uint32_t nfull = (uint32_t)(nvec / TV);            // tiles of a row that need no bounds checks
   const uint32_t row_step = ntiles % (uint32_t)STAGES;     // how far a row moves the ring position of tile 0
-  uint32_t s_row = (uint32_t)gq % (uint32_t)STAGES;        // stage of this group's first tile of the current row
+  uint32_t s_row = 0u;                  // stage of tile 0 of the current row
   uint32_t fphase = 0u;                 // per stage: phase bit of this group's full barrier
   int lr = 0;
   for (int64_t it = blockIdx.x; it < n_rows; it += gridDim.x, ++lr) {
@@ -939,8 +949,11 @@ __device__ void consumer_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int c
       return true;
     };
     {
-      uint32_t s = s_row;
-      for (uint32_t tile = gq; tile < ntiles; tile += NG) {
+      const uint32_t g0 = sm.g0[p];          // written by the slot's top-k warp before it opened the slot
+      const uint32_t first = ((uint32_t)gq + (uint32_t)NG - g0) % (uint32_t)NG;   // this group's first tile of the row
+      uint32_t s = s_row + first;
+      if (s >= (uint32_t)STAGES) s -= (uint32_t)STAGES;
+      for (uint32_t tile = first; tile < ntiles; tile += NG) {
         if (!consume_tile(tile, s)) { raise_timeout(sm, A.sc); return; }
         s += NG;
         if (s >= (uint32_t)STAGES) s -= (uint32_t)STAGES;
@@ -1034,6 +1047,7 @@ __device__ void topk_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int t, in
       }
     }
     uint32_t seen = 0u;                       // candidates counted into the histogram so far
+    if (t == 0 && lane == 0) sm.g0[p] = first_group(rrow);
     __syncwarp();
     if (lane == 0) mbar_arrive(&sm.slot_ready[p]);
 
