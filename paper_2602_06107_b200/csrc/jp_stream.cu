@@ -867,7 +867,7 @@ __device__ void consumer_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int c
   const int tail = (int)(A.V - nvec * N);
   const uint32_t ntiles = nvec > 0 ? (uint32_t)((nvec + TV - 1) / TV) : 1u;
   const uint32_t idmask = 0xffffffffu >> __clz(ntiles * (uint32_t)TP - 1u);   // covers every pass id of a row
-  const int gq = cw / WPT;              // this warp's group: it takes tiles gq, gq + NG, ...
+  const int gq = cw / WPT;              // this warp's group: it takes every NG-th tile of a row
   const int wq = cw % WPT;              // its place among the warps that share a tile
   static_assert(HV == 2, "a pass takes its maximum over two vectors");
   const uint32_t nfull = (uint32_t)(nvec / TV);            // tiles of a row that need no bounds checks
