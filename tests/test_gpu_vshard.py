@@ -24,7 +24,7 @@ pytestmark = pytest.mark.gpu
 @pytest.fixture(scope="module")
 def ranks():
     jp_build.build()
-    cs = [B.Context(0) for _ in range(8)]
+    cs = [B.Context(0) for _ in range(17)]
     yield cs
     for c in cs:
         c.close()
@@ -68,7 +68,8 @@ def same_bits(a, b):
 
 
 @pytest.mark.parametrize("dtype,T,V,n,k", [("bf16", 300, 20000, 4, 16), ("bf16", 96, 151936, 8, 32),
-                                           ("f32", 130, 4099, 3, 8), ("bf16", 64, 50001, 2, 128)])
+                                           ("f32", 130, 4099, 3, 8), ("bf16", 64, 50001, 2, 128),
+                                           ("bf16", 24, 16 * 1024, 16, 128)])     # n * k at the merge's limit
 def test_shards_match_oracle_on_the_whole_vocabulary(ranks, dtype, T, V, n, k):
     align = 8 if dtype == "bf16" else 4
     ld = -(-V // align) * align
@@ -241,3 +242,20 @@ def test_pushed_lines_equal_the_gathered_ones(ranks):
     with pytest.raises(B.JackpotError, match="16"):
         B.jp_vshard_local_push(ranks[0], B.make_desc(za[:, :hi]), za[:, :hi], zp[:, :hi], tok, mask, 0, V, k, 0,
                                [bufs[0]] * 17)
+
+
+def test_shards_of_an_empty_batch(ranks):
+    c = ranks[0]
+    za = torch.empty((0, 4096), dtype=torch.bfloat16, device="cuda")
+    tok = torch.empty(0, dtype=torch.int32, device="cuda")
+    buf = torch.empty((0, B.jp_vshard_record_floats(8)), device="cuda")
+    d = B.jp_obrs_desc()
+    d.T, d.V, d.ld, d.dtype = 0, 4096, 4096, B.JP_BF16
+    B.jp_vshard_local(c, d, za, za, tok, None, 0, 8192, 8, buf)
+    B.jp_vshard_merge(c, 2, 0, buf, 0, 8192, 8)
+    out = runner._alloc_outputs(1, "cuda")
+    B.jp_batch_finalize(c, B.jp_obrs_desc(), 1.0, B.JP_LAMBDA_FIXED, 0, out["accept"], out["weight"],
+                        out["logp_actor"], out["logp_policy"], out["stats_buf"])
+    torch.cuda.synchronize()
+    st = B.read_stats(out["stats_buf"])
+    assert st["n_valid"] == 0 and st["status"] == 0
