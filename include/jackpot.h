@@ -267,8 +267,8 @@ jp_status jp_obrs_apply_kappa(jp_ctx* ctx, double kappa, float c1, float* out_we
  * gathered_of_shard is a HOST array of n_shards DEVICE pointers, entry p being shard p's gathered
  * buffer [n_shards, T, words] as this device can address it (its own buffer, and the peers'
  * through peer-mapped memory: CUDA IPC or symmetric memory, set up by the caller); the kernel
- * stores this shard's lines at [my_shard] of every one of them with plain stores (no multicast,
- * no bulk copies).  n_shards <= 16.  The caller makes sure every shard's push has completed
+ * stores this shard's lines at [my_shard] of every one of them with plain global stores and
+ * nothing else.  n_shards <= 16.  The caller makes sure every shard's push has completed
  * (its stream reached the end of the call, then a barrier over the devices) before any shard
  * runs jp_vshard_merge on its gathered buffer, and that no shard is still merging the previous
  * batch from a buffer that is pushed to again. */
