@@ -99,8 +99,17 @@ __global__ void __launch_bounds__(VS_NT) vshard_merge_kernel(int n_shards, int m
   const int64_t W = vshard_words(k);
   auto line = [&](int s) { return g + ((int64_t)s * T + r) * W; };
 
+  // entry e of the 2 n: tensor t, shard s, place j (n <= 2048, so the quotient by k is exact in fp32)
+  const float inv_k = 1.f / (float)k;
+  auto split = [&](int e, int& t, int& s, int& j) {
+    t = e >= n ? 1 : 0;
+    const int x = e - t * n;
+    s = (int)(((float)x + 0.5f) * inv_k);
+    j = x - s * k;
+  };
   for (int e = tid; e < 2 * n; e += VS_NT) {
-    const int t = e / n, x = e % n, s = x / k, j = x % k;
+    int t, s, j;
+    split(e, t, s, j);
     const float* o = line(s);
     const int32_t idx = __float_as_int(o[kVshardHeader + t * k + j]);
     const float v = o[kVshardHeader + (t == 0 ? 2 * k : 4 * k) + t * k + j];
@@ -119,7 +128,8 @@ __global__ void __launch_bounds__(VS_NT) vshard_merge_kernel(int n_shards, int m
     for (int e = tid; e < 2 * n; e += VS_NT) {
       const unsigned long long key = keys[e];
       if (key == 0ull) continue;
-      const int t = e / n, x = e % n, s = x / k, j = x % k;
+      int t, s, j;
+      split(e, t, s, j);
       // every shard's list is sorted best first (empty slots, key 0, at its end): the keys above
       // this one are a prefix of each list, found by bisection
       const unsigned long long* kt = keys + t * n;
