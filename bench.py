@@ -1,22 +1,36 @@
 #!/usr/bin/env python
 """Benchmark of the OBRS token pass (libjackpot) on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfg2_qwen3]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload cfg2_qwen3|cfg3_batch|cfg4_sweep|cfg5_train]
 
-A step is one forward pass of the whole path (row stream with online softmax and
-both top-k lists, acceptance, decision, Z_approx, kappa, weights) over one batch
-of synthetic logits of the Qwen3 shape: T=4096 tokens, V=151936, bf16, k=32,
-lambda=2.0.  The same JSON line also reports the forward+backward step on the
-same batch (fused logit gradients for both tensors), the roofline of the row
-stream kernel, the end-to-end rate from host buffers, and the CPU oracle timed
-on the machine's host cores.  With --gpus N (torchrun) each rank runs its own batch
-(rows are independent; weak scaling, no data-path collective).
+A step is one pass of the whole path over one batch of synthetic logits:
+
+  cfg2_qwen3 (default)  one jp_obrs_forward over T=4096 tokens, V=151936, bf16, k=32, lambda=2
+                        (row stream with online softmax and both top-k lists, acceptance, decision,
+                        Z_approx, kappa, weights); the line also carries forward+backward on the
+                        same batch, the end-to-end rate from host buffers and the CPU oracle;
+  cfg3_batch            64 padded responses (131,072 rows, ~58 % valid) streamed in 16 chunks of 8192
+                        rows, lambda from an acceptance budget of 0.6, k=64 (jp_batch_begin / chunk /
+                        finalize); the unit is a valid token;
+  cfg4_sweep            16,384 rows at three actor/policy mismatches and k in {8, 32, 128, V}: twelve
+                        forwards per step, Z_approx against the exact Z and throughput per point;
+  cfg5_train            32,768 rows in 4 chunks: chunked forward with a budget of 0.5 and a weight
+                        clip, then one fused backward per chunk (bf16 gradients of both tensors).
+
+Every workload prints one JSON line with `roofline` (the dominant kernel, timed per launch by CUDA
+events on the stream it runs on), `cpu_baseline` (the oracle on a bounded sample, all host cores and
+one) and `e2e` (host buffers through jp_obrs_forward_host, or null with the reason).  With --gpus N
+every rank runs its own batch of the same shape (rows are independent: weak scaling, no data-path
+collective); started without torchrun, the script starts its N ranks itself.
 """
 from __future__ import annotations
 
 import argparse
+import glob
 import json
 import os
+import socket
 import subprocess
 import sys
 import tempfile
@@ -26,8 +40,10 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-METRIC = "obrs_forward_tokens_per_s"
 UNIT = "tokens/s"
+METRICS = {"cfg2_qwen3": "obrs_forward_tokens_per_s", "cfg3_batch": "obrs_forward_tokens_per_s",
+           "cfg4_sweep": "obrs_forward_tokens_per_s", "cfg5_train": "obrs_fwd_bwd_tokens_per_s"}
+DATASHEET_GBS = 8000.0
 
 
 def _peaks():
@@ -40,7 +56,7 @@ def _peaks():
 
 
 class ClockSampler:
-    """nvidia-smi clock / throttle-reason samples taken during the timed region."""
+    """nvidia-smi clock / throttle-reason samples, taken from start() to stop()."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
          "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
@@ -50,7 +66,7 @@ class ClockSampler:
         self.p = None
         try:
             self.p = subprocess.Popen(["nvidia-smi", "-i", str(gpu_index), f"--query-gpu={self.Q}",
-                                       "--format=csv,noheader,nounits", "-lms", "50"],
+                                       "--format=csv,noheader,nounits", "-lms", "20"],
                                       stdout=self.f, stderr=subprocess.DEVNULL)
         except OSError:
             self.p = None
@@ -66,17 +82,21 @@ class ClockSampler:
             self.p.kill()
         self.f.flush()
         self.f.seek(0)
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in self.f.read().splitlines():
             c = [x.strip() for x in line.split(",")]
             if len(c) < 9:
                 continue
             try:
-                sm.append(float(c[1]))
-                mx.append(float(c[2]))
+                s_, m_, p_ = float(c[1]), float(c[2]), float(c[3])
             except ValueError:
                 continue
+            if p_ < 300.0:            # an idle sample between two timed regions says nothing about the load
+                continue
+            sm.append(s_)
+            mx.append(m_)
+            pw.append(p_)
             for n, v in zip(names, c[5:9]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
@@ -84,47 +104,118 @@ class ClockSampler:
         os.unlink(self.f.name)
         if sm:
             sm.sort()
-            out.update(sm_mhz=sm[len(sm) // 2], sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+            out.update(sm_mhz=sm[len(sm) // 2], sm_mhz_min=sm[0], sm_max_mhz=max(mx), power_w_max=max(pw),
+                       reasons=sorted(reasons), samples=len(sm), note="samples under load (board power >= 300 W)")
         return out
+
+
+def _recipe(r0, T, seed, sigma=None):
+    from paper_2602_06107_b200.inputs import LogitRecipe
+    return LogitRecipe(T=T, V=r0.V, dtype=r0.dtype, sigma0=r0.sigma0, peaks=r0.peaks, peak_lo=r0.peak_lo,
+                       peak_hi=r0.peak_hi, sigma=r0.sigma if sigma is None else sigma, seed=seed)
 
 
 def _workload(name):
     from paper_2602_06107_b200.inputs import CONFIGS
-    cfg = CONFIGS[name]
-    return cfg
+    if name not in METRICS:
+        raise SystemExit(f"bench.py: workload {name!r} is not a bench line (choose from {sorted(METRICS)}); "
+                         "the tiny exact-check shape is a parity test, see tests/")
+    return CONFIGS[name]
+
+
+# ---------------------------------------------------------------------------------------------------
+# the oracle on the host cores (cpu_baseline leg and the reference arm)
+
+def _oracle_sample(name, cfg, rows, device="cpu"):
+    """`rows` rows of the workload (its first chunk / first sweep point), as the oracle takes them."""
+    from paper_2602_06107_b200.inputs import make_lengths_mask, make_logits, to_numpy_bits
+    r0 = cfg["recipe"]
+    za, zp, tok = make_logits(_recipe(r0, rows, r0.seed), device, block_rows=rows)
+    mask = None
+    if name == "cfg3_batch":
+        m, _ = make_lengths_mask(cfg["n_resp"], cfg["max_len"], cfg["min_len"], seed=cfg["seed"], device="cpu")
+        mask = m[:rows].numpy().copy()
+    return to_numpy_bits(za), to_numpy_bits(zp), tok.cpu().numpy(), mask
+
+
+def _oracle_step(name, cfg, za, zp, tok, mask):
+    """One pass of the oracle over the sample, with the workload's own parameters; returns the
+    number of units (tokens, valid tokens for the padded batch) it processed."""
+    import numpy as np
+
+    import oracle
+    n = za.shape[0]
+    if name == "cfg2_qwen3":
+        oracle.forward(za, zp, tok, None, lam=cfg["lam"], k=cfg["k"], seed=cfg["seed"])
+        return n
+    if name == "cfg3_batch":
+        oracle.forward(za, zp, tok, mask, budget=cfg["budget"], k=cfg["k"], seed=cfg["seed"])
+        return int((mask != 0).sum())
+    if name == "cfg4_sweep":
+        for k in cfg["ks"]:
+            oracle.forward(za, zp, tok, None, lam=cfg["lam"], k=min(k, za.shape[1]), seed=cfg["seed"])
+        return n * len(cfg["ks"])
+    ref = oracle.forward(za, zp, tok, None, budget=cfg["budget"], k=cfg["k"], seed=cfg["seed"], c1=cfg["c1"])
+    adv = np.ones(n, np.float32)
+    oracle.grad_rows(np.arange(n), za, zp, tok, ref["accept"], ref["w"], ref["lse_a"], ref["lse_p"],
+                     float(ref["stats"]["n_valid"]), adv=adv, lambda_distill=cfg["lambda_distill"])
+    return n
+
+
+def _time_oracle(name, cfg, sample, seconds, threads=None):
+    import oracle
+    all_threads = oracle.num_threads()
+    if threads is not None:
+        oracle.set_num_threads(threads)
+    try:
+        _oracle_step(name, cfg, *[None if x is None else x[:8] for x in sample])
+        t0, units, reps = time.perf_counter(), 0, 0
+        while time.perf_counter() - t0 < seconds:
+            units += _oracle_step(name, cfg, *sample)
+            reps += 1
+        dt = time.perf_counter() - t0
+        return units / dt, reps, dt, oracle.num_threads()
+    finally:
+        if threads is not None:
+            oracle.set_num_threads(all_threads)
+
+
+def cpu_baseline_for(name, cfg, sample):
+    rows = sample[0].shape[0]
+    v, reps, dt, cores = _time_oracle(name, cfg, sample, 8.0)
+    one = [None if x is None else x[:max(8, rows // 8)] for x in sample]
+    v1, reps1, dt1, _ = _time_oracle(name, cfg, one, 6.0, threads=1)
+    what = {"cfg2_qwen3": "forward", "cfg3_batch": "forward with the budget solve, valid tokens",
+            "cfg4_sweep": "the four k of one sweep point", "cfg5_train": "forward + both gradients"}[name]
+    return {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"first {rows} rows of the workload, {what}, {reps} passes, {dt:.1f} s",
+            "single_thread": {"value": v1, "unit": UNIT, "cores": 1,
+                              "sample": f"first {one[0].shape[0]} rows, {reps1} passes, {dt1:.1f} s"}}
 
 
 def run_reference(args, rank):
-    """The reference arm: the CPU oracle, as it stands, on this machine's host cores,
-    each step a bounded sample of the workload's rows."""
+    """The reference arm: the CPU oracle, as it stands, on this machine's host cores, each step a
+    bounded sample of the workload's rows."""
     if rank != 0:
         return
-    import numpy as np
-    import torch
-
     import oracle
-    from paper_2602_06107_b200.inputs import LogitRecipe, make_logits, to_numpy_bits
     cfg = _workload(args.workload)
     r = cfg["recipe"]
     rows = args.ref_rows
-    sample = LogitRecipe(T=rows, V=r.V, dtype=r.dtype, sigma0=r.sigma0, peaks=r.peaks, peak_lo=r.peak_lo,
-                         peak_hi=r.peak_hi, sigma=r.sigma, seed=r.seed)
-    za, zp, tok = make_logits(sample, "cpu", block_rows=rows)
-    za, zp, tok = to_numpy_bits(za), to_numpy_bits(zp), tok.numpy()
-    k, lam = cfg.get("k", 32), cfg.get("lam", 2.0)
+    sample = _oracle_sample(args.workload, cfg, rows)
     for _ in range(args.warmup):
-        oracle.forward(za, zp, tok, None, lam=lam, k=k, seed=cfg["seed"])
-    t0 = time.perf_counter()
+        _oracle_step(args.workload, cfg, *sample)
+    t0, units = time.perf_counter(), 0
     for _ in range(args.steps):
-        oracle.forward(za, zp, tok, None, lam=lam, k=k, seed=cfg["seed"])
+        units += _oracle_step(args.workload, cfg, *sample)
     dt = time.perf_counter() - t0
-    val = rows * args.steps / dt
+    val = units / dt
     cores = oracle.num_threads()
-    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+    line = {"impl": "reference", "metric": METRICS[args.workload], "value": val, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
             "data": "synthetic",
-            "config": {"workload": args.workload, "T": r.T, "V": r.V, "logits": r.dtype, "k": k, "lambda": lam,
+            "config": {"workload": args.workload, "T": r.T, "V": r.V, "logits": r.dtype,
                        "sample": f"{rows} rows of the workload per step"},
             "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle",
                              "sample": f"{rows} rows x {args.steps} steps of {args.workload}"},
@@ -133,222 +224,465 @@ def run_reference(args, rank):
     print(json.dumps(line))
 
 
-def run_ours(args, rank, world, local_rank):
-    import torch
-    import torch.distributed as dist
+# ---------------------------------------------------------------------------------------------------
+# the library on the GPU
 
-    from paper_2602_06107_b200 import binding as B
-    from paper_2602_06107_b200 import build as jp_build
-    from paper_2602_06107_b200 import runner
-    from paper_2602_06107_b200.inputs import LogitRecipe, make_logits
+class Bench:
+    """What every workload needs: device, ranks, context, timing."""
 
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py: no CUDA device; libjackpot has no CPU path")
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
-    if rank == 0:
-        jp_build.build()
-    if world > 1:
-        dist.barrier()
-    cfg = _workload(args.workload)
-    r0 = cfg["recipe"]
-    T = args.T or r0.T
-    r = LogitRecipe(T=T, V=r0.V, dtype=r0.dtype, sigma0=r0.sigma0, peaks=r0.peaks, peak_lo=r0.peak_lo,
-                    peak_hi=r0.peak_hi, sigma=r0.sigma, seed=r0.seed + 1000 * rank)
-    k, lam, seed = cfg.get("k", 32), cfg.get("lam", 2.0), cfg["seed"]
-    za, zp, tok = make_logits(r, dev)
-    V = r.V
-    esize = za.element_size()
-    ctx = B.Context(local_rank)
-    B.jp_reserve(ctx, T, V, k)
-    out = runner._alloc_outputs(T, dev)
-    desc = B.make_desc(za)
+    def __init__(self, args, rank, world, local_rank):
+        import torch
+        import torch.distributed as dist
 
-    def fwd():
-        B.jp_obrs_forward(ctx, desc, za, zp, tok, None, lam, k, seed, out["accept"], out["weight"],
-                          out["logp_actor"], out["logp_policy"], out["stats_buf"])
-
-    def sync_all():
-        torch.cuda.synchronize(dev)
+        from paper_2602_06107_b200 import binding as B
+        from paper_2602_06107_b200 import build as jp_build
+        self.torch, self.dist, self.B = torch, dist, B
+        self.args, self.rank, self.world = args, rank, world
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py: no CUDA device; libjackpot has no CPU path")
+        torch.cuda.set_device(local_rank)
+        self.dev = torch.device("cuda", local_rank)
+        if world > 1:
+            dist.init_process_group("nccl", device_id=self.dev)
+        if rank == 0:
+            jp_build.build()
         if world > 1:
             dist.barrier()
-            torch.cuda.synchronize(dev)
+        self.ctx = B.Context(local_rank)
+        self.local_rank = local_rank
+        self.peak, self.peak_kind = _peaks()
+        self.sampler = None
 
-    def timed(fn, steps, warmup):
+    def sync_all(self):
+        self.torch.cuda.synchronize(self.dev)
+        if self.world > 1:
+            self.dist.barrier()
+            self.torch.cuda.synchronize(self.dev)
+
+    def max_over_ranks(self, x):
+        if self.world > 1:
+            t = self.torch.tensor([x], device=self.dev, dtype=self.torch.float64)
+            self.dist.all_reduce(t, op=self.dist.ReduceOp.MAX)
+            x = float(t.item())
+        return x
+
+    def timed(self, fn, steps, warmup):
+        """Device time of `steps` calls (CUDA events on the stream the library launches on, which is
+        torch's current stream), barrier and device sync on both sides, max over ranks."""
+        torch = self.torch
         for _ in range(warmup):
             fn()
-        sync_all()
+        self.sync_all()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for _ in range(steps):
             fn()
         e1.record()
-        sync_all()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        self.sync_all()
+        return self.max_over_ranks(e0.elapsed_time(e1))
 
-    # ---- forward (the headline): device-resident inputs, per-launch stream-kernel times
-    B.jp_enable_kernel_timing(ctx, True)
-    sampler = ClockSampler(local_rank) if rank == 0 else None
-    l0 = ctx.launch_count()
-    ms = timed(fwd, args.steps, args.warmup)
-    launches = (ctx.launch_count() - l0) * args.steps // (args.steps + args.warmup)
-    clocks = sampler.stop() if sampler else None
-    kt = B.jp_stream_kernel_times(ctx, min(args.steps, 256))
-    B.jp_enable_kernel_timing(ctx, False)
+    def timed_with_kernel_times(self, fn, steps, warmup, launches_per_step):
+        """timed(), plus the device time of every row-stream launch of the timed steps."""
+        B = self.B
+        B.jp_enable_kernel_timing(self.ctx, True)
+        l0 = self.ctx.launch_count()
+        ms = self.timed(fn, steps, warmup)
+        launches = (self.ctx.launch_count() - l0) // (steps + warmup)
+        n = min(steps, 256 // launches_per_step) * launches_per_step
+        kt = B.jp_stream_kernel_times(self.ctx, n)
+        B.jp_enable_kernel_timing(self.ctx, False)
+        return ms, launches, kt
+
+    def roofline(self, kernel, alg_bytes, kernel_ms, **extra):
+        achieved = alg_bytes / (kernel_ms * 1e-3) / 1e9
+        r = {"bound": "hbm", "achieved": achieved, "peak": self.peak, "unit": "GB/s", "frac": achieved / self.peak,
+             "traffic": None, "peak_kind": f"of {self.peak_kind} (copy bandwidth; the 80 % target is judged on this one)",
+             "frac_of_datasheet_8tbs": achieved / DATASHEET_GBS, "kernel": kernel, "kernel_ms": kernel_ms,
+             "algorithmic_bytes": alg_bytes}
+        r.update(extra)
+        return r
+
+    def add_probe_rates(self, roof, a, b):
+        """This GPU's plain streaming rates, measured now with the library's probe kernel: the forward
+        only reads its logits, so the read-only rate is the tighter reference beside the copy rate."""
+        try:
+            ro = self.B.jp_probe_stream(a, None, reps=20)
+            roof["read_only_gbs_now"] = ro
+            roof["copy_gbs_now"] = self.B.jp_probe_stream(a, b, reps=10)
+            roof["frac_of_read_only_now"] = roof["achieved"] / ro
+        except Exception as exc:                               # a measurement aid must not lose the line
+            roof["probe_error"] = str(exc)
+
+    def add_traffic(self, roof, key, units):
+        """DRAM bytes per launch of the row stream, from an ncu capture of a smaller case scaled by
+        rows (traffic is proportional to the rows streamed); null unless the capture was taken
+        from the kernel source as it stands."""
+        tr = os.path.join(ROOT, "profiles", "traffic.json")
+        if not os.path.exists(tr):
+            return
+        with open(tr) as f:
+            t = json.load(f)
+        import hashlib
+        with open(os.path.join(ROOT, "paper_2602_06107_b200", "csrc", "jp_stream.cu"), "rb") as f:
+            digest = hashlib.sha256(f.read()).hexdigest()[:16]
+        ent = t.get(key)
+        if ent and ent.get("source_sha256_16") == digest:
+            roof["traffic"] = ent["dram_bytes_per_row"] * units
+
+    def stream_kernel_name(self, dtype, k, V):
+        if k >= V:
+            return f"prep_rows_kernel + stream_kernel<{dtype}, no top-k> (exact mode; exact_z_kernel follows)"
+        kpl = 1 if k <= 32 else 2 if k <= 64 else 4
+        return f"prep_rows_kernel + stream_kernel<{dtype}, {32 * kpl}-entry lists> (k = {k})"
+
+
+def wl_cfg2(b: Bench, cfg):
+    torch, B, args = b.torch, b.B, b.args
+    from paper_2602_06107_b200 import runner
+    from paper_2602_06107_b200.inputs import make_logits
+    r0 = cfg["recipe"]
+    T = args.T or r0.T
+    r = _recipe(r0, T, r0.seed + 1000 * b.rank)
+    k, lam, seed = cfg["k"], cfg["lam"], cfg["seed"]
+    za, zp, tok = make_logits(r, b.dev)
+    V, esize = r.V, za.element_size()
+    B.jp_reserve(b.ctx, T, V, k)
+    out = runner._alloc_outputs(T, b.dev)
+    desc = B.make_desc(za)
+
+    def fwd():
+        B.jp_obrs_forward(b.ctx, desc, za, zp, tok, None, lam, k, seed, out["accept"], out["weight"],
+                          out["logp_actor"], out["logp_policy"], out["stats_buf"])
+
+    ms, launches, kt = b.timed_with_kernel_times(fwd, args.steps, args.warmup, 1)
     stats = B.read_stats(out["stats_buf"])
-    ms_per_step = ms / args.steps
-    value = world * T * args.steps / (ms * 1e-3)
-    peak, peak_kind = _peaks()
     k_ms = sum(kt) / len(kt)
-    alg_bytes = 2.0 * stats["n_valid"] * V * esize
-    achieved = alg_bytes / (k_ms * 1e-3) / 1e9
+    alg = 2.0 * stats["n_valid"] * V * esize
+    roof = b.roofline(b.stream_kernel_name(r.dtype, k, V) + ": one forward's row stream", alg, k_ms,
+                      kernel_ms_min=min(kt), kernel_ms_max=max(kt))
+    b.add_probe_rates(roof, za, zp)
+    b.add_traffic(roof, "cfg2_qwen3", stats["n_valid"])
 
-    # ---- forward + backward on the same batch (fused gradients of both tensors)
-    adv = torch.randn(T, device=dev)
-    d_a = torch.empty_like(za)
-    d_p = torch.empty_like(zp)
+    # forward + backward on the same batch (fused gradients of both tensors)
+    adv = torch.randn(T, device=b.dev)
+    d_a, d_p = torch.empty_like(za), torch.empty_like(zp)
     bwd = B.make_bwd_desc(adv, 1.0, 1.0, 0, 0)
+
+    def bwd_only():
+        B.jp_obrs_backward(b.ctx, desc, bwd, za, zp, tok, None, out["accept"], out["weight"], d_a, d_p)
 
     def fwd_bwd():
         fwd()
-        B.jp_obrs_backward(ctx, desc, bwd, za, zp, tok, None, out["accept"], out["weight"], d_a, d_p)
-
-    def bwd_only():
-        B.jp_obrs_backward(ctx, desc, bwd, za, zp, tok, None, out["accept"], out["weight"], d_a, d_p)
+        bwd_only()
 
     steps_b = max(3, min(args.steps // 2, 100))
-    ms_fb = timed(fwd_bwd, steps_b, 3)
-    ms_b = timed(bwd_only, steps_b, 3)
+    ms_fb = b.timed(fwd_bwd, steps_b, 3)
+    ms_b = b.timed(bwd_only, steps_b, 3)
     del d_a, d_p
-    fb = {"value": world * T * steps_b / (ms_fb * 1e-3), "unit": UNIT, "ms_per_step": ms_fb / steps_b,
-          "backward_ms": ms_b / steps_b,
-          "backward_gbs": 4.0 * T * V * esize / (ms_b / steps_b * 1e-3) / 1e9,
-          "backward_frac_of_peak": 4.0 * T * V * esize / (ms_b / steps_b * 1e-3) / 1e9 / peak}
+    bw_gbs = 4.0 * T * V * esize / (ms_b / steps_b * 1e-3) / 1e9
+    fb = {"value": b.world * T * steps_b / (ms_fb * 1e-3), "unit": UNIT, "ms_per_step": ms_fb / steps_b,
+          "backward_ms": ms_b / steps_b, "backward_gbs": bw_gbs, "backward_frac_of_peak": bw_gbs / b.peak}
 
-    # ---- end to end from pinned host buffers through the host-buffer entry point
+    # end to end from pinned host buffers through the host-buffer entry point
     e2e = None
     if not args.no_e2e:
-        hza = za.cpu().pin_memory()
-        hzp = zp.cpu().pin_memory()
-        htok = tok.cpu().pin_memory()
+        hza, hzp, htok = za.cpu().pin_memory(), zp.cpu().pin_memory(), tok.cpu().pin_memory()
         hacc = torch.empty(T, dtype=torch.uint8).pin_memory()
-        hw = torch.empty(T, dtype=torch.float32).pin_memory()
-        hlq = torch.empty(T, dtype=torch.float32).pin_memory()
-        hlp = torch.empty(T, dtype=torch.float32).pin_memory()
+        hw, hlq, hlp = (torch.empty(T, dtype=torch.float32).pin_memory() for _ in range(3))
         hst = torch.zeros(B.STATS_BYTES, dtype=torch.uint8).pin_memory()
         hdesc = B.make_desc(hza)
 
         def e2e_step():
-            B.jp_obrs_forward_host(ctx, hdesc, hza, hzp, htok, None, lam, k, seed, hacc, hw, hlq, hlp, hst, 0)
+            B.jp_obrs_forward_host(b.ctx, hdesc, hza, hzp, htok, None, lam, k, seed, hacc, hw, hlq, hlp, hst, 0)
 
         e2e_steps = max(2, min(args.steps, 5))
         for _ in range(2):
             e2e_step()
-        sync_all()
+        b.sync_all()
         t0 = time.perf_counter()
         for _ in range(e2e_steps):
             e2e_step()
-        sync_all()
-        dt = time.perf_counter() - t0
-        if world > 1:
-            t = torch.tensor([dt], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            dt = float(t.item())
-        e2e = {"value": world * T * e2e_steps / dt, "unit": UNIT,
+        b.sync_all()
+        dt = b.max_over_ranks(time.perf_counter() - t0)
+        e2e = {"value": b.world * T * e2e_steps / dt, "unit": UNIT,
                "h2d_bytes_per_step": int(2 * T * V * esize + 4 * T),
                "d2h_bytes_per_step": int(T * 13 + B.STATS_BYTES), "ms_per_step": 1e3 * dt / e2e_steps}
-        assert torch.equal(hacc.to(dev), out["accept"]), "host-buffer path disagrees with the device path"
+        assert torch.equal(hacc.to(b.dev), out["accept"]), "host-buffer path disagrees with the device path"
         del hza, hzp
+    return dict(ms=ms, units_per_step=T, launches=launches, roofline=roof, e2e=e2e, extra={"fwd_bwd": fb},
+                config={"T": T, "V": V, "logits": r.dtype, "k": k, "lambda": lam, "seed": seed,
+                        "l2": f"inputs {2 * T * V * esize / 1e9:.2f} GB per step exceed the 126 MB L2; no flush needed",
+                        "stats": {n: stats[n] for n in ("alpha_hat", "kappa", "z_approx_mean")}})
 
+
+E2E_NULL = ("not measured for this workload: its host buffers would be {gb:.0f} GB of pinned memory per rank; the "
+            "host-buffer entry point is PCIe-bound and its rate is the default workload's e2e figure")
+
+
+def wl_cfg3(b: Bench, cfg):
+    torch, B, args = b.torch, b.B, b.args
+    from paper_2602_06107_b200 import runner
+    from paper_2602_06107_b200.inputs import make_lengths_mask, make_logits
+    r0, chunk, k = cfg["recipe"], cfg["chunk"], cfg["k"]
+    T, V = r0.T, r0.V
+    mask, _ = make_lengths_mask(cfg["n_resp"], cfg["max_len"], cfg["min_len"], seed=cfg["seed"] + 1000 * b.rank,
+                                device=b.dev)
+    n_valid = int(mask.sum().item())
+    parts = [make_logits(_recipe(r0, chunk, r0.seed + 17 * c + 1000 * b.rank), b.dev, block_rows=2048)
+             for c in range(T // chunk)]
+    B.jp_reserve(b.ctx, T, V, k)
+    out = runner._alloc_outputs(T, b.dev)
+    descs = [B.make_desc(p[0], token_offset=c * chunk) for c, p in enumerate(parts)]
+    masks = [mask[c * chunk:(c + 1) * chunk] for c in range(len(parts))]
+    fdesc = B.jp_obrs_desc()
+
+    def step():
+        B.jp_batch_begin(b.ctx, T, V, B.JP_BF16, k, 0.0)
+        for d, (za, zp, tok), m in zip(descs, parts, masks):
+            B.jp_batch_chunk(b.ctx, d, za, zp, tok, m)
+        B.jp_batch_finalize(b.ctx, fdesc, cfg["budget"], B.JP_LAMBDA_FROM_BUDGET, cfg["seed"], out["accept"],
+                            out["weight"], out["logp_actor"], out["logp_policy"], out["stats_buf"])
+
+    nch = len(parts)
+    ms, launches, kt = b.timed_with_kernel_times(step, args.steps, args.warmup, nch)
+    stats = B.read_stats(out["stats_buf"])
+    assert stats["n_valid"] == n_valid and stats["status"] == 0
+    k_ms = sum(kt) / (len(kt) // nch)                        # the sixteen launches of one step
+    alg = 2.0 * n_valid * V * 2
+    per_chunk = [sum(kt[i::nch]) / len(kt[i::nch]) for i in range(nch)]
+    roof = b.roofline(b.stream_kernel_name(r0.dtype, k, V) + f": the {nch} row-stream launches of one step", alg, k_ms,
+                      chunk_ms=per_chunk, chunk_valid_rows=[int(m.sum().item()) for m in masks])
+    b.add_probe_rates(roof, parts[0][0], parts[0][1])
+    b.add_traffic(roof, "cfg3_batch", n_valid)
+    return dict(ms=ms, units_per_step=n_valid, launches=launches, roofline=roof,
+                e2e={"value": None, "reason": E2E_NULL.format(gb=2 * T * V * 2 / 1e9)}, extra={},
+                config={"T": T, "valid_tokens": n_valid, "V": V, "logits": r0.dtype, "k": k, "budget": cfg["budget"],
+                        "chunks": nch, "unit": "valid tokens (padding rows are not read)",
+                        "padded_rows_per_s": b.world * T * args.steps / (ms * 1e-3),
+                        "l2": f"inputs {2 * T * V * 2 / 1e9:.1f} GB resident, {alg / 1e9:.1f} GB read per step: far beyond L2",
+                        "stats": {n: stats[n] for n in ("lambda_used", "alpha_hat", "mean_accept_prob", "kappa")}})
+
+
+def wl_cfg4(b: Bench, cfg):
+    torch, B, args = b.torch, b.B, b.args
+    from paper_2602_06107_b200 import runner
+    from paper_2602_06107_b200.inputs import make_logits
+    r0, lam, seed = cfg["recipe"], cfg["lam"], cfg["seed"]
+    T, V = r0.T, r0.V
+    B.jp_reserve(b.ctx, T, V, 128)
+    data = [make_logits(_recipe(r0, T, r0.seed + si + 1000 * b.rank, sigma=s), b.dev, block_rows=2048)
+            for si, s in enumerate(cfg["sigmas"])]
+    out = runner._alloc_outputs(T, b.dev)
+    zk = torch.empty(T, dtype=torch.float32, device=b.dev)
+    points = [(si, k) for si in range(len(data)) for k in cfg["ks"]]
+    descs = {}
+    for si, (za, _, _) in enumerate(data):
+        d = B.make_desc(za)
+        d.z_approx = zk.data_ptr()
+        descs[si] = d
+
+    def point(si, k):
+        za, zp, tok = data[si]
+        B.jp_obrs_forward(b.ctx, descs[si], za, zp, tok, None, lam, k, seed, out["accept"], out["weight"],
+                          out["logp_actor"], out["logp_policy"], out["stats_buf"])
+
+    def step():
+        for si, k in points:
+            point(si, k)
+
+    npt = len(points)
+    ms, launches, kt = b.timed_with_kernel_times(step, args.steps, args.warmup, npt)
+    per_point_ms = [sum(kt[i::npt]) / len(kt[i::npt]) for i in range(npt)]
+    # outside the timed region: every point once more on its own (CUDA events around the whole
+    # forward), and the normaliser error against the exact value
+    table, zx = [], {}
+    for si in range(len(data)):
+        point(si, V)
+        torch.cuda.synchronize()
+        zx[si] = zk.double().clone()
+    for i, (si, k) in enumerate(points):
+        one = b.timed(lambda: point(si, k), 5, 2) / 5
+        st = B.read_stats(out["stats_buf"])
+        passes = 2 if k >= V else 1
+        gbs = passes * 2.0 * T * V * 2 / (one * 1e-3) / 1e9
+        table.append({"sigma": cfg["sigmas"][si], "k": int(k), "forward_ms": one, "stream_kernel_ms": per_point_ms[i],
+                      "tokens_per_s": T / (one * 1e-3), "gb_per_s": gbs, "frac": gbs / b.peak,
+                      "stream_kernel_frac": 2.0 * T * V * 2 / (per_point_ms[i] * 1e-3) / 1e9 / b.peak,
+                      "mean_abs_zk_over_z_minus_1": float(((zk.double() / zx[si]) - 1.0).abs().mean().item()),
+                      "kappa": st["kappa"], "alpha_hat": st["alpha_hat"]})
+    k_ms = sum(per_point_ms)
+    alg = npt * 2.0 * T * V * 2
+    roof = b.roofline(f"prep_rows_kernel + stream_kernel<{r0.dtype}> at k in {list(cfg['ks'])}: the {npt} row-stream "
+                      "launches of one step (exact mode's second pass, exact_z_kernel, is not in this figure)",
+                      alg, k_ms)
+    b.add_probe_rates(roof, data[0][0], data[0][1])
+    return dict(ms=ms, units_per_step=T * npt, launches=launches, roofline=roof,
+                e2e={"value": None, "reason": E2E_NULL.format(gb=len(data) * 2 * T * V * 2 / 1e9)},
+                extra={"sweep": table},
+                config={"T": T, "V": V, "logits": r0.dtype, "lambda": lam, "sigmas": list(cfg["sigmas"]),
+                        "ks": [int(k) for k in cfg["ks"]], "forwards_per_step": npt,
+                        "l2": "every forward reads 9.96 GB (19.9 GB in exact mode): far beyond L2"})
+
+
+def wl_cfg5(b: Bench, cfg):
+    torch, B, args = b.torch, b.B, b.args
+    from paper_2602_06107_b200 import runner
+    from paper_2602_06107_b200.inputs import make_logits
+    r0, chunk, k = cfg["recipe"], cfg["chunk"], cfg["k"]
+    T, V = r0.T, r0.V
+    B.jp_reserve(b.ctx, T, V, k)
+    parts = [make_logits(_recipe(r0, chunk, r0.seed + 31 * c + 1000 * b.rank), b.dev, block_rows=2048)
+             for c in range(T // chunk)]
+    grads = [(torch.empty_like(za), torch.empty_like(zp)) for za, zp, _ in parts]
+    g = torch.Generator(device="cpu").manual_seed(cfg["seed"])
+    adv = torch.randn(T // chunk, generator=g).repeat_interleave(chunk).to(b.dev)      # one draw per response
+    out = runner._alloc_outputs(T, b.dev)
+    nch = len(parts)
+    descs = [B.make_desc(p[0], token_offset=c * chunk) for c, p in enumerate(parts)]
+    fdesc = B.jp_obrs_desc()
+    fdesc.c1 = cfg["c1"]
+    bdescs = [B.make_bwd_desc(adv[c * chunk:(c + 1) * chunk], cfg["lambda_distill"], 1.0, 0, c * chunk)
+              for c in range(nch)]
+
+    def forward():
+        B.jp_batch_begin(b.ctx, T, V, B.JP_BF16, k, 0.0)
+        for d, (za, zp, tok) in zip(descs, parts):
+            B.jp_batch_chunk(b.ctx, d, za, zp, tok, None)
+        B.jp_batch_finalize(b.ctx, fdesc, cfg["budget"], B.JP_LAMBDA_FROM_BUDGET, cfg["seed"], out["accept"],
+                            out["weight"], out["logp_actor"], out["logp_policy"], out["stats_buf"])
+
+    def backward():
+        for c, (za, zp, tok) in enumerate(parts):
+            sl = slice(c * chunk, (c + 1) * chunk)
+            B.jp_obrs_backward(b.ctx, descs[c], bdescs[c], za, zp, tok, None, out["accept"][sl], out["weight"][sl],
+                               grads[c][0], grads[c][1])
+
+    def step():
+        forward()
+        backward()
+
+    ms, launches, kt = b.timed_with_kernel_times(step, args.steps, args.warmup, nch)
+    stats = B.read_stats(out["stats_buf"])
+    assert stats["status"] == 0
+    steps2 = max(3, min(args.steps, 20))
+    ms_b = b.timed(backward, steps2, 2) / steps2
+    ms_f = b.timed(forward, steps2, 2) / steps2
+    alg_b = 4.0 * T * V * 2
+    roof = b.roofline("grad_kernel<bf16> (reads both rows, writes both bf16 gradient rows): the "
+                      f"{nch} backward launches of one step", alg_b, ms_b)
+    k_ms = sum(kt) / (len(kt) // nch)
+    fw = b.roofline(b.stream_kernel_name(r0.dtype, k, V) + f": the {nch} row-stream launches of one step",
+                    2.0 * T * V * 2, k_ms, forward_ms=ms_f)
+    b.add_probe_rates(fw, parts[0][0], parts[0][1])
+    roof["copy_gbs_now"] = fw.get("copy_gbs_now")
+    return dict(ms=ms, units_per_step=T, launches=launches, roofline=roof,
+                e2e={"value": None, "reason": E2E_NULL.format(gb=2 * T * V * 2 / 1e9)},
+                extra={"forward_roofline": fw, "forward_ms": ms_f, "backward_ms": ms_b,
+                       "ideal_tokens_per_s_at_peak": b.peak * 1e9 / (6.0 * V * 2)},
+                config={"T": T, "V": V, "logits": r0.dtype, "k": k, "budget": cfg["budget"], "c1": cfg["c1"],
+                        "lambda_distill": cfg["lambda_distill"], "chunks": nch,
+                        "l2": f"{6 * T * V * 2 / 1e9:.1f} GB moved per step: far beyond L2",
+                        "stats": {n: stats[n] for n in ("lambda_used", "alpha_hat", "kappa")}})
+
+
+WORKLOADS = {"cfg2_qwen3": wl_cfg2, "cfg3_batch": wl_cfg3, "cfg4_sweep": wl_cfg4, "cfg5_train": wl_cfg5}
+
+
+def _nccl_summary(log_dir, world):
+    """What the communicator's own log says: ranks, and whether in-switch reduction is on."""
+    if not log_dir:
+        return None
+    text = ""
+    for p in glob.glob(os.path.join(log_dir, "*")):
+        try:
+            with open(p, errors="replace") as f:
+                text += f.read()
+        except OSError:
+            pass
+    return {"init_complete_lines": text.count("Init COMPLETE"), "nranks_expected": world,
+            "nvls_mentioned": "NVLS" in text}
+
+
+def run_ours(args, rank, world, local_rank):
+    cfg = _workload(args.workload)
+    b = Bench(args, rank, world, local_rank)
+    sampler = ClockSampler(local_rank) if rank == 0 else None       # alive across every timed region
+    res = WORKLOADS[args.workload](b, cfg)
+    clocks = sampler.stop() if sampler else None
     if rank != 0:
         return
-    # ---- the oracle on this machine's host cores, on a bounded sample of the same workload
     cpu_baseline = None
     if not args.no_cpu_baseline:
-        import oracle
-        from paper_2602_06107_b200.inputs import to_numpy_bits
-        n = min(args.ref_rows, T)
-        hz_a, hz_p, ht = to_numpy_bits(za[:n]), to_numpy_bits(zp[:n]), tok[:n].cpu().numpy()
-        oracle.forward(hz_a[:8], hz_p[:8], ht[:8], None, lam=lam, k=k, seed=seed)
-        t0 = time.perf_counter()
-        reps = 0
-        while time.perf_counter() - t0 < 10.0:
-            oracle.forward(hz_a, hz_p, ht, None, lam=lam, k=k, seed=seed)
-            reps += 1
-        dt = time.perf_counter() - t0
-        cpu_baseline = {"value": n * reps / dt, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-                        "sample": f"first {n} rows of the batch, {reps} passes, {dt:.1f} s"}
-
-    line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": args.workload, "T": T, "V": V, "logits": r.dtype, "k": k, "lambda": lam,
-                   "seed": seed, "parallelism": f"rows x{world}" if world > 1 else "1 gpu",
-                   "l2": f"inputs {2 * T * V * esize / 1e9:.2f} GB per step exceed the 126 MB L2; no flush needed",
-                   "stats": {"alpha_hat": stats["alpha_hat"], "kappa": stats["kappa"],
-                             "z_approx_mean": stats["z_approx_mean"]}},
-        "clocks": clocks,
-        "e2e": e2e,
-        "gpu_launches": int(launches),
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": None, "peak_kind": f"of {peak_kind}", "kernel": "prep_rows_kernel + stream_kernel<bf16,k<=32> (one forward's row stream)",
-                     "kernel_ms": k_ms, "kernel_ms_min": min(kt), "kernel_ms_max": max(kt),
-                     "algorithmic_bytes": alg_bytes},
-        "fwd_bwd": fb,
-        "cpu_baseline": cpu_baseline,
-    }
-    # this GPU's plain streaming rates, measured now with the library's probe kernel: the forward
-    # only reads its logits, so the read-only rate is the tighter reference beside the copy rate
-    try:
-        line["roofline"]["read_only_gbs_now"] = B.jp_probe_stream(za, None, reps=20)
-        line["roofline"]["copy_gbs_now"] = B.jp_probe_stream(za, zp, reps=10)
-    except Exception as exc:                                   # a measurement aid must not lose the line
-        line["roofline"]["probe_error"] = str(exc)
-    # DRAM bytes per launch of the row stream, from an ncu capture of a smaller case
-    # scaled by rows (traffic is proportional to the rows streamed); null unless the
-    # capture was taken from the kernel source as it stands
-    tr = os.path.join(ROOT, "profiles", "traffic.json")
-    if os.path.exists(tr):
-        with open(tr) as f:
-            t = json.load(f)
-        src = os.path.join(ROOT, "paper_2602_06107_b200", "csrc", "jp_stream.cu")
-        import hashlib
-        with open(src, "rb") as f:
-            digest = hashlib.sha256(f.read()).hexdigest()[:16]
-        ent = t.get(args.workload)
-        if ent and ent.get("source_sha256_16") == digest:
-            line["roofline"]["traffic"] = ent["dram_bytes_per_row"] * stats["n_valid"]
+        cpu_baseline = cpu_baseline_for(args.workload, cfg, _oracle_sample(args.workload, cfg, args.ref_rows))
+    ms = res["ms"]
+    roof = res["roofline"]
+    if clocks and clocks.get("sm_mhz"):
+        roof["kernel_ms_x_sm_mhz"] = roof["kernel_ms"] * clocks["sm_mhz"]
+    config = {"workload": args.workload}
+    config.update(res["config"])
+    config["parallelism"] = f"rows x{world}: every rank its own batch" if world > 1 else "1 gpu"
+    if world > 1:
+        config["nccl"] = _nccl_summary(os.environ.get("JP_BENCH_NCCL_LOG_DIR"), world)
+    line = {"metric": METRICS[args.workload], "value": world * res["units_per_step"] * args.steps / (ms * 1e-3),
+            "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic", "config": config, "clocks": clocks, "e2e": res["e2e"],
+            "gpu_launches": int(res["launches"]), "roofline": roof}
+    line.update(res["extra"])
+    line["cpu_baseline"] = cpu_baseline
     print(json.dumps(line))
+
+
+def _free_port():
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    return port
+
+
+def relaunch_with_ranks(args):
+    """`python bench.py --gpus N` without a launcher: start the N ranks here (one process per GPU,
+    rendezvous on 127.0.0.1) and pass their output through; rank 0 prints the one line."""
+    env = dict(os.environ)
+    log_dir = tempfile.mkdtemp(prefix="jp_bench_nccl_")
+    env.setdefault("NCCL_DEBUG", "INFO")
+    env.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+    env.setdefault("NCCL_DEBUG_FILE", os.path.join(log_dir, "nccl.%h.%p.log"))   # keeps stdout to the one JSON line
+    env["JP_BENCH_NCCL_LOG_DIR"] = log_dir
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(_free_port()), os.path.abspath(__file__)] + sys.argv[1:]
+    raise SystemExit(subprocess.call(cmd, env=env))
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--steps", type=int, default=0, help="timed steps (default: 1000 for cfg2_qwen3, 10 for the others)")
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2_qwen3")
-    ap.add_argument("--T", type=int, default=0, help="override the workload's row count")
+    ap.add_argument("--T", type=int, default=0, help="override the row count (cfg2_qwen3 only)")
     ap.add_argument("--ref-rows", type=int, default=256, help="rows in the CPU oracle's bounded sample")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
+    if args.steps <= 0:
+        args.steps = (1000 if args.workload == "cfg2_qwen3" else 10) if args.impl == "ours" else 20
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.T and args.workload != "cfg2_qwen3":
+        raise SystemExit("bench.py: --T applies to cfg2_qwen3 only")
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if args.impl == "reference":
         run_reference(args, rank)
         return
-    if world != args.gpus and world == 1 and args.gpus > 1:
-        raise SystemExit("bench.py: launch with torch.distributed.run for --gpus > 1")
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        relaunch_with_ranks(args)
+    if world != args.gpus:
+        raise SystemExit(f"bench.py: --gpus {args.gpus} but the launcher started {world} ranks")
     run_ours(args, rank, world, local_rank)
 
 

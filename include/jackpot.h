@@ -20,7 +20,8 @@
  *     cudaMalloc on first use or by jp_reserve; it grows, never shrinks.
  *   - Return value: JP_OK or a negative jp_status; jp_last_error(ctx) gives a
  *     sentence.  Conditions found on the device (token id out of range,
- *     non-finite rows) never trap: they are counted in jp_stats.
+ *     non-finite rows) never trap: such rows are counted in jp_stats and
+ *     treated as masked, so the other rows' results do not depend on them.
  *   - A context is thread-compatible, not thread-safe.
  *   - Rows with mask[t] == 0 are not read; their outputs are accept = 0,
  *     weight = 0, logp = 0 and zero gradient rows.
@@ -54,6 +55,8 @@ typedef enum { JP_LAMBDA_FIXED = 0, JP_LAMBDA_FROM_BUDGET = 1 } jp_lambda_mode;
 
 enum { JP_MAX_TOPK = 128 };
 enum { JP_STATIC_MAX_ROWS = 131072 };   /* row limit of jp_budget_lambda_static */
+enum { JP_DESC_KL = 1 };                /* jp_obrs_desc.flags: also compute KL(p_target || p_inf) per row (one more
+                                           pass over the rows) and report its batch mean in jp_stats.mean_kl_p_q */
 
 /* Shapes, dtype, mode and optional outputs of one forward / backward call.
  * Zero-initialise, then set T, V and what differs from the defaults. */
@@ -66,7 +69,7 @@ typedef struct {
   int32_t dtype;         /* jp_dtype of the logits; gradients are always bf16            */
   int32_t lambda_mode;   /* jp_lambda_mode: meaning of lambda_or_budget                  */
   float c1;              /* clip on w_OBRS (Algorithm 1, step 3); <= 0 means no clip     */
-  int32_t reserved0;
+  int32_t flags;         /* 0, or JP_DESC_KL                                             */
   int64_t token_offset;  /* global index of row 0: the accept draw of row t is keyed on
                             (seed, token_offset + t)                                     */
   /* Optional per-token outputs (device pointers, NULL to skip). */
@@ -84,16 +87,20 @@ typedef struct {
 
 /* Batch statistics, written to DEVICE memory by the last kernel of a forward. */
 typedef struct {
-  int64_t n_valid;       /* N: rows with mask != 0 and a token id inside [0, V)            */
+  int64_t n_valid;       /* N: rows with mask != 0, a token id inside [0, V) and usable numbers (see n_nonfinite) */
   int64_t n_accept;      /* accepted among them                                           */
   int64_t n_bad_token;   /* unmasked rows whose token id was outside [0, V): treated as masked */
-  int64_t n_nonfinite;   /* valid rows whose log-sum-exp came out non-finite              */
+  int64_t n_nonfinite;   /* unmasked rows with a NaN or +inf logit, or whose sampled token has probability 0
+                            under the rollout model: treated as masked.  (log p_target(a_t) = -inf is a
+                            legal row: the ratio is 0 and the token is rejected.)                       */
   double alpha_hat;      /* n_accept / n_valid (Section 4.4.2)                            */
   double mean_accept_prob; /* mean of a(x_t) over valid rows                              */
   double z_approx_mean;  /* mean of Z_approx over valid rows                              */
   double kappa;          /* alpha_hat / z_approx_mean; 1 if n_valid == 0 or the mean is 0 */
   double lambda_used;    /* the fixed lambda, or the one solved from the budget           */
-  double reserved;
+  double mean_kl_p_q;    /* mean over valid rows of KL(p_target(.|s_t) || p_inf(.|s_t)), the actor-policy
+                            divergence the paper tracks during training; NaN unless JP_DESC_KL was set
+                            (in a chunked batch: on every chunk)                                     */
   int32_t status;        /* 0, or a jp_status raised on the device                        */
   int32_t pad;
 } jp_stats;
@@ -215,14 +222,24 @@ jp_status jp_batch_finalize(jp_ctx* ctx, const jp_obrs_desc* desc_outputs, float
  * rows are still streamed once. */
 jp_status jp_batch_logprobs(jp_ctx* ctx, float* out_logp_actor, float* out_logp_policy, uint8_t* out_valid);
 
-/* Weights with a calibration factor supplied by the caller (Section 4.4.2: kappa
- * is a batch-wide scalar).  A batch whose rows are spread over several devices
- * runs the forward on each shard, sums (n_valid, n_accept, n_valid *
- * z_approx_mean) of the shards' jp_stats over all of them, forms
- * kappa = (sum n_accept / sum n_valid) / (sum of Z_approx / sum n_valid) and
- * calls this on every shard: out_weight [rows of the last forward / batch] fp32
- * gets min(kappa Z_approx max(lambda, p/q), c1) from the context's records
- * (c1 <= 0: no clip).  JP_ERR_STATE without records. */
+/* A batch whose rows are spread over several devices (Section 4.4.2: the calibration
+ * factor kappa is batch-wide).  Every device runs the forward on its shard, then
+ *   jp_batch_totals       copies the shard's sums (N, accepted, sum of Z_approx, sum of
+ *                         a(x_t)) to out_totals, [4] doubles in DEVICE memory;
+ *   (the caller adds the shards' totals element-wise: one all-reduce of 32 bytes)
+ *   jp_obrs_apply_totals  forms kappa = (accepted / N) / (sum of Z_approx / N) from the
+ *                         summed totals (DEVICE, [4]; kappa = 1 if N = 0 or the sum is 0,
+ *                         the rule of the one-device forward) and rewrites out_weight
+ *                         [rows of the last forward / batch] = min(kappa Z_approx
+ *                         max(lambda, p/q), c1) from the context's records (c1 <= 0: no
+ *                         clip); out_stats (DEVICE, may be NULL) gets the batch-wide N,
+ *                         accepted, alpha_hat, mean acceptance, mean Z_approx and kappa
+ *                         beside this shard's own counters.
+ * Both enqueue on the context's stream and do not wait.  JP_ERR_STATE without records.
+ * jp_obrs_apply_kappa does the same with a kappa the caller already has. */
+jp_status jp_batch_totals(jp_ctx* ctx, double* out_totals);
+jp_status jp_obrs_apply_totals(jp_ctx* ctx, const double* totals, float c1, float* out_weight,
+                               jp_stats* out_stats);
 jp_status jp_obrs_apply_kappa(jp_ctx* ctx, double kappa, float c1, float* out_weight);
 
 /* Vocabulary-parallel forward (Section 4.4 names the [tokens, vocabulary] logits as the

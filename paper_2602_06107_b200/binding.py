@@ -20,11 +20,12 @@ JP_LAMBDA_FIXED, JP_LAMBDA_FROM_BUDGET = 0, 1
 JP_MAX_TOPK = 128
 JP_STATIC_MAX_ROWS = 131072
 JP_ERR_TOO_LARGE = -8
+JP_DESC_KL = 1
 
 EXPORTS = (
     "jp_create", "jp_destroy", "jp_set_stream", "jp_obrs_workspace_bytes", "jp_reserve",
     "jp_obrs_forward", "jp_obrs_backward", "jp_batch_begin", "jp_batch_chunk", "jp_batch_finalize",
-    "jp_obrs_forward_host", "jp_obrs_apply_kappa", "jp_batch_logprobs", "jp_obrs_row_lambda", "jp_vshard_record_floats", "jp_vshard_local", "jp_vshard_local_push", "jp_vshard_merge", "jp_vshard_backward", "jp_budget_lambda_static", "jp_probe_stream", "jp_status_string", "jp_last_error", "jp_launch_count",
+    "jp_obrs_forward_host", "jp_obrs_apply_kappa", "jp_batch_totals", "jp_obrs_apply_totals", "jp_batch_logprobs", "jp_obrs_row_lambda", "jp_vshard_record_floats", "jp_vshard_local", "jp_vshard_local_push", "jp_vshard_merge", "jp_vshard_backward", "jp_budget_lambda_static", "jp_probe_stream", "jp_status_string", "jp_last_error", "jp_launch_count",
     "jp_enable_kernel_timing", "jp_stream_kernel_times",
 )
 
@@ -37,7 +38,7 @@ class jp_obrs_desc(ctypes.Structure):
     _fields_ = [
         ("T", ctypes.c_int64), ("V", ctypes.c_int64), ("ld", ctypes.c_int64),
         ("dtype", ctypes.c_int32), ("lambda_mode", ctypes.c_int32),
-        ("c1", ctypes.c_float), ("reserved0", ctypes.c_int32),
+        ("c1", ctypes.c_float), ("flags", ctypes.c_int32),
         ("token_offset", ctypes.c_int64),
         ("topk_idx_actor", ctypes.c_void_p), ("topk_idx_policy", ctypes.c_void_p),
         ("topk_val_actor", ctypes.c_void_p), ("topk_val_policy", ctypes.c_void_p),
@@ -53,12 +54,15 @@ class jp_stats(ctypes.Structure):
         ("n_bad_token", ctypes.c_int64), ("n_nonfinite", ctypes.c_int64),
         ("alpha_hat", ctypes.c_double), ("mean_accept_prob", ctypes.c_double),
         ("z_approx_mean", ctypes.c_double), ("kappa", ctypes.c_double),
-        ("lambda_used", ctypes.c_double), ("reserved", ctypes.c_double),
+        ("lambda_used", ctypes.c_double), ("mean_kl_p_q", ctypes.c_double),
         ("status", ctypes.c_int32), ("pad", ctypes.c_int32),
     ]
 
     def as_dict(self):
-        return {n: getattr(self, n) for n, _ in self._fields_ if n not in ("reserved", "pad")}
+        d = {n: getattr(self, n) for n, _ in self._fields_ if n != "pad"}
+        if d["mean_kl_p_q"] != d["mean_kl_p_q"]:      # NaN in the struct: the divergence was not asked for
+            d["mean_kl_p_q"] = None
+        return d
 
 
 class jp_obrs_bwd_desc(ctypes.Structure):
@@ -100,6 +104,8 @@ def load():
                                      vp, vp, vp, vp, vp, vp, vp, vp]
     lib.jp_obrs_apply_kappa.argtypes = [vp, ctypes.c_double, f32, vp]
     lib.jp_batch_logprobs.argtypes = [vp, vp, vp, vp]
+    lib.jp_batch_totals.argtypes = [vp, vp]
+    lib.jp_obrs_apply_totals.argtypes = [vp, vp, f32, vp, vp]
     lib.jp_obrs_row_lambda.argtypes = [vp, ctypes.POINTER(jp_obrs_desc), vp, vp, vp, f32, vp, vp, vp, vp]
     lib.jp_vshard_record_floats.argtypes = [ctypes.c_int]
     lib.jp_vshard_record_floats.restype = ctypes.c_size_t
@@ -180,7 +186,7 @@ class Context:
 
 
 def make_desc(logits: torch.Tensor, *, lambda_mode=JP_LAMBDA_FIXED, c1=0.0, token_offset=0, aux=None,
-              T=None) -> jp_obrs_desc:
+              T=None, flags=0) -> jp_obrs_desc:
     d = jp_obrs_desc()
     d.T = logits.shape[0] if T is None else T
     d.V = logits.shape[1]
@@ -189,6 +195,7 @@ def make_desc(logits: torch.Tensor, *, lambda_mode=JP_LAMBDA_FIXED, c1=0.0, toke
     d.lambda_mode = lambda_mode
     d.c1 = c1
     d.token_offset = token_offset
+    d.flags = flags
     for name, t in (aux or {}).items():
         setattr(d, name, t.data_ptr() if t is not None else None)
     return d
@@ -268,6 +275,14 @@ def jp_batch_logprobs(ctx: Context, out_logp_actor, out_logp_policy, out_valid):
 
 def jp_obrs_apply_kappa(ctx: Context, kappa: float, c1: float, out_weight):
     ctx.check(ctx.lib.jp_obrs_apply_kappa(ctx.h, kappa, c1, _ptr(out_weight)))
+
+
+def jp_batch_totals(ctx: Context, out_totals):
+    ctx.check(ctx.lib.jp_batch_totals(ctx.h, _ptr(out_totals)))
+
+
+def jp_obrs_apply_totals(ctx: Context, totals, c1: float, out_weight, out_stats=None):
+    ctx.check(ctx.lib.jp_obrs_apply_totals(ctx.h, _ptr(totals), c1, _ptr(out_weight), _ptr(out_stats)))
 
 
 def jp_budget_lambda_static(logp_actor, logp_policy, mask, T: int, budget: float, out_lambda, stream=None) -> int:

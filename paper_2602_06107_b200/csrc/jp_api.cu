@@ -30,6 +30,7 @@ struct jp_ctx {
   int64_t rec_rows = 0;          // rows covered (T of the forward / T_total of the batch)
   int64_t rec_V = 0;
   int rec_k = 0;                 // 0 = exact mode
+  bool rec_kl = false;           // the records hold KL(p || q) of every streamed row
   int32_t rec_dtype = 0;
   bool batch_open = false;
   bool batch_exact = false;
@@ -54,7 +55,7 @@ namespace {
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
-  size_t scalars, partials, idx, za, zp, f[9], flag, ratio, dval, list, spill, vtok, vmask, total;
+  size_t scalars, partials, idx, za, zp, f[10], flag, ratio, dval, list, spill, vtok, vmask, total;
 };
 
 Layout layout_for(int64_t rows, int k) {
@@ -67,7 +68,7 @@ Layout layout_for(int64_t rows, int k) {
   L.idx = take(cand * 4);
   L.za = take(cand * 4);
   L.zp = take(cand * 4);
-  for (int i = 0; i < 9; ++i) L.f[i] = take((size_t)rows * 4);
+  for (int i = 0; i < 10; ++i) L.f[i] = take((size_t)rows * 4);
   L.flag = take((size_t)rows);
   L.ratio = take((size_t)rows * 8);
   L.dval = take((size_t)rows * 4);
@@ -128,6 +129,7 @@ jp_status ensure_workspace(jp_ctx* c, int64_t rows, int k) {
   c->rec.a = (float*)(b + L.f[6]);
   c->rec.lse_a_lo = (float*)(b + L.f[7]);
   c->rec.lse_p_lo = (float*)(b + L.f[8]);
+  c->rec.kl = (float*)(b + L.f[9]);
   c->rec.flag = (uint8_t*)(b + L.flag);
   c->rec.ratio = (double*)(b + L.ratio);
   c->rec.dval = (float*)(b + L.dval);
@@ -168,10 +170,26 @@ jp_status check_lambda(jp_ctx* c, float v, int32_t mode) {
   return JP_OK;
 }
 
+// One more pass over a block of rows: the exact Z (into z_out) and / or KL(p || q).
+jp_status extra_pass(jp_ctx* c, const jp_obrs_desc* d, int64_t ld, int64_t record_offset, const void* za,
+                     const void* zp, float* z_out, bool want_kl) {
+  if (d->T == 0 || (!z_out && !want_kl)) return JP_OK;
+  cudaError_t e = cudaMemsetAsync(&c->sc->row_counter2, 0, sizeof(int32_t), c->stream);   // the pass's work queue
+  if (e != cudaSuccess) return cuda_fail(c, e, "cudaMemsetAsync");
+  ExactZArgs x{};
+  x.za = za; x.zp = zp; x.T = d->T; x.V = d->V; x.ld = ld; x.dtype = d->dtype;
+  x.record_offset = record_offset; x.rec = c->rec; x.sc = c->sc;
+  x.out = z_out;
+  x.out_kl = want_kl ? c->rec.kl : nullptr;
+  e = launch_exact_z(x, c->stream, c->sms);
+  if (e != cudaSuccess) return cuda_fail(c, e, "exact-Z / KL kernel launch");
+  c->launches += 1;
+  return JP_OK;
+}
+
 // Streams one block of rows into the records at record_offset.
 jp_status stream_rows(jp_ctx* c, const jp_obrs_desc* d, int64_t ld, int k_eff, int64_t record_offset,
-                      const void* za, const void* zp, const int32_t* tokens, const uint8_t* mask,
-                      bool exact_now, bool exact_to_zx) {
+                      const void* za, const void* zp, const int32_t* tokens, const uint8_t* mask) {
   if (d->T == 0) return JP_OK;
   if (!za || !zp || !tokens) return fail(c, JP_ERR_INVALID_ARG, "logits or tokens pointer is NULL");
   if (!aligned16(za) || !aligned16(zp)) return fail(c, JP_ERR_ALIGNMENT, "logit base pointers must be 16-byte aligned");
@@ -188,15 +206,6 @@ jp_status stream_rows(jp_ctx* c, const jp_obrs_desc* d, int64_t ld, int k_eff, i
   if (c->timing) { cudaEventRecord(c->ev1[slot], c->stream); c->ev_count += 1; }
   if (e != cudaSuccess) return cuda_fail(c, e, "stream kernel launch");
   c->launches += 2;
-  if (exact_now) {
-    ExactZArgs x{};
-    x.za = za; x.zp = zp; x.T = d->T; x.V = d->V; x.ld = ld; x.dtype = d->dtype;
-    x.record_offset = record_offset; x.rec = c->rec; x.sc = c->sc;
-    x.out = exact_to_zx ? c->rec.zx : c->rec.zk;
-    e = launch_exact_z(x, c->stream, c->sms);
-    if (e != cudaSuccess) return cuda_fail(c, e, "exact-Z kernel launch");
-    c->launches += 1;
-  }
   return JP_OK;
 }
 
@@ -210,6 +219,7 @@ EpilogueArgs epilogue_args(jp_ctx* c, const jp_obrs_desc* d, int64_t T, int k_ef
   a.n_part = (int32_t)(np < 1 ? 1 : (np > kMaxPartials ? kMaxPartials : np));
   a.out_accept = out_accept; a.out_weight = out_weight; a.out_lq = out_lq; a.out_lp = out_lp;
   a.out_stats = out_stats;
+  a.have_kl = c->rec_kl ? 1 : 0;
   if (d) {
     a.aux_idx_a = d->topk_idx_actor; a.aux_idx_p = d->topk_idx_policy;
     a.aux_val_a = d->topk_val_actor; a.aux_val_p = d->topk_val_policy;
@@ -335,29 +345,24 @@ jp_status jp_obrs_forward(jp_ctx* c, const jp_obrs_desc* d, const void* za, cons
   const bool want_zx = d->z_exact != nullptr && !exact;
   if ((st = ensure_workspace(c, d->T > 0 ? d->T : 1, k_eff)) != JP_OK) return st;
   const bool budget = d->lambda_mode == JP_LAMBDA_FROM_BUDGET;
+  const bool want_kl = (d->flags & JP_DESC_KL) != 0;
   cudaError_t e = launch_reset(c->sc, budget ? 1.0f : lambda_or_budget, c->stream);
   if (e != cudaSuccess) return cuda_fail(c, e, "reset launch");
   c->launches += 1;
   c->have_records = false;
-  // exact Z needs lambda: with a budget it has to wait for the solve
-  const bool exact_pass = exact || want_zx;
-  st = stream_rows(c, d, ld, k_eff, 0, za, zp, tokens, mask, exact_pass && !budget, want_zx);
+  c->rec_kl = want_kl;
+  st = stream_rows(c, d, ld, k_eff, 0, za, zp, tokens, mask);
   if (st != JP_OK) return st;
+  // the exact Z needs lambda: with a budget it has to wait for the solve; the divergence does not
+  float* z_out = exact ? c->rec.zk : (want_zx ? c->rec.zx : nullptr);
+  if ((st = extra_pass(c, d, ld, 0, za, zp, budget ? nullptr : z_out, want_kl)) != JP_OK) return st;
   EpilogueArgs ea = epilogue_args(c, d, d->T, k_eff, seed, d->token_offset, d->c1, out_accept,
                                   out_weight, out_lq, out_lp, out_stats);
   int nl = 0;
   if (budget) {
     e = launch_budget_solve(ea, (double)lambda_or_budget, c->stream, &nl);
     if (e != cudaSuccess) return cuda_fail(c, e, "budget solve launch");
-    if (exact_pass && d->T > 0) {
-      ExactZArgs x{};
-      x.za = za; x.zp = zp; x.T = d->T; x.V = d->V; x.ld = ld; x.dtype = d->dtype;
-      x.record_offset = 0; x.rec = c->rec; x.sc = c->sc;
-      x.out = want_zx ? c->rec.zx : c->rec.zk;
-      e = launch_exact_z(x, c->stream, c->sms);
-      if (e != cudaSuccess) return cuda_fail(c, e, "exact-Z kernel launch");
-      nl += 1;
-    }
+    if ((st = extra_pass(c, d, ld, 0, za, zp, z_out, false)) != JP_OK) return st;
   }
   e = launch_epilogue(ea, c->stream, &nl);
   c->launches += nl;
@@ -388,6 +393,7 @@ jp_status jp_batch_begin(jp_ctx* c, int64_t T_total, int64_t V, int32_t dtype, i
   c->batch_open = true;
   c->batch_exact = exact;
   c->have_records = false;
+  c->rec_kl = T_total > 0;       // stays true only if every chunk asks for the divergence
   c->rec_rows = T_total; c->rec_V = V; c->rec_k = k_eff; c->rec_dtype = dtype;
   return JP_OK;
 }
@@ -406,7 +412,10 @@ jp_status jp_batch_chunk(jp_ctx* c, const jp_obrs_desc* d, const void* za, const
   // the row list restarts for every chunk; the other scalars accumulate
   cudaError_t e = cudaMemsetAsync(&c->sc->n_list, 0, 2 * sizeof(int32_t), c->stream);
   if (e != cudaSuccess) return cuda_fail(c, e, "cudaMemsetAsync");
-  return stream_rows(c, d, ld, c->rec_k, d->token_offset, za, zp, tokens, mask, c->batch_exact, false);
+  const bool want_kl = (d->flags & JP_DESC_KL) != 0;
+  if (!want_kl && d->T > 0) c->rec_kl = false;
+  if ((st = stream_rows(c, d, ld, c->rec_k, d->token_offset, za, zp, tokens, mask)) != JP_OK) return st;
+  return extra_pass(c, d, ld, d->token_offset, za, zp, c->batch_exact ? c->rec.zk : nullptr, want_kl);
 }
 
 jp_status jp_batch_finalize(jp_ctx* c, const jp_obrs_desc* dout, float lambda_or_budget,
@@ -473,7 +482,7 @@ jp_status vshard_local_impl(jp_ctx* c, const jp_obrs_desc* d, const void* za, co
     e = launch_vshard_localize(d->T, tokens, mask, vocab_offset, d->V, V_total, 0, c->vtok, c->vmask, c->sc, c->stream);
     if (e != cudaSuccess) return cuda_fail(c, e, "shard token launch");
     c->launches += 1;
-    if ((st = stream_rows(c, d, ld, k, 0, za, zp, c->vtok, c->vmask, false, false)) != JP_OK) return st;
+    if ((st = stream_rows(c, d, ld, k, 0, za, zp, c->vtok, c->vmask)) != JP_OK) return st;
     e = launch_vshard_export(d->T, k, c->rec, za, zp, ld, d->dtype, c->vtok, c->vmask, vocab_offset, dests, line0,
                              c->stream);
     if (e != cudaSuccess) return cuda_fail(c, e, "shard export launch");
@@ -528,6 +537,7 @@ jp_status jp_vshard_merge(jp_ctx* c, int n_shards, int my_shard, const float* ga
   c->vshard_local_done = false;
   c->batch_open = true;
   c->batch_exact = false;
+  c->rec_kl = false;             // the divergence needs whole rows
   c->rec_rows = T; c->rec_V = V_total; c->rec_k = k;
   return JP_OK;
 }
@@ -577,6 +587,28 @@ jp_status jp_obrs_apply_kappa(jp_ctx* c, double kappa, float c1, float* out_weig
   cudaError_t e = launch_reweight(c->rec_rows, c->rec, c->sc, kappa, c1, out_weight, c->stream);
   if (e != cudaSuccess) return cuda_fail(c, e, "reweight launch");
   if (c->rec_rows > 0) c->launches += 1;
+  return JP_OK;
+}
+
+jp_status jp_batch_totals(jp_ctx* c, double* out_totals) {
+  if (!c) return JP_ERR_INVALID_ARG;
+  if (!c->have_records) return fail(c, JP_ERR_STATE, "no forward records in this context: run the forward (or finalize the batch) first");
+  if (!out_totals) return fail(c, JP_ERR_INVALID_ARG, "out_totals is NULL");
+  cudaSetDevice(c->device);
+  cudaError_t e = cudaMemcpyAsync(out_totals, c->sc->totals, 4 * sizeof(double), cudaMemcpyDeviceToDevice, c->stream);
+  if (e != cudaSuccess) return cuda_fail(c, e, "cudaMemcpyAsync(totals)");
+  return JP_OK;
+}
+
+jp_status jp_obrs_apply_totals(jp_ctx* c, const double* totals, float c1, float* out_weight, jp_stats* out_stats) {
+  if (!c) return JP_ERR_INVALID_ARG;
+  if (!c->have_records) return fail(c, JP_ERR_STATE, "no forward records in this context: run the forward (or finalize the batch) first");
+  if (!totals) return fail(c, JP_ERR_INVALID_ARG, "totals is NULL");
+  if (!out_weight && c->rec_rows > 0) return fail(c, JP_ERR_INVALID_ARG, "out_weight is NULL");
+  cudaSetDevice(c->device);
+  cudaError_t e = launch_reweight_totals(c->rec_rows, c->rec, c->sc, totals, c1, out_weight, out_stats, c->stream);
+  if (e != cudaSuccess) return cuda_fail(c, e, "reweight launch");
+  c->launches += 1;
   return JP_OK;
 }
 

@@ -89,7 +89,7 @@ __global__ void __launch_bounds__(GNT, GCTAS_PER_SM) grad_kernel(GradArgs A) {
     const int64_t rrow = A.record_offset + row;
     uint4* oa = (uint4*)((char*)A.d_actor + row * A.ld * 2);
     uint4* op = (uint4*)((char*)A.d_policy + row * A.ld * 2);
-    bool valid = (A.mask == nullptr || A.mask[row] != 0) && A.rec.flag[rrow] != 0 && g_over_n != 0.f;
+    bool valid = (A.mask == nullptr || A.mask[row] != 0) && A.rec.flag[rrow] == kRowValid && g_over_n != 0.f;
     const int64_t x = A.tokens[row];
     if (!valid) {
       if (tid == 0) {
@@ -126,10 +126,11 @@ __global__ void __launch_bounds__(GNT, GCTAS_PER_SM) grad_kernel(GradArgs A) {
         if (A.tis_cap > 0.f) F = fmin(F, (double)A.tis_cap);
       }
       const double s_o = ppo_surrogate(r_o, (double)adv, A.clip, (double)A.eps_lo, (double)A.eps_hi, &slope_o);
-      cp = (float)(-(double)g_over_n * m * rho * slope_t * r_t);
+      // (a rejected token contributes nothing, whatever its ratios: p_new(a_t) = 0 makes rho infinite)
+      cp = m != 0.0 ? (float)(-(double)g_over_n * rho * slope_t * r_t) : 0.f;
       ca = (float)(-(double)g_over_n * F * slope_o * r_o);
       if (tid == 0) {
-        if (A.out_obj_policy) A.out_obj_policy[row] = (float)(m * rho * s_t);
+        if (A.out_obj_policy) A.out_obj_policy[row] = m != 0.0 ? (float)(rho * s_t) : 0.f;
         if (A.out_obj_actor) A.out_obj_actor[row] = (float)(F * s_o);
       }
     }

@@ -22,7 +22,10 @@ struct Records {
   float* zk;        // [cap] Z_approx (or exact Z when k >= V)
   float* zx;        // [cap] exact Z when asked for beside Z_approx
   float* a;         // [cap] acceptance probability
-  uint8_t* flag;    // [cap] 1 = valid row with records, 0 = masked / bad / never streamed
+  float* kl;        // [cap] KL(p_target || p_inf) of the row, when the caller asked for it
+  uint8_t* flag;    // [cap] 1 = valid row with records, 0 = masked / bad token / never streamed,
+                    //       2 = streamed, but a log-sum-exp or a log-prob of the sampled token is not finite:
+                    //       counted in n_nonfinite and otherwise treated as masked
   double* ratio;    // [cap] p(a_t)/q(a_t) in double, compacted, for the budget solve
   float* dval;      // [cap] lp - lq of the compacted valid rows
 };
@@ -34,19 +37,24 @@ struct Scalars {
   int32_t n_compact;       // number of valid rows found by the ratio kernel
   int32_t status;
   unsigned long long n_bad_token;
-  unsigned long long n_nonfinite;
   float lambda;            // lambda in use (fixed, or written by the budget solve)
   float pad;
   double lambda64;
+  double totals[4];        // the last forward's batch sums: N, accepted, sum of Z_approx, sum of a(x_t)
   jp_stats stats;          // the last forward's batch statistics
 };
+
+constexpr uint8_t kRowValid = 1;      // values of Records::flag
+constexpr uint8_t kRowNonFinite = 2;
 
 constexpr int kMaxPartials = 256;
 struct Partials {
   long long n_valid[kMaxPartials];
   long long n_accept[kMaxPartials];
+  long long n_nonfinite[kMaxPartials];
   double sum_zk[kMaxPartials];
   double sum_a[kMaxPartials];
+  double sum_kl[kMaxPartials];
 };
 
 struct StreamArgs {
@@ -78,7 +86,8 @@ struct ExactZArgs {
   int64_t record_offset;
   Records rec;
   Scalars* sc;
-  float* out;              // rec.zk or rec.zx
+  float* out;              // rec.zk or rec.zx; null = no exact Z in this pass
+  float* out_kl;           // rec.kl; null = no KL(p || q) in this pass
 };
 
 struct EpilogueArgs {
@@ -91,6 +100,7 @@ struct EpilogueArgs {
   Scalars* sc;
   Partials* part;
   int32_t n_part;
+  int32_t have_kl;         // rec.kl holds KL(p || q) of every valid row: sum it into the statistics
   // outputs, all [T] (any may be null)
   uint8_t* out_accept;
   float* out_weight;
@@ -153,6 +163,8 @@ cudaError_t launch_budget_solve(const EpilogueArgs& a, double budget, cudaStream
 cudaError_t launch_epilogue(const EpilogueArgs& a, cudaStream_t s, int* n_launch);
 cudaError_t launch_reweight(int64_t T, const Records& rec, const Scalars* sc, double kappa, float c1,
                             float* out_weight, cudaStream_t s);
+cudaError_t launch_reweight_totals(int64_t T, const Records& rec, Scalars* sc, const double* totals, float c1,
+                                   float* out_weight, jp_stats* out_stats, cudaStream_t s);
 cudaError_t launch_logprobs(int64_t T, const Records& rec, float* out_lq, float* out_lp, uint8_t* out_valid,
                             cudaStream_t s);
 cudaError_t launch_row_lambda(const RowLambdaArgs& a, cudaStream_t s, int sms);

@@ -51,39 +51,25 @@
 
 namespace jp {
 
-#ifndef JP_NC
-#define JP_NC 16
-#endif
-#ifndef JP_VPL
-#define JP_VPL 4
-#endif
-#ifndef JP_NG
-#define JP_NG 2
-#endif
-#ifndef JP_SAMPLE_VPL
-#define JP_SAMPLE_VPL 32
-#endif
-#ifndef JP_TAU_NS
-#define JP_TAU_NS 200
-#endif
-constexpr int NC = JP_NC;                 // consumer warps
-constexpr int NG = JP_NG;                 // consumer groups: a row's tiles go to them in turn, starting with first_group(row)
+constexpr int NC = 16;                    // consumer warps
+constexpr int NG = 2;                     // consumer groups: a row's tiles go to them in turn, starting with first_group(row)
 constexpr int WPT = NC / NG;              // warps that share one tile
-constexpr int VPL = JP_VPL;               // 16-byte vectors per lane per tensor per tile
+constexpr int VPL = 4;                    // 16-byte vectors per lane per tensor per tile
 constexpr int TV = WPT * 32 * VPL;        // vectors per tensor per tile
 constexpr int HV = 2;                     // vectors per tensor a lane holds at a time
-static_assert(JP_VPL % HV == 0, "a tile is taken in passes of HV vectors");
-static_assert(JP_NG == 2, "tiles go to consumer groups by parity; the producer keeps two phase masks");
+static_assert(VPL % HV == 0, "a tile is taken in passes of HV vectors");
+static_assert(NG == 2, "tiles go to consumer groups by parity; the producer keeps two phase masks");
 static_assert(NC % NG == 0, "consumer groups must divide the warps");
 constexpr int NSLOT = 4;                  // rows in flight between the consumers and the top-k warps
 constexpr int SCAP = 288;                 // keys a top-k warp buffers before it sorts them into the list
 constexpr int NB = 256;                   // histogram bins
 constexpr int TP = TV / HV;               // passes per tensor per tile
-constexpr int SAMPLE = 32 * JP_SAMPLE_VPL;  // vectors of a row its top-k warp looks at before the row starts
+constexpr int SAMPLE = 32 * 32;            // vectors of a row its top-k warp looks at before the row starts
 constexpr int NTOPK = NSLOT * 2;          // top-k warps: (slot, tensor)
 constexpr int NWARPS = 1 + NC + NTOPK;
 constexpr int NTHREADS = NWARPS * 32;
 constexpr long long kSpinLimit = 4000000000ll;   // clock cycles a wait may last (about 2 s)
+constexpr uint32_t kTauPollNs = 200u;     // how long a top-k warp sleeps between two looks at its row's candidates
 
 // NSTAGES: depth of the ring.  NCAND: candidate passes a row may collect before it
 // falls back to a re-scan.  The kernel for k <= 64 takes 5 stages and 1024 candidates;
@@ -126,6 +112,11 @@ __device__ __forceinline__ void mbar_init(unsigned long long* bar, uint32_t coun
 }
 __device__ __forceinline__ void mbar_arrive(unsigned long long* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// Arrival that cannot be issued before `dep` has been computed: the value is an input
+// of the statement, though the instruction does not use it.
+__device__ __forceinline__ void mbar_arrive_after(unsigned long long* bar, uint32_t dep) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];  // after %1" ::"r"(smem_u32(bar)), "r"(dep) : "memory");
 }
 __device__ __forceinline__ void mbar_arrive_expect_tx(unsigned long long* bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
@@ -267,37 +258,6 @@ struct Online {
   unsigned long long s2;
 };
 
-#ifndef JP_POLY_WORDS
-#define JP_POLY_WORDS 0
-#endif
-// 2^x for two x <= ~0 without the special-function unit, folded into the running
-// sums: returns s + 2^x (both lanes).  x is rounded to the nearest integer n with the
-// 1.5 * 2^23 trick, 2^(x - n) comes from a degree-5 polynomial on [-0.5, 0.5] (fitted
-// for the smallest maximum relative error, 1.7e-7, about that of ex2.approx) and 2^n
-// is built in the exponent field.  x is clamped at -125 so that the exponent stays
-// valid: terms below 2^-125 count as 2^-125, far below one ulp of any sum that holds
-// a term near 1.  A NaN stays a NaN.
-__device__ __forceinline__ unsigned long long add_exp2_poly2(unsigned long long s2, unsigned long long x2) {
-  float x0, x1;
-  unpack2(x2, x0, x1);
-  asm("max.NaN.f32 %0, %0, %1;" : "+f"(x0) : "f"(-125.f));
-  asm("max.NaN.f32 %0, %0, %1;" : "+f"(x1) : "f"(-125.f));
-  x2 = pack2(x0, x1);
-  const unsigned long long t2 = fadd2(x2, pack2(12582912.f, 12582912.f));
-  const unsigned long long n2 = fadd2(t2, pack2(-12582912.f, -12582912.f));
-  const unsigned long long f2 = ffma2(n2, pack2(-1.f, -1.f), x2);
-  unsigned long long p2 = ffma2(pack2(1.326462603e-03f, 1.326462603e-03f), f2, pack2(9.671481326e-03f, 9.671481326e-03f));
-  p2 = ffma2(p2, f2, pack2(5.550733581e-02f, 5.550733581e-02f));
-  p2 = ffma2(p2, f2, pack2(2.402224243e-01f, 2.402224243e-01f));
-  p2 = ffma2(p2, f2, pack2(6.931470037e-01f, 6.931470037e-01f));
-  p2 = ffma2(p2, f2, pack2(1.f, 1.f));
-  float t0, t1;
-  unpack2(t2, t0, t1);
-  const float sc0 = __int_as_float((__float_as_int(t0) << 23) + 0x3f800000);
-  const float sc1 = __int_as_float((__float_as_int(t1) << 23) + 0x3f800000);
-  return ffma2(p2, pack2(sc0, sc1), s2);
-}
-
 // Makes sure the reference exponent covers a maximum vm: moves it (and the sums,
 // by an exact power of two) when vm is beyond the limit.
 __device__ __forceinline__ void raise_max(float vm, Online& o) {
@@ -323,15 +283,9 @@ __device__ __forceinline__ void add_terms(const uint4& v, Online& o) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       unsigned long long a = ffma2(pack2(__uint_as_float(w[i] << 16), __uint_as_float(w[i] & 0xffff0000u)), L2, nm2);
-      if (i >= 4 - JP_POLY_WORDS) {
-        // a share of the exponentials runs on the FMA pipe: one ex2 per logit would
-        // saturate the special-function unit before HBM
-        o.s2 = add_exp2_poly2(o.s2, a);
-      } else {
-        float a0, a1;
-        unpack2(a, a0, a1);
-        o.s2 = fadd2(o.s2, pack2(ex2_approx(a0), ex2_approx(a1)));
-      }
+      float a0, a1;
+      unpack2(a, a0, a1);
+      o.s2 = fadd2(o.s2, pack2(ex2_approx(a0), ex2_approx(a1)));
     }
   } else {
     unsigned long long a = ffma2(pack2(__uint_as_float(v.x), __uint_as_float(v.y)), L2, nm2);
@@ -349,6 +303,22 @@ template <int DT>
 __device__ __forceinline__ void accumulate(const uint4& v, float vm, Online& o) {
   raise_max(vm, o);
   add_terms<DT>(v, o);
+}
+
+// Hands a ring stage back to the producer once this warp has consumed its part of the tile.
+// The stage may be overwritten (by the copy engine) as soon as the arrival is counted, so
+// every shared-memory load of the tile must have returned its value by then.  That is made
+// a data dependence rather than a matter of instruction order: the running sums take in
+// every loaded word, the vote below takes in the sums of all 32 lanes, and the arrival takes
+// the vote's result as an operand.  A load whose value has been consumed has been performed,
+// and the arrival (release) / the producer's wait (acquire) order the copy after it.
+// (An arrival placed right after the loads was seen to overtake one that was still queued
+// behind a burst of shared-memory atomics: the lane then read the next tile's bytes.)
+__device__ __forceinline__ void release_stage(unsigned long long* empty_bar, const Online& oa, const Online& op,
+                                              int lane) {
+  const uint32_t mix = (uint32_t)oa.s2 ^ (uint32_t)(oa.s2 >> 32) ^ (uint32_t)op.s2 ^ (uint32_t)(op.s2 >> 32);
+  const uint32_t vote = __ballot_sync(0xffffffffu, mix == 0x7fc00001u);   // any predicate of the sums will do
+  if (lane == 0) mbar_arrive_after(empty_bar, vote);
 }
 
 // The ragged end of a row (fewer than one 16-byte vector) as a -inf padded vector.
@@ -915,11 +885,7 @@ __device__ void consumer_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int c
             if (mp >= tp) record_hit<CAP>(&sm.ncand[p][1], sm.cand[p][1], A.spill, 2 * p + 1, id, idmask, mp);
           }
         }
-        // Free the stage only now that arithmetic has consumed every loaded vector.  An arrival
-        // issued right after the last loads can overtake them: a load still queued behind a burst
-        // of shared-memory atomics was seen to return the next tile's bytes.
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sm.empty[s]);
+        release_stage(&sm.empty[s], oa, op, lane);
       } else {
         // the row's last, partial tile: bounds checked
         const uint32_t v0 = tile * TV + wq * 32 + lane;
@@ -943,8 +909,7 @@ __device__ void consumer_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int c
             if (mp >= tp) record_hit<CAP>(&sm.ncand[p][1], sm.cand[p][1], A.spill, 2 * p + 1, id, idmask, mp);
           }
         }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sm.empty[s]);
+        release_stage(&sm.empty[s], oa, op, lane);
       }
       return true;
     };
@@ -1054,7 +1019,7 @@ __device__ void topk_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int t, in
     // while the row streams: raise tau to the highest bin with k candidates at or above it
     {
       long long t0 = 0;
-      for (uint32_t i = 0; !mbar_try_wait_for(&sm.row_done[p], ph, (uint32_t)JP_TAU_NS); ++i) {
+      for (uint32_t i = 0; !mbar_try_wait_for(&sm.row_done[p], ph, kTauPollNs); ++i) {
         if (TOPK) {
           const uint32_t nc = lds_volatile_u32(&sm.ncand[p][t]);
           const uint32_t n = nc < (uint32_t)CAP ? nc : (uint32_t)CAP;
@@ -1157,9 +1122,8 @@ __device__ void topk_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int t, in
       const float lsef = (float)lse;
       const float lpx = (float)((double)zx - lse);
       const float lo = (float)(lse - (double)lsef);
-      if (t == 0) { A.rec.lse_a[rrow] = lsef; A.rec.lse_a_lo[rrow] = lo; A.rec.lq[rrow] = lpx; A.rec.flag[rrow] = 1; }
+      if (t == 0) { A.rec.lse_a[rrow] = lsef; A.rec.lse_a_lo[rrow] = lo; A.rec.lq[rrow] = lpx; A.rec.flag[rrow] = kRowValid; }
       else        { A.rec.lse_p[rrow] = lsef; A.rec.lse_p_lo[rrow] = lo; A.rec.lp[rrow] = lpx; }
-      if (!isfinite(lsef)) atomicAdd(&A.sc->n_nonfinite, 1ull);
     }
     __syncwarp();
   }
@@ -1253,18 +1217,29 @@ __device__ __forceinline__ void load_tile(uint4 (&va)[XUNROLL], uint4 (&vp)[XUNR
   }
 }
 
-// Exact normaliser: Z_t = sum_v min(q_t(v), p_t(v)/lambda), one more pass over the
-// row with the log-sum-exps known (Eq. obrs_dist; Appendix A, Z_C).
-template <int DT>
+// One more pass over the rows with the log-sum-exps known.
+//   WANT_Z : the exact normaliser Z_t = sum_v min(q_t(v), p_t(v) / lambda) (Eq. obrs_dist;
+//            Appendix A, Z_C)
+//   WANT_KL: KL(p_t || q_t) = sum_v p_t(v) (zp_v - za_v) - lse_p + lse_a, the divergence
+//            between target and rollout distribution that the paper tracks during training
+// Exponents are taken relative to integers M near lse log2(e), so that the fused
+// multiply-add z log2(e) - M is rounded once and the fractional remainder is a factor
+// common to the row, applied in double at the end.  The remainder also carries the share
+// of the fp32 constant's shortfall (log2(e) - kLog2e) that matters, taken at z = lse, where
+// the terms that dominate the sums lie.
+template <int DT, bool WANT_Z, bool WANT_KL>
 __global__ void __launch_bounds__(XNT, XCTAS_PER_SM) exact_z_kernel(ExactZArgs A) {
-  __shared__ float red[XNWARP];
+  __shared__ float red[2][XNWARP];
   __shared__ int s_row;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   constexpr int N = Vec<DT>::N;
+  constexpr double kLog2e64 = 1.4426950408889634074;
+  const double kLog2eShort = kLog2e64 - (double)kLog2e;      // what the fp32 constant lacks
   const int64_t nvec = A.V / N;
   const int tail = (int)(A.V - nvec * N);
   const int64_t nvt = nvec + (tail > 0 ? 1 : 0);
-  const float log2_lambda = log2f(A.sc->lambda);
+  const double lambda = WANT_Z ? (double)A.sc->lambda : 1.0;
+  const double log2_lambda = log2(lambda);
   for (;;) {
     if (tid == 0) s_row = atomicAdd(&A.sc->row_counter2, 1);
     __syncthreads();
@@ -1272,15 +1247,25 @@ __global__ void __launch_bounds__(XNT, XCTAS_PER_SM) exact_z_kernel(ExactZArgs A
     __syncthreads();
     if (row >= A.T) break;
     const int64_t rrow = A.record_offset + row;
-    if (!A.rec.flag[rrow]) {
-      if (tid == 0) A.out[rrow] = 0.f;
+    if (A.rec.flag[rrow] != kRowValid) {
+      if (tid == 0) {
+        if (WANT_Z) A.out[rrow] = 0.f;
+        if (WANT_KL) A.out_kl[rrow] = 0.f;
+      }
       continue;
     }
     const char* ra = (const char*)A.za + row * A.ld * Vec<DT>::ESIZE;
     const char* rp = (const char*)A.zp + row * A.ld * Vec<DT>::ESIZE;
-    const float ca = A.rec.lse_a[rrow] * kLog2e;
-    const float cp = A.rec.lse_p[rrow] * kLog2e + log2_lambda;
-    float acc = 0.f;
+    const double lse_a = (double)A.rec.lse_a[rrow] + (double)A.rec.lse_a_lo[rrow];
+    const double lse_p = (double)A.rec.lse_p[rrow] + (double)A.rec.lse_p_lo[rrow];
+    const double ca = lse_a * kLog2e64, cp = lse_p * kLog2e64 + log2_lambda;
+    // the clamp keeps M an integer that fp32 holds exactly; rows that far out are non-finite anyway
+    const float Ma = (float)rint(fmin(fmax(ca, -16777216.0), 16777216.0));
+    const float Mp = (float)rint(fmin(fmax(cp, -16777216.0), 16777216.0));
+    const double fq = exp2(((double)Ma - ca) + lse_a * kLog2eShort);     // q = fq 2^(za kLog2e - Ma)
+    const double fp = exp2(((double)Mp - cp) + lse_p * kLog2eShort);     // p / lambda = fp 2^(zp kLog2e - Mp)
+    const float ratio = (float)(fp / fq);
+    float acc = 0.f, kl = 0.f;
     for (int64_t v0 = 0; v0 < nvt; v0 += (int64_t)XNT * XUNROLL) {
       uint4 va[XUNROLL], vp[XUNROLL];
       load_tile<DT>(va, vp, ra, rp, v0, nvec, tail, tid);
@@ -1288,20 +1273,28 @@ __global__ void __launch_bounds__(XNT, XCTAS_PER_SM) exact_z_kernel(ExactZArgs A
       for (int j = 0; j < XUNROLL; ++j) {
 #pragma unroll
         for (int e = 0; e < N; ++e) {
-          float q = ex2_approx(fmaf(Vec<DT>::get(va[j], e), kLog2e, -ca));
-          float p = ex2_approx(fmaf(Vec<DT>::get(vp[j], e), kLog2e, -cp));
-          acc += fminf(q, p);
+          const float za = Vec<DT>::get(va[j], e), zp = Vec<DT>::get(vp[j], e);
+          const float p = ex2_approx(fmaf(zp, kLog2e, -Mp));
+          if (WANT_Z) {
+            const float q = ex2_approx(fmaf(za, kLog2e, -Ma));
+            acc += fminf(q, p * ratio);
+          }
+          if (WANT_KL && p > 0.f) kl = fmaf(p, zp - za, kl);
         }
       }
     }
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-    if (lane == 0) red[warp] = acc;
+    for (int off = 16; off > 0; off >>= 1) {
+      acc += __shfl_xor_sync(0xffffffffu, acc, off);
+      kl += __shfl_xor_sync(0xffffffffu, kl, off);
+    }
+    if (lane == 0) { red[0][warp] = acc; red[1][warp] = kl; }
     __syncthreads();
     if (tid == 0) {
-      double S = 0.0;
-      for (int w = 0; w < XNWARP; ++w) S += (double)red[w];
-      A.out[rrow] = (float)S;
+      double S = 0.0, K = 0.0;
+      for (int w = 0; w < XNWARP; ++w) { S += (double)red[0][w]; K += (double)red[1][w]; }
+      if (WANT_Z) A.out[rrow] = (float)(S * fq);
+      if (WANT_KL) A.out_kl[rrow] = (float)(K * fp * lambda - lse_p + lse_a);
     }
     __syncthreads();
   }
@@ -1347,12 +1340,19 @@ cudaError_t launch_stream(const StreamArgs& a, cudaStream_t s, int sms) {
   }
 }
 
+template <int DT>
+static void launch_exact_z_dt(const ExactZArgs& a, int g, cudaStream_t s) {
+  if (a.out && a.out_kl) exact_z_kernel<DT, true, true><<<g, XNT, 0, s>>>(a);
+  else if (a.out) exact_z_kernel<DT, true, false><<<g, XNT, 0, s>>>(a);
+  else exact_z_kernel<DT, false, true><<<g, XNT, 0, s>>>(a);
+}
+
 cudaError_t launch_exact_z(const ExactZArgs& a, cudaStream_t s, int sms) {
-  if (a.T <= 0) return cudaSuccess;
+  if (a.T <= 0 || (!a.out && !a.out_kl)) return cudaSuccess;
   const int grid = sms * XCTAS_PER_SM;
   int g = (int)(a.T < grid ? a.T : grid);
-  if (a.dtype == JP_BF16) exact_z_kernel<JP_BF16><<<g, XNT, 0, s>>>(a);
-  else exact_z_kernel<JP_F32><<<g, XNT, 0, s>>>(a);
+  if (a.dtype == JP_BF16) launch_exact_z_dt<JP_BF16>(a, g, s);
+  else launch_exact_z_dt<JP_F32>(a, g, s);
   return cudaGetLastError();
 }
 

@@ -55,7 +55,7 @@ __global__ void __launch_bounds__(VS_NT) vshard_export_kernel(int64_t T, int k, 
   auto put = [&](int64_t w, float v) {
     for (int p = 0; p < dests.n; ++p) dests.dst[p][o + w] = v;
   };
-  const bool flag = rec.flag[r] != 0;
+  const bool flag = rec.flag[r] != 0;      // a non-finite slice travels as it is: the merged row is then non-finite too
   if (lane == 0) {
     const bool owner = flag && mask_local[r] == 2;
     float xa = 0.f, xp = 0.f;
@@ -178,11 +178,7 @@ __global__ void __launch_bounds__(VS_NT) vshard_merge_kernel(int n_shards, int m
       rec.lse_p[r] = lpf; rec.lse_p_lo[r] = (float)(lp - (double)lpf);
       rec.lq[r] = (float)(xa - la);
       rec.lp[r] = (float)(xp - lp);
-      rec.flag[r] = 1;
-      // a row that only another shard found non-finite counts here as well
-      const float* mine = line(my_shard);
-      if ((!isfinite(laf) || !isfinite(lpf)) && isfinite(mine[2]) && isfinite(mine[4]))
-        atomicAdd(&sc->n_nonfinite, 1ull);
+      rec.flag[r] = kRowValid;      // a non-finite merged row is found and counted by the finalize step
     }
   }
 }

@@ -4,9 +4,11 @@ Token rows are independent (rejection is per token), so a batch shards over
 ranks by contiguous row ranges and every rank streams its own rows.  The
 accept draw of a row is keyed on its global index (desc.token_offset), so the
 decisions do not depend on how the batch was split.  The one batch-wide
-quantity is the calibration factor kappa (Section 4.4.2): 24 bytes per rank,
-summed with one all-reduce, after which every rank rewrites its weights with
-jp_obrs_apply_kappa.  Nothing here does arithmetic on per-token data.
+quantity is the calibration factor kappa (Section 4.4.2): the library writes a
+shard's four batch sums to device memory (jp_batch_totals), one all-reduce adds
+them up (32 bytes per rank), and the library forms kappa from the sums and
+rewrites the shard's weights (jp_obrs_apply_totals).  Nothing here does any of
+the method's arithmetic.
 """
 from __future__ import annotations
 
@@ -23,28 +25,23 @@ def shard_rows(T: int, world: int, rank: int):
     return lo, lo + q + (1 if rank < r else 0)
 
 
-def batch_totals(stats: dict) -> torch.Tensor:
-    """The three sums kappa is made of, from one shard's jp_stats (float64; counts below 2^53 are exact)."""
-    n = float(stats["n_valid"])
-    return torch.tensor([n, float(stats["n_accept"]), n * float(stats["z_approx_mean"])], dtype=torch.float64)
-
-
-def kappa_from_totals(tot) -> float:
-    n, acc, szk = (float(x) for x in tot)
-    if n <= 0 or szk <= 0:
-        return 1.0
-    return (acc / n) / (szk / n)
-
-
-def global_kappa(stats: dict, group=None, device=None) -> tuple[float, torch.Tensor]:
-    """All-reduces the shard totals; returns (kappa of the whole batch, the summed totals)."""
-    tot = batch_totals(stats)
-    if device is not None:
-        tot = tot.to(device)
+def all_reduce_totals(totals: torch.Tensor, group=None) -> torch.Tensor:
+    """Sums the shards' batch totals (the four doubles jp_batch_totals writes) over the ranks, in place."""
     if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
-        dist.all_reduce(tot, op=dist.ReduceOp.SUM, group=group)
-    tot = tot.cpu()
-    return kappa_from_totals(tot), tot
+        dist.all_reduce(totals, op=dist.ReduceOp.SUM, group=group)
+    return totals
+
+
+def apply_global_kappa(ctx, out_weight: torch.Tensor, c1: float = 0.0, group=None, out_stats=None) -> torch.Tensor:
+    """After every rank's forward on its shard: exchanges the batch totals (32 bytes, one all-reduce on
+    device memory) and lets the library form the batch-wide kappa and rewrite this shard's weights
+    (jp_batch_totals -> all-reduce -> jp_obrs_apply_totals).  Returns the summed totals (device)."""
+    from . import binding as B
+    totals = torch.empty(4, dtype=torch.float64, device=out_weight.device)
+    B.jp_batch_totals(ctx, totals)
+    all_reduce_totals(totals, group)
+    B.jp_obrs_apply_totals(ctx, totals, c1, out_weight, out_stats)
+    return totals
 
 
 def max_over_ranks(value: float, group=None, device=None) -> float:

@@ -52,6 +52,12 @@ def check_forward(out, ref, k, V, mask=None, c1=0.0, exact_too=False):
         assert np.array_equal(g["topk_idx_actor"][valid], ref["topk_idx_a"][valid])
         assert np.array_equal(g["topk_idx_policy"][valid], ref["topk_idx_p"][valid])
         assert np.all(g["topk_idx_actor"][~valid] == -1)
+        # the published values are the rows' own logits at the published indices, widened exactly
+        za_h, zp_h = ref.get("za_f32"), ref.get("zp_f32")
+        if za_h is not None:
+            rows = np.nonzero(valid)[0][:, None]
+            assert np.array_equal(g["topk_val_actor"][valid], za_h[rows, ref["topk_idx_a"][valid]])
+            assert np.array_equal(g["topk_val_policy"][valid], zp_h[rows, ref["topk_idx_p"][valid]])
     assert np.array_equal(g["uniform"], ref["u"])
     close(g["accept_prob"], ref["a"])
     diff = g["accept"] != ref["accept"]
@@ -86,6 +92,7 @@ def run_case(ctx, za, zp, tok, mask=None, *, lam=None, budget=None, k, seed, c1=
     m = None if mask is None else mask.cpu().numpy()
     ref = oracle.forward(to_numpy_bits(za), to_numpy_bits(zp), tok.cpu().numpy(), m, lam=lam, budget=budget,
                          k=k, seed=seed, c1=c1, token_offset=token_offset, exact=exact_too)
+    ref["za_f32"], ref["zp_f32"] = za.float().cpu().numpy(), zp.float().cpu().numpy()   # exact widening
     if budget is not None:
         # lambda parity first, then everything else with lambda forced to the oracle's value so
         # that a last-bit difference in lambda cannot leak into the accept bits
@@ -253,6 +260,7 @@ def test_chunked_batch_matches_monolithic_and_oracle(ctx):
     ch = runner.forward_chunked(ctx, chunks, T, V, B.JP_BF16, budget=0.6, k=k, seed=5, aux=True)
     for n in ("accept", "weight", "logp_actor", "logp_policy", "z_approx", "uniform", "topk_idx_actor"):
         assert torch.equal(mono[n], ch[n]), n
+    assert mono["stats"]["mean_kl_p_q"] is None            # not asked for
     assert mono["stats"] == ch["stats"]
     ref = oracle.forward(to_numpy_bits(za), to_numpy_bits(zp), tok.cpu().numpy(), mask.cpu().numpy(),
                          budget=0.6, k=k, seed=5)
@@ -306,18 +314,28 @@ def test_row_shards_with_a_batch_wide_kappa_match_the_undivided_batch(ctx):
     mask = (torch.arange(T, device="cuda") % 4 != 1).to(torch.uint8)
     whole = runner.forward(ctx, za, zp, tok, mask, lam=1.4, k=k, seed=3, c1=2.5)
     ctxs = [B.Context(0), B.Context(0)]
-    outs, tot = [], torch.zeros(3, dtype=torch.float64)
+    outs, tot = [], torch.zeros(4, dtype=torch.float64, device="cuda")
     for rank, c in enumerate(ctxs):
         lo, hi = parallel.shard_rows(T, 2, rank)
         o = runner.forward(c, za[lo:hi], zp[lo:hi], tok[lo:hi], mask[lo:hi], lam=1.4, k=k, seed=3, c1=2.5,
                            token_offset=lo)
         outs.append(o)
-        tot += parallel.batch_totals(o["stats"])
-    kappa = parallel.kappa_from_totals(tot)
-    close(kappa, whole["stats"]["kappa"], rtol=1e-12)
+        t = torch.empty(4, dtype=torch.float64, device="cuda")
+        B.jp_batch_totals(c, t)
+        tot += t                                  # what the all-reduce over the ranks does
+    gstats = []
     for c, o in zip(ctxs, outs):
-        B.jp_obrs_apply_kappa(c, kappa, 2.5, o["weight"])
+        sb = B.new_stats_buffer("cuda")
+        B.jp_obrs_apply_totals(c, tot, 2.5, o["weight"], sb)
+        gstats.append(sb)
     torch.cuda.synchronize()
+    for sb in gstats:                             # every shard ends with the undivided batch's statistics
+        gs = B.read_stats(sb)
+        close(gs["kappa"], whole["stats"]["kappa"], rtol=1e-12)
+        assert gs["n_valid"] == whole["stats"]["n_valid"] and gs["n_accept"] == whole["stats"]["n_accept"]
+        close(gs["z_approx_mean"], whole["stats"]["z_approx_mean"], rtol=1e-12)
+        close(gs["mean_accept_prob"], whole["stats"]["mean_accept_prob"], rtol=1e-12)
+    kappa = B.read_stats(gstats[0])["kappa"]
     assert torch.equal(torch.cat([o["accept"] for o in outs]), whole["accept"])
     w = torch.cat([o["weight"] for o in outs])
     assert torch.equal(w, whole["weight"])
@@ -354,7 +372,7 @@ def test_row_shards_in_budget_mode_share_one_lambda(ctx):
     # what the all-gather would hand to every rank
     lam = parallel.solve_on_device(torch.cat(lqs), torch.cat(lps), torch.cat(vs), budget)
     close(lam, whole["stats"]["lambda_used"], rtol=1e-6)
-    outs, tot = [], torch.zeros(3, dtype=torch.float64)
+    outs, tot = [], torch.zeros(4, dtype=torch.float64, device="cuda")
     for (lo, hi), c in zip(shards, ctxs):
         n = hi - lo
         o = runner._alloc_outputs(n, "cuda")
@@ -366,11 +384,14 @@ def test_row_shards_in_budget_mode_share_one_lambda(ctx):
         torch.cuda.synchronize()
         o["stats"] = B.read_stats(o["stats_buf"])
         outs.append(o)
-        tot += parallel.batch_totals(o["stats"])
-    kappa = parallel.kappa_from_totals(tot)
+        t = torch.empty(4, dtype=torch.float64, device="cuda")
+        B.jp_batch_totals(c, t)
+        tot += t
+    sb = B.new_stats_buffer("cuda")
     for c, o in zip(ctxs, outs):
-        B.jp_obrs_apply_kappa(c, kappa, 2.5, o["weight"])
+        B.jp_obrs_apply_totals(c, tot, 2.5, o["weight"], sb)
     torch.cuda.synchronize()
+    kappa = B.read_stats(sb)["kappa"]
     if float(np.float32(lam)) == float(np.float32(whole["stats"]["lambda_used"])):
         assert torch.equal(torch.cat([o["accept"] for o in outs]), whole["accept"])
         close(kappa, whole["stats"]["kappa"], rtol=1e-9)
@@ -426,27 +447,96 @@ def test_large_magnitude_logits(ctx):
     assert np.array_equal(out["topk_idx_actor"].cpu().numpy(), ref["topk_idx_a"])
     assert np.array_equal(out["topk_idx_policy"].cpu().numpy(), ref["topk_idx_p"])
     close(out["z_approx"].cpu().numpy(), ref["zk"])
+    # the normalisers and the weights hang on exp(z - lse): a log-sum-exp held in one fp32 word would
+    # put ulp(1500)/2 = 6e-5 on every one of them
+    flips, out, ref = run_case(ctx, za, zp, tok, lam=1.0, k=k, seed=1, exact_too=True)
+    flips, out, ref = run_case(ctx, za, zp, tok, lam=0.7, k=V, seed=1)
 
 
 def test_nonfinite_rows_are_counted_and_do_not_disturb_the_others(ctx):
-    """+inf and NaN logits: the row is counted in n_nonfinite and its results are unspecified; nothing
-    traps or waits, and every other row is what it would be without them."""
+    """+inf and NaN logits, and a sampled token of probability 0: the row is counted in n_nonfinite and
+    treated as masked; nothing traps or waits, and every other row, the batch statistics, kappa, the
+    weights and a budget-derived lambda are what they are with those rows masked out."""
     T, V, k = 64, 30000, 8
     r = LogitRecipe(T=T, V=V, dtype="bf16", sigma0=2.5, peaks=4, sigma=1.0, seed=63)
     za, zp, tok = make_logits(r, "cuda")
-    clean = runner.forward(ctx, za, zp, tok, None, lam=1.3, k=k, seed=2)
     za2, zp2 = za.clone(), zp.clone()
     za2[5, 100] = float("inf")
     zp2[9, 29999] = float("nan")
     za2[20, :] = float("nan")
-    out = runner.forward(ctx, za2, zp2, tok, None, lam=1.3, k=k, seed=2)
-    st = out["stats"]
-    assert st["status"] == 0 and st["n_nonfinite"] >= 3
+    zp2[31, :] = float("nan")
+    za2[31, 7] = float("nan")
+    za2[40, int(tok[40])] = float("-inf")          # the sampled token has probability 0 under the actor
+    bad_rows = [5, 9, 20, 31, 40]
     good = torch.ones(T, dtype=torch.bool, device="cuda")
-    good[[5, 9, 20]] = False
-    for n in ("logp_actor", "logp_policy", "lse_actor", "lse_policy", "z_approx", "accept_prob", "uniform",
-              "topk_idx_actor", "topk_idx_policy"):
-        assert torch.equal(out[n][good], clean[n][good]), n
+    good[bad_rows] = False
+    mask = good.to(torch.uint8)
+    names = ("logp_actor", "logp_policy", "lse_actor", "lse_policy", "z_approx", "accept_prob", "uniform",
+             "topk_idx_actor", "topk_idx_policy", "accept", "weight")
+    for kw in (dict(lam=1.3), dict(budget=0.55)):
+        for kk in (k, V):
+            clean = runner.forward(ctx, za, zp, tok, mask, k=kk, seed=2, c1=4.0, **kw)
+            out = runner.forward(ctx, za2, zp2, tok, None, k=kk, seed=2, c1=4.0, **kw)
+            st, cs = out["stats"], clean["stats"]
+            assert st["status"] == 0 and st["n_nonfinite"] == len(bad_rows) and cs["n_nonfinite"] == 0
+            for n in ("n_valid", "n_accept", "alpha_hat", "mean_accept_prob", "z_approx_mean", "kappa", "lambda_used"):
+                assert st[n] == cs[n], (n, st[n], cs[n])
+            for n in names:
+                if n in out:
+                    assert torch.equal(out[n][good], clean[n][good]), n
+            assert out["weight"][~good].abs().sum().item() == 0 and out["accept"][~good].sum().item() == 0
+            assert out["accept_prob"][~good].abs().sum().item() == 0 and out["z_approx"][~good].abs().sum().item() == 0
+    # and against the oracle with those rows masked
+    out = runner.forward(ctx, za2, zp2, tok, None, lam=1.3, k=k, seed=2)
+    ref = oracle.forward(to_numpy_bits(za), to_numpy_bits(zp), tok.cpu().numpy(), mask.cpu().numpy(), lam=1.3, k=k,
+                         seed=2)
+    check_forward(out, ref, k, V, mask.cpu().numpy())
+    # the gradient rows of such a row are zero
+    da, dp = runner.backward(ctx, za2, zp2, tok, None, out["accept"], out["weight"], lambda_distill=1.0)
+    torch.cuda.synchronize()
+    assert da[~good].float().abs().sum().item() == 0 and dp[~good].float().abs().sum().item() == 0
+    assert torch.isfinite(da[good].float()).all() and torch.isfinite(dp[good].float()).all()
+
+
+def test_mean_kl_statistic_on_request(ctx):
+    """jp_stats.mean_kl_p_q: the batch mean of KL(p_target || p_inf) per row (the actor-policy divergence
+    the paper tracks during training), computed by one more pass when the descriptor asks for it, NaN
+    otherwise; monolithic, chunked, and in exact mode."""
+    T, V, k = 300, 20008, 12
+    r = LogitRecipe(T=T, V=V, dtype="bf16", sigma0=2.5, peaks=4, sigma=1.1, seed=65)
+    za, zp, tok = make_logits(r, "cuda")
+    mask = (torch.arange(T, device="cuda") % 6 != 2).to(torch.uint8)
+    ref = oracle.forward(to_numpy_bits(za), to_numpy_bits(zp), tok.cpu().numpy(), mask.cpu().numpy(), lam=1.2, k=k,
+                         seed=4, want_kl=True)
+    o = runner._alloc_outputs(T, "cuda")
+
+    def run(kk, flags, **kw):
+        mode = B.JP_LAMBDA_FROM_BUDGET if "budget" in kw else B.JP_LAMBDA_FIXED
+        d = B.make_desc(za, flags=flags, lambda_mode=mode)
+        B.jp_obrs_forward(ctx, d, za, zp, tok, mask, kw.get("budget", kw.get("lam")), kk, 4, o["accept"], o["weight"],
+                          o["logp_actor"], o["logp_policy"], o["stats_buf"])
+        torch.cuda.synchronize()
+        return B.read_stats(o["stats_buf"])
+
+    assert run(k, 0, lam=1.2)["mean_kl_p_q"] is None
+    for st in (run(k, B.JP_DESC_KL, lam=1.2), run(V, B.JP_DESC_KL, lam=1.2), run(k, B.JP_DESC_KL, budget=0.6),
+               run(V, B.JP_DESC_KL, budget=0.6)):
+        close(st["mean_kl_p_q"], ref["stats"]["mean_kl_p_q"], rtol=1e-4, atol=5e-6)
+    # chunked: reported only if every chunk asked
+    for flags_last, want in ((B.JP_DESC_KL, True), (0, False)):
+        B.jp_batch_begin(ctx, T, V, B.JP_BF16, k, 0.0)
+        for off in range(0, T, 100):
+            fl = B.JP_DESC_KL if off < 200 else flags_last
+            B.jp_batch_chunk(ctx, B.make_desc(za[off:off + 100], token_offset=off, flags=fl), za[off:off + 100],
+                             zp[off:off + 100], tok[off:off + 100], mask[off:off + 100])
+        B.jp_batch_finalize(ctx, B.jp_obrs_desc(), 1.2, B.JP_LAMBDA_FIXED, 4, o["accept"], o["weight"],
+                            o["logp_actor"], o["logp_policy"], o["stats_buf"])
+        torch.cuda.synchronize()
+        got = B.read_stats(o["stats_buf"])["mean_kl_p_q"]
+        if want:
+            close(got, ref["stats"]["mean_kl_p_q"], rtol=1e-4, atol=5e-6)
+        else:
+            assert got is None
 
 
 def test_host_buffer_entry_point_equals_the_device_path(ctx):

@@ -1,9 +1,10 @@
 """GPU parity of jp_obrs_row_lambda (Theorem 3.4 per distribution) against the oracle.
 
-Bars: lambda_t within rtol 5e-5 of the oracle's exact sort-based solve (the GPU solves
-Z(lambda) = budget in fp32 sums of ex2.approx terms, each good to 2^-22; the root's
-condition number is at most 1); both KL values within rtol 1e-4 / atol 5e-6 (sums of
-V fp32 terms with cancellation against the log-sum-exps)."""
+Bars: lambda_t within rtol 1e-5 of the oracle's exact sort-based solve, the bar of every other
+lambda in this library (the root is ill-conditioned at budgets near 1, where most of the accepted
+mass sits on capped entries, so the kernel takes its normalisers and its last step in double);
+both KL values within rtol 1e-4 / atol 5e-6 (sums of V fp32 terms with cancellation against the
+log-sum-exps)."""
 import numpy as np
 import pytest
 import torch
@@ -36,7 +37,7 @@ def run(ctx, za, zp, mask, budget):
 
 
 @pytest.mark.parametrize("dtype,V", [("bf16", 20000), ("f32", 4099), ("bf16", 151936)])
-@pytest.mark.parametrize("budget", [0.3, 0.7, 0.95])
+@pytest.mark.parametrize("budget", [0.3, 0.7, 0.95, 0.995])
 def test_row_lambda_matches_oracle(ctx, dtype, V, budget):
     T = 24 if V > 100000 else 96
     ld = (V + 7) // 8 * 8
@@ -47,7 +48,7 @@ def test_row_lambda_matches_oracle(ctx, dtype, V, budget):
     lam, kb, ka, it = run(ctx, za, zp, mask, budget)
     ref = oracle.row_lambda(to_numpy_bits(za.contiguous()), to_numpy_bits(zp.contiguous()), budget,
                             mask=mask.cpu().numpy())
-    assert np.allclose(lam, ref["lam"], rtol=5e-5, atol=0), np.abs(lam / np.maximum(ref["lam"], 1e-30) - 1).max()
+    assert np.allclose(lam, ref["lam"], rtol=1e-5, atol=0), np.abs(lam / np.maximum(ref["lam"], 1e-30) - 1).max()
     assert np.allclose(kb, ref["kl_before"], rtol=1e-4, atol=5e-6)
     assert np.allclose(ka, ref["kl_after"], rtol=1e-4, atol=5e-6)
     valid = mask.cpu().numpy() != 0
@@ -61,11 +62,11 @@ def test_row_lambda_special_cases(ctx):
     za, zp, _ = make_logits(r, "cuda")
     # p == q: Z(lambda) = min(1, 1/lambda), so lambda = 1 / budget and nothing changes
     lam, kb, ka, _ = run(ctx, za, za, None, 0.4)
-    assert np.allclose(lam, 2.5, rtol=5e-5) and np.allclose(kb, 0, atol=5e-6) and np.allclose(ka, 0, atol=5e-6)
+    assert np.allclose(lam, 2.5, rtol=1e-5) and np.allclose(kb, 0, atol=5e-6) and np.allclose(ka, 0, atol=5e-6)
     # budget 1: the smallest ratio p/q
     lam, _, _, _ = run(ctx, za, zp, None, 1.0)
     ref = oracle.row_lambda(to_numpy_bits(za), to_numpy_bits(zp), 1.0)
-    assert np.allclose(lam, ref["lam"], rtol=5e-5)
+    assert np.allclose(lam, ref["lam"], rtol=1e-5)
     with pytest.raises(B.JackpotError, match="budget"):
         run(ctx, za, zp, None, 0.0)
     with pytest.raises(B.JackpotError, match="budget"):

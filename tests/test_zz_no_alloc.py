@@ -8,9 +8,11 @@ cudaMalloc).  For them the library offers one call whose scratch is a fixed
 array inside the library image.  This test drives it through the C ABI twice in
 a row -- the second call finds the first call's leftovers in the shared array --
 and checks both answers against the lambda that the ordinary forward solves from
-the same log-probabilities, within the tolerance the other parity tests use for
-lambda (rtol 1e-5 / atol 1e-6).  It also checks that nothing was allocated and
-that sizes beyond the fixed maximum are refused.
+the same log-probabilities, against the CPU oracle's exact sort-based solve, and
+against the defining equation itself, within the tolerance the other parity tests
+use for lambda (rtol 1e-5 / atol 1e-6).  It also checks that nothing was
+allocated, that the far end of the fixed array works (a batch of exactly the
+maximum size) and that sizes beyond the maximum are refused.
 
 The file name sorts last on purpose: a run that stops at the first failure has
 then already run every other test.
@@ -19,6 +21,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2602_06107_b200 import binding as B
 from paper_2602_06107_b200 import build as jp_build
 from paper_2602_06107_b200 import runner
@@ -30,6 +33,18 @@ RTOL, ATOL = 1e-5, 1e-6
 
 def _close(a, b):
     assert abs(a - b) <= ATOL + RTOL * abs(b), (a, b)
+
+
+def _check_against_the_definition(lam, lq, lp, mask, budget):
+    """lambda against the oracle's solve on the same fp32 log-probs, and the equation it solves,
+    (1/N) sum_t min(1, (p/q)(x_t) / lambda) = budget, evaluated directly in double."""
+    lq, lp = lq.cpu().numpy(), lp.cpu().numpy()
+    m = None if mask is None else mask.cpu().numpy()
+    _close(lam, oracle.lambda_from_budget(lq, lp, budget, m))
+    take = np.ones(lq.shape[0], bool) if m is None else m != 0
+    r = np.exp(lp[take].astype(np.float64) - lq[take].astype(np.float64))
+    if budget < 1.0:
+        assert abs(np.minimum(1.0, r / lam).mean() - budget) <= 2e-5 * budget
 
 
 def test_static_budget_lambda_matches_forward_twice_in_a_row():
@@ -56,12 +71,15 @@ def test_static_budget_lambda_matches_forward_twice_in_a_row():
         assert st == 0
         assert free_after == free_before, "a call after the first changed the device's free memory"
         _close(float(lam_out.item()), out["stats"]["lambda_used"])
+        _check_against_the_definition(float(lam_out.item()), out["logp_actor"], out["logp_policy"], mask, c["budget"])
         # no mask = all rows: same as a forward without a mask
         out_all = runner.forward(ctx, za, zp, tok, None, budget=c["budget"], k=8, seed=1)
         assert B.jp_budget_lambda_static(out_all["logp_actor"], out_all["logp_policy"], None, c["T"], c["budget"],
                                          lam_out) == 0
         torch.cuda.synchronize()
         _close(float(lam_out.item()), out_all["stats"]["lambda_used"])
+        _check_against_the_definition(float(lam_out.item()), out_all["logp_actor"], out_all["logp_policy"], None,
+                                      c["budget"])
     # budget 1: the largest lambda with full acceptance
     assert B.jp_budget_lambda_static(out_all["logp_actor"], out_all["logp_policy"], None, cases[-1]["T"], 1.0,
                                      lam_out) == 0
@@ -69,6 +87,22 @@ def test_static_budget_lambda_matches_forward_twice_in_a_row():
     d = (out_all["logp_policy"] - out_all["logp_actor"]).double()
     _close(float(lam_out.item()), float(torch.exp(d.min()).item()))
     ctx.close()
+
+
+def test_static_budget_lambda_at_the_maximum_size():
+    """A batch of exactly JP_STATIC_MAX_ROWS rows uses the fixed array to its last element; the log-probs
+    are synthetic (the solve only sees them), every seventh row masked."""
+    jp_build.build()
+    T = B.JP_STATIC_MAX_ROWS
+    g = torch.Generator(device="cuda").manual_seed(73)
+    lq = -torch.rand(T, generator=g, device="cuda") * 6.0
+    lp = lq + 1.5 * torch.randn(T, generator=g, device="cuda")
+    mask = (torch.arange(T, device="cuda") % 7 != 3).to(torch.uint8)
+    lam_out = torch.zeros(1, dtype=torch.float32, device="cuda")
+    for budget in (0.6, 0.25):
+        assert B.jp_budget_lambda_static(lq, lp, mask, T, budget, lam_out) == 0
+        torch.cuda.synchronize()
+        _check_against_the_definition(float(lam_out.item()), lq, lp, mask, budget)
 
 
 def test_static_entry_point_limits_and_arguments():
