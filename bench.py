@@ -282,14 +282,17 @@ class Bench:
         return self.max_over_ranks(e0.elapsed_time(e1))
 
     def timed_with_kernel_times(self, fn, steps, warmup, launches_per_step):
-        """timed(), plus the device time of every row-stream launch of the timed steps."""
+        """timed(), then the device time of every row-stream launch over the last steps again, with the
+        library's per-launch events on (they are off while the headline figure is taken: two event
+        records per launch cost a little stream time)."""
         B = self.B
-        B.jp_enable_kernel_timing(self.ctx, True)
         l0 = self.ctx.launch_count()
         ms = self.timed(fn, steps, warmup)
         launches = (self.ctx.launch_count() - l0) // (steps + warmup)
-        n = min(steps, 256 // launches_per_step) * launches_per_step
-        kt = B.jp_stream_kernel_times(self.ctx, n)
+        n_steps = min(steps, 256 // launches_per_step)
+        B.jp_enable_kernel_timing(self.ctx, True)
+        self.timed(fn, n_steps, 0)
+        kt = B.jp_stream_kernel_times(self.ctx, n_steps * launches_per_step)
         B.jp_enable_kernel_timing(self.ctx, False)
         return ms, launches, kt
 

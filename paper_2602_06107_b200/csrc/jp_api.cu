@@ -25,6 +25,7 @@ struct jp_ctx {
   int32_t* vtok = nullptr;       // a vocabulary shard's view of the call: local token ids ...
   uint8_t* vmask = nullptr;      // ... and row validity (2 = this shard holds the sampled token)
   Partials* part = nullptr;
+  SolvePartials* solve = nullptr;
   // state of the records
   bool have_records = false;
   int64_t rec_rows = 0;          // rows covered (T of the forward / T_total of the batch)
@@ -55,7 +56,7 @@ namespace {
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct Layout {
-  size_t scalars, partials, idx, za, zp, f[10], flag, ratio, dval, list, spill, vtok, vmask, total;
+  size_t scalars, partials, solve, idx, za, zp, f[10], flag, ratio, dval, list, spill, vtok, vmask, total;
 };
 
 Layout layout_for(int64_t rows, int k) {
@@ -64,6 +65,7 @@ Layout layout_for(int64_t rows, int k) {
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
   L.scalars = take(sizeof(Scalars));
   L.partials = take(sizeof(Partials));
+  L.solve = take(sizeof(SolvePartials));
   size_t cand = (size_t)rows * 2 * (size_t)(k > 0 ? k : 1);
   L.idx = take(cand * 4);
   L.za = take(cand * 4);
@@ -117,6 +119,7 @@ jp_status ensure_workspace(jp_ctx* c, int64_t rows, int k) {
   char* b = c->ws;
   c->sc = (Scalars*)(b + L.scalars);
   c->part = (Partials*)(b + L.partials);
+  c->solve = (SolvePartials*)(b + L.solve);
   c->rec.idx = (int32_t*)(b + L.idx);
   c->rec.za = (float*)(b + L.za);
   c->rec.zp = (float*)(b + L.zp);
@@ -214,7 +217,7 @@ EpilogueArgs epilogue_args(jp_ctx* c, const jp_obrs_desc* d, int64_t T, int k_ef
                            float* out_lq, float* out_lp, jp_stats* out_stats) {
   EpilogueArgs a{};
   a.T = T; a.k = k_eff; a.seed = seed; a.rng_base = rng_base; a.c1 = c1;
-  a.rec = c->rec; a.sc = c->sc; a.part = c->part;
+  a.rec = c->rec; a.sc = c->sc; a.part = c->part; a.solve = c->solve;
   int64_t np = (T + 7) / 8;
   a.n_part = (int32_t)(np < 1 ? 1 : (np > kMaxPartials ? kMaxPartials : np));
   a.out_accept = out_accept; a.out_weight = out_weight; a.out_lq = out_lq; a.out_lp = out_lp;

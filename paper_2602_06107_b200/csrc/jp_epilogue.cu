@@ -18,6 +18,8 @@ __global__ void reset_kernel(Scalars* sc, float lambda_fixed) {
   sc->n_bad_token = 0ull;
   sc->lambda = lambda_fixed;
   sc->lambda64 = (double)lambda_fixed;
+  sc->bs_ticket = 0;
+  sc->bs_done = 0;
 }
 
 __global__ void clear_flags_kernel(uint8_t* flag, int64_t n) {
@@ -54,90 +56,150 @@ __global__ void ratio_kernel(int64_t T, Records rec) {
   }
 }
 
-constexpr int SOLVE_NT = 1024;
+// ---- lambda from an acceptance budget ------------------------------------------------------
+// Solves (1/N) sum_t min(1, r_t / lambda) = budget for lambda.
+// g(lambda) = (1/N)[#{r >= lambda} + (1/lambda) sum_{r < lambda} r] is non-increasing.
+// The d_t = log r_t are fp32, so a search over the ordered fp32 bit patterns finds the two
+// adjacent floats x_lo < x_hi with g(e^{x_lo}) >= budget > g(e^{x_hi}); no d_t lies strictly
+// between them, so the set {d_t < x_hi} is the partially accepted set and
+// lambda = S / (N budget - #{d >= x_hi}) in closed form.
+// The search is 16-way: one launch evaluates g at 15 thresholds that split the current
+// bracket evenly, so 32 bits take at most 9 launches (plus one that counts N, sums all
+// ratios and finds the smallest).  Every launch spreads the rows over many blocks; each
+// block leaves its partial counts and sums, and the block that finishes last (a ticket
+// counter: no block ever waits) adds them up in block order and narrows the bracket.  The
+// sums therefore do not depend on timing.
+constexpr int BS_NT = 256;
+constexpr int BS_PER_THREAD = 4;
+constexpr int BS_ROUNDS = 10;
 
-struct CountSum {
-  long long c;
-  double s;
-};
-
-__device__ __forceinline__ CountSum block_count_sum(long long c, double s, long long* sc, double* ss) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+__device__ __forceinline__ void warp_sum_cs(long long& c, double& s) {
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) {
     c += __shfl_xor_sync(0xffffffffu, c, off);
     s += __shfl_xor_sync(0xffffffffu, s, off);
   }
-  __syncthreads();
-  if (lane == 0) { sc[warp] = c; ss[warp] = s; }
-  __syncthreads();
-  CountSum r{0, 0.0};
-  for (int w = 0; w < SOLVE_NT / 32; ++w) { r.c += sc[w]; r.s += ss[w]; }
-  return r;
 }
 
-// Solves (1/N) sum_t min(1, r_t / lambda) = budget for lambda.
-// g(lambda) = (1/N)[#{r >= lambda} + (1/lambda) sum_{r < lambda} r] is non-increasing.
-// The d_t are fp32, so a binary search over the ordered fp32 bit patterns finds
-// the two adjacent floats x_lo < x_hi with g(e^{x_lo}) >= budget > g(e^{x_hi});
-// no d_t lies strictly between them, so the set {d_t < x_hi} is the partially
-// accepted set and lambda = S / (N budget - #{d >= x_hi}) in closed form.
-__global__ void __launch_bounds__(SOLVE_NT) budget_solve_kernel(int64_t T, Records rec, Scalars* sc,
-                                                                double budget) {
-  __shared__ long long s_c[SOLVE_NT / 32];
-  __shared__ double s_s[SOLVE_NT / 32];
-  const int tid = threadIdx.x;
-  long long c = 0;
-  double mn = 1e300;
-  for (int64_t i = tid; i < T; i += SOLVE_NT)
-    if (rec.flag[i] == kRowValid) { c += 1; mn = fmin(mn, rec.ratio[i]); }
-  CountSum tot = block_count_sum(c, 0.0, s_c, s_s);
-  const long long N = tot.c;
-  double lam;
-  if (N == 0) {
-    lam = 1.0;
-  } else if (budget >= 1.0) {
-    // largest lambda with full acceptance: min_t r_t
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) mn = fmin(mn, __shfl_xor_sync(0xffffffffu, mn, off));
-    __syncthreads();
-    if ((tid & 31) == 0) s_s[tid >> 5] = mn;
-    __syncthreads();
-    lam = s_s[0];
-    for (int w = 1; w < SOLVE_NT / 32; ++w) lam = fmin(lam, s_s[w]);
-  } else {
-    uint32_t lo = f32_order_bits(JP_NEG_INF);                 // g = 1 >= budget there
-    uint32_t hi = f32_order_bits(__int_as_float(0x7f800000));  // g = 0 <  budget there
-    long long c_hi = 0;
-    double s_hi = 0.0;
-    {
-      double s = 0.0;
-      for (int64_t i = tid; i < T; i += SOLVE_NT)
-        if (rec.flag[i] == kRowValid) s += rec.ratio[i];
-      s_hi = block_count_sum(0, s, s_c, s_s).s;   // at +inf: nothing >= x, every r below
-    }
-    while (hi - lo > 1u) {
-      uint32_t mid = lo + ((hi - lo) >> 1);
-      float x = order_bits_f32(mid);
-      long long cg = 0;
-      double sl = 0.0;
-      for (int64_t i = tid; i < T; i += SOLVE_NT) {
-        if (rec.flag[i] == kRowValid) {
-          if (rec.dval[i] >= x) cg += 1;
-          else sl += rec.ratio[i];
-        }
-      }
-      CountSum r = block_count_sum(cg, sl, s_c, s_s);
-      double lx = exp((double)x);
-      double g = ((double)r.c + (r.s > 0.0 ? r.s / lx : 0.0)) / (double)N;
-      if (g < budget) { hi = mid; c_hi = r.c; s_hi = r.s; }
-      else lo = mid;
-    }
-    lam = s_hi / ((double)N * budget - (double)c_hi);
+// True in exactly one block per launch: the one whose ticket is the last.  The partials
+// written before the call are visible to that block afterwards.
+__device__ __forceinline__ bool last_block_done(Scalars* sc, int* s_flag) {
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const uint32_t t = atomicAdd(&sc->bs_ticket, 1u);
+    *s_flag = (t == gridDim.x - 1) ? 1 : 0;
   }
+  __syncthreads();
+  if (*s_flag) __threadfence();
+  return *s_flag != 0;
+}
+
+__global__ void __launch_bounds__(BS_NT) budget_init_kernel(int64_t T, Records rec, Scalars* sc, SolvePartials* part,
+                                                            double budget) {
+  __shared__ long long s_c[BS_NT / 32];
+  __shared__ double s_s[BS_NT / 32], s_m[BS_NT / 32];
+  __shared__ int s_flag;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  long long c = 0;
+  double s = 0.0, mn = 1e300;
+  for (int64_t i = (int64_t)blockIdx.x * BS_NT + tid; i < T; i += (int64_t)gridDim.x * BS_NT)
+    if (rec.flag[i] == kRowValid) { c += 1; s += rec.ratio[i]; mn = fmin(mn, rec.ratio[i]); }
+  warp_sum_cs(c, s);
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) mn = fmin(mn, __shfl_xor_sync(0xffffffffu, mn, off));
+  if (lane == 0) { s_c[warp] = c; s_s[warp] = s; s_m[warp] = mn; }
+  __syncthreads();
   if (tid == 0) {
-    sc->lambda64 = lam;
-    sc->lambda = (float)lam;
+    for (int w = 1; w < BS_NT / 32; ++w) { c += s_c[w]; s += s_s[w]; mn = fmin(mn, s_m[w]); }
+    part->c[blockIdx.x][0] = c; part->s[blockIdx.x][0] = s; part->s[blockIdx.x][1] = mn;
+  }
+  if (!last_block_done(sc, &s_flag)) return;
+  if (tid == 0) {
+    long long N = 0;
+    double S = 0.0, m = 1e300;
+    for (unsigned b = 0; b < gridDim.x; ++b) { N += part->c[b][0]; S += part->s[b][0]; m = fmin(m, part->s[b][1]); }
+    sc->bs_N = N;
+    sc->bs_lo = f32_order_bits(JP_NEG_INF);                     // g = 1 >= budget there
+    sc->bs_hi = f32_order_bits(__int_as_float(0x7f800000));      // g = 0 <  budget there
+    sc->bs_c_hi = 0;                                             // at +inf: nothing >= x, every r below
+    sc->bs_s_hi = S;
+    sc->bs_done = 0;
+    if (N == 0) { sc->lambda64 = 1.0; sc->lambda = 1.f; sc->bs_done = 1; }
+    else if (budget >= 1.0) { sc->lambda64 = m; sc->lambda = (float)m; sc->bs_done = 1; }   // largest lambda with full acceptance
+    sc->bs_ticket = 0;
+  }
+}
+
+__global__ void __launch_bounds__(BS_NT) budget_round_kernel(int64_t T, Records rec, Scalars* sc, SolvePartials* part,
+                                                             double budget) {
+  __shared__ long long s_c[BS_NT / 32][kSolveWays];
+  __shared__ double s_s[BS_NT / 32][kSolveWays];
+  __shared__ int s_flag;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (sc->bs_done) return;                       // every block reads the state the previous launch left
+  const uint32_t lo = sc->bs_lo, hi = sc->bs_hi;
+  const uint32_t span = hi - lo;                 // >= 2 while not done
+  const int nth = span - 1u < (uint32_t)(kSolveWays - 1) ? (int)(span - 1u) : kSolveWays - 1;
+  const uint32_t step = span / (uint32_t)(nth + 1);
+  // thresholds m_j = lo + j step, j = 1 .. nth, all strictly inside (lo, hi)
+  long long cg[kSolveWays];
+  double sl[kSolveWays];
+#pragma unroll
+  for (int j = 0; j < kSolveWays; ++j) { cg[j] = 0; sl[j] = 0.0; }
+  for (int64_t i = (int64_t)blockIdx.x * BS_NT + tid; i < T; i += (int64_t)gridDim.x * BS_NT) {
+    if (rec.flag[i] != kRowValid) continue;
+    const uint32_t ob = f32_order_bits(rec.dval[i]);
+    const double r = rec.ratio[i];
+#pragma unroll
+    for (int j = 1; j < kSolveWays; ++j) {
+      if (j <= nth) {
+        if (ob >= lo + (uint32_t)j * step) cg[j] += 1;
+        else sl[j] += r;
+      }
+    }
+  }
+#pragma unroll
+  for (int j = 1; j < kSolveWays; ++j) {
+    warp_sum_cs(cg[j], sl[j]);
+    if (lane == 0) { s_c[warp][j] = cg[j]; s_s[warp][j] = sl[j]; }
+  }
+  __syncthreads();
+  if (tid >= 1 && tid < kSolveWays) {
+    long long c = 0;
+    double s = 0.0;
+    for (int w = 0; w < BS_NT / 32; ++w) { c += s_c[w][tid]; s += s_s[w][tid]; }
+    part->c[blockIdx.x][tid] = c;
+    part->s[blockIdx.x][tid] = s;
+  }
+  if (!last_block_done(sc, &s_flag)) return;
+  if (tid >= 1 && tid < kSolveWays) {
+    long long c = 0;
+    double s = 0.0;
+    for (unsigned b = 0; b < gridDim.x; ++b) { c += part->c[b][tid]; s += part->s[b][tid]; }
+    s_c[0][tid] = c; s_s[0][tid] = s;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    const double N = (double)sc->bs_N;
+    uint32_t nlo = lo, nhi = hi;
+    long long c_hi = sc->bs_c_hi;
+    double s_hi = sc->bs_s_hi;
+    for (int j = 1; j <= nth; ++j) {              // g falls along the thresholds: the first one below the budget is the new hi
+      const uint32_t m = lo + (uint32_t)j * step;
+      const double lx = exp((double)order_bits_f32(m));
+      const double g = ((double)s_c[0][j] + (s_s[0][j] > 0.0 ? s_s[0][j] / lx : 0.0)) / N;
+      if (g < budget) { nhi = m; c_hi = s_c[0][j]; s_hi = s_s[0][j]; break; }
+      nlo = m;
+    }
+    sc->bs_lo = nlo; sc->bs_hi = nhi; sc->bs_c_hi = c_hi; sc->bs_s_hi = s_hi;
+    if (nhi - nlo <= 1u) {
+      const double lam = s_hi / (N * budget - (double)c_hi);
+      sc->lambda64 = lam;
+      sc->lambda = (float)lam;
+      sc->bs_done = 1;
+    }
+    sc->bs_ticket = 0;
   }
 }
 
@@ -271,18 +333,18 @@ __global__ void __launch_bounds__(EPI_NT) finalize_kernel(EpilogueArgs A) {
   __shared__ double s_kappa;
   __shared__ long long s_nv[EPI_NT], s_na[EPI_NT], s_nf[EPI_NT];
   __shared__ double s_zk[EPI_NT], s_a[EPI_NT], s_kl[EPI_NT];
-  static_assert(kMaxPartials <= EPI_NT, "one thread per partial sum");
-  // every block folds the same partial sums in the same fixed tree (so all blocks get
-  // the same bits): thread i starts from partial i, halves are added pairwise
+  static_assert(kMaxPartials % EPI_NT == 0, "every thread starts from the same number of partial sums");
+  // every block folds the same partial sums in the same fixed order (so all blocks get the
+  // same bits): thread i adds up partials i, i + EPI_NT, ... in turn, then halves are added pairwise
   {
     const int i = threadIdx.x;
-    const bool have = i < A.n_part;
-    s_nv[i] = have ? A.part->n_valid[i] : 0;
-    s_na[i] = have ? A.part->n_accept[i] : 0;
-    s_nf[i] = have ? A.part->n_nonfinite[i] : 0;
-    s_zk[i] = have ? A.part->sum_zk[i] : 0.0;
-    s_a[i] = have ? A.part->sum_a[i] : 0.0;
-    s_kl[i] = have ? A.part->sum_kl[i] : 0.0;
+    long long nv = 0, na = 0, nf = 0;
+    double zk = 0.0, a = 0.0, kl = 0.0;
+    for (int j = i; j < A.n_part; j += EPI_NT) {
+      nv += A.part->n_valid[j]; na += A.part->n_accept[j]; nf += A.part->n_nonfinite[j];
+      zk += A.part->sum_zk[j]; a += A.part->sum_a[j]; kl += A.part->sum_kl[j];
+    }
+    s_nv[i] = nv; s_na[i] = na; s_nf[i] = nf; s_zk[i] = zk; s_a[i] = a; s_kl[i] = kl;
   }
   __syncthreads();
   for (int half = EPI_NT / 2; half > 0; half >>= 1) {
@@ -396,8 +458,12 @@ cudaError_t launch_clear_flags(uint8_t* flag, int64_t n, cudaStream_t s) {
 cudaError_t launch_budget_solve(const EpilogueArgs& a, double budget, cudaStream_t s, int* n_launch) {
   if (a.T <= 0) return cudaSuccess;
   ratio_kernel<<<(unsigned)((a.T + 255) / 256), 256, 0, s>>>(a.T, a.rec);
-  budget_solve_kernel<<<1, SOLVE_NT, 0, s>>>(a.T, a.rec, a.sc, budget);
-  *n_launch += 2;
+  int64_t blocks = (a.T + BS_NT * BS_PER_THREAD - 1) / (BS_NT * BS_PER_THREAD);
+  if (blocks > kSolveMaxBlocks) blocks = kSolveMaxBlocks;
+  budget_init_kernel<<<(unsigned)blocks, BS_NT, 0, s>>>(a.T, a.rec, a.sc, a.solve, budget);
+  for (int r = 0; r < BS_ROUNDS; ++r)
+    budget_round_kernel<<<(unsigned)blocks, BS_NT, 0, s>>>(a.T, a.rec, a.sc, a.solve, budget);
+  *n_launch += 2 + BS_ROUNDS;
   return cudaGetLastError();
 }
 

@@ -41,13 +41,18 @@ struct Scalars {
   float pad;
   double lambda64;
   double totals[4];        // the last forward's batch sums: N, accepted, sum of Z_approx, sum of a(x_t)
+  // state of the budget solve between its launches: the bracket [lo, hi] in ordered fp32 bit
+  // patterns, count and ratio sum at hi, the number of valid rows, the last-block ticket
+  uint32_t bs_lo, bs_hi, bs_ticket, bs_done;
+  long long bs_N, bs_c_hi;
+  double bs_s_hi;
   jp_stats stats;          // the last forward's batch statistics
 };
 
 constexpr uint8_t kRowValid = 1;      // values of Records::flag
 constexpr uint8_t kRowNonFinite = 2;
 
-constexpr int kMaxPartials = 256;
+constexpr int kMaxPartials = 1024;
 struct Partials {
   long long n_valid[kMaxPartials];
   long long n_accept[kMaxPartials];
@@ -55,6 +60,14 @@ struct Partials {
   double sum_zk[kMaxPartials];
   double sum_a[kMaxPartials];
   double sum_kl[kMaxPartials];
+};
+
+// Per-block partial counts and sums of one launch of the budget solve.
+constexpr int kSolveMaxBlocks = 256;
+constexpr int kSolveWays = 16;
+struct SolvePartials {
+  long long c[kSolveMaxBlocks][kSolveWays];
+  double s[kSolveMaxBlocks][kSolveWays];
 };
 
 struct StreamArgs {
@@ -99,6 +112,7 @@ struct EpilogueArgs {
   Records rec;
   Scalars* sc;
   Partials* part;
+  SolvePartials* solve;    // scratch of the budget solve
   int32_t n_part;
   int32_t have_kl;         // rec.kl holds KL(p || q) of every valid row: sum it into the statistics
   // outputs, all [T] (any may be null)

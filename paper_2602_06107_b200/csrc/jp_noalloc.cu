@@ -17,11 +17,12 @@ namespace {
 
 constexpr int64_t kMaxRows = JP_STATIC_MAX_ROWS;
 constexpr size_t kOffScalars = 0;                                        // Scalars
-constexpr size_t kOffRatio = 1024;                                       // double[kMaxRows]
+constexpr size_t kOffSolve = 1024;                                       // SolvePartials
+constexpr size_t kOffRatio = kOffSolve + sizeof(SolvePartials);          // double[kMaxRows]
 constexpr size_t kOffDval = kOffRatio + sizeof(double) * kMaxRows;       // float[kMaxRows]
 constexpr size_t kOffFlag = kOffDval + sizeof(float) * kMaxRows;         // uint8_t[kMaxRows]
 constexpr size_t kScratchBytes = kOffFlag + kMaxRows;
-static_assert(sizeof(Scalars) <= kOffRatio, "the scalar block must fit before the arrays");
+static_assert(sizeof(Scalars) <= kOffSolve, "the scalar block must fit before the arrays");
 
 // 1.7 MB held by every device that loads the library, until the process exits.
 static __device__ __align__(256) unsigned char g_static_scratch[kScratchBytes];
@@ -64,6 +65,7 @@ extern "C" jp_status jp_budget_lambda_static(const float* logp_actor, const floa
   EpilogueArgs a{};
   a.T = T;
   a.sc = sc;
+  a.solve = (SolvePartials*)(base + kOffSolve);
   a.rec.ratio = (double*)(base + kOffRatio);
   a.rec.dval = (float*)(base + kOffDval);
   a.rec.flag = (uint8_t*)(base + kOffFlag);
