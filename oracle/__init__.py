@@ -156,6 +156,64 @@ def z_exact(za, zp, lse_a, lse_p, lam, mask=None, bad=None):
     return z
 
 
+def z_sparse(zp, inf_idx, inf_logp, new_idx, lse_p, lam, mask=None, bad=None):
+    """Z_approx when the rollout model is known only through its stored top-k log-probs
+    (Algorithm 1 Phase 1 / Phase 2 step 2): returns (z_lo, z_hi), see jo_z_sparse."""
+    T, V = _check2d(zp)
+    inf_idx = np.ascontiguousarray(inf_idx, np.int32)
+    inf_logp = np.ascontiguousarray(inf_logp, np.float32)
+    new_idx = np.ascontiguousarray(new_idx, np.int32)
+    lo, hi = np.zeros(T), np.zeros(T)
+    lib().jo_z_sparse(ctypes.c_int64(T), ctypes.c_int64(V), ctypes.c_int64(V), ctypes.c_int(_dtype_code(zp)),
+                      _vp(zp), _p(mask, ctypes.c_uint8), _p(bad, ctypes.c_uint8), ctypes.c_int(inf_idx.shape[1]),
+                      _p(inf_idx, ctypes.c_int32), _p(inf_logp, ctypes.c_float), ctypes.c_int(new_idx.shape[1]),
+                      _p(new_idx, ctypes.c_int32), _p(lse_p, ctypes.c_double), ctypes.c_double(lam),
+                      _p(lo, ctypes.c_double), _p(hi, ctypes.c_double))
+    return lo, hi
+
+
+def rollout_record(za, tokens, k_inf, mask=None):
+    """What Algorithm 1 Phase 1 stores per token from the rollout model's forward: log p_inf(a_t) and
+    the k_inf most likely tokens with their log-probabilities (fp32, best first)."""
+    T, V = _check2d(za)
+    r = lse_gather(za, za, tokens, mask)
+    idx = topk(za, k_inf, mask)
+    if za.dtype == np.uint16:
+        zf = (za.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+    else:
+        zf = za.astype(np.float64)
+    safe = np.maximum(idx, 0)
+    logp = (np.take_along_axis(zf, safe, axis=1) - r["lse_a"][:, None]).astype(np.float32)
+    logp[idx < 0] = 0.0
+    return r["lq"], idx, logp
+
+
+def forward_sparse(zp, tokens, logp_inf_token, inf_idx, inf_logp, mask=None, *, lam=None, budget=None, k=20, seed=0,
+                   token_offset=0, c1=0.0, cap=False):
+    """The forward steps with the rollout model known only through the stored record: the policy's
+    log-softmax and top-k from its logits, acceptance from the stored log p_inf(a_t), Z from
+    jo_z_sparse (z_lo, or z_hi with cap=True), then the batch correction and weights as usual."""
+    assert (lam is None) != (budget is None)
+    T, V = _check2d(zp)
+    mask = None if mask is None else np.ascontiguousarray(mask, np.uint8)
+    r = lse_gather(zp, zp, tokens, mask)
+    bad = r["bad"]
+    r["lq"] = np.ascontiguousarray(logp_inf_token, np.float32).copy()
+    r["lq"][(bad != 0) | (np.zeros(T, bool) if mask is None else mask == 0)] = 0.0
+    r["lq64"] = r["lq"].astype(np.float64)
+    r["topk_idx_p"] = topk(zp, k, mask)
+    if budget is not None:
+        lam = float(np.float32(lambda_from_budget(r["lq"], r["lp"], budget, mask, bad)))
+    lam = float(np.float32(lam))
+    r["lambda"] = lam
+    r["a"], r["u"], r["accept"] = accept(r["lq"], r["lp"], lam, seed, token_offset, mask, bad)
+    r["z_lo"], r["z_hi"] = z_sparse(zp, inf_idx, inf_logp, r["topk_idx_p"], r["lse_p"], lam, mask, bad)
+    r["zk"] = r["z_hi"] if cap else r["z_lo"]
+    r["w"], r["w64"], r["stats"] = batch_weights(r["lq"], r["lp"], r["accept"], r["a"], r["zk"], lam, c1, mask, bad)
+    r["stats"]["n_bad_token"] = int(bad.sum())
+    return r
+
+
 _STAT_KEYS = ("n_valid", "n_accept", "alpha_hat", "mean_accept_prob", "z_approx_mean", "kappa",
               "lambda_used")
 

@@ -251,6 +251,54 @@ void jo_z_topk(int64_t T, int64_t V, int64_t ld, int dtype, const void* za, cons
   }
 }
 
+// Step 7a, with the rollout model known only through what Algorithm 1 Phase 1 stores: per token
+// the log-probabilities of its k_inf most likely tokens, inf_idx / inf_logp [T, k_inf] (index
+// -1 = empty place).  Phase 2 step 2 sums min(p_inf(x), p_new(x)/lambda) over
+// V_k = TopK_inf U TopK_new.  For x in TopK_inf the term is as printed.  For x in TopK_new that
+// the rollout did not store, p_inf(x) is not known (the paper does not say what to take); two
+// readings, both returned:
+//   z_lo  the term is left out: a lower bound of the Z_approx of the dense path, so the
+//         inequality Z_approx <= Z on which Section 4.4.2 builds its correction still holds;
+//   z_hi  p_inf(x) is replaced by what is known about it, p_inf(x) <= the smallest stored
+//         probability, and the unknown terms together by the mass the stored list leaves,
+//         1 - sum of the stored probabilities: an upper bound of the dense Z_approx.
+// new_idx [T, k] is TopK_new from jo_topk on the policy logits.
+void jo_z_sparse(int64_t T, int64_t V, int64_t ld, int dtype, const void* zp, const uint8_t* mask,
+                 const uint8_t* bad, int k_inf, const int32_t* inf_idx, const float* inf_logp, int k,
+                 const int32_t* new_idx, const double* lse_p, double lambda, double* z_lo, double* z_hi) {
+  (void)V;
+#pragma omp parallel for schedule(dynamic, 16)
+  for (int64_t t = 0; t < T; ++t) {
+    z_lo[t] = 0.0;
+    z_hi[t] = 0.0;
+    if (!row_valid(mask, t) || (bad && bad[t])) continue;
+    double stored_sum = 0.0, stored_mass = 0.0, p_min = 1.0;
+    int n_stored = 0;
+    for (int j = 0; j < k_inf; ++j) {
+      const int32_t x = inf_idx[t * k_inf + j];
+      if (x < 0) continue;
+      const double q = std::exp((double)inf_logp[t * k_inf + j]);
+      const double p = std::exp(logit_at(zp, dtype, t * ld + x) - lse_p[t]);
+      stored_sum += std::min(q, p / lambda);
+      stored_mass += q;
+      p_min = std::min(p_min, q);
+      ++n_stored;
+    }
+    double unknown = 0.0;
+    for (int j = 0; j < k; ++j) {
+      const int32_t x = new_idx[t * k + j];
+      if (x < 0) continue;
+      bool stored = false;
+      for (int i = 0; i < k_inf; ++i) stored = stored || inf_idx[t * k_inf + i] == x;
+      if (stored) continue;
+      const double p = std::exp(logit_at(zp, dtype, t * ld + x) - lse_p[t]);
+      unknown += std::min(n_stored > 0 ? p_min : 1.0, p / lambda);
+    }
+    z_lo[t] = stored_sum;
+    z_hi[t] = stored_sum + std::min(unknown, std::max(0.0, 1.0 - stored_mass));
+  }
+}
+
 // Step 7b: the exact normaliser Z = sum_{x'} min(p_inf(x'), p_target(x')/lambda)
 // over the whole vocabulary (Eq. obrs_dist; Appendix A, Z_C).
 void jo_z_exact(int64_t T, int64_t V, int64_t ld, int dtype, const void* za, const void* zp,

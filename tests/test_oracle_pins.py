@@ -599,3 +599,98 @@ def test_row_lambda_kl_before_and_after():
     m = np.ones(30, np.uint8); m[3] = 0
     rm = oracle.row_lambda(za, zp, 0.7, mask=m)
     assert rm["lam"][3] == 0 and rm["kl_after"][3] == 0 and rm["lam"][4] == r["lam"][4]
+
+
+# ------------------------------------------------- sparse actor (stored top-k of the rollout model)
+
+def _sparse_brute(zp64, q_full, inf_idx, new_idx, lam):
+    """z_lo / z_hi written from their definitions with python sets, on exact double inputs."""
+    p = scipy.special.softmax(zp64)
+    stored = [int(x) for x in inf_idx if x >= 0]
+    lo = sum(min(q_full[x], p[x] / lam) for x in stored)
+    p_min = min(q_full[x] for x in stored) if stored else 1.0
+    rest = 1.0 - sum(q_full[x] for x in stored)
+    unknown = sum(min(p_min, p[x] / lam) for x in set(int(x) for x in new_idx if x >= 0) - set(stored))
+    return lo, lo + min(unknown, max(rest, 0.0))
+
+
+def test_sparse_actor_normaliser_by_hand():
+    """V = 4, rollout stored its 2 best, policy top-2 holds one token the rollout did not store."""
+    q = np.array([0.5, 0.3, 0.15, 0.05])
+    p = np.array([0.1, 0.2, 0.6, 0.1])
+    zp = np.log(p).astype(np.float32)[None, :]
+    lse_p = np.array([np.log(np.exp(zp.astype(np.float64)).sum())])
+    inf_idx = np.array([[0, 1]], np.int32)
+    inf_logp = np.log(q[:2]).astype(np.float32)[None, :]
+    new_idx = oracle.topk(zp, 2)
+    assert new_idx.tolist() == [[2, 1]]
+    for lam in (1.0, 2.0):
+        lo, hi = oracle.z_sparse(zp, inf_idx, inf_logp, new_idx, lse_p, lam)
+        want_lo = min(0.5, 0.1 / lam) + min(0.3, 0.2 / lam)
+        # token 2 is unknown to the rollout record: at most the smallest stored probability (0.3), at most
+        # the mass the record leaves (0.2), at most p/lambda
+        want_hi = want_lo + min(min(0.3, 0.6 / lam), 0.2)
+        assert lo[0] == pytest.approx(want_lo, rel=1e-6) and hi[0] == pytest.approx(want_hi, rel=1e-6)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_sparse_actor_normaliser_brackets_the_dense_estimate(dtype):
+    T, V = 24, 600
+    za, zp, tok = _rand_rows(T, V, 91, sigma=1.0)
+    if dtype == "bf16":
+        za, zp = _to_bf16_bits(za), _to_bf16_bits(zp)
+        za64, zp64 = _bf16_bits_to_f64(za), _bf16_bits_to_f64(zp)
+    else:
+        za64, zp64 = za.astype(np.float64), zp.astype(np.float64)
+    lg = oracle.lse_gather(za, zp, tok)
+    q_full = scipy.special.softmax(za64, axis=1)
+    prev_lo = None
+    for k in (4, 16, 64, V):
+        lq, inf_idx, inf_logp = oracle.rollout_record(za, tok, k)
+        # the record is what the definitions give: top-k of the actor, its log-softmax at those places
+        assert np.array_equal(inf_idx, oracle.topk(za, k))
+        assert np.allclose(inf_logp, np.log(np.take_along_axis(q_full, inf_idx, axis=1)), rtol=0, atol=2e-6)
+        assert np.allclose(lq, np.log(q_full[np.arange(T), tok]), rtol=0, atol=2e-6)
+        new_idx = oracle.topk(zp, k)
+        for lam in (0.7, 1.0, 2.5):
+            lo, hi = oracle.z_sparse(zp, inf_idx, inf_logp, new_idx, lg["lse_p"], lam)
+            dense = oracle.z_topk(za, zp, inf_idx, new_idx, lg["lse_a"], lg["lse_p"], lam)
+            exact = oracle.z_exact(za, zp, lg["lse_a"], lg["lse_p"], lam)
+            for t in range(T):
+                # brute force on the rounded record (the oracle sees fp32 log-probs)
+                qs = q_full[t].copy()
+                qs[inf_idx[t]] = np.exp(inf_logp[t].astype(np.float64))
+                blo, bhi = _sparse_brute(zp64[t], qs, inf_idx[t], new_idx[t], lam)
+                assert lo[t] == pytest.approx(blo, rel=1e-12) and hi[t] == pytest.approx(bhi, rel=1e-12)
+            tol = 1e-6
+            assert np.all(lo <= dense * (1 + tol)) and np.all(dense <= hi * (1 + tol))     # the bracket
+            assert np.all(lo <= exact * (1 + tol))                                         # Z_approx <= Z survives
+            if k == V:                                                                     # everything stored: the dense path
+                assert np.allclose(lo, exact, rtol=1e-6) and np.allclose(hi, exact, rtol=1e-6)
+        lo1, _ = oracle.z_sparse(zp, inf_idx, inf_logp, new_idx, lg["lse_p"], 1.0)
+        if prev_lo is not None:
+            assert np.all(lo1 >= prev_lo * (1 - 1e-6))                                     # grows with the stored list
+        prev_lo = lo1
+
+
+def test_sparse_forward_reduces_to_the_dense_forward_when_everything_is_stored():
+    T, V, k = 40, 300, 12
+    za, zp, tok = _rand_rows(T, V, 92, sigma=0.9)
+    mask = (np.arange(T) % 5 != 1).astype(np.uint8)
+    lq, inf_idx, inf_logp = oracle.rollout_record(za, tok, V, mask)
+    dense = oracle.forward(za, zp, tok, mask, lam=1.3, k=V, seed=5, c1=3.0)
+    for cap in (False, True):
+        sp = oracle.forward_sparse(zp, tok, lq, inf_idx, inf_logp, mask, lam=1.3, k=k, seed=5, c1=3.0, cap=cap)
+        assert np.array_equal(sp["accept"], dense["accept"]) and np.array_equal(sp["u"], dense["u"])
+        assert np.allclose(sp["zk"], dense["zk"], rtol=2e-6)
+        assert np.allclose(sp["w64"], dense["w64"], rtol=2e-6)
+        assert sp["stats"]["kappa"] == pytest.approx(dense["stats"]["kappa"], rel=2e-6)
+    # with a short record the floor reading can only lose mass, and kappa makes up for it on average
+    lq, inf_idx, inf_logp = oracle.rollout_record(za, tok, k, mask)
+    sp = oracle.forward_sparse(zp, tok, lq, inf_idx, inf_logp, mask, lam=1.3, k=k, seed=5)
+    d2 = oracle.forward(za, zp, tok, mask, lam=1.3, k=k, seed=5)
+    assert np.all(sp["zk"] <= d2["zk"] * (1 + 1e-6))
+    assert sp["stats"]["kappa"] >= d2["stats"]["kappa"] * (1 - 1e-9)
+    assert sp["stats"]["kappa"] * sp["stats"]["z_approx_mean"] == pytest.approx(sp["stats"]["alpha_hat"], rel=1e-12)
+    b = oracle.forward_sparse(zp, tok, lq, inf_idx, inf_logp, mask, budget=0.6, k=k, seed=5)
+    assert b["stats"]["mean_accept_prob"] == pytest.approx(0.6, abs=1e-6)
