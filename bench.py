@@ -2,7 +2,7 @@
 """Benchmark of the OBRS token pass (libjackpot) on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload cfg2_qwen3|cfg3_batch|cfg4_sweep|cfg5_train]
+                    [--workload cfg2_qwen3|cfg3_batch|cfg4_sweep|cfg5_train|sparse_actor]
 
 A step is one pass of the whole path over one batch of synthetic logits:
 
@@ -17,6 +17,10 @@ A step is one pass of the whole path over one batch of synthetic logits:
                         forwards per step, Z_approx against the exact Z and throughput per point;
   cfg5_train            32,768 rows in 4 chunks: chunked forward with a budget of 0.5 and a weight
                         clip, then one fused backward per chunk (bf16 gradients of both tensors).
+
+  sparse_actor          the cfg2 shape through jp_obrs_forward_sparse_actor: only the policy tensor is
+                        streamed (303,872 B per token), the rollout model comes as the record the
+                        paper's rollout phase stores (log p_inf(a_t) and its 20 best log-probs).
 
 Every workload prints one JSON line with `roofline` (the dominant kernel, timed per launch by CUDA
 events on the stream it runs on), `cpu_baseline` (the oracle on a bounded sample, all host cores and
@@ -42,7 +46,9 @@ if ROOT not in sys.path:
 
 UNIT = "tokens/s"
 METRICS = {"cfg2_qwen3": "obrs_forward_tokens_per_s", "cfg3_batch": "obrs_forward_tokens_per_s",
-           "cfg4_sweep": "obrs_forward_tokens_per_s", "cfg5_train": "obrs_fwd_bwd_tokens_per_s"}
+           "cfg4_sweep": "obrs_forward_tokens_per_s", "cfg5_train": "obrs_fwd_bwd_tokens_per_s",
+           "sparse_actor": "obrs_forward_tokens_per_s"}
+SPARSE_K_INF = 20            # the rollout stores its 20 most likely tokens (the paper's default top-k count)
 DATASHEET_GBS = 8000.0
 
 
@@ -117,6 +123,8 @@ def _recipe(r0, T, seed, sigma=None):
 
 def _workload(name):
     from paper_2602_06107_b200.inputs import CONFIGS
+    if name == "sparse_actor":                 # the headline shape, the rollout model as a stored record
+        return CONFIGS["cfg2_qwen3"]
     if name not in METRICS:
         raise SystemExit(f"bench.py: workload {name!r} is not a bench line (choose from {sorted(METRICS)}); "
                          "the tiny exact-check shape is a parity test, see tests/")
@@ -147,6 +155,10 @@ def _oracle_step(name, cfg, za, zp, tok, mask):
     n = za.shape[0]
     if name == "cfg2_qwen3":
         oracle.forward(za, zp, tok, None, lam=cfg["lam"], k=cfg["k"], seed=cfg["seed"])
+        return n
+    if name == "sparse_actor":
+        lq, idx, logp = oracle.rollout_record(za, tok, SPARSE_K_INF)      # the rollout engine's part, not the path's
+        oracle.forward_sparse(zp, tok, lq, idx, logp, None, lam=cfg["lam"], k=cfg["k"], seed=cfg["seed"])
         return n
     if name == "cfg3_batch":
         oracle.forward(za, zp, tok, mask, budget=cfg["budget"], k=cfg["k"], seed=cfg["seed"])
@@ -185,7 +197,8 @@ def cpu_baseline_for(name, cfg, sample):
     v, reps, dt, cores = _time_oracle(name, cfg, sample, 8.0)
     one = [None if x is None else x[:max(8, rows // 8)] for x in sample]
     v1, reps1, dt1, _ = _time_oracle(name, cfg, one, 6.0, threads=1)
-    what = {"cfg2_qwen3": "forward", "cfg3_batch": "forward with the budget solve, valid tokens",
+    what = {"cfg2_qwen3": "forward", "sparse_actor": "forward from the policy logits and the stored record (making "
+            "the record from the actor's logits is inside the timed region: it costs about as much again)", "cfg3_batch": "forward with the budget solve, valid tokens",
             "cfg4_sweep": "the four k of one sweep point", "cfg5_train": "forward + both gradients"}[name]
     return {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"first {rows} rows of the workload, {what}, {reps} passes, {dt:.1f} s",
@@ -311,7 +324,8 @@ class Bench:
         try:
             ro = self.B.jp_probe_stream(a, None, reps=20)
             roof["read_only_gbs_now"] = ro
-            roof["copy_gbs_now"] = self.B.jp_probe_stream(a, b, reps=10)
+            if b is not None:
+                roof["copy_gbs_now"] = self.B.jp_probe_stream(a, b, reps=10)
             roof["frac_of_read_only_now"] = roof["achieved"] / ro
         except Exception as exc:                               # a measurement aid must not lose the line
             roof["probe_error"] = str(exc)
@@ -588,7 +602,52 @@ def wl_cfg5(b: Bench, cfg):
                         "stats": {n: stats[n] for n in ("lambda_used", "alpha_hat", "kappa")}})
 
 
-WORKLOADS = {"cfg2_qwen3": wl_cfg2, "cfg3_batch": wl_cfg3, "cfg4_sweep": wl_cfg4, "cfg5_train": wl_cfg5}
+def wl_sparse(b: Bench, cfg):
+    torch, B, args = b.torch, b.B, b.args
+    from paper_2602_06107_b200 import runner
+    from paper_2602_06107_b200.inputs import make_logits
+    r0 = cfg["recipe"]
+    T = r0.T
+    r = _recipe(r0, T, r0.seed + 1000 * b.rank)
+    k, lam, seed = cfg["k"], cfg["lam"], cfg["seed"]
+    za, zp, tok = make_logits(r, b.dev)
+    V, esize = r.V, zp.element_size()
+    # the rollout record (input data: what a rollout engine stores per token), then the actor's logits go
+    lq_all = torch.empty((T,), dtype=torch.float32, device=b.dev)
+    inf_idx = torch.empty((T, SPARSE_K_INF), dtype=torch.int32, device=b.dev)
+    inf_logp = torch.empty((T, SPARSE_K_INF), dtype=torch.float32, device=b.dev)
+    for o in range(0, T, 512):
+        lsm = torch.log_softmax(za[o:o + 512].float(), dim=1)
+        v, i = lsm.topk(SPARSE_K_INF, dim=1)
+        inf_idx[o:o + 512], inf_logp[o:o + 512] = i.to(torch.int32), v
+        lq_all[o:o + 512] = lsm.gather(1, tok[o:o + 512].long()[:, None])[:, 0]
+    del za, lsm
+    B.jp_reserve(b.ctx, T, V, k)
+    out = runner._alloc_outputs(T, b.dev)
+    desc = B.make_desc(zp)
+
+    def fwd():
+        B.jp_obrs_forward_sparse_actor(b.ctx, desc, zp, tok, None, lq_all, inf_idx, inf_logp, SPARSE_K_INF, lam, k, seed,
+                                       out["accept"], out["weight"], out["logp_policy"], None, None, out["stats_buf"])
+
+    ms, launches, kt = b.timed_with_kernel_times(fwd, args.steps, args.warmup, 1)
+    stats = B.read_stats(out["stats_buf"])
+    k_ms = sum(kt) / len(kt)
+    alg = 1.0 * stats["n_valid"] * V * esize
+    roof = b.roofline(f"prep_rows_kernel + stream_kernel<{r.dtype}, {32 if k <= 32 else 64 if k <= 64 else 128}-entry list, "
+                      f"policy tensor only> (k = {k}): one forward's row stream", alg, k_ms,
+                      kernel_ms_min=min(kt), kernel_ms_max=max(kt))
+    b.add_probe_rates(roof, zp, None)
+    e2e = {"value": None, "reason": "the host-buffer entry point exists for the dense forward only"}
+    return dict(ms=ms, units_per_step=T, launches=launches, roofline=roof, e2e=e2e, extra={},
+                config={"T": T, "V": V, "logits": r.dtype, "k": k, "k_inf": SPARSE_K_INF, "lambda": lam, "seed": seed,
+                        "record": "log p_inf(a_t) and the 20 best log-probs per token, from torch.log_softmax / topk "
+                                  "of the synthetic actor logits",
+                        "l2": f"inputs {T * V * esize / 1e9:.2f} GB per step exceed the 126 MB L2; no flush needed",
+                        "stats": {n: stats[n] for n in ("alpha_hat", "kappa", "z_approx_mean")}})
+
+
+WORKLOADS = {"sparse_actor": wl_sparse, "cfg2_qwen3": wl_cfg2, "cfg3_batch": wl_cfg3, "cfg4_sweep": wl_cfg4, "cfg5_train": wl_cfg5}
 
 
 def _nccl_summary(log_dir, world):

@@ -55,6 +55,7 @@ typedef enum { JP_LAMBDA_FIXED = 0, JP_LAMBDA_FROM_BUDGET = 1 } jp_lambda_mode;
 
 enum { JP_MAX_TOPK = 128 };
 enum { JP_STATIC_MAX_ROWS = 131072 };   /* row limit of jp_budget_lambda_static */
+enum { JP_DESC_SPARSE_CAP = 2 };        /* jp_obrs_desc.flags, jp_obrs_forward_sparse_actor only: see there */
 enum { JP_DESC_KL = 1 };                /* jp_obrs_desc.flags: also compute KL(p_target || p_inf) per row (one more
                                            pass over the rows) and report its batch mean in jp_stats.mean_kl_p_q */
 
@@ -140,6 +141,37 @@ jp_status jp_obrs_forward(jp_ctx* ctx, const jp_obrs_desc* desc, const void* act
                           float lambda_or_budget, int k, uint64_t seed, uint8_t* out_accept,
                           float* out_weight, float* out_logp_actor, float* out_logp_policy,
                           jp_stats* out_stats);
+
+/* Forward pass with the rollout model known only through what the rollout stored, as in the
+ * paper's own pipeline (Algorithm 1, Phase 1: per token log p_inf(a_t) and TopK_inf(s_t), the
+ * log-probabilities of its k_inf most likely tokens; Phase 2, step 2 builds V_k and Z_approx
+ * from that record).  Only the policy tensor is streamed: half the bytes of jp_obrs_forward.
+ *   policy_logits  : [T, ld] of desc->dtype (DEVICE), each row read once
+ *   logp_inf_token : [T] fp32, log p_inf(a_t)
+ *   topk_inf_idx   : [T, k_inf] int32 token ids of TopK_inf (any order; -1 = empty place)
+ *   topk_inf_logp  : [T, k_inf] fp32 log p_inf of those tokens;  1 <= k_inf <= JP_MAX_TOPK
+ *   k              : size of TopK_new, 1..JP_MAX_TOPK, k < V
+ * Everything else as in jp_obrs_forward: log p_new(a_t) from the streamed row, acceptance
+ * min(1, p_new(a_t) / (lambda p_inf(a_t))) (Eq. obrs_accept), lambda fixed or from a budget,
+ * the accept draws, kappa and the weights (Section 4.4.2, Algorithm 1 step 3).
+ * Z_approx = sum over V_k = TopK_inf U TopK_new of min(p_inf(x), p_new(x) / lambda).  For x in
+ * TopK_new that the record does not hold, p_inf(x) is unknown and the paper does not say what to
+ * take.  Default: the term is left out, so Z_approx stays a lower bound of Z, which the bias
+ * correction of Section 4.4.2 assumes.  With JP_DESC_SPARSE_CAP in desc->flags it is bounded
+ * instead: p_inf(x) <= the smallest stored probability, and all such terms together <= the
+ * mass the record leaves; that is an upper bound of the dense path's Z_approx and may exceed Z.
+ * out_z_lower / out_z_upper ([T] fp32, NULL to skip) give both.  With k_inf = V stored the two
+ * coincide with jp_obrs_forward's exact mode.
+ * Optional outputs of desc: topk_idx_policy, topk_val_policy, accept_prob, uniform, z_approx (the
+ * reading in use), lse_policy; the actor-side ones and JP_DESC_KL are JP_ERR_UNSUPPORTED.  The
+ * records this call leaves do not serve jp_obrs_backward (JP_ERR_STATE): the gradient with
+ * respect to the rollout model's logits needs those logits. */
+jp_status jp_obrs_forward_sparse_actor(jp_ctx* ctx, const jp_obrs_desc* desc, const void* policy_logits,
+                                       const int32_t* tokens, const uint8_t* mask, const float* logp_inf_token,
+                                       const int32_t* topk_inf_idx, const float* topk_inf_logp, int k_inf,
+                                       float lambda_or_budget, int k, uint64_t seed, uint8_t* out_accept,
+                                       float* out_weight, float* out_logp_policy, float* out_z_lower,
+                                       float* out_z_upper, jp_stats* out_stats);
 
 /* Parameters of the backward pass (Eq. obrs_ppo, Eq. ppo_rollout, Eq.
  * distill_loss combined as Eq. sys_joint_obj; the PPO terms are maximised and

@@ -21,10 +21,11 @@ JP_MAX_TOPK = 128
 JP_STATIC_MAX_ROWS = 131072
 JP_ERR_TOO_LARGE = -8
 JP_DESC_KL = 1
+JP_DESC_SPARSE_CAP = 2
 
 EXPORTS = (
     "jp_create", "jp_destroy", "jp_set_stream", "jp_obrs_workspace_bytes", "jp_reserve",
-    "jp_obrs_forward", "jp_obrs_backward", "jp_batch_begin", "jp_batch_chunk", "jp_batch_finalize",
+    "jp_obrs_forward", "jp_obrs_forward_sparse_actor", "jp_obrs_backward", "jp_batch_begin", "jp_batch_chunk", "jp_batch_finalize",
     "jp_obrs_forward_host", "jp_obrs_apply_kappa", "jp_batch_totals", "jp_obrs_apply_totals", "jp_batch_logprobs", "jp_obrs_row_lambda", "jp_vshard_record_floats", "jp_vshard_local", "jp_vshard_local_push", "jp_vshard_merge", "jp_vshard_backward", "jp_budget_lambda_static", "jp_probe_stream", "jp_status_string", "jp_last_error", "jp_launch_count",
     "jp_enable_kernel_timing", "jp_stream_kernel_times",
 )
@@ -99,6 +100,8 @@ def load():
     lib.jp_reserve.argtypes = [vp, i64, i64, ctypes.c_int]
     lib.jp_obrs_forward.argtypes = [vp, ctypes.POINTER(jp_obrs_desc), vp, vp, vp, vp, f32, ctypes.c_int, u64,
                                     vp, vp, vp, vp, vp]
+    lib.jp_obrs_forward_sparse_actor.argtypes = [vp, ctypes.POINTER(jp_obrs_desc), vp, vp, vp, vp, vp, vp, ctypes.c_int,
+                                                 f32, ctypes.c_int, u64, vp, vp, vp, vp, vp, vp]
     lib.jp_obrs_forward_host.argtypes = lib.jp_obrs_forward.argtypes + [i64]
     lib.jp_obrs_backward.argtypes = [vp, ctypes.POINTER(jp_obrs_desc), ctypes.POINTER(jp_obrs_bwd_desc),
                                      vp, vp, vp, vp, vp, vp, vp, vp]
@@ -212,6 +215,16 @@ def jp_obrs_forward(ctx: Context, desc: jp_obrs_desc, actor_logits, policy_logit
                                       _ptr(tokens), _ptr(mask), lambda_or_budget, k, seed,
                                       _ptr(out_accept), _ptr(out_weight), _ptr(out_logp_actor),
                                       _ptr(out_logp_policy), _ptr(out_stats)))
+
+
+def jp_obrs_forward_sparse_actor(ctx: Context, desc: jp_obrs_desc, policy_logits, tokens, mask, logp_inf_token,
+                                 topk_inf_idx, topk_inf_logp, k_inf: int, lambda_or_budget: float, k: int, seed: int,
+                                 out_accept, out_weight, out_logp_policy, out_z_lower, out_z_upper, out_stats):
+    ctx.check(ctx.lib.jp_obrs_forward_sparse_actor(ctx.h, ctypes.byref(desc), _ptr(policy_logits), _ptr(tokens),
+                                                   _ptr(mask), _ptr(logp_inf_token), _ptr(topk_inf_idx),
+                                                   _ptr(topk_inf_logp), k_inf, lambda_or_budget, k, seed,
+                                                   _ptr(out_accept), _ptr(out_weight), _ptr(out_logp_policy),
+                                                   _ptr(out_z_lower), _ptr(out_z_upper), _ptr(out_stats)))
 
 
 def jp_obrs_forward_host(ctx: Context, desc: jp_obrs_desc, actor_logits, policy_logits, tokens, mask,

@@ -32,6 +32,7 @@ struct jp_ctx {
   int64_t rec_V = 0;
   int rec_k = 0;                 // 0 = exact mode
   bool rec_kl = false;           // the records hold KL(p || q) of every streamed row
+  bool rec_sparse = false;       // the records come from the sparse-actor forward: no actor log-sum-exp in them
   int32_t rec_dtype = 0;
   bool batch_open = false;
   bool batch_exact = false;
@@ -192,12 +193,14 @@ jp_status extra_pass(jp_ctx* c, const jp_obrs_desc* d, int64_t ld, int64_t recor
 
 // Streams one block of rows into the records at record_offset.
 jp_status stream_rows(jp_ctx* c, const jp_obrs_desc* d, int64_t ld, int k_eff, int64_t record_offset,
-                      const void* za, const void* zp, const int32_t* tokens, const uint8_t* mask) {
+                      const void* za, const void* zp, const int32_t* tokens, const uint8_t* mask,
+                      const float* logp_inf = nullptr) {
   if (d->T == 0) return JP_OK;
-  if (!za || !zp || !tokens) return fail(c, JP_ERR_INVALID_ARG, "logits or tokens pointer is NULL");
+  // za == NULL with logp_inf: the policy tensor alone is streamed (sparse-actor forward)
+  if ((!za && !logp_inf) || !zp || !tokens) return fail(c, JP_ERR_INVALID_ARG, "logits or tokens pointer is NULL");
   if (!aligned16(za) || !aligned16(zp)) return fail(c, JP_ERR_ALIGNMENT, "logit base pointers must be 16-byte aligned");
   StreamArgs a{};
-  a.za = za; a.zp = zp; a.tokens = tokens; a.mask = mask;
+  a.za = za; a.zp = zp; a.tokens = tokens; a.mask = mask; a.logp_inf = logp_inf;
   a.T = d->T; a.V = d->V; a.ld = ld; a.dtype = d->dtype; a.k = k_eff;
   a.record_offset = record_offset; a.rec = c->rec; a.sc = c->sc; a.list = c->list; a.spill = c->spill;
   const int slot = (int)(c->ev_count % jp_ctx::kEvRing);
@@ -354,6 +357,7 @@ jp_status jp_obrs_forward(jp_ctx* c, const jp_obrs_desc* d, const void* za, cons
   c->launches += 1;
   c->have_records = false;
   c->rec_kl = want_kl;
+  c->rec_sparse = false;
   st = stream_rows(c, d, ld, k_eff, 0, za, zp, tokens, mask);
   if (st != JP_OK) return st;
   // the exact Z needs lambda: with a budget it has to wait for the solve; the divergence does not
@@ -372,6 +376,64 @@ jp_status jp_obrs_forward(jp_ctx* c, const jp_obrs_desc* d, const void* za, cons
   if (e != cudaSuccess) return cuda_fail(c, e, "epilogue launch");
   c->have_records = true;
   c->rec_rows = d->T; c->rec_V = d->V; c->rec_k = k_eff; c->rec_dtype = d->dtype;
+  return JP_OK;
+}
+
+jp_status jp_obrs_forward_sparse_actor(jp_ctx* c, const jp_obrs_desc* d, const void* zp, const int32_t* tokens,
+                                       const uint8_t* mask, const float* logp_inf_token, const int32_t* topk_inf_idx,
+                                       const float* topk_inf_logp, int k_inf, float lambda_or_budget, int k,
+                                       uint64_t seed, uint8_t* out_accept, float* out_weight, float* out_lp,
+                                       float* out_z_lower, float* out_z_upper, jp_stats* out_stats) {
+  if (!c) return JP_ERR_INVALID_ARG;
+  int64_t ld = 0;
+  jp_status st = check_shape(c, d, &ld);
+  if (st != JP_OK) return st;
+  if (k < 1 || k > JP_MAX_TOPK || (int64_t)k >= d->V)
+    return fail(c, JP_ERR_UNSUPPORTED, "the sparse-actor forward takes 1 <= k <= JP_MAX_TOPK, k < V");
+  if (k_inf < 1 || k_inf > JP_MAX_TOPK) return fail(c, JP_ERR_UNSUPPORTED, "1 <= k_inf <= JP_MAX_TOPK");
+  if ((st = check_lambda(c, lambda_or_budget, d->lambda_mode)) != JP_OK) return st;
+  if (c->batch_open) return fail(c, JP_ERR_STATE, "a chunked batch is open: finalize it first");
+  if (d->flags & JP_DESC_KL) return fail(c, JP_ERR_UNSUPPORTED, "KL(p || q) needs the rollout model's full logits");
+  if (d->topk_idx_actor || d->topk_val_actor || d->z_exact || d->lse_actor)
+    return fail(c, JP_ERR_UNSUPPORTED, "actor-side optional outputs do not exist without the actor's logits");
+  if (d->T > 0 && (!logp_inf_token || !topk_inf_idx || !topk_inf_logp))
+    return fail(c, JP_ERR_INVALID_ARG, "a pointer of the rollout record is NULL");
+  cudaSetDevice(c->device);
+  if ((st = ensure_workspace(c, d->T > 0 ? d->T : 1, k)) != JP_OK) return st;
+  const bool budget = d->lambda_mode == JP_LAMBDA_FROM_BUDGET;
+  cudaError_t e = launch_reset(c->sc, budget ? 1.0f : lambda_or_budget, c->stream);
+  if (e != cudaSuccess) return cuda_fail(c, e, "reset launch");
+  c->launches += 1;
+  c->have_records = false;
+  c->rec_kl = false;
+  c->rec_sparse = true;
+  if ((st = stream_rows(c, d, ld, k, 0, nullptr, zp, tokens, mask, logp_inf_token)) != JP_OK) return st;
+  // the epilogue takes Z_approx as given (k = 0): the kernel below has computed it from the record
+  jp_obrs_desc dd = *d;
+  dd.topk_idx_policy = nullptr; dd.topk_val_policy = nullptr;
+  EpilogueArgs ea = epilogue_args(c, &dd, d->T, 0, seed, d->token_offset, d->c1, out_accept, out_weight, nullptr,
+                                  out_lp, out_stats);
+  int nl = 0;
+  if (budget) {
+    e = launch_budget_solve(ea, (double)lambda_or_budget, c->stream, &nl);
+    if (e != cudaSuccess) return cuda_fail(c, e, "budget solve launch");
+  }
+  if (d->T > 0) {
+    SparseZArgs z{};
+    z.zp = zp; z.T = d->T; z.V = d->V; z.ld = ld; z.dtype = d->dtype; z.k = k; z.k_inf = k_inf;
+    z.cap = (d->flags & JP_DESC_SPARSE_CAP) ? 1 : 0;
+    z.inf_idx = topk_inf_idx; z.inf_logp = topk_inf_logp; z.rec = c->rec; z.sc = c->sc;
+    z.out_z_lower = out_z_lower; z.out_z_upper = out_z_upper;
+    z.out_idx_p = d->topk_idx_policy; z.out_val_p = d->topk_val_policy;
+    e = launch_sparse_z(z, c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e, "sparse Z launch");
+    nl += 1;
+  }
+  e = launch_epilogue(ea, c->stream, &nl);
+  c->launches += nl;
+  if (e != cudaSuccess) return cuda_fail(c, e, "epilogue launch");
+  c->have_records = true;
+  c->rec_rows = d->T; c->rec_V = d->V; c->rec_k = k; c->rec_dtype = d->dtype;
   return JP_OK;
 }
 
@@ -397,6 +459,7 @@ jp_status jp_batch_begin(jp_ctx* c, int64_t T_total, int64_t V, int32_t dtype, i
   c->batch_exact = exact;
   c->have_records = false;
   c->rec_kl = T_total > 0;       // stays true only if every chunk asks for the divergence
+  c->rec_sparse = false;
   c->rec_rows = T_total; c->rec_V = V; c->rec_k = k_eff; c->rec_dtype = dtype;
   return JP_OK;
 }
@@ -541,6 +604,7 @@ jp_status jp_vshard_merge(jp_ctx* c, int n_shards, int my_shard, const float* ga
   c->batch_open = true;
   c->batch_exact = false;
   c->rec_kl = false;             // the divergence needs whole rows
+  c->rec_sparse = false;
   c->rec_rows = T; c->rec_V = V_total; c->rec_k = k;
   return JP_OK;
 }
@@ -630,6 +694,7 @@ jp_status backward_impl(jp_ctx* c, const jp_obrs_desc* d, const jp_obrs_bwd_desc
   if (st != JP_OK) return st;
   if (!b) return fail(c, JP_ERR_INVALID_ARG, "bwd desc is NULL");
   if (!c->have_records) return fail(c, JP_ERR_STATE, "no forward records in this context: run the forward (or finalize the batch) first");
+  if (c->rec_sparse) return fail(c, JP_ERR_STATE, "the records come from jp_obrs_forward_sparse_actor: the gradients need both models' log-sum-exps (run jp_obrs_forward)");
   const bool slice = slice_offset >= 0;
   if (!slice && (d->V != c->rec_V || d->dtype != c->rec_dtype)) return fail(c, JP_ERR_STATE, "V / dtype differ from the forward that left the records");
   if (slice && d->dtype != c->rec_dtype) return fail(c, JP_ERR_STATE, "dtype differs from the forward that left the records");

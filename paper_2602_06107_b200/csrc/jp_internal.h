@@ -71,8 +71,9 @@ struct SolvePartials {
 };
 
 struct StreamArgs {
-  const void* za;
+  const void* za;          // null: only the policy tensor is streamed (sparse-actor forward)
   const void* zp;
+  const float* logp_inf;   // [T] log p_inf(a_t) from the rollout record (only with za == null)
   const int32_t* tokens;
   const uint8_t* mask;
   int64_t T, V, ld;
@@ -154,6 +155,23 @@ struct GradArgs {
   double* out_loss;
 };
 
+// Z_approx from a stored rollout record (jp_sparse.cu).
+struct SparseZArgs {
+  const void* zp;
+  int64_t T, V, ld;
+  int32_t dtype;
+  int32_t k, k_inf;
+  int32_t cap;             // 0: unknown actor terms left out; 1: capped by what the record implies
+  const int32_t* inf_idx;  // [T, k_inf]
+  const float* inf_logp;   // [T, k_inf]
+  Records rec;
+  Scalars* sc;
+  float* out_z_lower;      // [T] or null
+  float* out_z_upper;      // [T] or null
+  int32_t* out_idx_p;      // [T, k] or null
+  float* out_val_p;        // [T, k] or null
+};
+
 struct RowLambdaArgs {
   const void* za;
   const void* zp;
@@ -181,6 +199,7 @@ cudaError_t launch_reweight_totals(int64_t T, const Records& rec, Scalars* sc, c
                                    float* out_weight, jp_stats* out_stats, cudaStream_t s);
 cudaError_t launch_logprobs(int64_t T, const Records& rec, float* out_lq, float* out_lp, uint8_t* out_valid,
                             cudaStream_t s);
+cudaError_t launch_sparse_z(const SparseZArgs& a, cudaStream_t s);
 cudaError_t launch_row_lambda(const RowLambdaArgs& a, cudaStream_t s, int sms);
 
 // Vocabulary shards (jp_vshard.cu).  Packed per-row record of one shard, in 4-byte words:

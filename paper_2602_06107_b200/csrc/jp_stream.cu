@@ -773,7 +773,7 @@ __device__ __forceinline__ void raise_timeout(SM& sm, Scalars* sc) {
 }
 
 // ---- producer ---------------------------------------------------------------
-template <int DT, class SM>
+template <int DT, bool SINGLE, class SM>
 __device__ void producer_loop(const StreamArgs& A, SM& sm, int64_t n_rows) {
   constexpr int N = Vec<DT>::N;
   constexpr int STAGES = SM::STAGES;
@@ -801,8 +801,8 @@ __device__ void producer_loop(const StreamArgs& A, SM& sm, int64_t n_rows) {
       const uint32_t bytes = tile == ntiles - 1 ? last_bytes : (uint32_t)(TV * 16);
       const int grp = (tile + g0) % NG;
       if (bytes > 0) {
-        mbar_arrive_expect_tx(&sm.full[grp][s], 2u * bytes);
-        bulk_g2s(&sm.ring[s][0][0], ra, bytes, &sm.full[grp][s], policy);
+        mbar_arrive_expect_tx(&sm.full[grp][s], SINGLE ? bytes : 2u * bytes);
+        if (!SINGLE) bulk_g2s(&sm.ring[s][0][0], ra, bytes, &sm.full[grp][s], policy);
         bulk_g2s(&sm.ring[s][1][0], rp, bytes, &sm.full[grp][s], policy);
       } else {
         mbar_arrive(&sm.full[grp][s]);
@@ -829,7 +829,7 @@ __device__ void producer_loop(const StreamArgs& A, SM& sm, int64_t n_rows) {
 }
 
 // ---- consumers ----------------------------------------------------------------
-template <int DT, bool TOPK, bool UNROLL, class SM>
+template <int DT, bool TOPK, bool UNROLL, bool SINGLE, class SM>
 __device__ void consumer_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int cw, int lane) {
   constexpr int N = Vec<DT>::N;
   constexpr int STAGES = SM::STAGES, CAP = SM::CAP;
@@ -870,18 +870,22 @@ __device__ void consumer_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int c
         for (int h = 0; h < VPL / HV; ++h, sa += HV * WPT * 32, sp += HV * WPT * 32, id += WPT * 32) {
           uint4 va[HV], vp[HV];
 #pragma unroll
-          for (int j = 0; j < HV; ++j) { va[j] = sa[j * WPT * 32]; vp[j] = sp[j * WPT * 32]; }
+          for (int j = 0; j < HV; ++j) {
+            if (!SINGLE) va[j] = sa[j * WPT * 32];
+            vp[j] = sp[j * WPT * 32];
+          }
           // one maximum and one check against the reference exponent per tensor per pass
-          const float ma = Vec<DT>::vmax2(va[0], va[1]), mp = Vec<DT>::vmax2(vp[0], vp[1]);
-          raise_max(ma, oa);
+          float ma = JP_NEG_INF;
+          if (!SINGLE) { ma = Vec<DT>::vmax2(va[0], va[1]); raise_max(ma, oa); }
+          const float mp = Vec<DT>::vmax2(vp[0], vp[1]);
           raise_max(mp, op);
 #pragma unroll
           for (int j = 0; j < HV; ++j) {
-            add_terms<DT>(va[j], oa);
+            if (!SINGLE) add_terms<DT>(va[j], oa);
             add_terms<DT>(vp[j], op);
           }
           if (TOPK) {
-            if (ma >= ta) record_hit<CAP>(&sm.ncand[p][0], sm.cand[p][0], A.spill, 2 * p, id, idmask, ma);
+            if (!SINGLE && ma >= ta) record_hit<CAP>(&sm.ncand[p][0], sm.cand[p][0], A.spill, 2 * p, id, idmask, ma);
             if (mp >= tp) record_hit<CAP>(&sm.ncand[p][1], sm.cand[p][1], A.spill, 2 * p + 1, id, idmask, mp);
           }
         }
@@ -896,16 +900,16 @@ __device__ void consumer_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int c
           for (int j = 0; j < HV; ++j) {
             const int o = (h * HV + j) * WPT * 32;
             uint4 a4 = Vec<DT>::neg_inf(), p4 = Vec<DT>::neg_inf();
-            if ((int64_t)(v0 + o) < nvec) { a4 = sa[o]; p4 = sp[o]; }
+            if ((int64_t)(v0 + o) < nvec) { if (!SINGLE) a4 = sa[o]; p4 = sp[o]; }
             const float vm_a = Vec<DT>::vmax(a4), vm_p = Vec<DT>::vmax(p4);
-            accumulate<DT>(a4, vm_a, oa);
+            if (!SINGLE) accumulate<DT>(a4, vm_a, oa);
             accumulate<DT>(p4, vm_p, op);
             ma = fmaxf(ma, vm_a);
             mp = fmaxf(mp, vm_p);
           }
           // a pass with no vector inside the row holds nothing
           if (TOPK && (int64_t)(v0 + h * HV * WPT * 32) < nvec) {
-            if (ma >= ta) record_hit<CAP>(&sm.ncand[p][0], sm.cand[p][0], A.spill, 2 * p, id, idmask, ma);
+            if (!SINGLE && ma >= ta) record_hit<CAP>(&sm.ncand[p][0], sm.cand[p][0], A.spill, 2 * p, id, idmask, ma);
             if (mp >= tp) record_hit<CAP>(&sm.ncand[p][1], sm.cand[p][1], A.spill, 2 * p + 1, id, idmask, mp);
           }
         }
@@ -931,9 +935,11 @@ __device__ void consumer_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int c
       const int64_t row = A.list[it];
       const char* ra = (const char*)A.za + row * A.ld * Vec<DT>::ESIZE;
       const char* rp = (const char*)A.zp + row * A.ld * Vec<DT>::ESIZE;
-      const uint4 ta = load_tail_vector<DT>(ra, nvec * N, tail);
+      if (!SINGLE) {
+        const uint4 ta = load_tail_vector<DT>(ra, nvec * N, tail);
+        accumulate<DT>(ta, Vec<DT>::vmax(ta), oa);
+      }
       const uint4 tp = load_tail_vector<DT>(rp, nvec * N, tail);
-      accumulate<DT>(ta, Vec<DT>::vmax(ta), oa);
       accumulate<DT>(tp, Vec<DT>::vmax(tp), op);
     }
 
@@ -962,7 +968,7 @@ __device__ void consumer_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int c
 
 // ---- top-k warps ---------------------------------------------------------------
 // One warp per (row slot p, tensor t); it owns rows p, p + NSLOT, ... of the CTA.
-template <int DT, int KPL, class SM>
+template <int DT, int KPL, bool SINGLE, class SM>
 __device__ void topk_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int t, int p, int lane) {
   constexpr int N = Vec<DT>::N;
   constexpr int CAP = SM::CAP;
@@ -982,6 +988,15 @@ __device__ void topk_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int t, in
   for (int64_t it = (int64_t)blockIdx.x + (int64_t)p * gridDim.x; it < n_rows;
        it += (int64_t)NSLOT * gridDim.x, lr += NSLOT) {
     const uint32_t ph = (uint32_t)((lr / NSLOT) & 1);
+    if (SINGLE && t == 0) {
+      // one tensor only (the rollout model is known through its stored record): this warp has no
+      // list to build; it keeps the slot's hand-shake going
+      if (lane == 0) sm.g0[p] = first_group(A.record_offset + A.list[it]);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sm.slot_ready[p]);
+      if (!mbar_wait(&sm.row_done[p], ph, &sm.abort)) { raise_timeout(sm, A.sc); return; }
+      continue;
+    }
     if (TOPK && lr >= 2) {
       // Do not look at the row before the consumers are one row away from it (the row two
       // before it is done): the sample then still sits in L2 when the row streams, instead
@@ -1095,7 +1110,7 @@ __device__ void topk_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int t, in
           if (key != 0ull) {
             const uint32_t idx = key_index(key);
             A.rec.idx[o] = (int32_t)idx;
-            A.rec.za[o] = Vec<DT>::load_scalar(ra, idx);
+            A.rec.za[o] = SINGLE ? 0.f : Vec<DT>::load_scalar(ra, idx);
             A.rec.zp[o] = Vec<DT>::load_scalar(rp, idx);
           } else {
             A.rec.idx[o] = -1; A.rec.za[o] = 0.f; A.rec.zp[o] = 0.f;
@@ -1124,12 +1139,18 @@ __device__ void topk_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int t, in
       const float lo = (float)(lse - (double)lsef);
       if (t == 0) { A.rec.lse_a[rrow] = lsef; A.rec.lse_a_lo[rrow] = lo; A.rec.lq[rrow] = lpx; A.rec.flag[rrow] = kRowValid; }
       else        { A.rec.lse_p[rrow] = lsef; A.rec.lse_p_lo[rrow] = lo; A.rec.lp[rrow] = lpx; }
+      if (SINGLE) {
+        // log p_inf(a_t) comes from the rollout record, not from a row of logits
+        A.rec.lse_a[rrow] = 0.f; A.rec.lse_a_lo[rrow] = 0.f;
+        A.rec.lq[rrow] = A.logp_inf[row];
+        A.rec.flag[rrow] = kRowValid;
+      }
     }
     __syncwarp();
   }
 }
 
-template <int DT, int KPL>
+template <int DT, int KPL, bool SINGLE>
 __global__ void __launch_bounds__(NTHREADS, 1) stream_kernel(StreamArgs A) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   using SM = StreamSmemFor<KPL>;
@@ -1153,14 +1174,14 @@ __global__ void __launch_bounds__(NTHREADS, 1) stream_kernel(StreamArgs A) {
   const int64_t n_rows = A.sc->n_list;
 
   if (warp == 0) {
-    if (lane == 0) producer_loop<DT, SM>(A, sm, n_rows);
+    if (lane == 0) producer_loop<DT, SINGLE, SM>(A, sm, n_rows);
   } else if (warp <= NC) {
     // (unrolling a tile's two passes saves 3 % of the instructions; the kernel for the longest
     // lists is faster with them rolled)
-    consumer_loop<DT, (KPL > 0), (KPL != 4), SM>(A, sm, n_rows, warp - 1, lane);
+    consumer_loop<DT, (KPL > 0), (KPL != 4), SINGLE, SM>(A, sm, n_rows, warp - 1, lane);
   } else {
     const int tw = warp - 1 - NC;
-    topk_loop<DT, KPL, SM>(A, sm, n_rows, tw & 1, tw >> 1, lane);
+    topk_loop<DT, KPL, SINGLE, SM>(A, sm, n_rows, tw & 1, tw >> 1, lane);
   }
 }
 
@@ -1306,14 +1327,33 @@ int stream_grid_size(int device) {
   return sms;
 }
 
-template <int DT, int KPL>
+template <int DT, int KPL, bool SINGLE>
 static cudaError_t launch_stream_variant(const StreamArgs& a, cudaStream_t s, int grid) {
   // per device, and cheap: set on every launch rather than cached per process
-  cudaError_t e = cudaFuncSetAttribute(stream_kernel<DT, KPL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(stream_kernel<DT, KPL, SINGLE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)sizeof(StreamSmemFor<KPL>));
   if (e != cudaSuccess) return e;
-  stream_kernel<DT, KPL><<<grid, NTHREADS, sizeof(StreamSmemFor<KPL>), s>>>(a);
+  stream_kernel<DT, KPL, SINGLE><<<grid, NTHREADS, sizeof(StreamSmemFor<KPL>), s>>>(a);
   return cudaGetLastError();
+}
+
+template <int DT>
+static cudaError_t launch_stream_dt(const StreamArgs& a, cudaStream_t s, int grid) {
+  const int kpl = a.k <= 0 ? 0 : a.k <= 32 ? 1 : a.k <= 64 ? 2 : 4;
+  if (a.za == nullptr) {           // the policy tensor alone (the rollout model comes as a stored record)
+    switch (kpl) {
+      case 0: return cudaErrorInvalidValue;
+      case 1: return launch_stream_variant<DT, 1, true>(a, s, grid);
+      case 2: return launch_stream_variant<DT, 2, true>(a, s, grid);
+      default: return launch_stream_variant<DT, 4, true>(a, s, grid);
+    }
+  }
+  switch (kpl) {
+    case 0: return launch_stream_variant<DT, 0, false>(a, s, grid);
+    case 1: return launch_stream_variant<DT, 1, false>(a, s, grid);
+    case 2: return launch_stream_variant<DT, 2, false>(a, s, grid);
+    default: return launch_stream_variant<DT, 4, false>(a, s, grid);
+  }
 }
 
 cudaError_t launch_stream(const StreamArgs& a, cudaStream_t s, int sms) {
@@ -1323,21 +1363,7 @@ cudaError_t launch_stream(const StreamArgs& a, cudaStream_t s, int sms) {
   if (e != cudaSuccess) return e;
   int grid = (int)(a.T < sms ? a.T : sms);
   if (grid > kStreamMaxCtas) grid = kStreamMaxCtas;      // the spill area is laid out for that many CTAs
-  const int kpl = a.k <= 0 ? 0 : a.k <= 32 ? 1 : a.k <= 64 ? 2 : 4;
-  if (a.dtype == JP_BF16) {
-    switch (kpl) {
-      case 0: return launch_stream_variant<JP_BF16, 0>(a, s, grid);
-      case 1: return launch_stream_variant<JP_BF16, 1>(a, s, grid);
-      case 2: return launch_stream_variant<JP_BF16, 2>(a, s, grid);
-      default: return launch_stream_variant<JP_BF16, 4>(a, s, grid);
-    }
-  }
-  switch (kpl) {
-    case 0: return launch_stream_variant<JP_F32, 0>(a, s, grid);
-    case 1: return launch_stream_variant<JP_F32, 1>(a, s, grid);
-    case 2: return launch_stream_variant<JP_F32, 2>(a, s, grid);
-    default: return launch_stream_variant<JP_F32, 4>(a, s, grid);
-  }
+  return a.dtype == JP_BF16 ? launch_stream_dt<JP_BF16>(a, s, grid) : launch_stream_dt<JP_F32>(a, s, grid);
 }
 
 template <int DT>

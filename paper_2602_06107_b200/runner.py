@@ -90,3 +90,31 @@ def backward(ctx: B.Context, za, zp, tokens, mask, accept, weight, *, advantages
     else:
         B.jp_vshard_backward(ctx, desc, bwd, za, zp, tokens, mask, vocab_offset, accept, weight, d_actor, d_policy)
     return d_actor, d_policy
+
+
+def forward_sparse_actor(ctx: B.Context, zp, tokens, mask, logp_inf_token, topk_inf_idx, topk_inf_logp, *, lam=None,
+                         budget=None, k=20, seed=0, token_offset=0, c1=0.0, cap=False, aux=True):
+    """One jp_obrs_forward_sparse_actor call; returns a dict of device tensors plus ``stats``."""
+    assert (lam is None) != (budget is None)
+    T, V = zp.shape
+    dev = zp.device
+    out = _alloc_outputs(T, dev)
+    del out["logp_actor"]
+    out["z_lower"] = torch.empty(T, dtype=torch.float32, device=dev)
+    out["z_upper"] = torch.empty(T, dtype=torch.float32, device=dev)
+    auxd = {}
+    if aux:
+        auxd = {n: torch.empty(T, dtype=torch.float32, device=dev) for n in ("accept_prob", "uniform", "z_approx",
+                                                                              "lse_policy")}
+        auxd["topk_idx_policy"] = torch.empty((T, k), dtype=torch.int32, device=dev)
+        auxd["topk_val_policy"] = torch.empty((T, k), dtype=torch.float32, device=dev)
+    mode = B.JP_LAMBDA_FIXED if budget is None else B.JP_LAMBDA_FROM_BUDGET
+    desc = B.make_desc(zp, lambda_mode=mode, c1=c1, token_offset=token_offset, aux=auxd,
+                       flags=B.JP_DESC_SPARSE_CAP if cap else 0)
+    B.jp_obrs_forward_sparse_actor(ctx, desc, zp, tokens, mask, logp_inf_token, topk_inf_idx, topk_inf_logp,
+                                   topk_inf_idx.shape[1], lam if budget is None else budget, k, seed, out["accept"],
+                                   out["weight"], out["logp_policy"], out["z_lower"], out["z_upper"], out["stats_buf"])
+    out.update(auxd)
+    torch.cuda.synchronize(dev)
+    out["stats"] = B.read_stats(out["stats_buf"])
+    return out
