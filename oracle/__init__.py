@@ -214,6 +214,20 @@ def forward_sparse(zp, tokens, logp_inf_token, inf_idx, inf_logp, mask=None, *, 
     return r
 
 
+def lmhead_rows(rows, hidden, weight):
+    """fp32 logits of the given rows of an output layer: hidden [T, H] and weight [V, H] as bf16 bit
+    patterns (uint16); products and sums in double, one rounding."""
+    rows = np.ascontiguousarray(rows, dtype=np.int64)
+    assert hidden.dtype == np.uint16 and weight.dtype == np.uint16 and hidden.shape[1] == weight.shape[1]
+    hidden, weight = np.ascontiguousarray(hidden), np.ascontiguousarray(weight)
+    H, V = hidden.shape[1], weight.shape[0]
+    out = np.zeros((rows.shape[0], V), dtype=np.float32)
+    lib().jo_lmhead_rows(ctypes.c_int64(rows.shape[0]), _p(rows, ctypes.c_int64), ctypes.c_int64(H), ctypes.c_int64(V),
+                         _p(hidden, ctypes.c_uint16), ctypes.c_int64(H), _p(weight, ctypes.c_uint16),
+                         ctypes.c_int64(H), _p(out, ctypes.c_float))
+    return out
+
+
 _STAT_KEYS = ("n_valid", "n_accept", "alpha_hat", "mean_accept_prob", "z_approx_mean", "kappa",
               "lambda_used")
 

@@ -299,6 +299,24 @@ void jo_z_sparse(int64_t T, int64_t V, int64_t ld, int dtype, const void* zp, co
   }
 }
 
+// Logits of an output layer for a set of rows: z[t, v] = sum_h hidden[t, h] * weight[v, h], both
+// operands bf16 (every product is exact in double), summed in double in ascending h, rounded once
+// to fp32.  (Section 4.4: the logit tensor the method consumes is the output of this product; a
+// fused pass forms it tile by tile and never stores it.)
+void jo_lmhead_rows(int64_t n_rows, const int64_t* rows, int64_t H, int64_t V, const uint16_t* hidden,
+                    int64_t ld_hidden, const uint16_t* weight, int64_t ld_weight, float* out) {
+#pragma omp parallel for schedule(dynamic, 64) collapse(2)
+  for (int64_t i = 0; i < n_rows; ++i) {
+    for (int64_t v = 0; v < V; ++v) {
+      const uint16_t* hr = hidden + rows[i] * ld_hidden;
+      const uint16_t* wr = weight + v * ld_weight;
+      double acc = 0.0;
+      for (int64_t h = 0; h < H; ++h) acc += logit_at(hr, 0, h) * logit_at(wr, 0, h);
+      out[i * V + v] = (float)acc;
+    }
+  }
+}
+
 // Step 7b: the exact normaliser Z = sum_{x'} min(p_inf(x'), p_target(x')/lambda)
 // over the whole vocabulary (Eq. obrs_dist; Appendix A, Z_C).
 void jo_z_exact(int64_t T, int64_t V, int64_t ld, int dtype, const void* za, const void* zp,

@@ -694,3 +694,24 @@ def test_sparse_forward_reduces_to_the_dense_forward_when_everything_is_stored()
     assert sp["stats"]["kappa"] * sp["stats"]["z_approx_mean"] == pytest.approx(sp["stats"]["alpha_hat"], rel=1e-12)
     b = oracle.forward_sparse(zp, tok, lq, inf_idx, inf_logp, mask, budget=0.6, k=k, seed=5)
     assert b["stats"]["mean_accept_prob"] == pytest.approx(0.6, abs=1e-6)
+
+
+# ------------------------------------------------------------------ output layer (fused pass)
+
+def test_lmhead_rows_is_the_matrix_product():
+    """The oracle's logits of an output layer against numpy's matmul on the exactly widened operands
+    (every bf16 x bf16 product is exact in double; numpy's summation order may differ, hence 1e-12),
+    and against a hand-worked 2 x 3 case."""
+    rng = np.random.default_rng(93)
+    T, H, V = 7, 96, 37
+    hb = _to_bf16_bits(rng.normal(0, 1, (T, H)).astype(np.float32))
+    wb = _to_bf16_bits(rng.normal(0, 1, (V, H)).astype(np.float32))
+    rows = np.array([6, 0, 3])
+    z = oracle.lmhead_rows(rows, hb, wb)
+    want = _bf16_bits_to_f64(hb)[rows] @ _bf16_bits_to_f64(wb).T
+    assert z.dtype == np.float32 and z.shape == (3, V)
+    assert np.array_equal(z, want.astype(np.float32)) or np.allclose(z, want, rtol=1e-7, atol=1e-12)
+    h2 = _to_bf16_bits(np.array([[1.0, 2.0, -0.5], [0.25, 0.0, 4.0]], np.float32))
+    w2 = _to_bf16_bits(np.array([[2.0, 1.0, 1.0], [-1.0, 0.5, 8.0]], np.float32))
+    z2 = oracle.lmhead_rows(np.arange(2), h2, w2)
+    assert z2.tolist() == [[3.5, -4.0], [4.5, 31.75]]
