@@ -173,6 +173,30 @@ jp_status jp_obrs_forward_sparse_actor(jp_ctx* ctx, const jp_obrs_desc* desc, co
                                        float* out_weight, float* out_logp_policy, float* out_z_lower,
                                        float* out_z_upper, jp_stats* out_stats);
 
+/* The row pass fused into the output layer, for one model (Section 4.4 names the
+ * [tokens, vocabulary] logit tensor as the method's memory bottleneck; here it is never
+ * written).  logits z[t, v] = sum_h hidden[t, h] * weight[v, h]: bf16 operands, fp32
+ * accumulation on the tensor cores; the logits keep that fp32 value (they are not rounded to
+ * bf16 as a stored logit tensor would be).  Per row t the call yields
+ *   out_lse [T] fp32         log sum_v exp z[t, v]
+ *   out_logp_token [T] fp32  z[t, tokens[t]] - lse
+ *   out_topk_idx / out_topk_val [T, k]  the k largest logits, best first, equal values by lower
+ *                            index, and their values; 1 <= k <= 32
+ * which is what Algorithm 1 keeps of a forward pass (Phase 1: log p(a_t) and the top-k
+ * log-probabilities; Phase 2 step 1 likewise for the policy).
+ *   hidden : [T, ld_hidden] bf16, weight : [V, ld_weight] bf16 (the output layer's matrix, one row
+ *            per vocabulary entry), both DEVICE, 16-byte aligned, pitches multiples of 16 bytes
+ *            (ld = 0 means H); tokens [T] int32; mask [T] uint8 or NULL
+ *   out_status : one int32 in DEVICE memory (may be NULL): 0, or JP_ERR_TIMEOUT if a wait inside
+ *            the kernel ran out (results are then unspecified)
+ * Rows with mask 0 or a token id outside [0, V) give lse = logp = 0 and indices -1.  Work is
+ * enqueued on the context's stream; the context keeps a scratch buffer for partial results
+ * (cudaMalloc on first use or growth). */
+jp_status jp_lmhead_lse_topk(jp_ctx* ctx, const void* hidden, int64_t ld_hidden, const void* weight,
+                             int64_t ld_weight, const int32_t* tokens, const uint8_t* mask, int64_t T,
+                             int64_t H, int64_t V, int k, float* out_lse, float* out_logp_token,
+                             int32_t* out_topk_idx, float* out_topk_val, int32_t* out_status);
+
 /* Parameters of the backward pass (Eq. obrs_ppo, Eq. ppo_rollout, Eq.
  * distill_loss combined as Eq. sys_joint_obj; the PPO terms are maximised and
  * the distillation term minimised, so the loss is

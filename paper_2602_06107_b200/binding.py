@@ -25,7 +25,7 @@ JP_DESC_SPARSE_CAP = 2
 
 EXPORTS = (
     "jp_create", "jp_destroy", "jp_set_stream", "jp_obrs_workspace_bytes", "jp_reserve",
-    "jp_obrs_forward", "jp_obrs_forward_sparse_actor", "jp_obrs_backward", "jp_batch_begin", "jp_batch_chunk", "jp_batch_finalize",
+    "jp_obrs_forward", "jp_obrs_forward_sparse_actor", "jp_lmhead_lse_topk", "jp_obrs_backward", "jp_batch_begin", "jp_batch_chunk", "jp_batch_finalize",
     "jp_obrs_forward_host", "jp_obrs_apply_kappa", "jp_batch_totals", "jp_obrs_apply_totals", "jp_batch_logprobs", "jp_obrs_row_lambda", "jp_vshard_record_floats", "jp_vshard_local", "jp_vshard_local_push", "jp_vshard_merge", "jp_vshard_backward", "jp_budget_lambda_static", "jp_probe_stream", "jp_status_string", "jp_last_error", "jp_launch_count",
     "jp_enable_kernel_timing", "jp_stream_kernel_times",
 )
@@ -102,6 +102,7 @@ def load():
                                     vp, vp, vp, vp, vp]
     lib.jp_obrs_forward_sparse_actor.argtypes = [vp, ctypes.POINTER(jp_obrs_desc), vp, vp, vp, vp, vp, vp, ctypes.c_int,
                                                  f32, ctypes.c_int, u64, vp, vp, vp, vp, vp, vp]
+    lib.jp_lmhead_lse_topk.argtypes = [vp, vp, i64, vp, i64, vp, vp, i64, i64, i64, ctypes.c_int, vp, vp, vp, vp, vp]
     lib.jp_obrs_forward_host.argtypes = lib.jp_obrs_forward.argtypes + [i64]
     lib.jp_obrs_backward.argtypes = [vp, ctypes.POINTER(jp_obrs_desc), ctypes.POINTER(jp_obrs_bwd_desc),
                                      vp, vp, vp, vp, vp, vp, vp, vp]
@@ -225,6 +226,16 @@ def jp_obrs_forward_sparse_actor(ctx: Context, desc: jp_obrs_desc, policy_logits
                                                    _ptr(topk_inf_logp), k_inf, lambda_or_budget, k, seed,
                                                    _ptr(out_accept), _ptr(out_weight), _ptr(out_logp_policy),
                                                    _ptr(out_z_lower), _ptr(out_z_upper), _ptr(out_stats)))
+
+
+def jp_lmhead_lse_topk(ctx: Context, hidden, weight, tokens, mask, k: int, out_lse, out_logp_token, out_topk_idx,
+                       out_topk_val, out_status=None):
+    """hidden [T, H] and weight [V, H]: bf16 CUDA tensors (rows may be padded: the stride is passed on)."""
+    T, H = hidden.shape
+    V = weight.shape[0]
+    ctx.check(ctx.lib.jp_lmhead_lse_topk(ctx.h, _ptr(hidden), hidden.stride(0), _ptr(weight), weight.stride(0),
+                                         _ptr(tokens), _ptr(mask), T, H, V, k, _ptr(out_lse), _ptr(out_logp_token),
+                                         _ptr(out_topk_idx), _ptr(out_topk_val), _ptr(out_status)))
 
 
 def jp_obrs_forward_host(ctx: Context, desc: jp_obrs_desc, actor_logits, policy_logits, tokens, mask,

@@ -9,7 +9,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libjackpot.so")
-SOURCES = ["jp_api.cu", "jp_stream.cu", "jp_epilogue.cu", "jp_grad.cu", "jp_noalloc.cu", "jp_probe.cu", "jp_rowlambda.cu", "jp_vshard.cu", "jp_sparse.cu"]
+SOURCES = ["jp_api.cu", "jp_stream.cu", "jp_epilogue.cu", "jp_grad.cu", "jp_noalloc.cu", "jp_probe.cu", "jp_rowlambda.cu", "jp_vshard.cu", "jp_sparse.cu", "jp_lmhead.cu"]
 HEADERS = ["jp_common.cuh", "jp_internal.h"]
 
 

@@ -45,6 +45,8 @@ struct jp_ctx {
   cudaEvent_t ev0[kEvRing] = {}, ev1[kEvRing] = {};
   int64_t ev_count = 0;          // stream-kernel launches timed since timing was enabled
   // staging for the host-buffer entry point
+  char* lm_scratch = nullptr;    // partial results of the fused output-layer pass
+  size_t lm_bytes = 0;
   char* stage = nullptr;
   size_t stage_bytes = 0;
   cudaStream_t copy_stream = nullptr;
@@ -281,6 +283,7 @@ jp_status jp_destroy(jp_ctx* c) {
   cudaStreamSynchronize(c->stream);
   if (c->ws) cudaFree(c->ws);
   if (c->stage) cudaFree(c->stage);
+  if (c->lm_scratch) cudaFree(c->lm_scratch);
   for (int i = 0; i < jp_ctx::kEvRing; ++i) {
     if (c->ev0[i]) cudaEventDestroy(c->ev0[i]);
     if (c->ev1[i]) cudaEventDestroy(c->ev1[i]);
@@ -434,6 +437,44 @@ jp_status jp_obrs_forward_sparse_actor(jp_ctx* c, const jp_obrs_desc* d, const v
   if (e != cudaSuccess) return cuda_fail(c, e, "epilogue launch");
   c->have_records = true;
   c->rec_rows = d->T; c->rec_V = d->V; c->rec_k = k; c->rec_dtype = d->dtype;
+  return JP_OK;
+}
+
+jp_status jp_lmhead_lse_topk(jp_ctx* c, const void* hidden, int64_t ld_hidden, const void* weight, int64_t ld_weight,
+                             const int32_t* tokens, const uint8_t* mask, int64_t T, int64_t H, int64_t V, int k,
+                             float* out_lse, float* out_logp_token, int32_t* out_topk_idx, float* out_topk_val,
+                             int32_t* out_status) {
+  if (!c) return JP_ERR_INVALID_ARG;
+  if (T < 0 || H < 1 || V < 1 || V > (int64_t)0x7fffffff) return fail(c, JP_ERR_INVALID_ARG, "T < 0, H < 1 or V out of range");
+  if (k < 1 || k > kLmheadMaxK) return fail(c, JP_ERR_UNSUPPORTED, "the fused output-layer pass keeps lists of 1 <= k <= 32 entries");
+  if (ld_hidden == 0) ld_hidden = H;
+  if (ld_weight == 0) ld_weight = H;
+  if (ld_hidden < H || ld_weight < H) return fail(c, JP_ERR_INVALID_ARG, "leading dimension < H");
+  if ((ld_hidden * 2) % 16 != 0 || (ld_weight * 2) % 16 != 0)
+    return fail(c, JP_ERR_ALIGNMENT, "row pitches of hidden and weight must be multiples of 16 bytes");
+  if (T == 0) return JP_OK;
+  if (!hidden || !weight || !tokens || !out_lse || !out_logp_token || !out_topk_idx || !out_topk_val)
+    return fail(c, JP_ERR_INVALID_ARG, "a required pointer is NULL");
+  if (!aligned16(hidden) || !aligned16(weight)) return fail(c, JP_ERR_ALIGNMENT, "hidden and weight must be 16-byte aligned");
+  cudaSetDevice(c->device);
+  const int splits = lmhead_splits(T, V, c->sms);
+  const size_t need = lmhead_scratch_bytes(T, k, splits);
+  cudaError_t e;
+  if (need > c->lm_bytes) {
+    cudaStreamSynchronize(c->stream);
+    if (c->lm_scratch) cudaFree(c->lm_scratch);
+    c->lm_scratch = nullptr; c->lm_bytes = 0;
+    e = cudaMalloc((void**)&c->lm_scratch, need);
+    if (e != cudaSuccess) return fail(c, JP_ERR_WORKSPACE, std::string("scratch cudaMalloc: ") + cudaGetErrorString(e));
+    c->lm_bytes = need;
+  }
+  int32_t* status = out_status ? out_status : (int32_t*)(c->lm_scratch + need - 256);
+  e = cudaMemsetAsync(status, 0, sizeof(int32_t), c->stream);
+  if (e != cudaSuccess) return cuda_fail(c, e, "cudaMemsetAsync");
+  e = launch_lmhead(hidden, ld_hidden, weight, ld_weight, tokens, mask, T, H, V, k, splits, c->lm_scratch, status,
+                    out_lse, out_logp_token, out_topk_idx, out_topk_val, c->stream);
+  if (e != cudaSuccess) return cuda_fail(c, e, "fused output-layer launch");
+  c->launches += 2;
   return JP_OK;
 }
 
@@ -797,6 +838,7 @@ jp_status jp_obrs_forward_host(jp_ctx* c, const jp_obrs_desc* d, const void* za,
   if (need > c->stage_bytes) {
     cudaStreamSynchronize(c->stream);
     if (c->stage) cudaFree(c->stage);
+  if (c->lm_scratch) cudaFree(c->lm_scratch);
     c->stage = nullptr; c->stage_bytes = 0;
     e = cudaMalloc((void**)&c->stage, need);
     if (e != cudaSuccess) return fail(c, JP_ERR_WORKSPACE, std::string("staging cudaMalloc: ") + cudaGetErrorString(e));

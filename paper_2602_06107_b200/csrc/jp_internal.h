@@ -224,4 +224,13 @@ cudaError_t launch_vshard_merge(int n_shards, int my_shard, const float* gathere
                                 const Records& rec, Scalars* sc, cudaStream_t s);
 cudaError_t launch_grad(const GradArgs& a, cudaStream_t s, int sms, int* n_launch);
 
+// Output layer fused with the row pass (jp_lmhead.cu).
+constexpr int kLmheadMaxK = 32;
+size_t lmhead_scratch_bytes(int64_t T, int k, int splits);
+int lmhead_splits(int64_t T, int64_t V, int sms);
+cudaError_t launch_lmhead(const void* hidden, int64_t ldh, const void* weight, int64_t ldw, const int32_t* tokens,
+                          const uint8_t* mask, int64_t T, int64_t H, int64_t V, int k, int splits, void* scratch,
+                          int32_t* status, float* out_lse, float* out_logp, int32_t* out_idx, float* out_val,
+                          cudaStream_t s);
+
 }  // namespace jp
