@@ -2,7 +2,7 @@
 """Benchmark of the OBRS token pass (libjackpot) on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload cfg2_qwen3|cfg3_batch|cfg4_sweep|cfg5_train|sparse_actor]
+                    [--workload cfg2_qwen3|cfg3_batch|cfg4_sweep|cfg5_train|sparse_actor|lmhead_fused]
 
 A step is one pass of the whole path over one batch of synthetic logits:
 
@@ -21,6 +21,9 @@ A step is one pass of the whole path over one batch of synthetic logits:
   sparse_actor          the cfg2 shape through jp_obrs_forward_sparse_actor: only the policy tensor is
                         streamed (303,872 B per token), the rollout model comes as the record the
                         paper's rollout phase stores (log p_inf(a_t) and its 20 best log-probs).
+  lmhead_fused          one model's row pass fused into its output layer (jp_lmhead_lse_topk): 4096 hidden
+                        states of width 2048 against the [151936, 2048] bf16 output matrix on the tensor
+                        cores; log-sum-exp, token log-prob and top-20 straight from the accumulator.
 
 Every workload prints one JSON line with `roofline` (the dominant kernel, timed per launch by CUDA
 events on the stream it runs on), `cpu_baseline` (the oracle on a bounded sample, all host cores and
@@ -47,7 +50,8 @@ if ROOT not in sys.path:
 UNIT = "tokens/s"
 METRICS = {"cfg2_qwen3": "obrs_forward_tokens_per_s", "cfg3_batch": "obrs_forward_tokens_per_s",
            "cfg4_sweep": "obrs_forward_tokens_per_s", "cfg5_train": "obrs_fwd_bwd_tokens_per_s",
-           "sparse_actor": "obrs_forward_tokens_per_s"}
+           "sparse_actor": "obrs_forward_tokens_per_s", "lmhead_fused": "lmhead_row_pass_tokens_per_s"}
+LMHEAD = dict(T=4096, H=2048, k=20)    # hidden size of the paper's 1.7B rollout model; its default top-k count
 SPARSE_K_INF = 20            # the rollout stores its 20 most likely tokens (the paper's default top-k count)
 DATASHEET_GBS = 8000.0
 
@@ -88,7 +92,7 @@ class ClockSampler:
             self.p.kill()
         self.f.flush()
         self.f.seek(0)
-        sm, mx, pw, reasons = [], [], [], set()
+        sm, mx, pw, reasons, rows_all = [], [], [], set(), []
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in self.f.read().splitlines():
             c = [x.strip() for x in line.split(",")]
@@ -98,7 +102,8 @@ class ClockSampler:
                 s_, m_, p_ = float(c[1]), float(c[2]), float(c[3])
             except ValueError:
                 continue
-            if p_ < 300.0:            # an idle sample between two timed regions says nothing about the load
+            rows_all.append((s_, m_, p_, c[5:9]))
+            if p_ < 250.0:            # an idle sample between two timed regions says nothing about the load
                 continue
             sm.append(s_)
             mx.append(m_)
@@ -108,10 +113,20 @@ class ClockSampler:
                     reasons.add(n)
         self.f.close()
         os.unlink(self.f.name)
+        note = "samples under load (board power >= 250 W)"
+        if not sm and rows_all:       # a run too short for the power reading to rise: take what there is
+            note = "the timed regions were too short for a sample under load: all samples"
+            for s_, m_, p_, flags in rows_all:
+                sm.append(s_)
+                mx.append(m_)
+                pw.append(p_)
+                for n, v in zip(names, flags):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
         if sm:
             sm.sort()
             out.update(sm_mhz=sm[len(sm) // 2], sm_mhz_min=sm[0], sm_max_mhz=max(mx), power_w_max=max(pw),
-                       reasons=sorted(reasons), samples=len(sm), note="samples under load (board power >= 300 W)")
+                       reasons=sorted(reasons), samples=len(sm), note=note)
         return out
 
 
@@ -124,6 +139,8 @@ def _recipe(r0, T, seed, sigma=None):
 def _workload(name):
     from paper_2602_06107_b200.inputs import CONFIGS
     if name == "sparse_actor":                 # the headline shape, the rollout model as a stored record
+        return CONFIGS["cfg2_qwen3"]
+    if name == "lmhead_fused":
         return CONFIGS["cfg2_qwen3"]
     if name not in METRICS:
         raise SystemExit(f"bench.py: workload {name!r} is not a bench line (choose from {sorted(METRICS)}); "
@@ -138,6 +155,14 @@ def _oracle_sample(name, cfg, rows, device="cpu"):
     """`rows` rows of the workload (its first chunk / first sweep point), as the oracle takes them."""
     from paper_2602_06107_b200.inputs import make_lengths_mask, make_logits, to_numpy_bits
     r0 = cfg["recipe"]
+    if name == "lmhead_fused":
+        import torch
+        g = torch.Generator().manual_seed(11)
+        rows = min(rows, 16)                                     # 0.6 GFLOP per row in scalar double
+        h = torch.randn((rows, LMHEAD["H"]), generator=g).to(torch.bfloat16)
+        w = (torch.randn((r0.V, LMHEAD["H"]), generator=g) * (3.0 / LMHEAD["H"] ** 0.5)).to(torch.bfloat16)
+        tok = torch.randint(0, r0.V, (rows,), generator=g, dtype=torch.int32)
+        return to_numpy_bits(h), to_numpy_bits(w), tok.numpy(), None
     za, zp, tok = make_logits(_recipe(r0, rows, r0.seed), device, block_rows=rows)
     mask = None
     if name == "cfg3_batch":
@@ -156,6 +181,12 @@ def _oracle_step(name, cfg, za, zp, tok, mask):
     if name == "cfg2_qwen3":
         oracle.forward(za, zp, tok, None, lam=cfg["lam"], k=cfg["k"], seed=cfg["seed"])
         return n
+    if name == "lmhead_fused":
+        hb, wb = za, zp                                          # the sample carries hidden states and the matrix here
+        z = oracle.lmhead_rows(np.arange(hb.shape[0]), hb, wb)
+        oracle.lse_gather(z, z, tok, None)
+        oracle.topk(z, LMHEAD["k"], None)
+        return hb.shape[0]
     if name == "sparse_actor":
         lq, idx, logp = oracle.rollout_record(za, tok, SPARSE_K_INF)      # the rollout engine's part, not the path's
         oracle.forward_sparse(zp, tok, lq, idx, logp, None, lam=cfg["lam"], k=cfg["k"], seed=cfg["seed"])
@@ -180,7 +211,8 @@ def _time_oracle(name, cfg, sample, seconds, threads=None):
     if threads is not None:
         oracle.set_num_threads(threads)
     try:
-        _oracle_step(name, cfg, *[None if x is None else x[:8] for x in sample])
+        if name != "lmhead_fused":
+            _oracle_step(name, cfg, *[None if x is None else x[:8] for x in sample])
         t0, units, reps = time.perf_counter(), 0, 0
         while time.perf_counter() - t0 < seconds:
             units += _oracle_step(name, cfg, *sample)
@@ -196,8 +228,10 @@ def cpu_baseline_for(name, cfg, sample):
     rows = sample[0].shape[0]
     v, reps, dt, cores = _time_oracle(name, cfg, sample, 8.0)
     one = [None if x is None else x[:max(8, rows // 8)] for x in sample]
+    if name == "lmhead_fused":
+        one = [sample[0][:2], sample[1], sample[2][:2], None]       # the matrix stays whole: two rows of hidden states
     v1, reps1, dt1, _ = _time_oracle(name, cfg, one, 6.0, threads=1)
-    what = {"cfg2_qwen3": "forward", "sparse_actor": "forward from the policy logits and the stored record (making "
+    what = {"cfg2_qwen3": "forward", "lmhead_fused": "logits of the rows in double, then log-sum-exp and top-k", "sparse_actor": "forward from the policy logits and the stored record (making "
             "the record from the actor's logits is inside the timed region: it costs about as much again)", "cfg3_batch": "forward with the budget solve, valid tokens",
             "cfg4_sweep": "the four k of one sweep point", "cfg5_train": "forward + both gradients"}[name]
     return {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
@@ -216,6 +250,7 @@ def run_reference(args, rank):
     r = cfg["recipe"]
     rows = args.ref_rows
     sample = _oracle_sample(args.workload, cfg, rows)
+    rows = sample[0].shape[0]
     for _ in range(args.warmup):
         _oracle_step(args.workload, cfg, *sample)
     t0, units = time.perf_counter(), 0
@@ -647,7 +682,52 @@ def wl_sparse(b: Bench, cfg):
                         "stats": {n: stats[n] for n in ("alpha_hat", "kappa", "z_approx_mean")}})
 
 
-WORKLOADS = {"sparse_actor": wl_sparse, "cfg2_qwen3": wl_cfg2, "cfg3_batch": wl_cfg3, "cfg4_sweep": wl_cfg4, "cfg5_train": wl_cfg5}
+def wl_lmhead(b: Bench, cfg):
+    torch, B, args = b.torch, b.B, b.args
+    T, H, k = LMHEAD["T"], LMHEAD["H"], LMHEAD["k"]
+    V = cfg["recipe"].V
+    g = torch.Generator(device=b.dev).manual_seed(11 + 1000 * b.rank)
+    h = torch.randn((T, H), generator=g, device=b.dev).to(torch.bfloat16)
+    w = (torch.randn((V, H), generator=g, device=b.dev) * (3.0 / H ** 0.5)).to(torch.bfloat16)
+    tok = torch.randint(0, V, (T,), generator=g, device=b.dev, dtype=torch.int32)
+    lse, lp = torch.empty(T, device=b.dev), torch.empty(T, device=b.dev)
+    idx = torch.empty((T, k), dtype=torch.int32, device=b.dev)
+    val = torch.empty((T, k), device=b.dev)
+    st = torch.zeros(1, dtype=torch.int32, device=b.dev)
+
+    def step():
+        B.jp_lmhead_lse_topk(b.ctx, h, w, tok, None, k, lse, lp, idx, val, st)
+
+    l0 = b.ctx.launch_count()
+    ms = b.timed(step, args.steps, args.warmup)
+    launches = (b.ctx.launch_count() - l0) // (args.steps + args.warmup)
+    assert st.item() == 0, "a wait inside the fused kernel ran out"
+    flops = 2.0 * T * V * H
+    peaks = {}
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            peaks = json.load(f)
+    long_run = ms > 500.0                                     # longer than about half a second: the board's power limit rules
+    peak = float(peaks.get("bf16_tflops_sustained" if long_run else "bf16_tflops", 1404.0 if long_run else 1590.0))
+    achieved = flops / (ms / args.steps * 1e-3) / 1e12
+    roof = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+            "traffic": None, "peak_kind": ("of measured" if peaks else "of fallback") + (" (sustained)" if long_run else " (burst)"),
+            "frac_of_sustained": achieved / float(peaks.get("bf16_tflops_sustained", 1404.0)),
+            "kernel": "lmhead_kernel (tcgen05.mma 128x256x16 bf16 -> fp32 in TMEM, TMA operand ring, epilogue from the "
+                      "accumulator) + lmhead_merge_kernel; timed together by CUDA events around the call",
+            "kernel_ms": ms / args.steps, "algorithmic_flops": flops,
+            "operand_bytes": float(V * H * 2 + T * H * 2)}
+    return dict(ms=ms, units_per_step=T, launches=launches, roofline=roof,
+                e2e={"value": None, "reason": "inputs are a model's hidden states and output matrix, resident on the device in "
+                                              "any use of this call; there is no host-buffer entry point for it"},
+                extra={}, dtype="bf16",
+                config={"T": T, "H": H, "V": V, "k": k, "operands": "bf16 hidden [T, H] and weight [V, H], N(0,1) and "
+                        "N(0, 9/H) draws: logits ~ N(0, 9)", "logits_never_stored_bytes": float(T) * V * 2,
+                        "l2": f"the output matrix ({V * H * 2 / 1e6:.0f} MB) exceeds the 126 MB L2; no flush needed"})
+
+
+WORKLOADS = {"lmhead_fused": wl_lmhead, "sparse_actor": wl_sparse, "cfg2_qwen3": wl_cfg2, "cfg3_batch": wl_cfg3, "cfg4_sweep": wl_cfg4, "cfg5_train": wl_cfg5}
 
 
 def _nccl_summary(log_dir, world):
@@ -688,7 +768,7 @@ def run_ours(args, rank, world, local_rank):
     line = {"metric": METRICS[args.workload], "value": world * res["units_per_step"] * args.steps / (ms * 1e-3),
             "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f32", "data": "synthetic", "config": config, "clocks": clocks, "e2e": res["e2e"],
+            "dtype": res.get("dtype", "f32"), "data": "synthetic", "config": config, "clocks": clocks, "e2e": res["e2e"],
             "gpu_launches": int(res["launches"]), "roofline": roof}
     line.update(res["extra"])
     line["cpu_baseline"] = cpu_baseline
