@@ -2,7 +2,8 @@
 """Benchmark of the OBRS token pass (libjackpot) on B200.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--workload cfg2_qwen3|cfg3_batch|cfg4_sweep|cfg5_train|sparse_actor|lmhead_fused]
+                    [--workload cfg2_qwen3|cfg3_batch|cfg4_sweep|cfg5_train|sparse_actor|lmhead_fused|
+                                vocab_shards|vocab_widths]
 
 A step is one pass of the whole path over one batch of synthetic logits:
 
@@ -24,6 +25,10 @@ A step is one pass of the whole path over one batch of synthetic logits:
   lmhead_fused          one model's row pass fused into its output layer (jp_lmhead_lse_topk): 4096 hidden
                         states of width 2048 against the [151936, 2048] bf16 output matrix on the tensor
                         cores; log-sum-exp, token log-prob and top-20 straight from the accumulator.
+  vocab_shards          the cfg2 batch split by columns over 8 vocabulary shards: one rank's share (local
+                        pass of its slice, merge of all shards' records, finalize); 2 and 4 shards beside it.
+  vocab_widths          the row stream at vocabulary widths from 8 K to 262 K columns, rows scaled so that
+                        every point streams the same 2.4 GB.
 
 Every workload prints one JSON line with `roofline` (the dominant kernel, timed per launch by CUDA
 events on the stream it runs on), `cpu_baseline` (the oracle on a bounded sample, all host cores and
@@ -50,7 +55,8 @@ if ROOT not in sys.path:
 UNIT = "tokens/s"
 METRICS = {"cfg2_qwen3": "obrs_forward_tokens_per_s", "cfg3_batch": "obrs_forward_tokens_per_s",
            "cfg4_sweep": "obrs_forward_tokens_per_s", "cfg5_train": "obrs_fwd_bwd_tokens_per_s",
-           "sparse_actor": "obrs_forward_tokens_per_s", "lmhead_fused": "lmhead_row_pass_tokens_per_s"}
+           "sparse_actor": "obrs_forward_tokens_per_s", "lmhead_fused": "lmhead_row_pass_tokens_per_s",
+           "vocab_shards": "obrs_forward_tokens_per_s", "vocab_widths": "obrs_forward_tokens_per_s"}
 LMHEAD = dict(T=4096, H=2048, k=20)    # hidden size of the paper's 1.7B rollout model; its default top-k count
 SPARSE_K_INF = 20            # the rollout stores its 20 most likely tokens (the paper's default top-k count)
 DATASHEET_GBS = 8000.0
@@ -140,7 +146,7 @@ def _workload(name):
     from paper_2602_06107_b200.inputs import CONFIGS
     if name == "sparse_actor":                 # the headline shape, the rollout model as a stored record
         return CONFIGS["cfg2_qwen3"]
-    if name == "lmhead_fused":
+    if name in ("lmhead_fused", "vocab_shards", "vocab_widths"):
         return CONFIGS["cfg2_qwen3"]
     if name not in METRICS:
         raise SystemExit(f"bench.py: workload {name!r} is not a bench line (choose from {sorted(METRICS)}); "
@@ -179,6 +185,9 @@ def _oracle_step(name, cfg, za, zp, tok, mask):
     import oracle
     n = za.shape[0]
     if name == "cfg2_qwen3":
+        oracle.forward(za, zp, tok, None, lam=cfg["lam"], k=cfg["k"], seed=cfg["seed"])
+        return n
+    if name in ("vocab_shards", "vocab_widths"):             # the oracle knows whole rows of the headline shape only
         oracle.forward(za, zp, tok, None, lam=cfg["lam"], k=cfg["k"], seed=cfg["seed"])
         return n
     if name == "lmhead_fused":
@@ -231,7 +240,8 @@ def cpu_baseline_for(name, cfg, sample):
     if name == "lmhead_fused":
         one = [sample[0][:2], sample[1], sample[2][:2], None]       # the matrix stays whole: two rows of hidden states
     v1, reps1, dt1, _ = _time_oracle(name, cfg, one, 6.0, threads=1)
-    what = {"cfg2_qwen3": "forward", "lmhead_fused": "logits of the rows in double, then log-sum-exp and top-k", "sparse_actor": "forward from the policy logits and the stored record (making "
+    what = {"cfg2_qwen3": "forward", "vocab_shards": "forward on whole rows (the oracle does not shard)",
+            "vocab_widths": "forward at V = 151,936 only", "lmhead_fused": "logits of the rows in double, then log-sum-exp and top-k", "sparse_actor": "forward from the policy logits and the stored record (making "
             "the record from the actor's logits is inside the timed region: it costs about as much again)", "cfg3_batch": "forward with the budget solve, valid tokens",
             "cfg4_sweep": "the four k of one sweep point", "cfg5_train": "forward + both gradients"}[name]
     return {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
@@ -727,7 +737,132 @@ def wl_lmhead(b: Bench, cfg):
                         "l2": f"the output matrix ({V * H * 2 / 1e6:.0f} MB) exceeds the 126 MB L2; no flush needed"})
 
 
-WORKLOADS = {"lmhead_fused": wl_lmhead, "sparse_actor": wl_sparse, "cfg2_qwen3": wl_cfg2, "cfg3_batch": wl_cfg3, "cfg4_sweep": wl_cfg4, "cfg5_train": wl_cfg5}
+def wl_vocab_shards(b: Bench, cfg):
+    """One rank's share of the vocabulary-parallel forward.  The shards run one after the other on this
+    GPU to fill the gathered buffer (a rank has one of them); shard 0's three phases are what a step times."""
+    torch, B, args = b.torch, b.B, b.args
+    from paper_2602_06107_b200 import parallel, runner
+    from paper_2602_06107_b200.inputs import make_logits
+    r0 = cfg["recipe"]
+    r = _recipe(r0, r0.T, r0.seed + 1000 * b.rank)
+    za, zp, tok = make_logits(r, b.dev)
+    T, V = za.shape
+    k, lam, seed = cfg["k"], cfg["lam"], cfg["seed"]
+    words = B.jp_vshard_record_floats(k)
+    out = runner._alloc_outputs(T, b.dev)
+    fdesc = B.jp_obrs_desc()
+    table, headline = [], None
+    for n in (2, 4, 8):
+        bounds = [parallel.shard_columns(V, n, s) for s in range(n)]
+        gathered = torch.empty((n, T, words), device=b.dev)
+        for s_, (lo, hi) in enumerate(bounds):
+            zs, ps = za[:, lo:hi], zp[:, lo:hi]
+            B.jp_vshard_local(b.ctx, B.make_desc(zs), zs, ps, tok, None, lo, V, k, gathered[s_])
+        lo, hi = bounds[0]
+        zs, ps = za[:, lo:hi], zp[:, lo:hi]
+        d0 = B.make_desc(zs)
+
+        def local():
+            B.jp_vshard_local(b.ctx, d0, zs, ps, tok, None, lo, V, k, gathered[0])
+
+        def merge():
+            B.jp_vshard_merge(b.ctx, n, 0, gathered, T, V, k)
+
+        def finalize():
+            B.jp_batch_finalize(b.ctx, fdesc, lam, B.JP_LAMBDA_FIXED, seed, out["accept"], out["weight"],
+                                out["logp_actor"], out["logp_policy"], out["stats_buf"])
+
+        def step():
+            local()
+            merge()
+            finalize()
+
+        if n == 8:
+            ms, launches, kt = b.timed_with_kernel_times(step, args.steps, args.warmup, 1)
+            headline = (ms, launches, sum(kt) / len(kt), hi - lo)
+        reps = max(5, min(args.steps, 50))
+        # the phases one by one: events between the three calls of a step
+        for _ in range(2):
+            step()
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(reps)]
+        b.sync_all()
+        for e in ev:
+            e[0].record()
+            local()
+            e[1].record()
+            merge()
+            e[2].record()
+            finalize()
+            e[3].record()
+        b.sync_all()
+        t_local = sum(e[0].elapsed_time(e[1]) for e in ev) / reps
+        t_merge = sum(e[1].elapsed_time(e[2]) for e in ev) / reps
+        t_fin = sum(e[2].elapsed_time(e[3]) for e in ev) / reps
+        t_step = t_local + t_merge + t_fin
+        step()
+        torch.cuda.synchronize()
+        st = B.read_stats(out["stats_buf"])
+        gb = 2.0 * T * (hi - lo) * 2 / 1e9
+        table.append({"shards": n, "shard_columns": hi - lo, "local_ms": t_local, "local_gb_per_s": gb / (t_local * 1e-3),
+                      "local_frac": gb / (t_local * 1e-3) / b.peak, "merge_ms": t_merge, "finalize_ms": t_fin,
+                      "rank_total_ms": t_step, "all_gather_bytes_per_rank": T * words * 4,
+                      "tokens_per_s": T / (t_step * 1e-3), "n_accept": st["n_accept"], "kappa": st["kappa"]})
+    ms, launches, k_ms, width = headline
+    roof = b.roofline(b.stream_kernel_name(r.dtype, k, V) + f": the row stream of one slice of {width} columns (8 shards)",
+                      2.0 * T * width * 2, k_ms)
+    b.add_probe_rates(roof, za, zp)
+    return dict(ms=ms, units_per_step=T, launches=launches, roofline=roof,
+                e2e={"value": None, "reason": "the slices of a vocabulary-parallel output layer are device-resident by construction"},
+                extra={"shards": table},
+                config={"T": T, "V": V, "logits": r.dtype, "k": k, "lambda": lam, "shards": 8,
+                        "step": "shard 0's local pass, the merge of all 8 shards' records, finalize: one rank's share; the "
+                                "all-gather between local pass and merge is not in the timed region on one GPU",
+                        "l2": "the slice (311 MB) exceeds the 126 MB L2"})
+
+
+def wl_vocab_widths(b: Bench, cfg):
+    torch, B, args = b.torch, b.B, b.args
+    from paper_2602_06107_b200 import runner
+    from paper_2602_06107_b200.inputs import make_logits
+    r0 = cfg["recipe"]
+    k, lam, seed = cfg["k"], cfg["lam"], cfg["seed"]
+    widths = (8192, 18992, 32000, 50304, 65536, 128256, 151936, 262144)
+    points = []
+    for V in widths:
+        T = int(round(4096 * 151936 / V / 148)) * 148
+        r = _recipe(r0, T, r0.seed, None)
+        r = type(r)(T=T, V=V, dtype=r.dtype, sigma0=r.sigma0, peaks=r.peaks, peak_lo=r.peak_lo, peak_hi=r.peak_hi,
+                    sigma=r.sigma, seed=r.seed + 1000 * b.rank)
+        za, zp, tok = make_logits(r, b.dev, block_rows=2048)
+        out = runner._alloc_outputs(T, b.dev)
+        points.append((V, T, za, zp, tok, out, B.make_desc(za)))
+    B.jp_reserve(b.ctx, max(p[1] for p in points), 262144, k)
+
+    def point(i):
+        V, T, za, zp, tok, out, d = points[i]
+        B.jp_obrs_forward(b.ctx, d, za, zp, tok, None, lam, k, seed, out["accept"], out["weight"], out["logp_actor"],
+                          out["logp_policy"], out["stats_buf"])
+
+    def step():
+        for i in range(len(points)):
+            point(i)
+
+    npt = len(points)
+    ms, launches, kt = b.timed_with_kernel_times(step, args.steps, args.warmup, npt)
+    per = [sum(kt[i::npt]) / len(kt[i::npt]) for i in range(npt)]
+    table = [{"V": V, "rows": T, "stream_kernel_ms": per[i], "gb_per_s": 2.0 * T * V * 2 / (per[i] * 1e-3) / 1e9,
+              "frac": 2.0 * T * V * 2 / (per[i] * 1e-3) / 1e9 / b.peak,
+              "us_per_row_per_cta": per[i] * 1e3 / (T / 148)} for i, (V, T, *_rest) in enumerate(points)]
+    alg = sum(2.0 * T * V * 2 for V, T, *_r in points)
+    roof = b.roofline(f"prep_rows_kernel + stream_kernel<{r0.dtype}, 32-entry lists> over {npt} vocabulary widths", alg, sum(per))
+    return dict(ms=ms, units_per_step=sum(p[1] for p in points), launches=launches, roofline=roof,
+                e2e={"value": None, "reason": "a sweep of the row stream alone"}, extra={"widths": table},
+                config={"widths": list(widths), "k": k, "lambda": lam, "logits": r0.dtype,
+                        "rows": "scaled so that every width streams about 2.4 GB, a multiple of 148",
+                        "l2": "every point exceeds the 126 MB L2"})
+
+
+WORKLOADS = {"vocab_shards": wl_vocab_shards, "vocab_widths": wl_vocab_widths, "lmhead_fused": wl_lmhead, "sparse_actor": wl_sparse, "cfg2_qwen3": wl_cfg2, "cfg3_batch": wl_cfg3, "cfg4_sweep": wl_cfg4, "cfg5_train": wl_cfg5}
 
 
 def _nccl_summary(log_dir, world):

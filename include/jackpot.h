@@ -321,7 +321,7 @@ jp_status jp_obrs_apply_kappa(jp_ctx* ctx, double kappa, float c1, float* out_we
  * desc describes the slice: T rows, V = the slice's width (> k), ld, dtype.  tokens are ids in
  * [0, V_total) (others make the row invalid and are counted in n_bad_token); vocab_offset is
  * the slice's first column.  The slices of the shards must tile [0, V_total) without overlap.
- * 1 <= k <= JP_MAX_TOPK (no exact mode: JP_ERR_UNSUPPORTED); n_shards * k <= 2048
+ * 1 <= k <= JP_MAX_TOPK (no exact mode: JP_ERR_UNSUPPORTED); n_shards <= 128, n_shards * k <= 4096
  * (JP_ERR_TOO_LARGE).  A row is valid if every shard found it valid.  All pointers device
  * memory owned by the caller; the calls enqueue on the context's stream and return.  The
  * context's records afterwards describe the whole vocabulary; the gradients of a slice come

@@ -633,8 +633,9 @@ jp_status jp_vshard_merge(jp_ctx* c, int n_shards, int my_shard, const float* ga
   if (!c->vshard_local_done) return fail(c, JP_ERR_STATE, "jp_vshard_merge without jp_vshard_local");
   if (T != c->vshard_T || k != c->vshard_k) return fail(c, JP_ERR_INVALID_ARG, "T / k differ from jp_vshard_local");
   if (n_shards < 1 || my_shard < 0 || my_shard >= n_shards) return fail(c, JP_ERR_INVALID_ARG, "shard index out of range");
+  if (n_shards > kVshardMaxShards) return fail(c, JP_ERR_TOO_LARGE, "the merge takes at most 128 shards");
   if ((int64_t)n_shards * k > kVshardMaxEntries)
-    return fail(c, JP_ERR_TOO_LARGE, "n_shards * k beyond the merge kernel's 2048 entries per list");
+    return fail(c, JP_ERR_TOO_LARGE, "n_shards * k beyond the 4096 entries per list the merge holds in shared memory");
   if (T > 0 && !gathered) return fail(c, JP_ERR_INVALID_ARG, "gathered is NULL");
   cudaSetDevice(c->device);
   cudaError_t e = launch_vshard_merge(n_shards, my_shard, gathered, T, k, c->rec, c->sc, c->stream);

@@ -207,7 +207,8 @@ cudaError_t launch_row_lambda(const RowLambdaArgs& a, cudaStream_t s, int sms);
 // [6,7] the sampled token's two logits (owner only)  [8, 8+2k) global indices of the two lists
 // [8+2k, 8+4k) actor logits of the entries  [8+4k, 8+6k) policy logits of the entries.
 constexpr int kVshardHeader = 8;
-constexpr int kVshardMaxEntries = 2048;   // n_shards * k the merge kernel ranks in shared memory
+constexpr int kVshardMaxShards = 128;     // shards the merge kernel walks (four per lane of its warp)
+constexpr int kVshardMaxEntries = 4096;   // n_shards * k: the keys of one list of every shard, in a warp's shared memory
 constexpr int kVshardMaxDests = 16;       // shards a local pass can push its lines to
 struct VshardDests {
   float* dst[kVshardMaxDests];

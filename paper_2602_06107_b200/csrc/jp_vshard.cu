@@ -87,73 +87,115 @@ __global__ void __launch_bounds__(VS_NT) vshard_export_kernel(int64_t T, int k, 
   }
 }
 
-// One block per row.  Every entry of the shards' lists gets its rank among the entries of
-// its tensor by counting the keys above it in every shard's (sorted) list (keys are
-// distinct: the shards' columns are disjoint); ranks below k are the merged list.
+// One warp per row.  For each of the two lists the warp first copies every shard's k entries
+// into shared memory as 64-bit (order bits, ~index) keys (all loads in flight at once), then
+// lane s walks shard s's keys (and shards s + 32, ...: up to four per lane), which are sorted
+// best first: every round the best of the lanes' current heads under the row kernel's order
+// (higher logit first, equal logits by lower index; keys are distinct because the shards'
+// columns are disjoint) is the next entry of the merged list, and the winning lane moves on.
+// k rounds of one warp-wide maximum per list replace a rank count of every entry against every
+// shard's list; where each merged entry came from is noted, and both logits of the entries are
+// fetched at the end, again all at once.
 __global__ void __launch_bounds__(VS_NT) vshard_merge_kernel(int n_shards, int my_shard, const float* g, int64_t T,
-                                                             int k, Records rec, Scalars* sc) {
-  extern __shared__ unsigned long long keys[];      // [2][n_shards * k]
-  const int64_t r = blockIdx.x;
-  const int tid = threadIdx.x;
+                                                             int k, Records rec, Scalars* sc, int warps_per_block) {
+  extern __shared__ unsigned long long vs_smem[];            // per warp: n_shards * k keys, then k (shard, place) notes
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (warp >= warps_per_block) return;
+  const int64_t r = (int64_t)blockIdx.x * warps_per_block + warp;
+  if (r >= T) return;
   const int n = n_shards * k;
+  unsigned long long* keys = vs_smem + (size_t)warp * (size_t)(n + (k + 1) / 2);
+  uint32_t* from = reinterpret_cast<uint32_t*>(keys + n);    // (shard << 16) | place of merged entry j
   const int64_t W = vshard_words(k);
   auto line = [&](int s) { return g + ((int64_t)s * T + r) * W; };
 
-  // entry e of the 2 n: tensor t, shard s, place j (n <= 2048, so the quotient by k is exact in fp32)
-  const float inv_k = 1.f / (float)k;
-  auto split = [&](int e, int& t, int& s, int& j) {
-    t = e >= n ? 1 : 0;
-    const int x = e - t * n;
-    s = (int)(((float)x + 0.5f) * inv_k);
-    j = x - s * k;
-  };
-  for (int e = tid; e < 2 * n; e += VS_NT) {
-    int t, s, j;
-    split(e, t, s, j);
-    const float* o = line(s);
-    const int32_t idx = __float_as_int(o[kVshardHeader + t * k + j]);
-    const float v = o[kVshardHeader + (t == 0 ? 2 * k : 4 * k) + t * k + j];
-    keys[e] = idx >= 0 ? make_key(v, (uint32_t)idx) : 0ull;
-  }
-  for (int j = tid; j < 2 * k; j += VS_NT) {
-    const int64_t e = r * (2 * k) + j;
-    rec.idx[e] = -1; rec.za[e] = 0.f; rec.zp[e] = 0.f;
-  }
-  __syncthreads();
+  bool mine = true;
+  for (int s = lane; s < n_shards; s += 32) mine = mine && __float_as_int(line(s)[0]) != 0;
+  const bool all = __all_sync(0xffffffffu, mine);
 
-  bool all = true;
-  for (int s = 0; s < n_shards; ++s) all = all && __float_as_int(line(s)[0]) != 0;
-
-  if (all) {
-    for (int e = tid; e < 2 * n; e += VS_NT) {
-      const unsigned long long key = keys[e];
-      if (key == 0ull) continue;
-      int t, s, j;
-      split(e, t, s, j);
-      // every shard's list is sorted best first (empty slots, key 0, at its end): the keys above
-      // this one are a prefix of each list, found by bisection
-      const unsigned long long* kt = keys + t * n;
-      int above = 0;
-      for (int s2 = 0; s2 < n_shards && above < k; ++s2) {
-        const unsigned long long* Ls = kt + s2 * k;
-        int lo = 0, hi = k;
-        while (lo < hi) {
-          const int mid = (lo + hi) >> 1;
-          if (Ls[mid] > key) lo = mid + 1; else hi = mid;
+  for (int t = 0; t < 2; ++t) {
+    const int64_t dst0 = r * (2 * k) + (int64_t)t * k;
+    if (!all) {
+      for (int j = lane; j < k; j += 32) { rec.idx[dst0 + j] = -1; rec.za[dst0 + j] = 0.f; rec.zp[dst0 + j] = 0.f; }
+      continue;
+    }
+    __syncwarp();
+    for (int e = lane; e < n; e += 32) {
+      const int s = e / k, j = e - s * k;
+      const float* o = line(s);
+      const int32_t idx = __float_as_int(o[kVshardHeader + t * k + j]);
+      const float v = o[kVshardHeader + (t == 0 ? 2 * k : 4 * k) + t * k + j];
+      keys[e] = idx >= 0 ? make_key(v, (uint32_t)idx) : 0ull;
+    }
+    __syncwarp();
+    static_assert(kVshardMaxShards == 4 * 32, "four shards per lane");
+    if (n_shards <= 32) {
+      // one shard per lane: the head key stays in a register; the warp-wide maximum of the 64-bit
+      // keys is two 32-bit reductions (high words, then low words among the lanes that tie on top)
+      int head = 0;
+      unsigned long long key = lane < n_shards ? keys[lane * k] : 0ull;
+      for (int j = 0; j < k; ++j) {
+        const uint32_t hi = (uint32_t)(key >> 32), lo = (uint32_t)key;
+        const uint32_t mhi = __reduce_max_sync(0xffffffffu, hi);
+        const uint32_t mlo = __reduce_max_sync(0xffffffffu, hi == mhi ? lo : 0u);
+        if (mhi == 0u && mlo == 0u) {                         // the shards hold fewer than k entries in all
+          if (lane == 0) from[j] = 0xffffffffu;
+          continue;
         }
-        above += lo;
+        if (hi == mhi && lo == mlo) {                         // keys are distinct: exactly one lane
+          from[j] = ((uint32_t)lane << 16) | (uint32_t)head;
+          ++head;
+          key = head < k ? keys[lane * k + head] : 0ull;
+        }
       }
-      if (above < k) {
+    } else {
+      int head[4] = {0, 0, 0, 0};
+      for (int j = 0; j < k; ++j) {
+        unsigned long long key = 0ull;
+        int which = 0;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const int s = lane + 32 * q;
+          if (s < n_shards && head[q] < k) {
+            const unsigned long long kq = keys[s * k + head[q]];
+            if (kq > key) { key = kq; which = q; }
+          }
+        }
+        const uint32_t hi = (uint32_t)(key >> 32), lo = (uint32_t)key;
+        const uint32_t mhi = __reduce_max_sync(0xffffffffu, hi);
+        const uint32_t mlo = __reduce_max_sync(0xffffffffu, hi == mhi ? lo : 0u);
+        if (mhi == 0u && mlo == 0u) {
+          if (lane == 0) from[j] = 0xffffffffu;
+          continue;
+        }
+        if (hi == mhi && lo == mlo) {
+          int h = head[0];
+#pragma unroll
+          for (int q = 1; q < 4; ++q)
+            if (q == which) h = head[q];
+          from[j] = ((uint32_t)(lane + 32 * which) << 16) | (uint32_t)h;
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            if (q == which) head[q] += 1;
+        }
+      }
+    }
+    __syncwarp();
+    for (int j = lane; j < k; j += 32) {
+      const uint32_t f = from[j];
+      if (f == 0xffffffffu) {
+        rec.idx[dst0 + j] = -1; rec.za[dst0 + j] = 0.f; rec.zp[dst0 + j] = 0.f;
+      } else {
+        const int s = (int)(f >> 16), h = (int)(f & 0xffffu);
         const float* o = line(s);
-        const int64_t dst = r * (2 * k) + (int64_t)t * k + above;
-        rec.idx[dst] = (int32_t)key_index(key);
-        rec.za[dst] = o[kVshardHeader + 2 * k + t * k + j];
-        rec.zp[dst] = o[kVshardHeader + 4 * k + t * k + j];
+        rec.idx[dst0 + j] = __float_as_int(o[kVshardHeader + t * k + h]);
+        rec.za[dst0 + j] = o[kVshardHeader + 2 * k + t * k + h];
+        rec.zp[dst0 + j] = o[kVshardHeader + 4 * k + t * k + h];
       }
     }
   }
 
-  if (tid == 0) {
+  if (lane == 0) {
     if (!all) {
       rec.flag[r] = 0;
       rec.lse_a[r] = 0.f; rec.lse_p[r] = 0.f; rec.lse_a_lo[r] = 0.f; rec.lse_p_lo[r] = 0.f;
@@ -207,8 +249,13 @@ cudaError_t launch_vshard_export(int64_t T, int k, const Records& rec, const voi
 cudaError_t launch_vshard_merge(int n_shards, int my_shard, const float* gathered, int64_t T, int k,
                                 const Records& rec, Scalars* sc, cudaStream_t s) {
   if (T <= 0) return cudaSuccess;
-  const size_t smem = (size_t)2 * n_shards * k * sizeof(unsigned long long);   // <= 32 KB by kVshardMaxEntries
-  vshard_merge_kernel<<<(unsigned)T, VS_NT, smem, s>>>(n_shards, my_shard, gathered, T, k, rec, sc);
+  // per warp: the keys of one list of every shard and a note per merged entry; at most 32 KB + 256 B
+  const size_t per_warp = ((size_t)n_shards * k + (size_t)(k + 1) / 2) * sizeof(unsigned long long);
+  int wpb = (int)((size_t)(48 * 1024) / per_warp);
+  if (wpb > VS_NT / 32) wpb = VS_NT / 32;
+  if (wpb < 1) return cudaErrorInvalidValue;                 // excluded by kVshardMaxEntries
+  vshard_merge_kernel<<<(unsigned)((T + wpb - 1) / wpb), VS_NT, per_warp * wpb, s>>>(n_shards, my_shard, gathered, T, k,
+                                                                                   rec, sc, wpb);
   return cudaGetLastError();
 }
 

@@ -39,7 +39,7 @@ def run_shards(ctxs, za, zp, tok, mask, bounds, *, lam=None, budget=None, k, see
     gathered = torch.empty((n, T, words), dtype=torch.float32, device=za.device)
     for s, (lo, hi) in enumerate(bounds):
         zs, ps = za[:, lo:hi], zp[:, lo:hi]
-        B.jp_vshard_local(ctxs[s], B.make_desc(zs), zs, ps, tok, mask, lo, V, k, gathered[s])
+        B.jp_vshard_local(ctxs[s % len(ctxs)], B.make_desc(zs), zs, ps, tok, mask, lo, V, k, gathered[s])
     outs = []
     for s in finish:
         s = s % n
@@ -51,7 +51,7 @@ def run_shards(ctxs, za, zp, tok, mask, bounds, *, lam=None, budget=None, k, see
 
         # the rank's own local pass runs again inside (same bits), then the merge over all shards
         lo, hi = bounds[s]
-        out = parallel.forward_vocab_parallel(ctxs[s], za[:, lo:hi], zp[:, lo:hi], tok, mask, lo, V, lam=lam,
+        out = parallel.forward_vocab_parallel(ctxs[s % len(ctxs)], za[:, lo:hi], zp[:, lo:hi], tok, mask, lo, V, lam=lam,
                                               budget=budget, k=k, seed=seed, c1=c1, aux=True, gather=gather,
                                               shard_index=s)
         assert torch.equal(got["packed"].view(torch.int32), gathered[s].view(torch.int32))
@@ -69,7 +69,9 @@ def same_bits(a, b):
 
 @pytest.mark.parametrize("dtype,T,V,n,k", [("bf16", 300, 20000, 4, 16), ("bf16", 96, 151936, 8, 32),
                                            ("f32", 130, 4099, 3, 8), ("bf16", 64, 50001, 2, 128),
-                                           ("bf16", 24, 16 * 1024, 16, 128)])     # n * k at the merge's limit
+                                           ("bf16", 24, 16 * 1024, 16, 128),
+                                           ("bf16", 40, 8 * 1024, 40, 12),       # more shards than lanes in the merge's warp
+                                           ("f32", 20, 128 * 40, 128, 5)])       # the most shards the merge takes
 def test_shards_match_oracle_on_the_whole_vocabulary(ranks, dtype, T, V, n, k):
     align = 8 if dtype == "bf16" else 4
     ld = -(-V // align) * align
@@ -153,7 +155,7 @@ def test_shard_call_sequence_and_limits(ranks):
     with pytest.raises(B.JackpotError, match="outside"):
         B.jp_vshard_local(c, B.make_desc(za), za, zp, tok, None, 8, 4096, 16, buf)
     B.jp_vshard_local(c, B.make_desc(za), za, zp, tok, None, 0, 4096, 16, buf)
-    with pytest.raises(B.JackpotError, match="2048"):
+    with pytest.raises(B.JackpotError, match="128 shards"):
         B.jp_vshard_merge(c, 129, 0, buf, 8, 4096, 16)
     with pytest.raises(B.JackpotError, match="differ"):
         B.jp_vshard_merge(c, 1, 0, buf, 8, 4096, 8)
