@@ -3,7 +3,7 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
                     [--workload cfg2_qwen3|cfg3_batch|cfg4_sweep|cfg5_train|sparse_actor|lmhead_fused|
-                                vocab_shards|vocab_widths]
+                                fused_forward|vocab_shards|vocab_widths]
 
 A step is one pass of the whole path over one batch of synthetic logits:
 
@@ -25,6 +25,9 @@ A step is one pass of the whole path over one batch of synthetic logits:
   lmhead_fused          one model's row pass fused into its output layer (jp_lmhead_lse_topk): 4096 hidden
                         states of width 2048 against the [151936, 2048] bf16 output matrix on the tensor
                         cores; log-sum-exp, token log-prob and top-20 straight from the accumulator.
+  fused_forward         the whole forward with both models' output layers fused (jp_obrs_forward_lmhead): two
+                        such passes, the partner logits of the list entries, then acceptance, Z_approx, kappa
+                        and weights; neither logit tensor is stored.
   vocab_shards          the cfg2 batch split by columns over 8 vocabulary shards: one rank's share (local
                         pass of its slice, merge of all shards' records, finalize); 2 and 4 shards beside it.
   vocab_widths          the row stream at vocabulary widths from 8 K to 262 K columns, rows scaled so that
@@ -56,7 +59,8 @@ UNIT = "tokens/s"
 METRICS = {"cfg2_qwen3": "obrs_forward_tokens_per_s", "cfg3_batch": "obrs_forward_tokens_per_s",
            "cfg4_sweep": "obrs_forward_tokens_per_s", "cfg5_train": "obrs_fwd_bwd_tokens_per_s",
            "sparse_actor": "obrs_forward_tokens_per_s", "lmhead_fused": "lmhead_row_pass_tokens_per_s",
-           "vocab_shards": "obrs_forward_tokens_per_s", "vocab_widths": "obrs_forward_tokens_per_s"}
+           "vocab_shards": "obrs_forward_tokens_per_s", "vocab_widths": "obrs_forward_tokens_per_s",
+           "fused_forward": "obrs_forward_tokens_per_s"}
 LMHEAD = dict(T=4096, H=2048, k=20)    # hidden size of the paper's 1.7B rollout model; its default top-k count
 SPARSE_K_INF = 20            # the rollout stores its 20 most likely tokens (the paper's default top-k count)
 DATASHEET_GBS = 8000.0
@@ -146,7 +150,7 @@ def _workload(name):
     from paper_2602_06107_b200.inputs import CONFIGS
     if name == "sparse_actor":                 # the headline shape, the rollout model as a stored record
         return CONFIGS["cfg2_qwen3"]
-    if name in ("lmhead_fused", "vocab_shards", "vocab_widths"):
+    if name in ("lmhead_fused", "fused_forward", "vocab_shards", "vocab_widths"):
         return CONFIGS["cfg2_qwen3"]
     if name not in METRICS:
         raise SystemExit(f"bench.py: workload {name!r} is not a bench line (choose from {sorted(METRICS)}); "
@@ -161,7 +165,7 @@ def _oracle_sample(name, cfg, rows, device="cpu"):
     """`rows` rows of the workload (its first chunk / first sweep point), as the oracle takes them."""
     from paper_2602_06107_b200.inputs import make_lengths_mask, make_logits, to_numpy_bits
     r0 = cfg["recipe"]
-    if name == "lmhead_fused":
+    if name in ("lmhead_fused", "fused_forward"):
         import torch
         g = torch.Generator().manual_seed(11)
         rows = min(rows, 16)                                     # 0.6 GFLOP per row in scalar double
@@ -190,6 +194,12 @@ def _oracle_step(name, cfg, za, zp, tok, mask):
     if name in ("vocab_shards", "vocab_widths"):             # the oracle knows whole rows of the headline shape only
         oracle.forward(za, zp, tok, None, lam=cfg["lam"], k=cfg["k"], seed=cfg["seed"])
         return n
+    if name == "fused_forward":                              # both models' logits in double, then the dense forward
+        hb, wb = za, zp
+        z = oracle.lmhead_rows(np.arange(hb.shape[0]), hb, wb)
+        z2 = oracle.lmhead_rows(np.arange(hb.shape[0]), hb, wb)
+        oracle.forward(z, z2, tok, None, lam=1.0, k=LMHEAD["k"], seed=cfg["seed"])
+        return hb.shape[0]
     if name == "lmhead_fused":
         hb, wb = za, zp                                          # the sample carries hidden states and the matrix here
         z = oracle.lmhead_rows(np.arange(hb.shape[0]), hb, wb)
@@ -220,7 +230,7 @@ def _time_oracle(name, cfg, sample, seconds, threads=None):
     if threads is not None:
         oracle.set_num_threads(threads)
     try:
-        if name != "lmhead_fused":
+        if name not in ("lmhead_fused", "fused_forward"):
             _oracle_step(name, cfg, *[None if x is None else x[:8] for x in sample])
         t0, units, reps = time.perf_counter(), 0, 0
         while time.perf_counter() - t0 < seconds:
@@ -237,10 +247,10 @@ def cpu_baseline_for(name, cfg, sample):
     rows = sample[0].shape[0]
     v, reps, dt, cores = _time_oracle(name, cfg, sample, 8.0)
     one = [None if x is None else x[:max(8, rows // 8)] for x in sample]
-    if name == "lmhead_fused":
+    if name in ("lmhead_fused", "fused_forward"):
         one = [sample[0][:2], sample[1], sample[2][:2], None]       # the matrix stays whole: two rows of hidden states
     v1, reps1, dt1, _ = _time_oracle(name, cfg, one, 6.0, threads=1)
-    what = {"cfg2_qwen3": "forward", "vocab_shards": "forward on whole rows (the oracle does not shard)",
+    what = {"cfg2_qwen3": "forward", "fused_forward": "both models' logits of the rows in double, then the dense forward", "vocab_shards": "forward on whole rows (the oracle does not shard)",
             "vocab_widths": "forward at V = 151,936 only", "lmhead_fused": "logits of the rows in double, then log-sum-exp and top-k", "sparse_actor": "forward from the policy logits and the stored record (making "
             "the record from the actor's logits is inside the timed region: it costs about as much again)", "cfg3_batch": "forward with the budget solve, valid tokens",
             "cfg4_sweep": "the four k of one sweep point", "cfg5_train": "forward + both gradients"}[name]
@@ -862,7 +872,57 @@ def wl_vocab_widths(b: Bench, cfg):
                         "l2": "every point exceeds the 126 MB L2"})
 
 
-WORKLOADS = {"vocab_shards": wl_vocab_shards, "vocab_widths": wl_vocab_widths, "lmhead_fused": wl_lmhead, "sparse_actor": wl_sparse, "cfg2_qwen3": wl_cfg2, "cfg3_batch": wl_cfg3, "cfg4_sweep": wl_cfg4, "cfg5_train": wl_cfg5}
+def wl_fused_forward(b: Bench, cfg):
+    torch, B, args = b.torch, b.B, b.args
+    from paper_2602_06107_b200 import runner
+    T, H, k = LMHEAD["T"], LMHEAD["H"], LMHEAD["k"]
+    V, seed = cfg["recipe"].V, cfg["seed"]
+    g = torch.Generator(device=b.dev).manual_seed(12 + 1000 * b.rank)
+    ha = torch.randn((T, H), generator=g, device=b.dev).to(torch.bfloat16)
+    wa = (torch.randn((V, H), generator=g, device=b.dev) * (3.0 / H ** 0.5)).to(torch.bfloat16)
+    hp = ha.clone()
+    wp = (wa.float() + torch.randn((V, H), generator=g, device=b.dev) * (1.0 / H ** 0.5)).to(torch.bfloat16)
+    tok = torch.randint(0, V, (T,), generator=g, device=b.dev, dtype=torch.int32)
+    out = runner._alloc_outputs(T, b.dev)
+    d = B.jp_obrs_desc()
+    d.T, d.V = T, V
+
+    def step():
+        B.jp_obrs_forward_lmhead(b.ctx, d, ha, wa, hp, wp, tok, None, 1.0, k, seed, out["accept"], out["weight"],
+                                 out["logp_actor"], out["logp_policy"], out["stats_buf"])
+
+    l0 = b.ctx.launch_count()
+    ms = b.timed(step, args.steps, args.warmup)
+    launches = (b.ctx.launch_count() - l0) // (args.steps + args.warmup)
+    st = B.read_stats(out["stats_buf"])
+    assert st["status"] == 0
+    flops = 2.0 * 2.0 * T * V * H + 2.0 * T * 2 * k * H * 2          # two output layers, and the partner logits
+    peaks = {}
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            peaks = json.load(f)
+    long_run = ms > 500.0
+    peak = float(peaks.get("bf16_tflops_sustained" if long_run else "bf16_tflops", 1404.0 if long_run else 1590.0))
+    achieved = flops / (ms / args.steps * 1e-3) / 1e12
+    roof = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+            "peak_kind": ("of measured" if peaks else "of fallback") + (" (sustained)" if long_run else " (burst)"),
+            "frac_of_sustained": achieved / float(peaks.get("bf16_tflops_sustained", 1404.0)),
+            "kernel": "the whole step: 2 x (lmhead_kernel + lmhead_merge_kernel), fused_records_kernel, epilogue, finalize; "
+                      "timed together by CUDA events (the two tcgen05 kernels are 98 % of it)",
+            "kernel_ms": ms / args.steps, "algorithmic_flops": flops}
+    return dict(ms=ms, units_per_step=T, launches=launches, roofline=roof, dtype="bf16",
+                e2e={"value": None, "reason": "inputs are two models' hidden states and output matrices, resident on the device "
+                                              "in any use of this call"},
+                extra={},
+                config={"T": T, "H": H, "V": V, "k": k, "lambda": 1.0,
+                        "tokens": "uniform draws (the sampled token enters only O(T) scalars; kappa is not meaningful here)",
+                        "logits_never_stored_bytes": 2.0 * T * V * 2,
+                        "l2": "the output matrices (2 x 622 MB) exceed the 126 MB L2; no flush needed",
+                        "stats": {n: st[n] for n in ("alpha_hat", "kappa", "z_approx_mean")}})
+
+
+WORKLOADS = {"fused_forward": wl_fused_forward, "vocab_shards": wl_vocab_shards, "vocab_widths": wl_vocab_widths, "lmhead_fused": wl_lmhead, "sparse_actor": wl_sparse, "cfg2_qwen3": wl_cfg2, "cfg3_batch": wl_cfg3, "cfg4_sweep": wl_cfg4, "cfg5_train": wl_cfg5}
 
 
 def _nccl_summary(log_dir, world):

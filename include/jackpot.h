@@ -197,6 +197,31 @@ jp_status jp_lmhead_lse_topk(jp_ctx* ctx, const void* hidden, int64_t ld_hidden,
                              int64_t H, int64_t V, int k, float* out_lse, float* out_logp_token,
                              int32_t* out_topk_idx, float* out_topk_val, int32_t* out_status);
 
+/* The whole forward with both models' row passes fused into their output layers: neither
+ * [T, V] logit tensor is ever stored (Section 4.4).  Each model's logits are
+ * hidden[t, :] . weight[v, :] as in jp_lmhead_lse_topk (bf16 operands, fp32 accumulation, one
+ * pass per model); for every entry of the two top-k lists the other model's logit is one more
+ * dot product of a hidden state with a row of that model's output matrix; from there lambda
+ * (fixed or from a budget), acceptance (Eq. obrs_accept), the accept draws, Z_approx over the
+ * union of the two lists (Section 4.4.1), kappa and the weights (Section 4.4.2, Algorithm 1
+ * step 3) run exactly as in jp_obrs_forward.
+ *   desc : T, V (vocabulary), lambda_mode, c1, token_offset and the optional outputs are used;
+ *          dtype and ld are ignored.  z_exact and JP_DESC_KL are JP_ERR_UNSUPPORTED (they need
+ *          whole rows of logits).
+ *   hidden_actor [T, ld_ha] / weight_actor [V, ld_wa] with hidden size H_actor, and the same for
+ *   the policy (the two models may differ in hidden size): bf16, DEVICE, 16-byte aligned,
+ *   pitches multiples of 16 bytes (ld = 0 means H).  1 <= k <= 32, k < V.
+ * Outputs as in jp_obrs_forward.  The logits keep the precision of the fp32 accumulator, so
+ * log-probs agree with a forward over stored bf16 logits only to the rounding of those.  The
+ * records this call leaves do not serve jp_obrs_backward (JP_ERR_STATE). */
+jp_status jp_obrs_forward_lmhead(jp_ctx* ctx, const jp_obrs_desc* desc, const void* hidden_actor, int64_t ld_ha,
+                                 const void* weight_actor, int64_t ld_wa, int64_t H_actor,
+                                 const void* hidden_policy, int64_t ld_hp, const void* weight_policy,
+                                 int64_t ld_wp, int64_t H_policy, const int32_t* tokens, const uint8_t* mask,
+                                 float lambda_or_budget, int k, uint64_t seed, uint8_t* out_accept,
+                                 float* out_weight, float* out_logp_actor, float* out_logp_policy,
+                                 jp_stats* out_stats);
+
 /* Parameters of the backward pass (Eq. obrs_ppo, Eq. ppo_rollout, Eq.
  * distill_loss combined as Eq. sys_joint_obj; the PPO terms are maximised and
  * the distillation term minimised, so the loss is

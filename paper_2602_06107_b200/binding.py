@@ -25,7 +25,7 @@ JP_DESC_SPARSE_CAP = 2
 
 EXPORTS = (
     "jp_create", "jp_destroy", "jp_set_stream", "jp_obrs_workspace_bytes", "jp_reserve",
-    "jp_obrs_forward", "jp_obrs_forward_sparse_actor", "jp_lmhead_lse_topk", "jp_obrs_backward", "jp_batch_begin", "jp_batch_chunk", "jp_batch_finalize",
+    "jp_obrs_forward", "jp_obrs_forward_sparse_actor", "jp_lmhead_lse_topk", "jp_obrs_forward_lmhead", "jp_obrs_backward", "jp_batch_begin", "jp_batch_chunk", "jp_batch_finalize",
     "jp_obrs_forward_host", "jp_obrs_apply_kappa", "jp_batch_totals", "jp_obrs_apply_totals", "jp_batch_logprobs", "jp_obrs_row_lambda", "jp_vshard_record_floats", "jp_vshard_local", "jp_vshard_local_push", "jp_vshard_merge", "jp_vshard_backward", "jp_budget_lambda_static", "jp_probe_stream", "jp_status_string", "jp_last_error", "jp_launch_count",
     "jp_enable_kernel_timing", "jp_stream_kernel_times",
 )
@@ -103,6 +103,8 @@ def load():
     lib.jp_obrs_forward_sparse_actor.argtypes = [vp, ctypes.POINTER(jp_obrs_desc), vp, vp, vp, vp, vp, vp, ctypes.c_int,
                                                  f32, ctypes.c_int, u64, vp, vp, vp, vp, vp, vp]
     lib.jp_lmhead_lse_topk.argtypes = [vp, vp, i64, vp, i64, vp, vp, i64, i64, i64, ctypes.c_int, vp, vp, vp, vp, vp]
+    lib.jp_obrs_forward_lmhead.argtypes = [vp, ctypes.POINTER(jp_obrs_desc), vp, i64, vp, i64, i64, vp, i64, vp, i64, i64,
+                                           vp, vp, f32, ctypes.c_int, u64, vp, vp, vp, vp, vp]
     lib.jp_obrs_forward_host.argtypes = lib.jp_obrs_forward.argtypes + [i64]
     lib.jp_obrs_backward.argtypes = [vp, ctypes.POINTER(jp_obrs_desc), ctypes.POINTER(jp_obrs_bwd_desc),
                                      vp, vp, vp, vp, vp, vp, vp, vp]
@@ -236,6 +238,17 @@ def jp_lmhead_lse_topk(ctx: Context, hidden, weight, tokens, mask, k: int, out_l
     ctx.check(ctx.lib.jp_lmhead_lse_topk(ctx.h, _ptr(hidden), hidden.stride(0), _ptr(weight), weight.stride(0),
                                          _ptr(tokens), _ptr(mask), T, H, V, k, _ptr(out_lse), _ptr(out_logp_token),
                                          _ptr(out_topk_idx), _ptr(out_topk_val), _ptr(out_status)))
+
+
+def jp_obrs_forward_lmhead(ctx: Context, desc: jp_obrs_desc, hidden_actor, weight_actor, hidden_policy, weight_policy,
+                           tokens, mask, lambda_or_budget: float, k: int, seed: int, out_accept, out_weight,
+                           out_logp_actor, out_logp_policy, out_stats):
+    """hidden_* [T, H_*] and weight_* [V, H_*]: bf16 CUDA tensors (strides are passed on); desc carries T and V."""
+    ctx.check(ctx.lib.jp_obrs_forward_lmhead(
+        ctx.h, ctypes.byref(desc), _ptr(hidden_actor), hidden_actor.stride(0), _ptr(weight_actor), weight_actor.stride(0),
+        hidden_actor.shape[1], _ptr(hidden_policy), hidden_policy.stride(0), _ptr(weight_policy),
+        weight_policy.stride(0), hidden_policy.shape[1], _ptr(tokens), _ptr(mask), lambda_or_budget, k, seed,
+        _ptr(out_accept), _ptr(out_weight), _ptr(out_logp_actor), _ptr(out_logp_policy), _ptr(out_stats)))
 
 
 def jp_obrs_forward_host(ctx: Context, desc: jp_obrs_desc, actor_logits, policy_logits, tokens, mask,

@@ -478,6 +478,100 @@ jp_status jp_lmhead_lse_topk(jp_ctx* c, const void* hidden, int64_t ld_hidden, c
   return JP_OK;
 }
 
+jp_status jp_obrs_forward_lmhead(jp_ctx* c, const jp_obrs_desc* d, const void* hidden_actor, int64_t ld_ha,
+                                 const void* weight_actor, int64_t ld_wa, int64_t H_actor, const void* hidden_policy,
+                                 int64_t ld_hp, const void* weight_policy, int64_t ld_wp, int64_t H_policy,
+                                 const int32_t* tokens, const uint8_t* mask, float lambda_or_budget, int k,
+                                 uint64_t seed, uint8_t* out_accept, float* out_weight, float* out_lq, float* out_lp,
+                                 jp_stats* out_stats) {
+  if (!c) return JP_ERR_INVALID_ARG;
+  if (!d) return fail(c, JP_ERR_INVALID_ARG, "desc is NULL");
+  const int64_t T = d->T, V = d->V;
+  if (T < 0 || V < 1 || V > (int64_t)0x7fffffff || H_actor < 1 || H_policy < 1)
+    return fail(c, JP_ERR_INVALID_ARG, "T < 0, V out of range or a hidden size < 1");
+  if (k < 1 || k > kLmheadMaxK || (int64_t)k >= V)
+    return fail(c, JP_ERR_UNSUPPORTED, "the fused output-layer pass keeps lists of 1 <= k <= 32 entries, k < V");
+  jp_status st = check_lambda(c, lambda_or_budget, d->lambda_mode);
+  if (st != JP_OK) return st;
+  if (c->batch_open) return fail(c, JP_ERR_STATE, "a chunked batch is open: finalize it first");
+  if (d->flags & JP_DESC_KL) return fail(c, JP_ERR_UNSUPPORTED, "KL(p || q) needs whole rows of logits, which this path never forms");
+  if (d->z_exact) return fail(c, JP_ERR_UNSUPPORTED, "the exact Z needs whole rows of logits, which this path never forms");
+  if (ld_ha == 0) ld_ha = H_actor;
+  if (ld_wa == 0) ld_wa = H_actor;
+  if (ld_hp == 0) ld_hp = H_policy;
+  if (ld_wp == 0) ld_wp = H_policy;
+  if (ld_ha < H_actor || ld_wa < H_actor || ld_hp < H_policy || ld_wp < H_policy)
+    return fail(c, JP_ERR_INVALID_ARG, "a leading dimension is smaller than the hidden size");
+  if ((ld_ha * 2) % 16 || (ld_wa * 2) % 16 || (ld_hp * 2) % 16 || (ld_wp * 2) % 16)
+    return fail(c, JP_ERR_ALIGNMENT, "row pitches of hidden states and output matrices must be multiples of 16 bytes");
+  if (T > 0 && (!hidden_actor || !weight_actor || !hidden_policy || !weight_policy || !tokens))
+    return fail(c, JP_ERR_INVALID_ARG, "a required pointer is NULL");
+  if (!aligned16(hidden_actor) || !aligned16(weight_actor) || !aligned16(hidden_policy) || !aligned16(weight_policy))
+    return fail(c, JP_ERR_ALIGNMENT, "hidden states and output matrices must be 16-byte aligned");
+  cudaSetDevice(c->device);
+  if ((st = ensure_workspace(c, T > 0 ? T : 1, k)) != JP_OK) return st;
+  const bool budget = d->lambda_mode == JP_LAMBDA_FROM_BUDGET;
+  cudaError_t e = launch_reset(c->sc, budget ? 1.0f : lambda_or_budget, c->stream);
+  if (e != cudaSuccess) return cuda_fail(c, e, "reset launch");
+  c->launches += 1;
+  c->have_records = false;
+  c->rec_kl = false;
+  c->rec_sparse = true;                       // no logits behind these records either: no backward from them
+  if (T > 0) {
+    const int splits = lmhead_splits(T, V, c->sms);
+    const size_t part = (lmhead_scratch_bytes(T, k, splits) + 255) / 256 * 256;
+    const size_t per_model = ((size_t)T * (8 + 8 * (size_t)k) + 255) / 256 * 256;   // lse, logp, idx[k], val[k]
+    const size_t need = part + 2 * per_model;
+    if (need > c->lm_bytes) {
+      cudaStreamSynchronize(c->stream);
+      if (c->lm_scratch) cudaFree(c->lm_scratch);
+      c->lm_scratch = nullptr; c->lm_bytes = 0;
+      e = cudaMalloc((void**)&c->lm_scratch, need);
+      if (e != cudaSuccess) return fail(c, JP_ERR_WORKSPACE, std::string("scratch cudaMalloc: ") + cudaGetErrorString(e));
+      c->lm_bytes = need;
+    }
+    // the device status word of the row kernels doubles as the fused kernels' (JP_ERR_TIMEOUT lands in jp_stats.status)
+    int32_t* status = &c->sc->status;
+    float* res[2][4];
+    for (int m = 0; m < 2; ++m) {
+      char* b = c->lm_scratch + part + (size_t)m * per_model;
+      res[m][0] = (float*)b;                                  // lse
+      res[m][1] = (float*)(b + (size_t)T * 4);                // log-prob of the token
+      res[m][2] = (float*)(b + (size_t)T * 8);                // idx (int32)
+      res[m][3] = (float*)(b + (size_t)T * 8 + (size_t)T * k * 4);
+    }
+    e = launch_lmhead(hidden_actor, ld_ha, weight_actor, ld_wa, tokens, mask, T, H_actor, V, k, splits, c->lm_scratch,
+                      status, res[0][0], res[0][1], (int32_t*)res[0][2], res[0][3], c->stream);
+    if (e == cudaSuccess)
+      e = launch_lmhead(hidden_policy, ld_hp, weight_policy, ld_wp, tokens, mask, T, H_policy, V, k, splits,
+                        c->lm_scratch, status, res[1][0], res[1][1], (int32_t*)res[1][2], res[1][3], c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e, "fused output-layer launch");
+    FusedRecordArgs fa{};
+    fa.hidden_a = hidden_actor; fa.weight_a = weight_actor; fa.hidden_p = hidden_policy; fa.weight_p = weight_policy;
+    fa.ld_ha = ld_ha; fa.ld_wa = ld_wa; fa.ld_hp = ld_hp; fa.ld_wp = ld_wp; fa.H_a = H_actor; fa.H_p = H_policy;
+    fa.tokens = tokens; fa.mask = mask; fa.T = T; fa.V = V; fa.k = k;
+    fa.lse_a = res[0][0]; fa.lq = res[0][1]; fa.idx_a = (const int32_t*)res[0][2]; fa.val_a = res[0][3];
+    fa.lse_p = res[1][0]; fa.lp = res[1][1]; fa.idx_p = (const int32_t*)res[1][2]; fa.val_p = res[1][3];
+    fa.rec = c->rec; fa.sc = c->sc;
+    e = launch_fused_records(fa, c->stream);
+    if (e != cudaSuccess) return cuda_fail(c, e, "fused records launch");
+    c->launches += 5;
+  }
+  EpilogueArgs ea = epilogue_args(c, d, T, k, seed, d->token_offset, d->c1, out_accept, out_weight, out_lq, out_lp,
+                                  out_stats);
+  int nl = 0;
+  if (budget) {
+    e = launch_budget_solve(ea, (double)lambda_or_budget, c->stream, &nl);
+    if (e != cudaSuccess) return cuda_fail(c, e, "budget solve launch");
+  }
+  e = launch_epilogue(ea, c->stream, &nl);
+  c->launches += nl;
+  if (e != cudaSuccess) return cuda_fail(c, e, "epilogue launch");
+  c->have_records = true;
+  c->rec_rows = T; c->rec_V = V; c->rec_k = k; c->rec_dtype = JP_BF16;
+  return JP_OK;
+}
+
 jp_status jp_batch_begin(jp_ctx* c, int64_t T_total, int64_t V, int32_t dtype, int k,
                          float fixed_lambda_for_exact_mode) {
   if (!c) return JP_ERR_INVALID_ARG;
@@ -736,7 +830,7 @@ jp_status backward_impl(jp_ctx* c, const jp_obrs_desc* d, const jp_obrs_bwd_desc
   if (st != JP_OK) return st;
   if (!b) return fail(c, JP_ERR_INVALID_ARG, "bwd desc is NULL");
   if (!c->have_records) return fail(c, JP_ERR_STATE, "no forward records in this context: run the forward (or finalize the batch) first");
-  if (c->rec_sparse) return fail(c, JP_ERR_STATE, "the records come from jp_obrs_forward_sparse_actor: the gradients need both models' log-sum-exps (run jp_obrs_forward)");
+  if (c->rec_sparse) return fail(c, JP_ERR_STATE, "the records come from a forward without both logit tensors (sparse-actor or fused output layer): the gradients need the logits (run jp_obrs_forward)");
   const bool slice = slice_offset >= 0;
   if (!slice && (d->V != c->rec_V || d->dtype != c->rec_dtype)) return fail(c, JP_ERR_STATE, "V / dtype differ from the forward that left the records");
   if (slice && d->dtype != c->rec_dtype) return fail(c, JP_ERR_STATE, "dtype differs from the forward that left the records");

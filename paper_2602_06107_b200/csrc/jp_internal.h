@@ -227,6 +227,18 @@ cudaError_t launch_grad(const GradArgs& a, cudaStream_t s, int sms, int* n_launc
 
 // Output layer fused with the row pass (jp_lmhead.cu).
 constexpr int kLmheadMaxK = 32;
+struct FusedRecordArgs {
+  const void* hidden_a; const void* weight_a; const void* hidden_p; const void* weight_p;   // bf16, row-major
+  int64_t ld_ha, ld_wa, ld_hp, ld_wp, H_a, H_p;
+  const int32_t* tokens; const uint8_t* mask;
+  int64_t T, V;
+  int32_t k;
+  const float* lse_a; const float* lq; const int32_t* idx_a; const float* val_a;   // the actor pass's results
+  const float* lse_p; const float* lp; const int32_t* idx_p; const float* val_p;   // the policy pass's
+  Records rec;
+  Scalars* sc;
+};
+cudaError_t launch_fused_records(const FusedRecordArgs& a, cudaStream_t s);
 size_t lmhead_scratch_bytes(int64_t T, int k, int splits);
 int lmhead_splits(int64_t T, int64_t V, int sms);
 cudaError_t launch_lmhead(const void* hidden, int64_t ldh, const void* weight, int64_t ldw, const int32_t* tokens,

@@ -464,6 +464,73 @@ bool make_map(EncodeTiledFn enc, CUtensorMap* map, const void* base, int64_t row
 
 }  // namespace
 
+namespace {
+// Dot product of two bf16 rows of length H by one warp (16-byte loads where the rows allow it,
+// fp32 sums, a fixed shuffle tree): the logit of one vocabulary entry under one model.
+__device__ __forceinline__ float warp_dot_bf16(const __nv_bfloat16* a, const __nv_bfloat16* b, int64_t H, int lane) {
+  float acc = 0.f;
+  const int64_t nvec = H / 8;
+  const uint4* a4 = reinterpret_cast<const uint4*>(a);
+  const uint4* b4 = reinterpret_cast<const uint4*>(b);
+  for (int64_t i = lane; i < nvec; i += 32) {
+    const uint4 x = a4[i], y = b4[i];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc = fmaf(Vec<JP_BF16>::get(x, e), Vec<JP_BF16>::get(y, e), acc);
+  }
+  for (int64_t i = nvec * 8 + lane; i < H; i += 32) acc = fmaf(__bfloat162float(a[i]), __bfloat162float(b[i]), acc);
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+  return acc;
+}
+
+// The records of the forward from two fused output-layer passes (Section 4.4.1: V_k is the
+// union of the two top-k sets and Z_approx needs both models' probabilities on it): per row
+// the two log-sum-exps, the sampled token's two log-probs, the two lists, and for every list
+// entry the logit of the *other* model, one dot product of a hidden state with one row of
+// that model's output matrix.  One warp per row.
+__global__ void __launch_bounds__(128) fused_records_kernel(FusedRecordArgs A) {
+  const int lane = threadIdx.x & 31;
+  const int64_t r = (int64_t)blockIdx.x * 4 + (threadIdx.x >> 5);
+  if (r >= A.T) return;
+  const int k = A.k;
+  const int32_t tok = A.tokens[r];
+  const bool bad = tok < 0 || (int64_t)tok >= A.V;
+  const bool valid = (A.mask == nullptr || A.mask[r] != 0) && !bad;
+  if (lane == 0) {
+    A.rec.flag[r] = valid ? kRowValid : 0;
+    A.rec.lse_a[r] = valid ? A.lse_a[r] : 0.f; A.rec.lse_a_lo[r] = 0.f;
+    A.rec.lse_p[r] = valid ? A.lse_p[r] : 0.f; A.rec.lse_p_lo[r] = 0.f;
+    A.rec.lq[r] = valid ? A.lq[r] : 0.f;
+    A.rec.lp[r] = valid ? A.lp[r] : 0.f;
+    if (bad && (A.mask == nullptr || A.mask[r] != 0)) atomicAdd(&A.sc->n_bad_token, 1ull);
+  }
+  const __nv_bfloat16* ha = (const __nv_bfloat16*)A.hidden_a + r * A.ld_ha;
+  const __nv_bfloat16* hp = (const __nv_bfloat16*)A.hidden_p + r * A.ld_hp;
+  for (int j = 0; j < 2 * k; ++j) {
+    const int64_t dst = r * (2 * k) + j;
+    const bool from_actor = j < k;
+    const int32_t idx = valid ? (from_actor ? A.idx_a[r * k + j] : A.idx_p[r * k + (j - k)]) : -1;
+    float za = 0.f, zp = 0.f;
+    if (idx >= 0) {                                           // uniform over the warp
+      if (from_actor) {
+        za = A.val_a[r * k + j];
+        zp = warp_dot_bf16(hp, (const __nv_bfloat16*)A.weight_p + (int64_t)idx * A.ld_wp, A.H_p, lane);
+      } else {
+        zp = A.val_p[r * k + (j - k)];
+        za = warp_dot_bf16(ha, (const __nv_bfloat16*)A.weight_a + (int64_t)idx * A.ld_wa, A.H_a, lane);
+      }
+    }
+    if (lane == 0) { A.rec.idx[dst] = idx; A.rec.za[dst] = za; A.rec.zp[dst] = zp; }
+  }
+}
+}  // namespace
+
+cudaError_t launch_fused_records(const FusedRecordArgs& a, cudaStream_t s) {
+  if (a.T <= 0) return cudaSuccess;
+  fused_records_kernel<<<(unsigned)((a.T + 3) / 4), 128, 0, s>>>(a);
+  return cudaGetLastError();
+}
+
 size_t lmhead_scratch_bytes(int64_t T, int k, int splits) {
   // part_s (double) first, then part_m, part_zx, part_val, part_idx
   return (size_t)splits * (size_t)T * (8 + 4 + 4 + (size_t)k * 8) + 256;

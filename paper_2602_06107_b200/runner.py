@@ -118,3 +118,26 @@ def forward_sparse_actor(ctx: B.Context, zp, tokens, mask, logp_inf_token, topk_
     torch.cuda.synchronize(dev)
     out["stats"] = B.read_stats(out["stats_buf"])
     return out
+
+
+def forward_lmhead(ctx: B.Context, h_actor, w_actor, h_policy, w_policy, tokens, mask=None, *, lam=None, budget=None, k=20,
+                   seed=0, token_offset=0, c1=0.0):
+    """One jp_obrs_forward_lmhead call; returns a dict of device tensors plus ``stats``."""
+    assert (lam is None) != (budget is None)
+    T, V = h_actor.shape[0], w_actor.shape[0]
+    dev = h_actor.device
+    out = _alloc_outputs(T, dev)
+    auxd = _alloc_aux(T, k, V, dev, False)
+    d = B.jp_obrs_desc()
+    d.T, d.V = T, V
+    d.lambda_mode = B.JP_LAMBDA_FIXED if budget is None else B.JP_LAMBDA_FROM_BUDGET
+    d.c1, d.token_offset = c1, token_offset
+    for n, t in auxd.items():
+        setattr(d, n, t.data_ptr())
+    B.jp_obrs_forward_lmhead(ctx, d, h_actor, w_actor, h_policy, w_policy, tokens, mask,
+                             lam if budget is None else budget, k, seed, out["accept"], out["weight"],
+                             out["logp_actor"], out["logp_policy"], out["stats_buf"])
+    out.update(auxd)
+    torch.cuda.synchronize(dev)
+    out["stats"] = B.read_stats(out["stats_buf"])
+    return out

@@ -115,3 +115,89 @@ def test_fused_output_layer_arguments(ctx):
     hp = torch.zeros((16, 68), dtype=torch.bfloat16, device="cuda")[:, :64]       # pitch 136 bytes
     with pytest.raises(B.JackpotError, match="16 bytes"):
         run(ctx, hp, w, tok, None, 4)
+
+
+# ---- the whole forward with both models' output layers fused ------------------------------------
+
+def _two_models(T, V, Ha, Hp, seed, noise=1.0):
+    """Actor and policy as hidden states and output matrices whose logits are N(0, 9) and differ by
+    N(0, noise^2) (same hidden states, perturbed matrix) when the hidden sizes agree, unrelated otherwise."""
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    ha = torch.randn((T, Ha), generator=g, device="cuda").to(torch.bfloat16)
+    wa = (torch.randn((V, Ha), generator=g, device="cuda") * (3.0 / Ha ** 0.5)).to(torch.bfloat16)
+    if Hp == Ha:
+        hp = ha.clone()
+        wp = (wa.float() + torch.randn((V, Ha), generator=g, device="cuda") * (noise / Ha ** 0.5)).to(torch.bfloat16)
+    else:
+        hp = torch.randn((T, Hp), generator=g, device="cuda").to(torch.bfloat16)
+        wp = (torch.randn((V, Hp), generator=g, device="cuda") * (3.0 / Hp ** 0.5)).to(torch.bfloat16)
+    za = ha.float() @ wa.float().t()
+    gum = -torch.log(-torch.log(torch.rand((T, V), generator=g, device="cuda").clamp_(1e-30, 1 - 1e-7)))
+    tok = (za + gum).argmax(1).to(torch.int32)               # a draw from (about) the actor's distribution
+    return ha, wa, hp, wp, tok
+
+
+def _check_fused_forward(ctx, ha, wa, hp, wp, tok, mask, rows, k, seed, lam=None, budget=None, c1=0.0, whole_batch=True):
+    from paper_2602_06107_b200 import runner
+    out = runner.forward_lmhead(ctx, ha, wa, hp, wp, tok, mask, lam=lam, budget=budget, k=k, seed=seed, c1=c1)
+    assert out["stats"]["status"] == 0
+    za = oracle.lmhead_rows(rows, to_numpy_bits(ha.contiguous()), to_numpy_bits(wa.contiguous()))
+    zp = oracle.lmhead_rows(rows, to_numpy_bits(hp.contiguous()), to_numpy_bits(wp.contiguous()))
+    m = None if mask is None else mask.cpu().numpy()[rows]
+    lam_used = float(np.float32(out["stats"]["lambda_used"]))
+    if budget is not None and whole_batch:
+        ref_b = oracle.forward(za, zp, tok.cpu().numpy()[rows], m, budget=budget, k=k, seed=seed, c1=c1)
+        assert abs(lam_used - ref_b["lambda"]) <= 2e-4 * ref_b["lambda"]      # the ratios carry the logits' 2e-5
+    # everything else with lambda forced to the library's value; rows are consecutive from rows[0]
+    ref = oracle.forward(za, zp, tok.cpu().numpy()[rows], m, lam=lam_used, k=k, seed=seed, c1=c1, token_offset=int(rows[0]))
+    valid = (np.ones(len(rows), bool) if m is None else m != 0) & (ref["bad"] == 0)
+    g = {n: t.cpu().numpy()[rows] for n, t in out.items() if isinstance(t, torch.Tensor) and t.shape[:1] == tok.shape}
+    tol = lambda x, r=RTOL, a=ATOL: a + r * np.abs(x)
+    for got, want in ((g["logp_actor"], ref["lq64"]), (g["logp_policy"], ref["lp64"]), (g["lse_actor"], ref["lse_a"]),
+                      (g["lse_policy"], ref["lse_p"])):
+        assert np.all(np.abs(got[valid] - want[valid]) <= tol(want[valid]))
+    assert np.array_equal(g["uniform"], ref["u"])
+    assert np.all(np.abs(g["accept_prob"] - ref["a"]) <= 1e-4 * np.maximum(ref["a"], 1e-3))
+    flips = g["accept"] != ref["accept"]
+    near = np.abs(ref["u"].astype(np.float64) - ref["a"]) < 1e-4
+    assert not (flips & ~near).any()
+    assert np.all(np.abs(g["z_approx"] - ref["zk"]) <= 1e-6 + 3e-4 * ref["zk"])
+    same_lists = sum(int(np.array_equal(g["topk_idx_actor"][i], ref["topk_idx_a"][i]) and
+                         np.array_equal(g["topk_idx_policy"][i], ref["topk_idx_p"][i])) for i in range(len(rows)) if valid[i])
+    assert same_lists >= 0.9 * valid.sum(), (same_lists, valid.sum())
+    assert np.all(g["weight"][~valid] == 0) and np.all(g["accept"][~valid] == 0)
+    if whole_batch:
+        st, rs = out["stats"], ref["stats"]
+        assert st["n_valid"] == rs["n_valid"] and st["n_bad_token"] == rs["n_bad_token"]
+        assert abs(st["z_approx_mean"] - rs["z_approx_mean"]) <= 3e-4 * rs["z_approx_mean"]
+        assert abs(st["mean_accept_prob"] - rs["mean_accept_prob"]) <= 1e-4
+        if not flips.any():
+            assert abs(st["kappa"] - rs["kappa"]) <= 5e-4 * rs["kappa"]
+            assert np.all(np.abs(g["weight"] - ref["w64"]) <= 1e-6 + 6e-4 * np.abs(ref["w64"]))
+    return out
+
+
+def test_fused_forward_small(ctx):
+    for (T, V, Ha, Hp, k) in ((160, 3000, 256, 256, 16), (100, 777, 128, 192, 8)):
+        ha, wa, hp, wp, tok = _two_models(T, V, Ha, Hp, seed=T)
+        tok[5] = V + 2
+        mask = (torch.arange(T, device="cuda") % 6 != 1).to(torch.uint8)
+        rows = np.arange(T)
+        _check_fused_forward(ctx, ha, wa, hp, wp, tok, mask, rows, k, seed=3, lam=1.3, c1=3.0)
+        _check_fused_forward(ctx, ha, wa, hp, wp, tok, None, rows, k, seed=3, budget=0.6)
+    # its records do not serve the backward
+    from paper_2602_06107_b200 import runner
+    ha, wa, hp, wp, tok = _two_models(32, 1024, 64, 64, seed=1)
+    out = runner.forward_lmhead(ctx, ha, wa, hp, wp, tok, None, lam=1.0, k=8)
+    z = torch.zeros((ha.shape[0], wa.shape[0]), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(B.JackpotError, match="without both logit tensors"):
+        runner.backward(ctx, z, z, tok, None, out["accept"], out["weight"])
+
+
+def test_fused_forward_full_vocabulary(ctx):
+    T, V, H, k = 512, 151936, 1024, 20
+    ha, wa, hp, wp, tok = _two_models(T, V, H, H, seed=9)
+    rows = np.arange(200, 216)
+    out = _check_fused_forward(ctx, ha, wa, hp, wp, tok, None, rows, k, seed=4, lam=1.0, whole_batch=False)
+    st = out["stats"]
+    assert st["n_valid"] == T and abs(st["kappa"] * st["z_approx_mean"] - st["alpha_hat"]) < 1e-12
