@@ -74,13 +74,16 @@ constexpr uint32_t kTauPollNs = 200u;     // how long a top-k warp sleeps betwee
 // NSTAGES: depth of the ring.  NCAND: candidate passes a row may collect before it
 // falls back to a re-scan.  The kernel for k <= 64 takes 5 stages and 1024 candidates;
 // for k <= 128 (about k (1 + ln(passes / k)) candidates per row) 4 stages and 2048.
-template <int NSTAGES, int NCAND>
+// NT: tensors a stage holds.  With one tensor streamed (the sparse-actor forward) the ring has
+// twice the stages of half the size: the same bytes in flight as with two tensors.
+template <int NSTAGES, int NCAND, int NT>
 struct __align__(128) StreamSmemT {
   static constexpr int STAGES = NSTAGES;
+  static constexpr int TENSORS = NT;
   static constexpr int CAP = NCAND;
   static_assert(NG < NSTAGES, "every consumer group needs a stage of its own and one must be in flight");
   static_assert(SAMPLE <= NCAND, "the sample's vector maxima are parked in the candidate buffer");
-  uint4 ring[STAGES][2][TV];              // [stage][tensor][vector]
+  uint4 ring[STAGES][NT][TV];             // [stage][tensor][vector]
   unsigned long long skeys[NSLOT][2][SCAP];  // [slot][tensor] keys waiting to be sorted into the list
   uint32_t cand[NSLOT][2][CAP];           // [slot][tensor] candidate passes: high bits of the maximum's order bits | pass id; 0 = not written yet
   uint32_t hist[NSLOT][2][NB];            // [slot][tensor] candidate passes per bin of their maximum (kept by the top-k warp)
@@ -98,9 +101,10 @@ struct __align__(128) StreamSmemT {
   int abort;
 };
 
-template <int KPL>
-using StreamSmemFor = StreamSmemT<(KPL == 4 ? 4 : 5), (KPL == 4 ? 2048 : 1024)>;
-static_assert(sizeof(StreamSmemFor<1>) <= 232448 && sizeof(StreamSmemFor<4>) <= 232448,
+template <int KPL, bool SINGLE = false>
+using StreamSmemFor = StreamSmemT<(KPL == 4 ? 4 : 5) * (SINGLE ? 2 : 1), (KPL == 4 ? 2048 : 1024), (SINGLE ? 1 : 2)>;
+static_assert(sizeof(StreamSmemFor<1>) <= 232448 && sizeof(StreamSmemFor<4>) <= 232448 &&
+                  sizeof(StreamSmemFor<1, true>) <= 232448 && sizeof(StreamSmemFor<4, true>) <= 232448,
               "the CTA's shared memory exceeds the 227 KB an sm_100 CTA can have");
 
 // ---- mbarrier / bulk-copy wrappers ----------------------------------------
@@ -803,7 +807,7 @@ __device__ void producer_loop(const StreamArgs& A, SM& sm, int64_t n_rows) {
       if (bytes > 0) {
         mbar_arrive_expect_tx(&sm.full[grp][s], SINGLE ? bytes : 2u * bytes);
         if (!SINGLE) bulk_g2s(&sm.ring[s][0][0], ra, bytes, &sm.full[grp][s], policy);
-        bulk_g2s(&sm.ring[s][1][0], rp, bytes, &sm.full[grp][s], policy);
+        bulk_g2s(&sm.ring[s][SM::TENSORS - 1][0], rp, bytes, &sm.full[grp][s], policy);
       } else {
         mbar_arrive(&sm.full[grp][s]);
       }
@@ -860,7 +864,7 @@ __device__ void consumer_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int c
       if (!mbar_wait(&sm.full[gq][s], (fphase >> s) & 1u, &sm.abort)) return false;
       fphase ^= 1u << s;
       const uint4* sa = &sm.ring[s][0][wq * 32 + lane];
-      const uint4* sp = &sm.ring[s][1][wq * 32 + lane];
+      const uint4* sp = &sm.ring[s][SM::TENSORS - 1][wq * 32 + lane];
       float ta = 0.f, tp = 0.f;
       if (TOPK) { ta = lds_volatile_f32(&sm.tau[p][0]); tp = lds_volatile_f32(&sm.tau[p][1]); }
       uint32_t id = tile * (uint32_t)TP + (uint32_t)(wq * 32 + lane);
@@ -1153,7 +1157,7 @@ __device__ void topk_loop(const StreamArgs& A, SM& sm, int64_t n_rows, int t, in
 template <int DT, int KPL, bool SINGLE>
 __global__ void __launch_bounds__(NTHREADS, 1) stream_kernel(StreamArgs A) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
-  using SM = StreamSmemFor<KPL>;
+  using SM = StreamSmemFor<KPL, SINGLE>;
   constexpr int STAGES = SM::STAGES;
   SM& sm = *reinterpret_cast<SM*>(smem_raw);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -1331,9 +1335,9 @@ template <int DT, int KPL, bool SINGLE>
 static cudaError_t launch_stream_variant(const StreamArgs& a, cudaStream_t s, int grid) {
   // per device, and cheap: set on every launch rather than cached per process
   cudaError_t e = cudaFuncSetAttribute(stream_kernel<DT, KPL, SINGLE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (int)sizeof(StreamSmemFor<KPL>));
+                                       (int)sizeof(StreamSmemFor<KPL, SINGLE>));
   if (e != cudaSuccess) return e;
-  stream_kernel<DT, KPL, SINGLE><<<grid, NTHREADS, sizeof(StreamSmemFor<KPL>), s>>>(a);
+  stream_kernel<DT, KPL, SINGLE><<<grid, NTHREADS, sizeof(StreamSmemFor<KPL, SINGLE>), s>>>(a);
   return cudaGetLastError();
 }
 
