@@ -214,6 +214,10 @@ __global__ void __launch_bounds__(EPI_NT) epilogue_kernel(EpilogueArgs A) {
   __shared__ double s_zk[EPI_WARPS], s_a[EPI_WARPS], s_kl[EPI_WARPS];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int k = A.k;
+  // launched as a programmatic dependent of the kernel before it (the row stream, or the last
+  // step of the budget solve): nothing is read before that kernel has finished
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const float lambda = A.sc->lambda;
   const float log_lambda = logf(lambda);
   const double log_lambda64 = log((double)lambda);
@@ -334,6 +338,7 @@ __global__ void __launch_bounds__(EPI_NT) finalize_kernel(EpilogueArgs A) {
   __shared__ long long s_nv[EPI_NT], s_na[EPI_NT], s_nf[EPI_NT];
   __shared__ double s_zk[EPI_NT], s_a[EPI_NT], s_kl[EPI_NT];
   static_assert(kMaxPartials % EPI_NT == 0, "every thread starts from the same number of partial sums");
+  asm volatile("griddepcontrol.wait;" ::: "memory");          // a programmatic dependent of epilogue_kernel
   // every block folds the same partial sums in the same fixed order (so all blocks get the
   // same bits): thread i adds up partials i, i + EPI_NT, ... in turn, then halves are added pairwise
   {
@@ -468,11 +473,23 @@ cudaError_t launch_budget_solve(const EpilogueArgs& a, double budget, cudaStream
 }
 
 cudaError_t launch_epilogue(const EpilogueArgs& a, cudaStream_t s, int* n_launch) {
-  epilogue_kernel<<<a.n_part, EPI_NT, 0, s>>>(a);
-  unsigned blocks = (unsigned)((a.T + EPI_NT - 1) / EPI_NT);
-  finalize_kernel<<<blocks < 1 ? 1 : blocks, EPI_NT, 0, s>>>(a);
+  // both may be set up while the kernel before them still runs (they wait for its end themselves)
+  cudaLaunchAttribute attr{};
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg{};
+  cfg.blockDim = dim3(EPI_NT);
+  cfg.stream = s;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  cfg.gridDim = dim3((unsigned)a.n_part);
+  cudaError_t e = cudaLaunchKernelEx(&cfg, epilogue_kernel, a);
+  if (e != cudaSuccess) return e;
+  const unsigned blocks = (unsigned)((a.T + EPI_NT - 1) / EPI_NT);
+  cfg.gridDim = dim3(blocks < 1 ? 1 : blocks);
+  e = cudaLaunchKernelEx(&cfg, finalize_kernel, a);
   *n_launch += 2;
-  return cudaGetLastError();
+  return e;
 }
 
 cudaError_t launch_logprobs(int64_t T, const Records& rec, float* out_lq, float* out_lp, uint8_t* out_valid,

@@ -1175,6 +1175,11 @@ __global__ void __launch_bounds__(NTHREADS, 1) stream_kernel(StreamArgs A) {
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
+  // The kernel is launched as a programmatic dependent of the row-list kernel: its CTAs are set up
+  // (shared memory carved, barriers initialised) while that kernel still runs; nothing it wrote
+  // is read before this point.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // whatever follows may be set up; it waits for this grid's end itself
   const int64_t n_rows = A.sc->n_list;
 
   if (warp == 0) {
@@ -1192,6 +1197,7 @@ __global__ void __launch_bounds__(NTHREADS, 1) stream_kernel(StreamArgs A) {
 // Splits the rows of one call into the list of valid rows the stream kernel walks
 // and the masked / out-of-range ones, whose records are cleared here.
 __global__ void __launch_bounds__(256) prep_rows_kernel(StreamArgs A) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the stream kernel may start setting up
   const int64_t row = (int64_t)blockIdx.x * 256 + threadIdx.x;
   const int lane = threadIdx.x & 31;
   bool valid = false, bad = false;
@@ -1337,8 +1343,17 @@ static cudaError_t launch_stream_variant(const StreamArgs& a, cudaStream_t s, in
   cudaError_t e = cudaFuncSetAttribute(stream_kernel<DT, KPL, SINGLE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)sizeof(StreamSmemFor<KPL, SINGLE>));
   if (e != cudaSuccess) return e;
-  stream_kernel<DT, KPL, SINGLE><<<grid, NTHREADS, sizeof(StreamSmemFor<KPL, SINGLE>), s>>>(a);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(NTHREADS);
+  cfg.dynamicSmemBytes = sizeof(StreamSmemFor<KPL, SINGLE>);
+  cfg.stream = s;
+  cudaLaunchAttribute attr{};
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may begin while the row-list kernel before it runs
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, stream_kernel<DT, KPL, SINGLE>, a);
 }
 
 template <int DT>
