@@ -460,6 +460,15 @@ jp_status jp_budget_lambda_static(const float* logp_actor, const float* logp_pol
                                   const uint8_t* mask, int64_t T, float budget, float* out_lambda,
                                   void* cuda_stream);
 
+/* Self-test of the bounded waits (the paper has no counterpart).  Every wait inside the kernels
+ * of this library (on a shared-memory barrier that the copy engine, another warp or the tensor
+ * cores complete) gives up after a fixed number of SM clock cycles, sets JP_ERR_TIMEOUT in a
+ * device status word and lets the kernel end instead of trapping or hanging.  This call runs
+ * that routine against a barrier nobody completes, with a limit of limit_cycles (1 .. 2e9:
+ * about a second at most): out_status (one int32, DEVICE) must read JP_ERR_TIMEOUT afterwards
+ * and the context must work as before.  Enqueued on the context's stream; does not wait. */
+jp_status jp_selftest_bounded_wait(jp_ctx* ctx, int64_t limit_cycles, int32_t* out_status);
+
 const char* jp_status_string(jp_status s);
 const char* jp_last_error(jp_ctx* ctx);
 /* Number of kernel launches this context has enqueued so far. */

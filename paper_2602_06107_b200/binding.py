@@ -26,7 +26,7 @@ JP_DESC_SPARSE_CAP = 2
 EXPORTS = (
     "jp_create", "jp_destroy", "jp_set_stream", "jp_obrs_workspace_bytes", "jp_reserve",
     "jp_obrs_forward", "jp_obrs_forward_sparse_actor", "jp_lmhead_lse_topk", "jp_obrs_forward_lmhead", "jp_obrs_backward", "jp_batch_begin", "jp_batch_chunk", "jp_batch_finalize",
-    "jp_obrs_forward_host", "jp_obrs_apply_kappa", "jp_batch_totals", "jp_obrs_apply_totals", "jp_batch_logprobs", "jp_obrs_row_lambda", "jp_vshard_record_floats", "jp_vshard_local", "jp_vshard_local_push", "jp_vshard_merge", "jp_vshard_backward", "jp_budget_lambda_static", "jp_probe_stream", "jp_status_string", "jp_last_error", "jp_launch_count",
+    "jp_obrs_forward_host", "jp_selftest_bounded_wait", "jp_obrs_apply_kappa", "jp_batch_totals", "jp_obrs_apply_totals", "jp_batch_logprobs", "jp_obrs_row_lambda", "jp_vshard_record_floats", "jp_vshard_local", "jp_vshard_local_push", "jp_vshard_merge", "jp_vshard_backward", "jp_budget_lambda_static", "jp_probe_stream", "jp_status_string", "jp_last_error", "jp_launch_count",
     "jp_enable_kernel_timing", "jp_stream_kernel_times",
 )
 
@@ -110,6 +110,7 @@ def load():
                                      vp, vp, vp, vp, vp, vp, vp, vp]
     lib.jp_obrs_apply_kappa.argtypes = [vp, ctypes.c_double, f32, vp]
     lib.jp_batch_logprobs.argtypes = [vp, vp, vp, vp]
+    lib.jp_selftest_bounded_wait.argtypes = [vp, i64, vp]
     lib.jp_batch_totals.argtypes = [vp, vp]
     lib.jp_obrs_apply_totals.argtypes = [vp, vp, f32, vp, vp]
     lib.jp_obrs_row_lambda.argtypes = [vp, ctypes.POINTER(jp_obrs_desc), vp, vp, vp, f32, vp, vp, vp, vp]
@@ -312,6 +313,10 @@ def jp_batch_logprobs(ctx: Context, out_logp_actor, out_logp_policy, out_valid):
 
 def jp_obrs_apply_kappa(ctx: Context, kappa: float, c1: float, out_weight):
     ctx.check(ctx.lib.jp_obrs_apply_kappa(ctx.h, kappa, c1, _ptr(out_weight)))
+
+
+def jp_selftest_bounded_wait(ctx: Context, limit_cycles: int, out_status):
+    ctx.check(ctx.lib.jp_selftest_bounded_wait(ctx.h, limit_cycles, _ptr(out_status)))
 
 
 def jp_batch_totals(ctx: Context, out_totals):

@@ -781,6 +781,18 @@ jp_status jp_batch_logprobs(jp_ctx* c, float* out_logp_actor, float* out_logp_po
   return JP_OK;
 }
 
+jp_status jp_selftest_bounded_wait(jp_ctx* c, int64_t limit_cycles, int32_t* out_status) {
+  if (!c) return JP_ERR_INVALID_ARG;
+  if (limit_cycles < 1 || limit_cycles > 2000000000ll) return fail(c, JP_ERR_INVALID_ARG, "limit_cycles must lie in [1, 2e9] (about a second at most)");
+  if (!out_status) return fail(c, JP_ERR_INVALID_ARG, "out_status is NULL");
+  cudaSetDevice(c->device);
+  cudaError_t e = cudaMemsetAsync(out_status, 0, sizeof(int32_t), c->stream);
+  if (e == cudaSuccess) e = launch_wait_selftest((long long)limit_cycles, out_status, c->stream);
+  if (e != cudaSuccess) return cuda_fail(c, e, "self-test launch");
+  c->launches += 1;
+  return JP_OK;
+}
+
 jp_status jp_obrs_apply_kappa(jp_ctx* c, double kappa, float c1, float* out_weight) {
   if (!c) return JP_ERR_INVALID_ARG;
   if (!c->have_records) return fail(c, JP_ERR_STATE, "no forward records in this context: run the forward (or finalize the batch) first");

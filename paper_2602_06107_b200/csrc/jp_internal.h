@@ -189,6 +189,7 @@ struct RowLambdaArgs {
 int stream_grid_size(int device);   // number of SMs
 cudaError_t launch_stream(const StreamArgs& a, cudaStream_t s, int sms);
 cudaError_t launch_exact_z(const ExactZArgs& a, cudaStream_t s, int sms);
+cudaError_t launch_wait_selftest(long long limit_cycles, int32_t* status, cudaStream_t s);
 cudaError_t launch_reset(Scalars* sc, float lambda_fixed, cudaStream_t s);
 cudaError_t launch_clear_flags(uint8_t* flag, int64_t n, cudaStream_t s);
 cudaError_t launch_budget_solve(const EpilogueArgs& a, double budget, cudaStream_t s, int* n_launch);

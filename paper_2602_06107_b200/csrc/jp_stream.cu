@@ -152,7 +152,8 @@ __device__ __forceinline__ bool mbar_try_wait_for(unsigned long long* bar, uint3
 // Bounded wait; false = gave up (or another warp did).  The first poll is inline;
 // the loop is out of line (the streaming code stays small).  The clock is read once
 // in 64 polls, each of which may itself suspend the thread for a while.
-__device__ __noinline__ bool mbar_wait_slow(unsigned long long* bar, uint32_t parity, volatile int* abort) {
+__device__ __noinline__ bool mbar_wait_slow(unsigned long long* bar, uint32_t parity, volatile int* abort,
+                                            long long limit = kSpinLimit) {
   long long t0 = 0;
   for (uint32_t i = 0;; ++i) {
     if (mbar_try_wait_for(bar, parity, 2000u)) return true;
@@ -160,7 +161,7 @@ __device__ __noinline__ bool mbar_wait_slow(unsigned long long* bar, uint32_t pa
       if (*abort) return false;
       const long long now = clock64();
       if (i == 0u) t0 = now;
-      else if (now - t0 > kSpinLimit) { *abort = 1; return false; }
+      else if (now - t0 > limit) { *abort = 1; return false; }
     }
   }
 }
@@ -1329,6 +1330,31 @@ __global__ void __launch_bounds__(XNT, XCTAS_PER_SM) exact_z_kernel(ExactZArgs A
     }
     __syncthreads();
   }
+}
+
+// Self-test of the bounded wait: one CTA whose warps wait, through the same routine as the row
+// kernel's roles, on a barrier that nobody ever arrives at, with a limit the caller gives.  The
+// wait must run out, raise the CTA's abort flag (which releases the warps still waiting), leave
+// JP_ERR_TIMEOUT in the status word and let the kernel end: no trap, no hang, the context stays
+// usable.
+__global__ void __launch_bounds__(128) wait_selftest_kernel(long long limit_cycles, int32_t* status) {
+  __shared__ unsigned long long bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  // warp 0 has the caller's limit; the others the kernel's own two seconds: they must be let go by
+  // the abort flag, as the row kernel's other roles are
+  const bool ok = mbar_wait_slow(&bar, 0u, &abort_flag, (threadIdx.x >> 5) == 0 ? limit_cycles : kSpinLimit);
+  if (!ok && (threadIdx.x & 31) == 0) atomicExch(status, (int)JP_ERR_TIMEOUT);
+}
+
+cudaError_t launch_wait_selftest(long long limit_cycles, int32_t* status, cudaStream_t s) {
+  wait_selftest_kernel<<<1, 128, 0, s>>>(limit_cycles, status);
+  return cudaGetLastError();
 }
 
 int stream_grid_size(int device) {

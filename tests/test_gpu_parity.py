@@ -614,3 +614,23 @@ def test_stream_probe_reports_a_plausible_rate():
     assert 1000.0 < rd < 12000.0 and 1000.0 < cp < 12000.0
     with pytest.raises(B.JackpotError):
         B.jp_probe_stream(x[1:], None, reps=1)          # not 16-byte aligned
+
+
+def test_a_wait_that_nothing_completes_runs_out_and_leaves_the_context_usable(ctx):
+    """The bounded wait of the kernels, against a barrier nobody arrives at, with a short limit (about
+    50 ms of SM clock): the kernel ends by itself, the status word reads JP_ERR_TIMEOUT, and the next
+    forward on the same context is unaffected."""
+    import time
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    B.jp_selftest_bounded_wait(ctx, 100_000_000, st)
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    assert st.item() == -6                                   # JP_ERR_TIMEOUT
+    assert 0.01 < dt < 1.5, dt
+    r = LogitRecipe(T=40, V=4096, dtype="bf16", sigma0=2.0, peaks=2, sigma=0.6, seed=77)
+    za, zp, tok = make_logits(r, "cuda")
+    run_case(ctx, za, zp, tok, lam=1.2, k=8, seed=1)
+    with pytest.raises(B.JackpotError, match="limit_cycles"):
+        B.jp_selftest_bounded_wait(ctx, 0, st)
