@@ -181,7 +181,7 @@ jp_status jp_obrs_forward_sparse_actor(jp_ctx* ctx, const jp_obrs_desc* desc, co
  *   out_lse [T] fp32         log sum_v exp z[t, v]
  *   out_logp_token [T] fp32  z[t, tokens[t]] - lse
  *   out_topk_idx / out_topk_val [T, k]  the k largest logits, best first, equal values by lower
- *                            index, and their values; 1 <= k <= 32
+ *                            index, and their values; 1 <= k <= 64
  * which is what Algorithm 1 keeps of a forward pass (Phase 1: log p(a_t) and the top-k
  * log-probabilities; Phase 2 step 1 likewise for the policy).
  *   hidden : [T, ld_hidden] bf16, weight : [V, ld_weight] bf16 (the output layer's matrix, one row
@@ -210,7 +210,7 @@ jp_status jp_lmhead_lse_topk(jp_ctx* ctx, const void* hidden, int64_t ld_hidden,
  *          whole rows of logits).
  *   hidden_actor [T, ld_ha] / weight_actor [V, ld_wa] with hidden size H_actor, and the same for
  *   the policy (the two models may differ in hidden size): bf16, DEVICE, 16-byte aligned,
- *   pitches multiples of 16 bytes (ld = 0 means H).  1 <= k <= 32, k < V.
+ *   pitches multiples of 16 bytes (ld = 0 means H).  1 <= k <= 64, k < V.
  * Outputs as in jp_obrs_forward.  The logits keep the precision of the fp32 accumulator, so
  * log-probs agree with a forward over stored bf16 logits only to the rounding of those.  The
  * records this call leaves do not serve jp_obrs_backward (JP_ERR_STATE). */

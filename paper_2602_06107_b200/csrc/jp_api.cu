@@ -446,7 +446,7 @@ jp_status jp_lmhead_lse_topk(jp_ctx* c, const void* hidden, int64_t ld_hidden, c
                              int32_t* out_status) {
   if (!c) return JP_ERR_INVALID_ARG;
   if (T < 0 || H < 1 || V < 1 || V > (int64_t)0x7fffffff) return fail(c, JP_ERR_INVALID_ARG, "T < 0, H < 1 or V out of range");
-  if (k < 1 || k > kLmheadMaxK) return fail(c, JP_ERR_UNSUPPORTED, "the fused output-layer pass keeps lists of 1 <= k <= 32 entries");
+  if (k < 1 || k > kLmheadMaxK) return fail(c, JP_ERR_UNSUPPORTED, "the fused output-layer pass keeps lists of 1 <= k <= 64 entries");
   if (ld_hidden == 0) ld_hidden = H;
   if (ld_weight == 0) ld_weight = H;
   if (ld_hidden < H || ld_weight < H) return fail(c, JP_ERR_INVALID_ARG, "leading dimension < H");
@@ -490,7 +490,7 @@ jp_status jp_obrs_forward_lmhead(jp_ctx* c, const jp_obrs_desc* d, const void* h
   if (T < 0 || V < 1 || V > (int64_t)0x7fffffff || H_actor < 1 || H_policy < 1)
     return fail(c, JP_ERR_INVALID_ARG, "T < 0, V out of range or a hidden size < 1");
   if (k < 1 || k > kLmheadMaxK || (int64_t)k >= V)
-    return fail(c, JP_ERR_UNSUPPORTED, "the fused output-layer pass keeps lists of 1 <= k <= 32 entries, k < V");
+    return fail(c, JP_ERR_UNSUPPORTED, "the fused output-layer pass keeps lists of 1 <= k <= 64 entries, k < V");
   jp_status st = check_lambda(c, lambda_or_budget, d->lambda_mode);
   if (st != JP_OK) return st;
   if (c->batch_open) return fail(c, JP_ERR_STATE, "a chunked batch is open: finalize it first");

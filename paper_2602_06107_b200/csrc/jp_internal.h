@@ -227,7 +227,7 @@ cudaError_t launch_vshard_merge(int n_shards, int my_shard, const float* gathere
 cudaError_t launch_grad(const GradArgs& a, cudaStream_t s, int sms, int* n_launch);
 
 // Output layer fused with the row pass (jp_lmhead.cu).
-constexpr int kLmheadMaxK = 32;
+constexpr int kLmheadMaxK = 64;
 struct FusedRecordArgs {
   const void* hidden_a; const void* weight_a; const void* hidden_p; const void* weight_p;   // bf16, row-major
   int64_t ld_ha, ld_wa, ld_hp, ld_wp, H_a, H_p;

@@ -38,7 +38,6 @@ constexpr int LM_BN = 256;                 // vocabulary columns per accumulator
 constexpr int LM_BK = 64;                  // K per stage: 64 bf16 = one 128-byte swizzle row
 constexpr int LM_UMMA_K = 16;              // K per tcgen05.mma of kind::f16
 constexpr int LM_THREADS = 192;
-constexpr int LM_KMAX = 32;                // longest list the epilogue keeps per row
 constexpr uint32_t LM_A_BYTES = LM_BM * LM_BK * 2;     // 16 KB
 constexpr uint32_t LM_B_BYTES = LM_BN * LM_BK * 2;     // 32 KB
 constexpr uint32_t LM_TMEM_COLS = 512;     // two accumulators of 256 columns
@@ -49,20 +48,23 @@ constexpr long long kLmSpin = 4000000000ll;
 // 32 KB per stage), one thread of the even CTA issues MMAs of M = 256 that read both CTAs' shared
 // memory and fill both CTAs' tensor memory.  Per SM the operand traffic of a tile falls by a
 // third, and six stages fit where four did.
-template <bool PAIR>
+// KMAX: the longest list a row keeps (32 or 64); the longer lists take the place of one stage.
+template <bool PAIR, int KMAX>
 struct __align__(1024) LmSmemT {
-  static constexpr int STAGES = PAIR ? 6 : 4;
+  static constexpr int STAGES = (PAIR ? 6 : 4) - (KMAX > 32 ? 1 : 0);
   static constexpr uint32_t B_BYTES = PAIR ? LM_B_BYTES / 2 : LM_B_BYTES;
   unsigned char a[STAGES][LM_A_BYTES];     // [stage] 128 rows x 128 B, swizzled by the copy engine
   unsigned char b[STAGES][B_BYTES];        // [stage] 256 (PAIR: 128) rows x 128 B
-  unsigned long long list[LM_KMAX][LM_BM]; // per row: the k best so far as (order bits, ~column) keys, unsorted
+  unsigned long long list[KMAX][LM_BM];    // per row: the k best so far as (order bits, ~column) keys, unsorted
                                            // (row fastest: no bank conflicts); 0 = empty place
   unsigned long long full[STAGES], empty[STAGES];
   unsigned long long acc_full[2], acc_empty[2];
   uint32_t tmem_base;
   int abort;
 };
-static_assert(sizeof(LmSmemT<false>) <= 231424 && sizeof(LmSmemT<true>) <= 231424, "beyond the 227 KB a CTA can have");
+static_assert(sizeof(LmSmemT<false, 32>) <= 231424 && sizeof(LmSmemT<true, 32>) <= 231424 &&
+                  sizeof(LmSmemT<false, 64>) <= 231424 && sizeof(LmSmemT<true, 64>) <= 231424,
+              "beyond the 227 KB a CTA can have");
 
 struct LmArgs {
   const int32_t* tokens;
@@ -244,11 +246,11 @@ __device__ __forceinline__ void list_sort(SM& sm, int row, int k) {
   }
 }
 
-template <bool PAIR>
+template <bool PAIR, int KMAX>
 __global__ void __launch_bounds__(LM_THREADS, 1) lmhead_kernel(const __grid_constant__ CUtensorMap map_a,
                                                                const __grid_constant__ CUtensorMap map_b, LmArgs A) {
   extern __shared__ unsigned char lm_raw[];
-  using SM = LmSmemT<PAIR>;
+  using SM = LmSmemT<PAIR, KMAX>;
   constexpr int LM_STAGES = SM::STAGES;
   SM& sm = *reinterpret_cast<SM*>(((uintptr_t)lm_raw + 1023) & ~(uintptr_t)1023);
   // in a pair the even CTA leads: it issues the MMAs and owns the barriers the copies are counted on
@@ -631,6 +633,25 @@ int lmhead_splits(int64_t T, int64_t V, int sms) {
   return (n_tiles + tps - 1) / tps;         // every split has at least one tile
 }
 
+template <bool PAIR, int KMAX>
+static cudaError_t launch_lmhead_variant(dim3 grid, const CUtensorMap& map_a, const CUtensorMap& map_b, const LmArgs& a,
+                                         cudaStream_t s) {
+  const size_t smem = sizeof(LmSmemT<PAIR, KMAX>) + 1024;
+  cudaError_t e = cudaFuncSetAttribute(lmhead_kernel<PAIR, KMAX>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(LM_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr{};
+  attr.id = cudaLaunchAttributeClusterDimension;
+  attr.val.clusterDim.x = PAIR ? 2 : 1; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, lmhead_kernel<PAIR, KMAX>, map_a, map_b, a);
+}
+
 cudaError_t launch_lmhead(const void* hidden, int64_t ldh, const void* weight, int64_t ldw, const int32_t* tokens,
                           const uint8_t* mask, int64_t T, int64_t H, int64_t V, int k, int splits, void* scratch,
                           int32_t* status, float* out_lse, float* out_logp, int32_t* out_idx, float* out_val,
@@ -666,26 +687,11 @@ cudaError_t launch_lmhead(const void* hidden, int64_t ldh, const void* weight, i
   if (pair) {
     // clusters of two CTAs along x: row blocks 2i and 2i + 1 (an odd count is rounded up: the extra
     // CTA works on rows beyond T, which read as zero and are never written)
-    const size_t smem = sizeof(LmSmemT<true>) + 1024;
-    e = cudaFuncSetAttribute(lmhead_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3((m_blocks + 1) / 2 * 2, (unsigned)splits);
-    cfg.blockDim = dim3(LM_THREADS);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = s;
-    cudaLaunchAttribute attr{};
-    attr.id = cudaLaunchAttributeClusterDimension;
-    attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
-    cfg.attrs = &attr;
-    cfg.numAttrs = 1;
-    e = cudaLaunchKernelEx(&cfg, lmhead_kernel<true>, map_a, map_b, a);
+    const dim3 grid((m_blocks + 1) / 2 * 2, (unsigned)splits);
+    e = k <= 32 ? launch_lmhead_variant<true, 32>(grid, map_a, map_b, a, s) : launch_lmhead_variant<true, 64>(grid, map_a, map_b, a, s);
   } else {
-    const size_t smem = sizeof(LmSmemT<false>) + 1024;
-    e = cudaFuncSetAttribute(lmhead_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    lmhead_kernel<false><<<dim3(m_blocks, (unsigned)splits), LM_THREADS, smem, s>>>(map_a, map_b, a);
-    e = cudaGetLastError();
+    const dim3 grid(m_blocks, (unsigned)splits);
+    e = k <= 32 ? launch_lmhead_variant<false, 32>(grid, map_a, map_b, a, s) : launch_lmhead_variant<false, 64>(grid, map_a, map_b, a, s);
   }
   if (e != cudaSuccess) return e;
   lmhead_merge_kernel<<<(unsigned)((T + 3) / 4), 128, 0, s>>>(a, out_lse, out_logp, out_idx, out_val);

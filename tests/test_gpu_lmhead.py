@@ -86,7 +86,8 @@ def check(ctx, h, w, tok, mask, k, rows):
 
 
 def test_fused_output_layer_small(ctx):
-    for (T, H, V, k) in ((200, 256, 1000, 8), (129, 192, 777, 32), (64, 64, 256, 1), (300, 520, 5003, 20)):
+    for (T, H, V, k) in ((200, 256, 1000, 8), (129, 192, 777, 32), (64, 64, 256, 1), (300, 520, 5003, 20), (260, 128, 2000, 40),
+                         (100, 256, 900, 64)):
         h, w, tok = make(T, H, V, seed=T + V, ldh=H + 8, ldw=H + 24)
         tok[3] = V + 1
         mask = (torch.arange(T, device="cuda") % 5 != 2).to(torch.uint8)
@@ -110,8 +111,8 @@ def test_fused_output_layer_full_vocabulary(ctx):
 
 def test_fused_output_layer_arguments(ctx):
     h, w, tok = make(16, 64, 300, seed=1)
-    with pytest.raises(B.JackpotError, match="32"):
-        run(ctx, h, w, tok, None, 33)
+    with pytest.raises(B.JackpotError, match="64"):
+        run(ctx, h, w, tok, None, 65)
     hp = torch.zeros((16, 68), dtype=torch.bfloat16, device="cuda")[:, :64]       # pitch 136 bytes
     with pytest.raises(B.JackpotError, match="16 bytes"):
         run(ctx, hp, w, tok, None, 4)
@@ -178,7 +179,7 @@ def _check_fused_forward(ctx, ha, wa, hp, wp, tok, mask, rows, k, seed, lam=None
 
 
 def test_fused_forward_small(ctx):
-    for (T, V, Ha, Hp, k) in ((160, 3000, 256, 256, 16), (100, 777, 128, 192, 8)):
+    for (T, V, Ha, Hp, k) in ((160, 3000, 256, 256, 16), (100, 777, 128, 192, 8), (200, 2000, 128, 128, 40)):
         ha, wa, hp, wp, tok = _two_models(T, V, Ha, Hp, seed=T)
         tok[5] = V + 2
         mask = (torch.arange(T, device="cuda") % 6 != 1).to(torch.uint8)
