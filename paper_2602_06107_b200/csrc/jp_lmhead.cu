@@ -7,8 +7,8 @@
 //
 // Shape of the kernel (one CTA per SM, 192 threads; with more than 128 rows the CTAs work in pairs,
 // see LmSmemT):
-//   warp 0      one lane issues the TMA loads (cp.async.bulk.tensor.2d, 128-byte swizzle, no
-//               multicast) of the next K-slab of both operands into a ring of shared-memory
+//   warp 0      one lane issues the TMA loads (cp.async.bulk.tensor.2d, 128-byte swizzle; every
+//               byte is fetched by exactly one CTA) of the next K-slab of both operands into a ring of shared-memory
 //               stages; completion is counted on an mbarrier per stage;
 //   warp 1      allocates tensor memory; one lane issues tcgen05.mma (M = 128 rows, N = 256
 //               columns, K = 16 per instruction, cta_group::1) into one of two accumulators of
