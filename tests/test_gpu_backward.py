@@ -56,7 +56,9 @@ def check_grads(da, dp, rows, za_np, zp_np, tok, mask, acc, w, lse_a, lse_p, n_v
     assert np.all(ga[~valid] == 0) and np.all(gp[~valid] == 0)
     rej = valid & (acc[rows] == 0)
     assert np.all(gp[rej] == 0), "a rejected token must not reach the policy gradient"
-    tol_sum = 2.0 ** -8 * np.abs(ra).sum(1) + 1e-12          # bf16 rounding of V terms
+    # bf16 rounding of V terms, plus the elementwise floor of the bar above summed over the row (where the
+    # gradients are tiny, A_t near 0, the floor and not the rounding is what bounds the elements)
+    tol_sum = 2.0 ** -8 * np.abs(ra).sum(1) + floor_a.sum(1) + 1e-12
     assert np.all(np.abs(ga.sum(1)) <= tol_sum + np.abs(ra.sum(1)))
     return needed_floor
 

@@ -80,3 +80,46 @@ def test_random_fused_output_layer_cases_against_the_oracle(ctx):
         h, w, tok = fused.make(T, H, V, seed=it, ldh=H + 8 * rng.randint(0, 2), ldw=H + 8 * rng.randint(0, 2))
         mask = None if it % 2 else (torch.arange(T, device="cuda") % 3 != 1).to(torch.uint8)
         fused.check(ctx, h, w, tok, mask, k, np.arange(T))
+
+
+def test_random_backward_cases_against_the_oracle(ctx):
+    """The fused gradients on random shapes (both dtypes, ragged widths, padded pitches, masks, in-place or
+    not, with and without the distillation term) against the oracle's double gradients at the backward's bar."""
+    from test_gpu_backward import check_grads
+    rng = random.Random(31)
+    for it in range(24):
+        dt = rng.choice(["bf16", "f32"])
+        V = rng.choice([rng.randint(40, 600), rng.randint(600, 20000)])
+        ld = -(-V // 8) * 8 + 8 * rng.choice([0, 0, 2])                  # gradients are bf16: pitch in units of 8
+        T = rng.randint(1, 120)
+        k = min(rng.choice([4, 16, 32]), V - 1)
+        r = LogitRecipe(T=T, V=ld, dtype=dt, sigma0=rng.choice([1.0, 2.5]), peaks=rng.choice([0, 4]), peak_lo=4.0, peak_hi=10.0,
+                        sigma=rng.choice([0.3, 1.0]), seed=rng.randint(0, 10 ** 6))
+        zaf, zpf, _ = make_logits(r, "cuda")
+        za, zp = zaf[:, :V], zpf[:, :V]
+        g = torch.Generator(device="cuda").manual_seed(100 + it)
+        gum = -torch.log(-torch.log(torch.rand((T, V), generator=g, device="cuda").clamp_(1e-30, 1 - 1e-7)))
+        tok = (za.float() + gum).argmax(1).to(torch.int32)
+        mask = None if rng.random() < 0.4 else (torch.rand(T, generator=g, device="cuda") > 0.25).to(torch.uint8)
+        adv = None if rng.random() < 0.3 else torch.randn(T, generator=g, device="cuda")
+        lam_d, gout = rng.choice([0.0, 1.0, 0.3]), rng.choice([1.0, 2.5])
+        out = runner.forward(ctx, za, zp, tok, mask, lam=rng.choice([0.7, 1.3]), k=k, seed=it, c1=rng.choice([0.0, 3.0]))
+        if out["stats"]["n_valid"] == 0:
+            continue
+        za_np, zp_np = to_numpy_bits(za.contiguous()), to_numpy_bits(zp.contiguous())
+        in_place = dt == "bf16" and rng.random() < 0.3
+        za_in = za.clone() if in_place else za                       # the in-place call overwrites its logits
+        zp_in = zp.clone() if in_place else zp
+        if in_place:
+            zfa, zfp = zaf.clone(), zpf.clone()
+            za_in, zp_in = zfa[:, :V], zfp[:, :V]
+        da, dp = runner.backward(ctx, za_in, zp_in, tok, mask, out["accept"], out["weight"], advantages=adv,
+                                 lambda_distill=lam_d, grad_out=gout, d_actor=za_in if in_place else None,
+                                 d_policy=zp_in if in_place else None)
+        torch.cuda.synchronize()
+        m = None if mask is None else mask.cpu().numpy()
+        lg = oracle.lse_gather(za_np, zp_np, tok.cpu().numpy(), m)
+        rows = np.arange(T)
+        check_grads(da, dp, rows, za_np, zp_np, tok.cpu().numpy(), m, out["accept"].cpu().numpy(),
+                    out["weight"].cpu().numpy(), lg["lse_a"], lg["lse_p"], out["stats"]["n_valid"],
+                    None if adv is None else adv.cpu().numpy(), lam_d, g=gout)
